@@ -1,0 +1,359 @@
+"""Pins for the fp64 oracle against what the paper and the mathematics fix.
+
+Each test names the passage it rests on.  Expected values are computed here with
+library routines (scipy softmax, numpy cumsum/searchsorted) or closed forms, never
+by calling the oracle on itself.
+"""
+import numpy as np
+import pytest
+from scipy import stats
+from scipy.special import softmax as sp_softmax
+
+import oracle
+
+EPS = 1e-10
+
+
+def tile(rows_t, rows_d, toks, B):
+    """Same (target, draft, tokens) for B sequences; only the random counters differ."""
+    t = np.broadcast_to(np.asarray(rows_t, np.float32), (B,) + np.shape(rows_t)).copy()
+    d = np.broadcast_to(np.asarray(rows_d, np.float32), (B,) + np.shape(rows_d)).copy()
+    x = np.broadcast_to(np.asarray(toks, np.int32), (B, len(toks))).copy()
+    return t, d, x
+
+
+def closed_form_accept(t_rows, d_rows, toks, T, beta):
+    """a_k = min(1, R_k + beta (1 - max P_t)): the acceptance region [0, R + Tol] of Sec. 3.2."""
+    a = []
+    for k, tok in enumerate(toks):
+        pt = sp_softmax(np.asarray(t_rows[k], np.float64) / T)
+        pd = sp_softmax(np.asarray(d_rows[k], np.float64) / T)
+        R = pt[tok] / max(pd[tok], EPS)
+        a.append(min(1.0, R + beta * (1.0 - pt.max())))
+    return np.array(a)
+
+
+# --------------------------------------------------------------------------- softmax
+def test_softmax_matches_library_routine():
+    rng = np.random.default_rng(1)
+    for V, T in [(7, 1.0), (1000, 0.7), (32000, 1.3)]:
+        l = rng.normal(0, 3, V)
+        p, m, Z = oracle.softmax(l, T)
+        np.testing.assert_allclose(p, sp_softmax(l / T), rtol=1e-12, atol=0)
+        assert m == l.max()
+        assert abs(p.sum() - 1) < 1e-12
+        assert abs(p.max() - 1.0 / Z) < 1e-15  # max P = exp(0)/Z: what the GPU path relies on
+        p2, _, _ = oracle.softmax(l + 123.25, T)  # shift invariance
+        np.testing.assert_allclose(p2, p, rtol=1e-9)
+
+
+def test_softmax_masked_and_bad_rows():
+    p, _, _ = oracle.softmax([0.0, -np.inf, 1.0], 1.0)
+    assert p[1] == 0.0 and abs(p.sum() - 1) < 1e-15
+    for bad in ([0.0, np.nan], [np.inf, 0.0], [-np.inf, -np.inf]):
+        with pytest.raises(ValueError):
+            oracle.softmax(bad, 1.0)
+
+
+# ----------------------------------------------------------------------- inverse CDF
+def test_inverse_cdf_matches_searchsorted():
+    rng = np.random.default_rng(2)
+    for V in (1, 2, 8, 1000):
+        r = rng.random(V)
+        r[rng.random(V) < 0.3] = 0.0
+        if r.sum() == 0:
+            r[0] = 1.0
+        C = np.cumsum(r)
+        for u in rng.random(200):
+            got = oracle.inverse_cdf(r, u)
+            want = int(np.searchsorted(C, u * C[-1], side="right"))
+            assert got["token"] == want
+            assert r[want] > 0
+            assert got["lo"] <= u < got["hi"] + 1e-15
+
+
+def test_inverse_cdf_hand_cases():
+    r = [0.0, 0.25, 0.0, 0.5, 0.25, 0.0]
+    assert oracle.inverse_cdf(r, 0.0)["token"] == 1          # u = 0 -> first positive mass
+    assert oracle.inverse_cdf(r, 0.2499999)["token"] == 1
+    assert oracle.inverse_cdf(r, 0.25)["token"] == 3         # boundary belongs to the next token (strict <)
+    assert oracle.inverse_cdf(r, 0.75)["token"] == 4
+    assert oracle.inverse_cdf(r, 1.0 - 2.0**-53)["token"] == 4
+    assert oracle.inverse_cdf([0, 0, 0], 0.5)["token"] == -1
+    near = oracle.inverse_cdf(r, 0.25 + 1e-9, band=1e-6)
+    assert (near["token"], near["band_lo"], near["band_hi"]) == (3, 1, 3)
+
+
+# -------------------------------------------------- closed-form acceptance probability
+@pytest.mark.parametrize("beta,T", [(0.0, 1.0), (0.1, 0.9), (0.5, 1.3), (1.0, 1.0)])
+def test_acceptance_probability_closed_form(beta, T):
+    """P(accept position k) = min(1, R_k + Tol_k) for U uniform (Sec. 3.2, acceptance region)."""
+    rng = np.random.default_rng(3)
+    K, V, B = 3, 6, 200_000
+    t_rows = rng.normal(0, 1.5, (K + 1, V))
+    d_rows = t_rows[:K] + rng.normal(0, 1.0, (K, V))
+    toks = [1, 4, 2]
+    t, d, x = tile(t_rows, d_rows, toks, B)
+    res = oracle.verify(t, d, x, T, beta, seed=5, offset=9, nthreads=4)
+    # float32 storage of the rows: recompute the closed form from what the oracle saw
+    a = closed_form_accept(t[0], d[0], toks, np.float32(T), np.float32(beta))
+    emp = (res.cls != 0).mean(axis=0)
+    sigma = np.sqrt(np.maximum(a * (1 - a), 1e-12) / B)
+    assert np.all(np.abs(emp - a) < 5 * sigma + 1e-9), (emp, a)
+    # first-rejection logic (Sec. 3.1): P(n = j) = prod_{i<j} a_i * (1 - a_j)
+    pn = np.array([np.prod(a[:j]) * (1 - a[j]) for j in range(K)] + [np.prod(a)])
+    counts = np.bincount(res.accept_len, minlength=K + 1)
+    keep = pn * B > 5
+    chi = ((counts[keep] - pn[keep] * B) ** 2 / (pn[keep] * B)).sum()
+    assert chi < stats.chi2.ppf(1 - 1e-5, max(keep.sum() - 1, 1)), (counts, pn * B)
+    assert counts[~keep].sum() <= 5 * (pn[~keep].sum() * B + 2)
+
+
+# ------------------------------------------------------------- output law, tiny vocab
+def _law(pt, pd, beta):
+    """Law of the token emitted at position 0 when x ~ P_d (refs [1],[2] with the EARS region)."""
+    a = np.minimum(1.0, pt / np.maximum(pd, EPS) + beta * (1 - pt.max()))
+    res = np.maximum(pt - pd, 0.0)
+    rej = (pd * (1 - a)).sum()
+    return pd * a + (rej * res / res.sum() if res.sum() > 0 else 0.0)
+
+
+@pytest.mark.parametrize("V,beta", [(4, 0.0), (8, 0.0), (8, 0.3)])
+def test_emitted_token_law_brute_force(V, beta):
+    """beta = 0 is standard speculative sampling, whose output law is exactly P_t
+    (Sec. 3.2 step 5 'identical to traditional'; refs [1],[2]); beta > 0 follows the
+    same enumeration with the widened acceptance region."""
+    rng = np.random.default_rng(40 + V)
+    B, T = 1_000_000, 1.0
+    t_rows = rng.normal(0, 1.2, (2, V)).astype(np.float32)
+    d_rows = (t_rows[:1] + rng.normal(0, 1.0, (1, V))).astype(np.float32)
+    pt = sp_softmax(t_rows[0].astype(np.float64))
+    pd = sp_softmax(d_rows[0].astype(np.float64))
+    law = _law(pt, pd, beta)
+    assert abs(law.sum() - 1) < 1e-12
+    if beta == 0.0:
+        np.testing.assert_allclose(law, pt, atol=1e-12)  # algebraic identity
+    x = rng.choice(V, size=(B, 1), p=pd).astype(np.int32)  # the draft model's own sampling
+    t = np.broadcast_to(t_rows, (B, 2, V)).copy()
+    d = np.broadcast_to(d_rows, (B, 1, V)).copy()
+    res = oracle.verify(t, d, x, T, beta, seed=77, offset=1, nthreads=4)
+    counts = np.bincount(res.tokens[:, 0], minlength=V)
+    chi, p = stats.chisquare(counts, law * B)
+    assert p > 1e-4, (chi, p, counts / B, law)
+    # prefix property: an accepted sequence repeats the draft token
+    acc = res.accept_len == 1
+    assert np.array_equal(res.tokens[acc, 0], x[acc, 0])
+    # a resampled token differs from the rejected one and has P_t > P_d there
+    rej = ~acc
+    assert np.all(res.tokens[rej, 0] != x[rej, 0])
+    assert np.all(pt[res.tokens[rej, 0]] > pd[res.tokens[rej, 0]])
+    assert np.all(res.tokens[rej, 1] == -1)
+
+
+def test_bonus_token_law():
+    """All drafts accepted (identical rows give R = 1): the extra token follows P_t of row K."""
+    rng = np.random.default_rng(6)
+    B, K, V, T = 400_000, 2, 8, 0.8
+    t_rows = rng.normal(0, 1.5, (K + 1, V)).astype(np.float32)
+    t, d, x = tile(t_rows, t_rows[:K], [3, 5], B)
+    res = oracle.verify(t, d, x, T, 0.0, seed=1, offset=2, nthreads=4)
+    assert np.all(res.accept_len == K)
+    assert np.all(res.tokens[:, :K] == x)
+    law = sp_softmax(t_rows[K].astype(np.float64) / np.float32(T))
+    chi, p = stats.chisquare(np.bincount(res.tokens[:, K], minlength=V), law * B)
+    assert p > 1e-4, (chi, p)
+    np.testing.assert_allclose(res.resid_mass, 1.0, atol=1e-12)
+
+
+# ------------------------------------------------------------------- tolerance term
+def test_one_hot_target_gives_zero_tolerance():
+    """max P_t = 1 makes Uncertainty = 0, so every beta decides like beta = 0 (Sec. 3.2)."""
+    rng = np.random.default_rng(7)
+    B, K, V = 2000, 3, 50
+    t = rng.normal(0, 1, (B, K + 1, V)).astype(np.float32)
+    hot = rng.integers(0, V, (B, K + 1))
+    np.put_along_axis(t, hot[..., None], 800.0, axis=2)
+    d = rng.normal(0, 1, (B, K, V)).astype(np.float32)
+    x = np.where(rng.random((B, K)) < 0.5, hot[:, :K], rng.integers(0, V, (B, K))).astype(np.int32)
+    base = oracle.verify(t, d, x, 1.0, 0.0, seed=3)
+    assert np.all(base.max_pt == 1.0)
+    for beta in (0.2, 1.0, 50.0):
+        r = oracle.verify(t, d, x, 1.0, beta, seed=3)
+        assert np.array_equal(r.cls != 0, base.cls != 0)
+        assert np.array_equal(r.margin, base.margin)
+        assert np.array_equal(r.tokens, base.tokens)
+        assert not np.any(r.cls == 2)  # no pardon without tolerance
+
+
+def test_accept_sets_nested_in_beta():
+    """Tolerance is proportional to beta, so with the same uniforms the accepted set only grows."""
+    rng = np.random.default_rng(8)
+    B, K, V = 500, 5, 300
+    t = rng.normal(0, 2, (B, K + 1, V)).astype(np.float32)
+    d = (t[:, :K] + rng.normal(0, 1.5, (B, K, V))).astype(np.float32)
+    x = rng.integers(0, V, (B, K)).astype(np.int32)
+    prev = None
+    for beta in (0.0, 0.05, 0.1, 0.2, 0.5, 1.0, 2.0):
+        r = oracle.verify(t, d, x, 1.0, beta, seed=11, offset=4)
+        if prev is not None:
+            assert np.all((prev.cls != 0) <= (r.cls != 0))
+            assert np.all(prev.accept_len <= r.accept_len)
+            assert np.array_equal(prev.cls == 1, r.cls == 1)  # the direct path ignores beta
+        prev = r
+    assert np.any(prev.cls == 2)
+
+
+def test_tolerance_grows_with_temperature():
+    """Higher temperature flattens P_t, lowers max P_t and so raises the tolerance (Sec. 4.3)."""
+    rng = np.random.default_rng(9)
+    B, K, V = 20, 2, 500
+    t = rng.normal(0, 2, (B, K + 1, V)).astype(np.float32)
+    d = rng.normal(0, 2, (B, K, V)).astype(np.float32)
+    x = rng.integers(0, V, (B, K)).astype(np.int32)
+    prev = None
+    for T in (0.5, 0.9, 1.0, 1.5, 3.0):
+        r = oracle.verify(t, d, x, T, 0.1)
+        if prev is not None:
+            assert np.all(r.max_pt < prev.max_pt)
+        prev = r
+
+
+def test_clamp_is_inert_and_eps_guard_applies():
+    """Sec. 3.3 item 2: threshold max(U - Tol, 0) and P_d^safe = max(P_d, 1e-10)."""
+    rng = np.random.default_rng(10)
+    B, K, V, beta = 5000, 1, 16, 1.0
+    t = rng.normal(0, 0.3, (B, K + 1, V)).astype(np.float32)   # flat target: Tol close to beta
+    d = rng.normal(0, 0.3, (B, K, V)).astype(np.float32)
+    x = rng.integers(0, V, (B, K)).astype(np.int32)
+    r = oracle.verify(t, d, x, 1.0, beta, seed=2)
+    U = np.array([oracle.uniform_accept(2, 0, b, 0) for b in range(B)])
+    tol = beta * (1 - r.max_pt[:, 0])
+    clamped = U - tol < 0
+    assert clamped.sum() > 100
+    assert np.all(r.cls[clamped, 0] != 0)                       # R >= 0 always clears a zero threshold
+    R = r.pt_tok[:, 0] / np.maximum(r.pd_tok[:, 0], EPS)
+    np.testing.assert_allclose(r.margin[clamped, 0], R[clamped], rtol=1e-12)
+    np.testing.assert_allclose(r.margin[~clamped, 0], (R - (U - tol))[~clamped], rtol=1e-9, atol=1e-12)
+    # a draft token whose draft probability is below eps: R uses eps, not P_d
+    t1 = np.zeros((1, 2, 4), np.float32)
+    t1[0, 0] = [0.0, 0.0, 0.0, -30.0]                           # P_t(tok 3) ~ 3e-14
+    d1 = np.zeros((1, 1, 4), np.float32)
+    d1[0, 0, 3] = -60.0                                         # P_d(tok 3) ~ 3e-27 < eps
+    r1 = oracle.verify(t1, d1, np.array([[3]], np.int32), 1.0, 0.0, seed=0)
+    assert r1.pd_tok[0, 0] < 1e-20
+    U0 = oracle.uniform_accept(0, 0, 0, 0)
+    assert abs((r1.margin[0, 0] + U0) - r1.pt_tok[0, 0] / EPS) < 1e-12
+    assert r1.accept_len[0] == 0                                # unguarded R = 1e13 would have accepted
+
+
+# ----------------------------------------------------------------------- invariants
+def test_invariants_on_random_batch():
+    rng = np.random.default_rng(12)
+    B, K, V, T, beta = 300, 4, 777, 1.1, 0.1
+    t = rng.normal(0, 2, (B, K + 1, V)).astype(np.float32)
+    d = (t[:, :K] + rng.normal(0, 1.0, (B, K, V))).astype(np.float32)
+    x = np.stack([[rng.choice(V, p=sp_softmax(d[b, k].astype(np.float64) / T)) for k in range(K)]
+                  for b in range(B)]).astype(np.int32)
+    r = oracle.verify(t, d, x, T, beta, seed=21, offset=3)
+    assert r.accept_len.min() >= 0 and r.accept_len.max() <= K
+    assert 0 < (r.accept_len < K).sum() < B
+    for b in range(B):
+        n = r.accept_len[b]
+        assert np.array_equal(r.tokens[b, :n], x[b, :n])
+        assert np.all(r.tokens[b, n + 1:] == -1)
+        assert 0 <= r.tokens[b, n] < V
+        # decisions recomputed from library softmax and the published uniform layout
+        for k in range(K):
+            pt = sp_softmax(t[b, k].astype(np.float64) / np.float32(T))
+            pd = sp_softmax(d[b, k].astype(np.float64) / np.float32(T))
+            np.testing.assert_allclose(r.pt_tok[b, k], pt[x[b, k]], rtol=1e-11)
+            np.testing.assert_allclose(r.pd_tok[b, k], pd[x[b, k]], rtol=1e-11)
+            np.testing.assert_allclose(r.max_pt[b, k], pt.max(), rtol=1e-12)
+        u = oracle.uniform_final(21, 3, b, K)
+        if n < K:
+            pt = sp_softmax(t[b, n].astype(np.float64) / np.float32(T))
+            pd = sp_softmax(d[b, n].astype(np.float64) / np.float32(T))
+            S = 0.5 * np.abs(pt - pd).sum()                      # total-variation identity
+            np.testing.assert_allclose(r.resid_mass[b], S, rtol=1e-10)
+            R = pt[x[b, n]] / pd[x[b, n]]
+            assert r.resid_mass[b] >= pd[x[b, n]] * (1 - R) - 1e-15
+            assert r.tokens[b, n] != x[b, n] and pt[r.tokens[b, n]] > pd[r.tokens[b, n]]
+            mass = np.maximum(pt - pd, 0)
+        else:
+            mass = sp_softmax(t[b, K].astype(np.float64) / np.float32(T))
+        C = np.cumsum(mass)
+        want = int(np.searchsorted(C, u * C[-1], side="right"))
+        if r.cdf_margin[b] > 1e-9:                               # away from a boundary the pick is unique
+            assert r.tokens[b, n] == want
+        else:
+            assert r.band_lo[b] <= want <= r.band_hi[b]
+    # first rejection = first position whose class is 0
+    first = np.array([np.argmax(np.append(r.cls[b] == 0, True)) for b in range(B)])
+    assert np.array_equal(first, r.accept_len)
+    # shifting every row by a constant changes nothing
+    r2 = oracle.verify(t + np.float32(8.0), d - np.float32(4.0), x, T, beta, seed=21, offset=3)
+    assert np.array_equal(r2.accept_len, r.accept_len)
+    assert (r2.tokens != r.tokens).mean() < 0.01   # +8 in fp32 re-rounds the logits slightly
+    # threads do not change results
+    r3 = oracle.verify(t, d, x, T, beta, seed=21, offset=3, nthreads=4)
+    assert np.array_equal(r3.tokens, r.tokens) and np.array_equal(r3.margin, r.margin)
+
+
+def test_identical_rows_accept_everything():
+    rng = np.random.default_rng(13)
+    B, K, V = 50, 6, 100
+    t = rng.normal(0, 3, (B, K + 1, V)).astype(np.float32)
+    x = rng.integers(0, V, (B, K)).astype(np.int32)
+    r = oracle.verify(t, t[:, :K].copy(), x, 0.9, 0.0, seed=5)
+    assert np.all(r.accept_len == K) and np.all(r.cls == 1)
+    np.testing.assert_allclose(r.pt_tok, r.pd_tok, rtol=0, atol=0)
+
+
+def test_batch_shards_reproduce_the_full_batch():
+    """The random counter carries the global sequence index, so shards agree with the whole."""
+    rng = np.random.default_rng(14)
+    B, K, V = 12, 3, 64
+    t = rng.normal(0, 2, (B, K + 1, V)).astype(np.float32)
+    d = (t[:, :K] + rng.normal(0, 1.5, (B, K, V))).astype(np.float32)
+    x = rng.integers(0, V, (B, K)).astype(np.int32)
+    full = oracle.verify(t, d, x, 1.0, 0.1, seed=9, offset=100)
+    for lo, hi in [(0, 5), (5, 12)]:
+        part = oracle.verify(t[lo:hi], d[lo:hi], x[lo:hi], 1.0, 0.1, seed=9, offset=100, b_first=lo)
+        assert np.array_equal(part.tokens, full.tokens[lo:hi])
+        assert np.array_equal(part.accept_len, full.accept_len[lo:hi])
+    other = oracle.verify(t, d, x, 1.0, 0.1, seed=9, offset=101)
+    assert not np.array_equal(other.margin, full.margin)
+
+
+def test_bf16_rows_widen_exactly():
+    import torch
+    g = torch.Generator().manual_seed(0)
+    B, K, V = 4, 2, 200
+    t = torch.randn(B, K + 1, V, generator=g).to(torch.bfloat16)
+    d = torch.randn(B, K, V, generator=g).to(torch.bfloat16)
+    x = torch.randint(0, V, (B, K), generator=g).to(torch.int32)
+    a = oracle.verify(t, d, x, 1.0, 0.2, seed=1)
+    b = oracle.verify(t.float(), d.float(), x, 1.0, 0.2, seed=1)
+    assert np.array_equal(a.tokens, b.tokens) and np.array_equal(a.pt_tok, b.pt_tok)
+
+
+def test_invalid_sequences_are_marked_not_fatal():
+    rng = np.random.default_rng(15)
+    B, K, V = 6, 2, 32
+    t = rng.normal(0, 1, (B, K + 1, V)).astype(np.float32)
+    d = rng.normal(0, 1, (B, K, V)).astype(np.float32)
+    x = rng.integers(0, V, (B, K)).astype(np.int32)
+    good = oracle.verify(t, d, x, 1.0, 0.1)
+    x[1, 0] = V
+    x[2, 1] = -1
+    t[3, 1, 5] = np.nan
+    d[4, 0, 7] = np.inf
+    t[5, K, :] = -np.inf
+    t[0, 0, 3] = -np.inf  # a masked vocabulary entry is legal
+    r = oracle.verify(t, d, x, 1.0, 0.1)
+    assert np.all(r.accept_len[1:] == -1) and np.all(r.tokens[1:] == -1)
+    assert r.accept_len[0] >= 0 and good.accept_len[0] >= 0
+    with pytest.raises(ValueError):
+        oracle.verify(t, d, x, 0.0, 0.1)
+    with pytest.raises(ValueError):
+        oracle.verify(t, d, x, 1.0, -0.1)
