@@ -1,0 +1,183 @@
+/*
+ * ears.h -- C ABI of the EARS speculative-decoding verification step for
+ * NVIDIA B200 (sm_100a).
+ *
+ * One call verifies K draft tokens for each of B independent sequences
+ * ("Efficient Adaptive Rejection Sampling", arXiv 2512.13194):
+ *
+ *   1. every target and draft logits row becomes a temperature softmax
+ *      (Sec. 3.1; temperature as discussed in Sec. 4.3);
+ *   2. draft token x_k is accepted iff
+ *          R_k >= max(U_k - Tolerance_k, 0),
+ *          R_k = P_t(x_k) / max(P_d(x_k), 1e-10),
+ *          Tolerance_k = beta * (1 - max_v P_t(v))
+ *      (Sec. 3.2: uncertainty, tolerance equation, acceptance condition;
+ *       Sec. 3.3 item 2: division guard and threshold clamp);
+ *   3. the first rejected position n ends the accepted prefix (Sec. 3.1);
+ *   4. position n receives a token drawn from normalize(max(0, P_t - P_d)) of
+ *      that position, or, when all K were accepted (n = K), a token drawn from
+ *      P_t of the extra target row.  The paper leaves this step to the target
+ *      model ("generate ... starting from position i", Sec. 3.1); the rule used
+ *      is the speculative-sampling one of its refs. [1], [2].
+ *
+ * Random numbers (not in the paper; fixed here so results are reproducible and
+ * independent of how a batch is split): Philox4x32-10 with
+ *     key     = (seed[31:0], seed[63:32])
+ *     counter = (offset[31:0], offset[63:32], b_global, slot)
+ *   slot k in [0,K): U_k = (word0 >> 8) * 2^-24              (exact in fp32)
+ *   slot K         : u   = ((word0 << 32 | word1) >> 11) * 2^-53, the uniform of
+ *                    the inverse-CDF draw in step 4 (token = smallest j with
+ *                    u*S < C_j, C_j the running sum of the masses, S their total).
+ * A caller advances `offset` by one per verification step.
+ *
+ * Conventions for every entry point unless stated otherwise:
+ *   - logits are row-major and contiguous: target [B, K+1, V], draft [B, K, V],
+ *     fp32 or bf16 (bit pattern of the upper half of an fp32); draft tokens [B, K]
+ *     int32.  -inf logits (masked vocabulary) are legal.
+ *   - pointers are DEVICE pointers owned by the caller; the library neither
+ *     retains nor frees them.  Logits must be aligned to their element size.
+ *     When both logits bases are 16-byte aligned and V * elem_size is a multiple
+ *     of 16 the rows are fetched with bulk asynchronous copies (TMA); otherwise a
+ *     slower element-wise loader is used with identical results.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls
+ *     enqueue work and return; they do not synchronise.
+ *   - outputs: out_accept_len[b] = n in [0, K]; out_tokens[b, 0:n] = the accepted
+ *     draft tokens, out_tokens[b, n] = the resampled (n < K) or bonus (n = K)
+ *     token, out_tokens[b, n+1:] = -1.
+ *   - a sequence whose data cannot be verified (draft token outside [0, V); a NaN
+ *     or +inf logit; a row with no finite logit) gets out_accept_len[b] = -1 and
+ *     out_tokens[b, :] = -1, and bit EARS_DEV_INVALID_INPUT is set in the device
+ *     status; other sequences are unaffected.  Nothing traps.
+ *   - the return value reports host-detectable errors only (enum below); 0 = enqueued.
+ */
+#ifndef EARS_H
+#define EARS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define EARS_VERSION 100
+
+enum {
+    EARS_OK = 0,
+    EARS_ERR_NULL = -1,      /* a required pointer is NULL */
+    EARS_ERR_SHAPE = -2,     /* B, K or V < 1; K > EARS_MAX_K; V > 2^30; sizes overflow */
+    EARS_ERR_PARAM = -3,     /* temperature not finite or <= 0; beta not finite or < 0; bad dtype */
+    EARS_ERR_ALIGN = -4,     /* logits not aligned to their element size; workspace not 256-byte aligned */
+    EARS_ERR_WORKSPACE = -5, /* caller workspace smaller than ears_workspace_bytes() */
+    EARS_ERR_CUDA = -6,      /* a CUDA runtime call failed (see ears_last_cuda_error) */
+    EARS_ERR_TIMEOUT = -7    /* a bounded device-side wait gave up (reported by ears_last_device_status) */
+};
+
+enum { EARS_DTYPE_F32 = 0, EARS_DTYPE_BF16 = 1 };
+
+/* bits of the sticky device status word */
+enum { EARS_DEV_INVALID_INPUT = 1, EARS_DEV_TIMEOUT = 2 };
+
+#define EARS_MAX_K 64
+
+/*
+ * The verification step as listed above, fp32 logits.  Uses a library-owned
+ * workspace cached per (device, stream); calls sharing a stream are ordered,
+ * calls on different streams are independent.
+ */
+int ears_verify_f32(const float* target_logits, const float* draft_logits,
+                    const int32_t* draft_tokens, int B, int K, int V,
+                    float temperature, float beta, uint64_t seed, uint64_t offset,
+                    int32_t* out_accept_len, int32_t* out_tokens, void* stream);
+
+/* Same, bf16 logits (pointer to 16-bit elements). */
+int ears_verify_bf16(const void* target_logits, const void* draft_logits,
+                     const int32_t* draft_tokens, int B, int K, int V,
+                     float temperature, float beta, uint64_t seed, uint64_t offset,
+                     int32_t* out_accept_len, int32_t* out_tokens, void* stream);
+
+/* Alias of ears_verify_f32 (the element type cannot be inferred from the arguments). */
+int ears_verify(const void* target_logits, const void* draft_logits,
+                const int32_t* draft_tokens, int B, int K, int V,
+                float temperature, float beta, uint64_t seed, uint64_t offset,
+                int32_t* out_accept_len, int32_t* out_tokens, void* stream);
+
+/*
+ * General form.  Beyond the arguments above:
+ *   dtype       EARS_DTYPE_F32 or EARS_DTYPE_BF16.
+ *   b_first     global index of local sequence 0; it enters the random counter so
+ *               that a batch sharded across GPUs (Sec. 3.3 item 3 treats all active
+ *               sequences independently) reproduces the unsharded result.
+ *   out_pt_tok, out_pd_tok, out_max_pt   [B,K] double, optional (NULL to skip):
+ *               P_t(x_k), P_d(x_k) and max_v P_t(v) of Sec. 3.2 step 1, for every
+ *               position (also those after the first rejection).
+ *   out_class   [B,K] uint8, optional: 0 reject, 1 direct accept (R >= U),
+ *               2 accept via the pardon path (Sec. 3.2 step 5).
+ *   out_resid_mass [B] double, optional: total mass S the final token was drawn
+ *               from (the residual mass, or ~1 for a bonus token).
+ *   workspace, workspace_bytes   caller-owned device scratch of at least
+ *               ears_workspace_bytes(B,K,V) bytes, 256-byte aligned, contents
+ *               arbitrary; or (NULL, 0) to use the library-owned one.  With a
+ *               caller workspace the call allocates nothing.  Two calls that may
+ *               overlap on the GPU must not share a workspace.
+ */
+int ears_verify_ex(int dtype, const void* target_logits, const void* draft_logits,
+                   const int32_t* draft_tokens, int B, int K, int V,
+                   float temperature, float beta, uint64_t seed, uint64_t offset,
+                   int64_t b_first, int32_t* out_accept_len, int32_t* out_tokens,
+                   double* out_pt_tok, double* out_pd_tok, double* out_max_pt,
+                   uint8_t* out_class, double* out_resid_mass,
+                   void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Same step with HOST buffers: copies the inputs to library-owned device staging
+ * buffers, runs the step, copies out_accept_len / out_tokens back and waits for
+ * completion.  All pointers are host memory (pinned memory makes the copies
+ * asynchronous and faster).  Returns a host error, or EARS_ERR_TIMEOUT if a device
+ * wait gave up; invalid sequences are reported in the outputs as above.
+ */
+int ears_verify_host(int dtype, const void* target_logits, const void* draft_logits,
+                     const int32_t* draft_tokens, int B, int K, int V,
+                     float temperature, float beta, uint64_t seed, uint64_t offset,
+                     int64_t b_first, int32_t* out_accept_len, int32_t* out_tokens,
+                     void* stream);
+
+/* Upper bound of the scratch bytes a call with these sizes needs (either dtype). */
+size_t ears_workspace_bytes(int B, int K, int V);
+
+/*
+ * Waits for `stream`, then returns and clears the sticky device status of the
+ * library-owned workspace of (current device, stream): an OR of EARS_DEV_* bits,
+ * or a negative EARS_ERR_* if the wait itself failed.
+ */
+int ears_last_device_status(void* stream);
+
+/* Same for a caller-owned workspace that was passed to ears_verify_ex on `stream`. */
+int ears_workspace_device_status(void* workspace, void* stream);
+
+/*
+ * Test hook for the device random stream: out[i, 0:4] = Philox4x32-10 of counter
+ * ctr_key[i, 0:4] and key ctr_key[i, 4:6]; both device pointers, n >= 0.
+ */
+int ears_philox_device(const uint32_t* ctr_key, uint32_t* out, int n, void* stream);
+
+/*
+ * Launch-plan override for tests (0 = automatic for every field):
+ *   loader 1 = bulk-copy (TMA) loader where alignment allows, 2 = element-wise loader;
+ *   parts_stats / parts_final = number of pieces each row is split into for the
+ *   statistics kernel / the final-token kernel (clamped to what the row allows).
+ * Results never depend on the plan except through floating-point summation order.
+ */
+int ears_set_plan(int loader, int parts_stats, int parts_final);
+
+const char* ears_status_string(int status);
+const char* ears_last_cuda_error(void); /* text of the last failing CUDA call on this thread, or "" */
+int ears_version(void);
+
+/* Frees every library-owned workspace and staging buffer (synchronises the devices used). */
+void ears_shutdown(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EARS_H */

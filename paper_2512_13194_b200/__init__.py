@@ -1,6 +1,23 @@
 """EARS speculative-decoding verification step, CUDA (sm_100a) implementation.
 
-``verify`` and friends call the C-ABI library built from ``csrc/``; there is no
-CPU fallback.  ``synth`` holds the seeded synthetic workloads.
+``verify`` and friends call the C-ABI library built from ``csrc/`` (declared in
+``include/ears.h``); there is no CPU fallback.  ``synth`` holds the seeded
+synthetic workloads, ``shard`` the batch partition used across GPUs.
 """
-from . import synth  # noqa: F401
+from . import shard, synth  # noqa: F401
+from .binding import (  # noqa: F401
+    DEV_INVALID_INPUT,
+    DEV_TIMEOUT,
+    EarsError,
+    last_device_status,
+    load_library,
+    philox_device,
+    set_plan,
+    shutdown,
+    verify,
+    verify_abi,
+    verify_host,
+    version,
+    workspace_bytes,
+    workspace_device_status,
+)

@@ -1,0 +1,216 @@
+"""ctypes binding of libears.so (include/ears.h).  Argument marshalling only:
+torch supplies device memory and streams, every step runs in the CUDA library.
+There is no fallback: a missing library or a failing call raises."""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+EARS_DTYPE_F32, EARS_DTYPE_BF16 = 0, 1
+DEV_INVALID_INPUT, DEV_TIMEOUT = 1, 2
+
+_lib = None
+
+
+class EarsError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"ears status {status}: {message}")
+        self.status = status
+
+
+def load_library(path: Optional[str] = None) -> ctypes.CDLL:
+    """Loads (and, when sources are newer, rebuilds) the in-tree CUDA library."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    if path is None:
+        path = _build.LIB
+        if not os.path.exists(path):
+            path = _build.build()
+    lib = ctypes.CDLL(path)
+    c = ctypes
+    common = [c.c_void_p, c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_int, c.c_float, c.c_float,
+              c.c_uint64, c.c_uint64]
+    for name in ("ears_verify_f32", "ears_verify_bf16", "ears_verify"):
+        fn = getattr(lib, name)
+        fn.argtypes = common + [c.c_void_p, c.c_void_p, c.c_void_p]
+        fn.restype = c.c_int
+    lib.ears_verify_ex.argtypes = ([c.c_int] + common + [c.c_int64] + [c.c_void_p] * 7
+                                   + [c.c_void_p, c.c_size_t, c.c_void_p])
+    lib.ears_verify_ex.restype = c.c_int
+    lib.ears_verify_host.argtypes = [c.c_int] + common + [c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p]
+    lib.ears_verify_host.restype = c.c_int
+    lib.ears_workspace_bytes.argtypes = [c.c_int, c.c_int, c.c_int]
+    lib.ears_workspace_bytes.restype = c.c_size_t
+    lib.ears_last_device_status.argtypes = [c.c_void_p]
+    lib.ears_last_device_status.restype = c.c_int
+    lib.ears_workspace_device_status.argtypes = [c.c_void_p, c.c_void_p]
+    lib.ears_workspace_device_status.restype = c.c_int
+    lib.ears_philox_device.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_void_p]
+    lib.ears_philox_device.restype = c.c_int
+    lib.ears_set_plan.argtypes = [c.c_int, c.c_int, c.c_int]
+    lib.ears_set_plan.restype = c.c_int
+    lib.ears_status_string.argtypes = [c.c_int]
+    lib.ears_status_string.restype = c.c_char_p
+    lib.ears_last_cuda_error.argtypes = []
+    lib.ears_last_cuda_error.restype = c.c_char_p
+    lib.ears_version.argtypes = []
+    lib.ears_version.restype = c.c_int
+    lib.ears_shutdown.argtypes = []
+    lib.ears_shutdown.restype = None
+    _lib = lib
+    return lib
+
+
+def _check(rc: int):
+    if rc != 0:
+        lib = load_library()
+        msg = lib.ears_status_string(rc).decode()
+        extra = lib.ears_last_cuda_error().decode()
+        raise EarsError(rc, msg + (f" ({extra})" if extra and rc == -6 else ""))
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return EARS_DTYPE_F32
+    if t.dtype == torch.bfloat16:
+        return EARS_DTYPE_BF16
+    raise TypeError(f"logits must be float32 or bfloat16, got {t.dtype}")
+
+
+def _shapes(target_logits, draft_logits, draft_tokens):
+    if target_logits.dim() != 3 or draft_logits.dim() != 3 or draft_tokens.dim() != 2:
+        raise ValueError("expected target [B,K+1,V], draft [B,K,V], tokens [B,K]")
+    B, K1, V = target_logits.shape
+    K = K1 - 1
+    if tuple(draft_logits.shape) != (B, K, V) or tuple(draft_tokens.shape) != (B, K):
+        raise ValueError("shape mismatch between target, draft and tokens")
+    if draft_logits.dtype != target_logits.dtype:
+        raise TypeError("target and draft logits must share a dtype")
+    return B, K, V
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def verify(target_logits: torch.Tensor, draft_logits: torch.Tensor, draft_tokens: torch.Tensor,
+           temperature: float, beta: float, seed: int = 0, offset: int = 0, *, b_first: int = 0,
+           stats: bool = False, workspace: Optional[torch.Tensor] = None, stream=None):
+    """One EARS verification step on the current CUDA device.
+
+    Returns (accept_len [B] int32, tokens [B,K+1] int32) and, with ``stats=True``, a dict with
+    pt_tok, pd_tok, max_pt [B,K] float64, cls [B,K] uint8 and resid_mass [B] float64.
+    The call is asynchronous on ``stream`` (default: torch's current stream).
+    """
+    lib = load_library()
+    B, K, V = _shapes(target_logits, draft_logits, draft_tokens)
+    dev = target_logits.device
+    if dev.type != "cuda" or draft_logits.device != dev or draft_tokens.device != dev:
+        raise ValueError("all inputs must live on the same CUDA device")
+    t = target_logits.contiguous()
+    d = draft_logits.contiguous()
+    x = draft_tokens.to(torch.int32).contiguous()
+    with torch.cuda.device(dev):
+        acc = torch.empty(B, dtype=torch.int32, device=dev)
+        tok = torch.empty((B, K + 1), dtype=torch.int32, device=dev)
+        st = None
+        ptrs = [None] * 5
+        if stats:
+            st = dict(pt_tok=torch.empty((B, K), dtype=torch.float64, device=dev),
+                      pd_tok=torch.empty((B, K), dtype=torch.float64, device=dev),
+                      max_pt=torch.empty((B, K), dtype=torch.float64, device=dev),
+                      cls=torch.empty((B, K), dtype=torch.uint8, device=dev),
+                      resid_mass=torch.zeros(B, dtype=torch.float64, device=dev))
+            ptrs = [st[k].data_ptr() for k in ("pt_tok", "pd_tok", "max_pt", "cls", "resid_mass")]
+        ws_ptr, ws_bytes = (None, 0) if workspace is None else (workspace.data_ptr(), workspace.numel() * workspace.element_size())
+        rc = lib.ears_verify_ex(_dtype_code(t), t.data_ptr(), d.data_ptr(), x.data_ptr(), B, K, V,
+                                float(temperature), float(beta), int(seed), int(offset), int(b_first),
+                                acc.data_ptr(), tok.data_ptr(), *ptrs, ws_ptr, ws_bytes, _stream_ptr(stream))
+    _check(rc)
+    return (acc, tok, st) if stats else (acc, tok)
+
+
+def verify_abi(name: str, target_logits, draft_logits, draft_tokens, temperature, beta, seed, offset,
+               stream=None):
+    """Calls one of the 13-argument entry points (ears_verify, ears_verify_f32, ears_verify_bf16) as is."""
+    lib = load_library()
+    B, K, V = _shapes(target_logits, draft_logits, draft_tokens)
+    dev = target_logits.device
+    acc = torch.empty(B, dtype=torch.int32, device=dev)
+    tok = torch.empty((B, K + 1), dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        rc = getattr(lib, name)(target_logits.data_ptr(), draft_logits.data_ptr(), draft_tokens.data_ptr(),
+                                B, K, V, float(temperature), float(beta), int(seed), int(offset),
+                                acc.data_ptr(), tok.data_ptr(), _stream_ptr(stream))
+    _check(rc)
+    return acc, tok
+
+
+def verify_host(target_logits: torch.Tensor, draft_logits: torch.Tensor, draft_tokens: torch.Tensor,
+                temperature: float, beta: float, seed: int = 0, offset: int = 0, *, b_first: int = 0,
+                out_accept_len: Optional[torch.Tensor] = None, out_tokens: Optional[torch.Tensor] = None,
+                stream=None):
+    """Same step with CPU tensors (pinned memory recommended): the library copies the inputs
+    to the device, runs the kernels, copies the results back and waits.  Returns CPU tensors."""
+    lib = load_library()
+    B, K, V = _shapes(target_logits, draft_logits, draft_tokens)
+    for a in (target_logits, draft_logits, draft_tokens):
+        if a.device.type != "cpu" or not a.is_contiguous():
+            raise ValueError("verify_host takes contiguous CPU tensors")
+    if draft_tokens.dtype != torch.int32:
+        raise TypeError("draft_tokens must be int32")
+    acc = out_accept_len if out_accept_len is not None else torch.empty(B, dtype=torch.int32)
+    tok = out_tokens if out_tokens is not None else torch.empty((B, K + 1), dtype=torch.int32)
+    rc = lib.ears_verify_host(_dtype_code(target_logits), target_logits.data_ptr(), draft_logits.data_ptr(),
+                              draft_tokens.data_ptr(), B, K, V, float(temperature), float(beta), int(seed),
+                              int(offset), int(b_first), acc.data_ptr(), tok.data_ptr(), _stream_ptr(stream))
+    _check(rc)
+    return acc, tok
+
+
+def workspace_bytes(B: int, K: int, V: int) -> int:
+    return int(load_library().ears_workspace_bytes(B, K, V))
+
+
+def last_device_status(stream=None) -> int:
+    rc = load_library().ears_last_device_status(_stream_ptr(stream))
+    if rc < 0:
+        _check(rc)
+    return rc
+
+
+def workspace_device_status(workspace: torch.Tensor, stream=None) -> int:
+    rc = load_library().ears_workspace_device_status(workspace.data_ptr(), _stream_ptr(stream))
+    if rc < 0:
+        _check(rc)
+    return rc
+
+
+def philox_device(ctr_key: torch.Tensor) -> torch.Tensor:
+    """ctr_key [n,6] int32/uint32 bit patterns on the GPU -> [n,4] words (int32 bit patterns)."""
+    lib = load_library()
+    ck = ctr_key.contiguous()
+    out = torch.empty((ck.shape[0], 4), dtype=torch.int32, device=ck.device)
+    with torch.cuda.device(ck.device):
+        _check(lib.ears_philox_device(ck.data_ptr(), out.data_ptr(), ck.shape[0], _stream_ptr(None)))
+    return out
+
+
+def set_plan(loader: int = 0, parts_stats: int = 0, parts_final: int = 0) -> None:
+    _check(load_library().ears_set_plan(loader, parts_stats, parts_final))
+
+
+def version() -> int:
+    return int(load_library().ears_version())
+
+
+def shutdown() -> None:
+    load_library().ears_shutdown()

@@ -1,0 +1,432 @@
+// C ABI of the EARS verification step (see include/ears.h): argument checks,
+// launch plan, workspace management and the two kernel launches.
+#include "../../include/ears.h"
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <utility>
+
+#include "ears_common.cuh"
+#include "ears_k1.cuh"
+#include "ears_k2.cuh"
+
+namespace {
+
+using namespace ears;
+
+constexpr int kStages1 = 6;  // 6 x 16 KB per CTA, two CTAs per SM
+constexpr int kStages2 = 3;  // 3 x 2 x 16 KB
+constexpr int kCtasPerSm = 2;
+constexpr int kUnitChunks = 16;  // 256 KB of one row per unit when there is plenty of work
+
+thread_local char g_cuda_error[256] = "";
+
+int cuda_fail(cudaError_t e, const char* what) {
+    snprintf(g_cuda_error, sizeof g_cuda_error, "%s: %s", what, cudaGetErrorString(e));
+    return EARS_ERR_CUDA;
+}
+#define EARS_CUDA(call)                                     \
+    do {                                                    \
+        cudaError_t e_ = (call);                            \
+        if (e_ != cudaSuccess) return cuda_fail(e_, #call); \
+    } while (0)
+
+struct PlanOverride { int loader = 0, parts1 = 0, parts2 = 0; };
+PlanOverride g_override;
+std::mutex g_mutex;
+
+struct DeviceInfo { int sms = 0; bool attrs_set = false; };
+std::map<int, DeviceInfo> g_devices;
+
+struct Buffer { void* ptr = nullptr; size_t bytes = 0; };
+std::map<std::pair<int, void*>, Buffer> g_workspaces;  // (device, stream) -> scratch
+std::map<std::pair<int, void*>, Buffer> g_staging;     // (device, stream) -> host-entry staging
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// pieces per row and chunks per piece for `items` rows of `chunks` chunks each
+void split_rows(long long items, int chunks, int sms, int forced_parts, int* parts, int* cpp) {
+    int c = kUnitChunks;
+    const long long want_units = 8LL * sms;
+    if (items * ((chunks + c - 1) / c) < want_units) {
+        long long per_row = (want_units + items - 1) / items;  // desired pieces per row
+        if (per_row > chunks) per_row = chunks;
+        c = (int)(chunks / per_row);
+        if (c < 1) c = 1;
+    }
+    if (forced_parts > 0) {
+        int fp = forced_parts > chunks ? chunks : forced_parts;
+        c = (chunks + fp - 1) / fp;
+    }
+    if (c > chunks) c = chunks;
+    *cpp = c;
+    *parts = (chunks + c - 1) / c;
+}
+
+Plan make_plan(int B, int K, int V, int esize, bool aligned, int sms, const PlanOverride& ov) {
+    Plan pl;
+    const int chunk_elems = kChunkBytes / esize;
+    const int chunks = (V + chunk_elems - 1) / chunk_elems;
+    pl.use_tma = aligned && ov.loader != 2;
+    split_rows((long long)B * (2 * K + 1), chunks, sms, ov.parts1, &pl.parts1, &pl.cpp1);
+    split_rows((long long)B, chunks, sms, ov.parts2, &pl.parts2, &pl.cpp2);
+    pl.nseg = (V + kSegElems - 1) / kSegElems;
+    return pl;
+}
+
+struct Layout {
+    size_t ticket1, ticket2, heads, counters_bytes;
+    size_t partial, rowstat, pt_tok, pd_tok, max_pt, cls, resid, segsum, total;
+};
+
+Layout make_layout(int B, int K, int V, int parts1) {
+    Layout L;
+    const size_t rows = (size_t)B * (2 * K + 1);
+    size_t o = 0;
+    L.heads = o; o += 16;  // fixed place: the status word is heads[2] of any workspace
+    L.ticket1 = o; o += (size_t)B * 4;
+    L.ticket2 = o; o += (size_t)B * 4;
+    L.counters_bytes = o;
+    o = align_up(o, 256);
+    L.partial = o; o = align_up(o + rows * parts1 * sizeof(float2), 256);
+    L.rowstat = o; o = align_up(o + rows * sizeof(float2), 256);
+    L.pt_tok = o; o = align_up(o + (size_t)B * K * 8, 256);
+    L.pd_tok = o; o = align_up(o + (size_t)B * K * 8, 256);
+    L.max_pt = o; o = align_up(o + (size_t)B * K * 8, 256);
+    L.cls = o; o = align_up(o + (size_t)B * K, 256);
+    L.resid = o; o = align_up(o + (size_t)B * 8, 256);
+    L.segsum = o; o = align_up(o + (size_t)B * ((V + kSegElems - 1) / kSegElems) * 8, 256);
+    L.total = o;
+    return L;
+}
+
+int check_shape(int B, int K, int V) {
+    if (B < 1 || K < 1 || V < 1) return EARS_ERR_SHAPE;
+    if (K > EARS_MAX_K || V > (1 << 30)) return EARS_ERR_SHAPE;
+    // element and unit counts must stay far inside 63 / 31 bits
+    const long double elems = (long double)B * (K + 1) * V;
+    if (elems * 4 > 4.0e18L) return EARS_ERR_SHAPE;
+    if ((long double)B * (2 * K + 1) * 64 > 2.0e9L) return EARS_ERR_SHAPE;
+    return EARS_OK;
+}
+
+int device_info(int dev, DeviceInfo** out) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceInfo& di = g_devices[dev];
+    if (di.sms == 0) {
+        int sms = 0;
+        EARS_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        di.sms = sms;
+    }
+    *out = &di;
+    return EARS_OK;
+}
+
+template <typename E>
+size_t smem1() { return sizeof(PipeSmem<kStages1, 1>) + 128; }
+template <typename E>
+size_t smem2() { return sizeof(PipeSmem<kStages2, 2>) + 128; }
+
+template <typename E>
+int set_attrs() {
+    EARS_CUDA(cudaFuncSetAttribute(k1_rowstats_decide<E, kStages1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)smem1<E>()));
+    EARS_CUDA(cudaFuncSetAttribute(k2_final_token<E, kStages2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)smem2<E>()));
+    return EARS_OK;
+}
+
+template <typename E>
+int launch(const Params& p, int sms, cudaStream_t stream) {
+    const long long units1 = (long long)p.B * (2 * p.K + 1) * p.plan.parts1;
+    const long long units2 = (long long)p.B * p.plan.parts2;
+    const long long cap = (long long)sms * kCtasPerSm;
+    const int grid1 = (int)(units1 < cap ? units1 : cap);
+    const int grid2 = (int)(units2 < cap ? units2 : cap);
+    k1_rowstats_decide<E, kStages1><<<grid1, kThreads, smem1<E>(), stream>>>(p);
+    EARS_CUDA(cudaGetLastError());
+    k2_final_token<E, kStages2><<<grid2, kThreads, smem2<E>(), stream>>>(p);
+    EARS_CUDA(cudaGetLastError());
+    return EARS_OK;
+}
+
+int get_buffer(std::map<std::pair<int, void*>, Buffer>& pool, int dev, void* stream, size_t bytes, void** out) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    Buffer& b = pool[std::make_pair(dev, stream)];
+    if (b.bytes < bytes) {
+        if (b.ptr) {
+            // work enqueued earlier on this stream may still use the old buffer
+            EARS_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+            EARS_CUDA(cudaFree(b.ptr));
+            b.ptr = nullptr;
+            b.bytes = 0;
+        }
+        const size_t want = align_up(bytes + bytes / 4, 1 << 20);
+        EARS_CUDA(cudaMalloc(&b.ptr, want));
+        b.bytes = want;
+    }
+    *out = b.ptr;
+    return EARS_OK;
+}
+
+int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B, int K, int V,
+                float temperature, float beta, uint64_t seed, uint64_t offset, int64_t b_first,
+                int32_t* out_len, int32_t* out_tok, double* o_pt, double* o_pd, double* o_max,
+                uint8_t* o_cls, double* o_resid, void* workspace, size_t workspace_bytes, void* stream_) {
+    if (!t || !d || !x || !out_len || !out_tok) return EARS_ERR_NULL;
+    if (dtype != EARS_DTYPE_F32 && dtype != EARS_DTYPE_BF16) return EARS_ERR_PARAM;
+    int rc = check_shape(B, K, V);
+    if (rc) return rc;
+    if (!(temperature > 0.0f) || !std::isfinite(temperature)) return EARS_ERR_PARAM;
+    if (!(beta >= 0.0f) || !std::isfinite(beta)) return EARS_ERR_PARAM;
+    if (b_first < 0 || (unsigned long long)b_first + (unsigned long long)B > 0xffffffffull) return EARS_ERR_PARAM;
+    const int esize = dtype == EARS_DTYPE_F32 ? 4 : 2;
+    if (((uintptr_t)t % esize) || ((uintptr_t)d % esize) || ((uintptr_t)x % 4)) return EARS_ERR_ALIGN;
+    if (workspace && ((uintptr_t)workspace % 256)) return EARS_ERR_ALIGN;
+    if (!workspace && workspace_bytes != 0) return EARS_ERR_WORKSPACE;
+
+    cudaStream_t stream = (cudaStream_t)stream_;
+    int dev = 0;
+    EARS_CUDA(cudaGetDevice(&dev));
+    DeviceInfo* di = nullptr;
+    rc = device_info(dev, &di);
+    if (rc) return rc;
+    if (!di->attrs_set) {
+        rc = set_attrs<float>();
+        if (rc) return rc;
+        rc = set_attrs<uint16_t>();
+        if (rc) return rc;
+        di->attrs_set = true;
+    }
+
+    const bool aligned = ((uintptr_t)t % 16 == 0) && ((uintptr_t)d % 16 == 0) && (((size_t)V * esize) % 16 == 0);
+    PlanOverride ov;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        ov = g_override;
+    }
+    const Plan plan = make_plan(B, K, V, esize, aligned, di->sms, ov);
+    const Layout L = make_layout(B, K, V, plan.parts1);
+    if (workspace) {
+        if (workspace_bytes < L.total) return EARS_ERR_WORKSPACE;
+    } else {
+        rc = get_buffer(g_workspaces, dev, stream_, L.total, &workspace);
+        if (rc) return rc;
+    }
+    char* w = (char*)workspace;
+    EARS_CUDA(cudaMemsetAsync(w, 0, L.counters_bytes, stream));
+
+    Params p;
+    p.t = t; p.d = d; p.x = x;
+    p.B = B; p.K = K; p.V = V;
+    p.c = (float)(1.4426950408889634 / (double)temperature);
+    p.T = (double)temperature;
+    p.beta = (double)beta;
+    p.seed = seed; p.offset = offset; p.b_first = b_first;
+    p.out_len = out_len; p.out_tok = out_tok;
+    p.pt_tok = o_pt ? o_pt : (double*)(w + L.pt_tok);
+    p.pd_tok = o_pd ? o_pd : (double*)(w + L.pd_tok);
+    p.max_pt = o_max ? o_max : (double*)(w + L.max_pt);
+    p.cls = o_cls ? o_cls : (uint8_t*)(w + L.cls);
+    p.resid = o_resid ? o_resid : (double*)(w + L.resid);
+    p.ticket1 = (int*)(w + L.ticket1);
+    p.ticket2 = (int*)(w + L.ticket2);
+    p.heads = (int*)(w + L.heads);
+    p.partial = (float2*)(w + L.partial);
+    p.rowstat = (float2*)(w + L.rowstat);
+    p.segsum = (double*)(w + L.segsum);
+    p.plan = plan;
+    return dtype == EARS_DTYPE_F32 ? launch<float>(p, di->sms, stream) : launch<uint16_t>(p, di->sms, stream);
+}
+
+size_t workspace_bound(int B, int K, int V) {
+    PlanOverride ov;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        ov = g_override;
+    }
+    size_t best = 0;
+    // the piece count depends on the SM count and element size; take the largest over both
+    // element sizes at a small and a large SM count (more SMs never ask for fewer pieces)
+    const int sm_counts[2] = {1, 1024};
+    for (int esize = 2; esize <= 4; esize += 2)
+        for (int s = 0; s < 2; ++s) {
+            const Plan pl = make_plan(B, K, V, esize, true, sm_counts[s], ov);
+            const size_t tot = make_layout(B, K, V, pl.parts1).total;
+            if (tot > best) best = tot;
+        }
+    return best;
+}
+
+__global__ void philox_kernel(const uint32_t* ctr_key, uint32_t* out, int n) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const uint32_t* c = ctr_key + (size_t)i * 6;
+    U32x4 r = philox4x32_10(U32x4{c[0], c[1], c[2], c[3]}, c[4], c[5]);
+    out[(size_t)i * 4 + 0] = r.w0;
+    out[(size_t)i * 4 + 1] = r.w1;
+    out[(size_t)i * 4 + 2] = r.w2;
+    out[(size_t)i * 4 + 3] = r.w3;
+}
+
+int read_status(int* heads, cudaStream_t stream) {
+    int status = 0;
+    EARS_CUDA(cudaMemcpyAsync(&status, heads + 2, sizeof(int), cudaMemcpyDeviceToHost, stream));
+    EARS_CUDA(cudaStreamSynchronize(stream));
+    return status;
+}
+
+}  // namespace
+
+extern "C" {
+
+int ears_verify_ex(int dtype, const void* target_logits, const void* draft_logits,
+                   const int32_t* draft_tokens, int B, int K, int V, float temperature, float beta,
+                   uint64_t seed, uint64_t offset, int64_t b_first, int32_t* out_accept_len,
+                   int32_t* out_tokens, double* out_pt_tok, double* out_pd_tok, double* out_max_pt,
+                   uint8_t* out_class, double* out_resid_mass, void* workspace, size_t workspace_bytes,
+                   void* stream) {
+    return verify_impl(dtype, target_logits, draft_logits, draft_tokens, B, K, V, temperature, beta, seed,
+                       offset, b_first, out_accept_len, out_tokens, out_pt_tok, out_pd_tok, out_max_pt,
+                       out_class, out_resid_mass, workspace, workspace_bytes, stream);
+}
+
+int ears_verify_f32(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
+                    int B, int K, int V, float temperature, float beta, uint64_t seed, uint64_t offset,
+                    int32_t* out_accept_len, int32_t* out_tokens, void* stream) {
+    return verify_impl(EARS_DTYPE_F32, target_logits, draft_logits, draft_tokens, B, K, V, temperature, beta,
+                       seed, offset, 0, out_accept_len, out_tokens, nullptr, nullptr, nullptr, nullptr, nullptr,
+                       nullptr, 0, stream);
+}
+
+int ears_verify_bf16(const void* target_logits, const void* draft_logits, const int32_t* draft_tokens,
+                     int B, int K, int V, float temperature, float beta, uint64_t seed, uint64_t offset,
+                     int32_t* out_accept_len, int32_t* out_tokens, void* stream) {
+    return verify_impl(EARS_DTYPE_BF16, target_logits, draft_logits, draft_tokens, B, K, V, temperature, beta,
+                       seed, offset, 0, out_accept_len, out_tokens, nullptr, nullptr, nullptr, nullptr, nullptr,
+                       nullptr, 0, stream);
+}
+
+int ears_verify(const void* target_logits, const void* draft_logits, const int32_t* draft_tokens,
+                int B, int K, int V, float temperature, float beta, uint64_t seed, uint64_t offset,
+                int32_t* out_accept_len, int32_t* out_tokens, void* stream) {
+    return ears_verify_f32((const float*)target_logits, (const float*)draft_logits, draft_tokens, B, K, V,
+                           temperature, beta, seed, offset, out_accept_len, out_tokens, stream);
+}
+
+int ears_verify_host(int dtype, const void* target_logits, const void* draft_logits,
+                     const int32_t* draft_tokens, int B, int K, int V, float temperature, float beta,
+                     uint64_t seed, uint64_t offset, int64_t b_first, int32_t* out_accept_len,
+                     int32_t* out_tokens, void* stream_) {
+    if (!target_logits || !draft_logits || !draft_tokens || !out_accept_len || !out_tokens) return EARS_ERR_NULL;
+    if (dtype != EARS_DTYPE_F32 && dtype != EARS_DTYPE_BF16) return EARS_ERR_PARAM;
+    int rc = check_shape(B, K, V);
+    if (rc) return rc;
+    const size_t esize = dtype == EARS_DTYPE_F32 ? 4 : 2;
+    const size_t tb = (size_t)B * (K + 1) * V * esize, db = (size_t)B * K * V * esize;
+    const size_t xb = (size_t)B * K * 4, lb = (size_t)B * 4, ob = (size_t)B * (K + 1) * 4;
+    size_t o_t = 0, o_d = align_up(o_t + tb, 256), o_x = align_up(o_d + db, 256);
+    size_t o_l = align_up(o_x + xb, 256), o_o = align_up(o_l + lb, 256), total = align_up(o_o + ob, 256);
+    cudaStream_t stream = (cudaStream_t)stream_;
+    int dev = 0;
+    EARS_CUDA(cudaGetDevice(&dev));
+    void* base = nullptr;
+    rc = get_buffer(g_staging, dev, stream_, total, &base);
+    if (rc) return rc;
+    char* s = (char*)base;
+    EARS_CUDA(cudaMemcpyAsync(s + o_t, target_logits, tb, cudaMemcpyHostToDevice, stream));
+    EARS_CUDA(cudaMemcpyAsync(s + o_d, draft_logits, db, cudaMemcpyHostToDevice, stream));
+    EARS_CUDA(cudaMemcpyAsync(s + o_x, draft_tokens, xb, cudaMemcpyHostToDevice, stream));
+    rc = verify_impl(dtype, s + o_t, s + o_d, (const int32_t*)(s + o_x), B, K, V, temperature, beta, seed, offset,
+                     b_first, (int32_t*)(s + o_l), (int32_t*)(s + o_o), nullptr, nullptr, nullptr, nullptr,
+                     nullptr, nullptr, 0, stream_);
+    if (rc) return rc;
+    EARS_CUDA(cudaMemcpyAsync(out_accept_len, s + o_l, lb, cudaMemcpyDeviceToHost, stream));
+    EARS_CUDA(cudaMemcpyAsync(out_tokens, s + o_o, ob, cudaMemcpyDeviceToHost, stream));
+    const int status = ears_last_device_status(stream_);
+    if (status < 0) return status;
+    return (status & EARS_DEV_TIMEOUT) ? EARS_ERR_TIMEOUT : EARS_OK;
+}
+
+size_t ears_workspace_bytes(int B, int K, int V) {
+    if (check_shape(B, K, V)) return 0;
+    return workspace_bound(B, K, V);
+}
+
+int ears_last_device_status(void* stream_) {
+    int dev = 0;
+    EARS_CUDA(cudaGetDevice(&dev));
+    void* ws = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        auto it = g_workspaces.find(std::make_pair(dev, stream_));
+        if (it != g_workspaces.end()) ws = it->second.ptr;
+    }
+    if (!ws) {
+        EARS_CUDA(cudaStreamSynchronize((cudaStream_t)stream_));
+        return 0;
+    }
+    return ears_workspace_device_status(ws, stream_);
+}
+
+int ears_workspace_device_status(void* workspace, void* stream_) {
+    if (!workspace) return EARS_ERR_NULL;
+    return read_status((int*)workspace, (cudaStream_t)stream_);
+}
+
+int ears_philox_device(const uint32_t* ctr_key, uint32_t* out, int n, void* stream) {
+    if (n < 0) return EARS_ERR_SHAPE;
+    if (n == 0) return EARS_OK;
+    if (!ctr_key || !out) return EARS_ERR_NULL;
+    philox_kernel<<<(n + 127) / 128, 128, 0, (cudaStream_t)stream>>>(ctr_key, out, n);
+    EARS_CUDA(cudaGetLastError());
+    return EARS_OK;
+}
+
+int ears_set_plan(int loader, int parts_stats, int parts_final) {
+    if (loader < 0 || loader > 2 || parts_stats < 0 || parts_final < 0) return EARS_ERR_PARAM;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    g_override.loader = loader;
+    g_override.parts1 = parts_stats;
+    g_override.parts2 = parts_final;
+    return EARS_OK;
+}
+
+const char* ears_status_string(int status) {
+    switch (status) {
+        case EARS_OK: return "ok";
+        case EARS_ERR_NULL: return "a required pointer is NULL";
+        case EARS_ERR_SHAPE: return "B, K or V out of range";
+        case EARS_ERR_PARAM: return "bad temperature, beta, dtype or sequence offset";
+        case EARS_ERR_ALIGN: return "pointer not aligned";
+        case EARS_ERR_WORKSPACE: return "workspace too small";
+        case EARS_ERR_CUDA: return "a CUDA call failed";
+        case EARS_ERR_TIMEOUT: return "a device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+const char* ears_last_cuda_error(void) { return g_cuda_error; }
+
+int ears_version(void) { return EARS_VERSION; }
+
+void ears_shutdown(void) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    int cur = 0;
+    cudaGetDevice(&cur);
+    for (auto* pool : {&g_workspaces, &g_staging}) {
+        for (auto& kv : *pool) {
+            if (!kv.second.ptr) continue;
+            cudaSetDevice(kv.first.first);
+            cudaDeviceSynchronize();
+            cudaFree(kv.second.ptr);
+        }
+        pool->clear();
+    }
+    cudaSetDevice(cur);
+}
+
+}  // extern "C"

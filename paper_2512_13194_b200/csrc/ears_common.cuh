@@ -1,0 +1,63 @@
+// Shapes, launch plan and workspace layout shared by the two kernels and the host API.
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace ears {
+
+constexpr int kConsumerWarps = 8;                    // warps that reduce the staged chunks
+constexpr int kConsumers = kConsumerWarps * 32;
+constexpr int kThreads = kConsumers + 32;            // + one loader warp
+constexpr int kChunkBytes = 16384;                   // bytes of one row staged per pipeline slot
+constexpr int kSegElems = 512;                       // elements per final-token segment sum
+constexpr double kEps = 1e-10;                       // division guard, Sec. 3.3 item 2
+constexpr double kTinyMass = 1e-300;                 // below this a residual is treated as empty
+
+// Device status bits (mirrors ears.h)
+constexpr int kDevInvalidInput = 1;
+constexpr int kDevTimeout = 2;
+
+struct Plan {
+    int use_tma;   // 1: bulk asynchronous copies, 0: element-wise loader
+    int parts1;    // pieces per row, statistics kernel
+    int cpp1;      // chunks per piece
+    int parts2;    // pieces per row, final-token kernel
+    int cpp2;
+    int nseg;      // segment sums per sequence
+};
+
+// Counter block at the start of the workspace, zeroed by one memset per call.
+//   ticket1[B] ticket2[B] head1 head2 status pad
+struct Params {
+    const void* t;        // target logits [B,K+1,V]
+    const void* d;        // draft logits  [B,K,V]
+    const int32_t* x;     // draft tokens  [B,K]
+    int B, K, V;
+    float c;              // log2(e) / temperature
+    double T;             // temperature
+    double beta;
+    unsigned long long seed, offset;
+    long long b_first;
+    int32_t* out_len;     // [B]
+    int32_t* out_tok;     // [B,K+1]
+    double* pt_tok;       // [B,K]
+    double* pd_tok;       // [B,K]
+    double* max_pt;       // [B,K]
+    uint8_t* cls;         // [B,K]
+    double* resid;        // [B]
+    int* ticket1;         // [B] arrivals of statistics pieces
+    int* ticket2;         // [B] arrivals of final-token pieces
+    int* heads;           // [0] statistics queue, [1] final-token queue, [2] status
+    float2* partial;      // [B*(2K+1)*parts1] (m, s) per row piece
+    float2* rowstat;      // [B*(2K+1)] (m, Z) per row
+    double* segsum;       // [B*nseg]
+    Plan plan;
+};
+
+// Row order inside a sequence: target k, draft k for k = 0..K-1, then the bonus
+// target row K.  ridx in [0, 2K].
+__host__ __device__ inline long long target_row(int b, int k, int K) { return (long long)b * (K + 1) + k; }
+__host__ __device__ inline long long draft_row(int b, int k, int K) { return (long long)b * K + k; }
+
+}  // namespace ears

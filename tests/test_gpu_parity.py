@@ -1,0 +1,199 @@
+"""GPU parity: the CUDA library (through its C ABI) against the fp64 oracle, element
+by element on the same seeded inputs."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2512_13194_b200 import synth
+from parity import Tally, assert_parity, compare
+
+pytestmark = pytest.mark.gpu
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "philox4x32_10_kat.txt")
+
+
+def run_both(ears, w, t, d, x, T, beta, seed=0, offset=0, b_first=0, nthreads=8):
+    dev = torch.device("cuda:0")
+    acc, tok, st = ears.verify(t.to(dev), d.to(dev), x.to(dev), T, beta, seed, offset, b_first=b_first, stats=True)
+    torch.cuda.synchronize()
+    assert ears.last_device_status() & ears.DEV_TIMEOUT == 0
+    ora = oracle.verify(t.cpu(), d.cpu(), x.cpu(), T, beta, seed=seed, offset=offset, b_first=b_first,
+                        nthreads=nthreads)
+    stats = {k: v.cpu().numpy() for k, v in st.items()}
+    tally = compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, w.K, stats)
+    # the mass the final token was drawn from
+    ok = ora.accept_len >= 0
+    np.testing.assert_allclose(stats["resid_mass"][ok], ora.resid_mass[ok], rtol=2e-5)
+    assert np.array_equal(stats["cls"][ok] != 0, ora.cls[ok] != 0) or tally.flagged_decisions > 0
+    return tally, acc, tok, ora
+
+
+def test_device_philox_known_answers(ears):
+    rows = []
+    with open(GOLDEN) as f:
+        for line in f:
+            if not line.startswith("#") and line.strip():
+                rows.append([int(v, 16) for v in line.split()])
+    ck = torch.from_numpy(np.array([r[:6] for r in rows], dtype=np.uint32).view(np.int32)).cuda()
+    out = ears.philox_device(ck).cpu().numpy().view(np.uint32)
+    assert out.tolist() == [r[6:] for r in rows]
+    rng = np.random.default_rng(0)
+    rnd = rng.integers(0, 2**32, (4096, 6), dtype=np.uint64).astype(np.uint32)
+    got = ears.philox_device(torch.from_numpy(rnd.view(np.int32)).cuda()).cpu().numpy().view(np.uint32)
+    for i in range(0, 4096, 97):
+        assert tuple(got[i].tolist()) == oracle.philox4x32_10(rnd[i, :4].tolist(), rnd[i, 4:].tolist())
+
+
+SHAPES = [
+    # B, K, V, dtype
+    (1, 1, 1, "fp32"), (2, 3, 7, "fp32"), (3, 2, 8, "bf16"), (2, 2, 9, "bf16"),
+    (2, 3, 1023, "fp32"), (3, 1, 1025, "bf16"), (2, 2, 4096, "fp32"), (2, 2, 4097, "fp32"),
+    (2, 2, 8192, "bf16"), (1, 4, 8200, "bf16"), (4, 5, 32000, "fp32"), (3, 4, 32001, "bf16"),
+    (2, 3, 70001, "fp32"), (5, 7, 50000, "bf16"), (1, 64, 515, "fp32"), (700, 2, 130, "fp32"),
+]
+
+
+@pytest.mark.parametrize("B,K,V,dtype", SHAPES)
+def test_parity_shapes(ears, B, K, V, dtype):
+    """Tiny to medium cases: several chunks, ragged tails, unaligned rows (element-wise loader)."""
+    tally = Tally()
+    for seed, (T, beta) in enumerate([(1.0, 0.0), (0.8, 0.3), (1.3, 1.0)]):
+        w, t, d, x = synth.tiny_inputs(B, K, V, dtype, seed=100 + seed, temperature=T)
+        tl, *_ = run_both(ears, w, t, d, x, T, beta, seed=seed, offset=7 * seed)
+        tally.merge(tl)
+    assert_parity(tally, max_explained=1)
+    assert tally.max_rel_prob_err < 1e-5
+
+
+@pytest.mark.parametrize("idx", [1, 2, 3, 4])
+def test_parity_workloads(ears, idx):
+    w = synth.workload(idx)
+    temps = w.temperatures or (w.temperature,)
+    betas = w.betas or (w.beta,)
+    tally = Tally()
+    lens = []
+    for T in temps:
+        t, d, x = synth.make_inputs(w, "cpu", temperature=T)
+        for beta in betas:
+            for offset in range(3):
+                tl, acc, tok, ora = run_both(ears, w, t, d, x, T, beta, seed=w.verify_seed, offset=offset)
+                tally.merge(tl)
+                lens.append(float(ora.accept_len.mean()))
+    assert_parity(tally)
+    assert tally.max_rel_prob_err < 1e-5
+    print(f"\n{w.name}: rows={tally.rows} explained={tally.explained} flagged_dec={tally.flagged_decisions} "
+          f"flagged_tok={tally.flagged_tokens} max_rel={tally.max_rel_prob_err:.2e} mean_len={np.mean(lens):.2f}")
+
+
+@pytest.mark.parametrize("beta", [1.0, 0.0])
+def test_parity_largest_workload(ears, beta):
+    """Full size of the largest configuration, in the launch configuration the benchmark times;
+    beta = 0 is added because at beta = 1 nearly everything is accepted and the residual path idles."""
+    w = synth.workload(5)
+    t, d, x = synth.make_inputs(w, "cuda:0")
+    acc, tok, st = ears.verify(t, d, x, w.temperature, beta, 0, 3, stats=True)
+    torch.cuda.synchronize()
+    assert ears.last_device_status() == 0
+    ora = oracle.verify(t.cpu(), d.cpu(), x.cpu(), w.temperature, beta, seed=0, offset=3,
+                        nthreads=oracle.max_threads())
+    tally = compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, w.K, {k: v.cpu().numpy() for k, v in st.items()})
+    assert_parity(tally)
+    assert tally.max_rel_prob_err < 1e-5
+    if beta == 0.0:
+        assert (ora.accept_len < w.K).mean() > 0.3
+    print(f"\ncfg5 beta={beta}: explained={tally.explained} flagged_tok={tally.flagged_tokens} "
+          f"max_rel={tally.max_rel_prob_err:.2e} mean_len={ora.accept_len.mean():.2f}")
+
+
+def test_launch_plans_agree(ears):
+    """Loader (bulk copy vs element-wise) and row splitting only change summation order."""
+    w, t, d, x = synth.tiny_inputs(6, 3, 40000, "bf16", seed=5)
+    try:
+        results = []
+        for plan in [(0, 0, 0), (1, 1, 1), (2, 0, 0), (1, 3, 2), (2, 5, 5), (1, 1000, 1000)]:
+            ears.set_plan(*plan)
+            tl, acc, tok, _ = run_both(ears, w, t, d, x, 1.0, 0.2, seed=3, offset=1)
+            assert_parity(tl, max_explained=1)
+            results.append((acc.cpu(), tok.cpu()))
+    finally:
+        ears.set_plan(0, 0, 0)
+    same = sum(torch.equal(r[1], results[0][1]) for r in results)
+    assert same >= len(results) - 1
+
+
+def test_invalid_sequences_are_marked(ears):
+    w, t, d, x = synth.tiny_inputs(8, 3, 5000, "fp32", seed=9)
+    t = t.clone(); d = d.clone(); x = x.clone()
+    x[1, 0] = 5000
+    x[2, 2] = -3
+    t[3, 1, 77] = float("nan")
+    d[4, 0, 4999] = float("inf")
+    t[5, 3, :] = float("-inf")
+    t[0, 0, 10:500] = float("-inf")   # masked vocabulary entries are legal
+    d[0, 0, 10:500] = float("-inf")
+    x[0, 0] = 5
+    dev = "cuda:0"
+    acc, tok = ears.verify(t.to(dev), d.to(dev), x.to(dev), 1.0, 0.1, 1, 2)
+    torch.cuda.synchronize()
+    assert ears.last_device_status() & ears.DEV_INVALID_INPUT
+    ora = oracle.verify(t, d, x, 1.0, 0.1, seed=1, offset=2)
+    assert ora.accept_len[1:6].tolist() == [-1] * 5
+    tl = compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, 3)
+    assert_parity(tl, max_explained=0)
+    # the next call starts from a clean status
+    acc, tok = ears.verify(t[6:].to(dev), d[6:].to(dev), x[6:].to(dev), 1.0, 0.1, 1, 2, b_first=6)
+    assert ears.last_device_status() == 0
+    assert torch.equal(acc.cpu(), torch.from_numpy(ora.accept_len[6:]))
+
+
+def test_batch_shards_match_full_batch(ears):
+    from paper_2512_13194_b200.shard import shard_range
+    w, t, d, x = synth.tiny_inputs(11, 4, 9000, "bf16", seed=21)
+    dev = "cuda:0"
+    full_len, full_tok = ears.verify(t.to(dev), d.to(dev), x.to(dev), 0.9, 0.1, 5, 17)
+    for world in (2, 3):
+        for rank in range(world):
+            lo, n = shard_range(11, rank, world)
+            a, k = ears.verify(t[lo:lo + n].to(dev), d[lo:lo + n].to(dev), x[lo:lo + n].to(dev), 0.9, 0.1, 5, 17,
+                               b_first=lo)
+            assert torch.equal(a, full_len[lo:lo + n]) and torch.equal(k, full_tok[lo:lo + n])
+
+
+def test_entry_points_agree(ears):
+    """13-argument symbols, caller-owned workspace, a side stream and the host-buffer entry."""
+    dev = "cuda:0"
+    for dtype, name in (("fp32", "ears_verify_f32"), ("bf16", "ears_verify_bf16"), ("fp32", "ears_verify")):
+        w, t, d, x = synth.tiny_inputs(5, 3, 12000, dtype, seed=33)
+        tg, dg, xg = t.to(dev), d.to(dev), x.to(dev)
+        ref_len, ref_tok = ears.verify(tg, dg, xg, 1.1, 0.2, 9, 4)
+        a, k = ears.verify_abi(name, tg, dg, xg, 1.1, 0.2, 9, 4)
+        assert torch.equal(a, ref_len) and torch.equal(k, ref_tok)
+        ws = torch.empty(ears.workspace_bytes(5, 3, 12000) + 256, dtype=torch.uint8, device=dev)
+        ws = ws[(-ws.data_ptr()) % 256:]
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            a, k = ears.verify(tg, dg, xg, 1.1, 0.2, 9, 4, workspace=ws, stream=side)
+        side.synchronize()
+        assert torch.equal(a, ref_len) and torch.equal(k, ref_tok)
+        assert ears.workspace_device_status(ws, side) == 0
+        with pytest.raises(ears.EarsError):
+            ears.verify(tg, dg, xg, 1.1, 0.2, 9, 4, workspace=ws[:256])
+        ha, hk = ears.verify_host(t.pin_memory(), d.pin_memory(), x.pin_memory(), 1.1, 0.2, 9, 4)
+        assert torch.equal(ha, ref_len.cpu()) and torch.equal(hk, ref_tok.cpu())
+        ha, hk = ears.verify_host(t, d, x, 1.1, 0.2, 9, 4)   # pageable memory works too
+        assert torch.equal(ha, ref_len.cpu()) and torch.equal(hk, ref_tok.cpu())
+
+
+def test_repeated_calls_are_reproducible(ears):
+    w, t, d, x = synth.tiny_inputs(9, 5, 20000, "fp32", seed=44)
+    dev = "cuda:0"
+    tg, dg, xg = t.to(dev), d.to(dev), x.to(dev)
+    first = ears.verify(tg, dg, xg, 1.0, 0.1, 1, 1)
+    for _ in range(5):
+        again = ears.verify(tg, dg, xg, 1.0, 0.1, 1, 1)
+        assert torch.equal(again[0], first[0]) and torch.equal(again[1], first[1])
+    other = ears.verify(tg, dg, xg, 1.0, 0.1, 1, 2)
+    assert not torch.equal(other[1], first[1])
