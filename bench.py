@@ -1,0 +1,315 @@
+#!/usr/bin/env python
+"""Benchmark of the EARS verification step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload 1..5]
+
+One step = one pass of the whole hot path (statistics + decisions + first-reject scan +
+final token) over one batch of synthetic logits.  The default workload is the largest
+configuration (B=512, K=3, V=256000, fp32: 3.67 GB of logits, far larger than L2, so every
+step streams from HBM).  With N > 1 (launched by torch.distributed.run, one rank per GPU)
+each rank verifies its own batch of the same size with its global sequence offset: batch
+sharding, no data-path collective, weak scaling.
+
+Rank 0 prints ONE JSON line.  `--impl reference` times the fp64 CPU oracle instead (a
+deliberately plain program) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "verify rows/s"
+UNIT = "rows/s"
+DATASHEET_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    REASONS = {
+        0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+        0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting",
+        0x100: "display_clock_setting", 0x10: "sync_boost",
+    }
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._halt = threading.Event()
+        self.error = None
+
+    def run(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM)
+            while not self._halt.is_set():
+                self.samples.append(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM))
+                mask = pynvml.nvmlDeviceGetCurrentClocksEventReasons(h) if hasattr(
+                    pynvml, "nvmlDeviceGetCurrentClocksEventReasons") else pynvml.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+                time.sleep(self.period)
+        except Exception as e:  # NVML missing: report it rather than guess
+            self.error = repr(e)
+
+    def stop(self):
+        self._halt.set()
+        self.join(timeout=2)
+        out = {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+               "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+        if self.error:
+            out["error"] = self.error
+        return out
+
+
+def physical_gpu_index(local_index: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_index])
+        except Exception:
+            return local_index
+    return local_index
+
+
+def resample_bytes(accept_len, K: int, V: int, esize: int) -> int:
+    """Bytes of the rows the final-token kernel reads: two rows after a rejection, one for a bonus."""
+    n = accept_len[accept_len >= 0]
+    return int(((n < K).sum().item() * 2 + (n >= K).sum().item()) * V * esize)
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2512_13194_b200 as ears
+    from paper_2512_13194_b200 import synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}: launch with torch.distributed.run")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the verification step has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    ears.load_library()
+
+    w = synth.workload(args.workload)
+    if args.batch:
+        w = w.with_batch(args.batch)
+    # every rank holds a batch of the configured size; rank r owns global sequences [r*B, (r+1)*B)
+    wr = w if world == 1 else dataclasses.replace(w, data_seed=w.data_seed + 7919 * rank)
+    t, d, x = synth.make_inputs(wr, dev)
+    b_first = rank * w.B
+    K, V, esize = w.K, w.V, w.elem_bytes
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        return ears.verify(t, d, x, w.temperature, w.beta, w.verify_seed, i, b_first=b_first)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(args.warmup, 3)):
+        acc, tok = step(i)
+    barrier()
+    if ears.last_device_status() != 0:
+        raise SystemExit("device status not clean after warm-up")
+
+    sampler = ClockSampler(physical_gpu_index(local)) if rank == 0 else None
+    if sampler:
+        sampler.start()
+        time.sleep(0.05)
+    ears.profile_begin(args.steps)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for i in range(args.steps):
+        acc, tok = step(1000 + i)
+    e1.record(stream)
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    k1_ms, k2_ms = ears.profile_end(args.steps)
+    clocks = sampler.stop() if sampler else None
+    if ears.last_device_status() != 0:
+        raise SystemExit("device status not clean after the timed region")
+
+    ms = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+    ms_step = ms.item() / args.steps
+    rows_total = w.rows * world
+    value = rows_total / (ms_step * 1e-3)
+
+    logits_bytes = w.logit_bytes
+    rs_bytes = resample_bytes(acc, K, V, esize)
+    step_bytes = logits_bytes + rs_bytes
+    k1_avg = statistics.fmean(k1_ms)
+    k2_avg = statistics.fmean(k2_ms)
+    peak, peak_kind = measured_peak()
+    achieved = logits_bytes / (k1_avg * 1e-3) / 1e9
+
+    # end to end through the host-buffer entry point: H2D of the inputs and D2H of the results every step
+    th, dh, xh = (a.cpu().pin_memory() for a in (t, d, x))
+    out_len = torch.empty(w.B, dtype=torch.int32).pin_memory()
+    out_tok = torch.empty((w.B, K + 1), dtype=torch.int32).pin_memory()
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    ears.verify_host(th, dh, xh, w.temperature, w.beta, w.verify_seed, 0, b_first=b_first,
+                     out_accept_len=out_len, out_tokens=out_tok)
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(e2e_steps):
+        ears.verify_host(th, dh, xh, w.temperature, w.beta, w.verify_seed, 1000 + i, b_first=b_first,
+                         out_accept_len=out_len, out_tokens=out_tok)
+    torch.cuda.synchronize()
+    e2e_s = torch.tensor([time.perf_counter() - t0], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(e2e_s, op=dist.ReduceOp.MAX)
+    e2e_value = rows_total / (e2e_s.item() / e2e_steps)
+    h2d = th.numel() * th.element_size() + dh.numel() * dh.element_size() + xh.numel() * 4
+    d2h = out_len.numel() * 4 + out_tok.numel() * 4
+    chk_len, chk_tok = step(1000 + e2e_steps - 1)
+    assert torch.equal(out_len, chk_len.cpu()) and torch.equal(out_tok, chk_tok.cpu()), \
+        "host entry disagrees with device entry"
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_baseline(w, th, dh, xh, args.cpu_sample)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic",
+            "config": {"workload": w.name, "B_per_gpu": w.B, "K": K, "V": V, "logits_dtype": w.dtype,
+                       "temperature": w.temperature, "beta": w.beta, "parallelism": f"batch-shard x{world}",
+                       "l2": "inputs (3.67 GB at the default workload) exceed L2; no flush needed"
+                             if logits_bytes > 512e6 else "inputs fit L2: warm-cache number",
+                       "mean_accept_len": float(acc.float().mean().item())},
+            "hbm_gbs_step": step_bytes / (ms_step * 1e-3) / 1e9,
+            "bytes_per_step": {"logits": logits_bytes, "final_token_rows": rs_bytes},
+            "kernel_ms": {"rowstats_decide": k1_avg, "final_token": k2_avg},
+            "roofline": {"bound": "hbm", "kernel": "k1_rowstats_decide", "achieved": achieved, "peak": peak,
+                         "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                         "frac_of_datasheet_8000": achieved / DATASHEET_HBM_GBS,
+                         "traffic": None},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": e2e_steps},
+            "gpu_launches": 2 * args.steps,
+            "clocks": clocks,
+        }
+        if cpu:
+            line["cpu_baseline"] = cpu
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def cpu_baseline(w, th, dh, xh, sample: int):
+    """The oracle as it stands on the host cores, on the first `sample` sequences of the workload."""
+    import oracle
+    n = min(sample, w.B)
+    cores = min(oracle.max_threads(), len(os.sched_getaffinity(0)))
+    t0 = time.perf_counter()
+    oracle.verify(th[:n], dh[:n], xh[:n], w.temperature, w.beta, seed=w.verify_seed, offset=1000, nthreads=cores)
+    dt = time.perf_counter() - t0
+    return {"value": n * (2 * w.K + 1) / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"first {n} of {w.B} sequences of {w.name}, one step, {dt:.2f} s wall"}
+
+
+def run_reference(args):
+    """The fp64 oracle on the host cores; each step verifies a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2512_13194_b200 import synth
+    w = synth.workload(args.workload)
+    if args.batch:
+        w = w.with_batch(args.batch)
+    cores = min(oracle.max_threads(), len(os.sched_getaffinity(0)))
+    warm = max(args.warmup, 1)
+    # size the per-step sample so that (steps + warm-up) oracle calls take about two minutes
+    probe_w = w.with_batch(min(w.B, 16))
+    t, d, x = synth.make_inputs(probe_w, "cpu")
+    t0 = time.perf_counter()
+    oracle.verify(t, d, x, w.temperature, w.beta, seed=w.verify_seed, offset=0, nthreads=cores)
+    per_seq = (time.perf_counter() - t0) / probe_w.B
+    budget = 120.0 / (args.steps + warm)
+    n = int(max(1, min(w.B, budget / max(per_seq, 1e-9))))
+    if n > probe_w.B:
+        n = (n // 16) * 16 or n
+        t, d, x = synth.make_inputs(w.with_batch(n), "cpu")
+    else:
+        t, d, x = t[:n], d[:n], x[:n]
+    for i in range(warm):
+        oracle.verify(t, d, x, w.temperature, w.beta, seed=w.verify_seed, offset=i, nthreads=cores)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        oracle.verify(t, d, x, w.temperature, w.beta, seed=w.verify_seed, offset=1000 + i, nthreads=cores)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = n * (2 * w.K + 1) / dt
+    sample = f"first {n} of {w.B} sequences of {w.name} per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": warm, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B_per_step": n, "K": w.K, "V": w.V, "logits_dtype": w.dtype,
+                   "temperature": w.temperature, "beta": w.beta},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", type=int, default=5, help="1..5; the default is the largest configuration")
+    ap.add_argument("--batch", type=int, default=0, help="override B (smaller cases for profiler captures)")
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--cpu-sample", type=int, default=512, help="sequences given to the CPU baseline")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -170,6 +170,18 @@ int ears_philox_device(const uint32_t* ctr_key, uint32_t* out, int n, void* stre
  */
 int ears_set_plan(int loader, int parts_stats, int parts_final);
 
+/*
+ * Per-kernel device timing for benchmarks.  After ears_profile_begin(max_calls) every
+ * verification call (up to max_calls) records CUDA events on its stream before the
+ * statistics kernel, between the two kernels and after the final-token kernel; nothing
+ * synchronises.  ears_profile_end waits for the last recorded event, writes the
+ * per-call durations in milliseconds (statistics kernel, final-token kernel) into the
+ * two host arrays of `capacity` floats, stores the number of calls timed in *n_calls
+ * and releases the events.  Not thread-safe against concurrent verification calls.
+ */
+int ears_profile_begin(int max_calls);
+int ears_profile_end(float* stats_ms, float* final_ms, int capacity, int* n_calls);
+
 const char* ears_status_string(int status);
 const char* ears_last_cuda_error(void); /* text of the last failing CUDA call on this thread, or "" */
 int ears_version(void);

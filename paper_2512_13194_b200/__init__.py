@@ -12,6 +12,8 @@ from .binding import (  # noqa: F401
     last_device_status,
     load_library,
     philox_device,
+    profile_begin,
+    profile_end,
     set_plan,
     shutdown,
     verify,

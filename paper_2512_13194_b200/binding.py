@@ -55,6 +55,10 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ears_philox_device.restype = c.c_int
     lib.ears_set_plan.argtypes = [c.c_int, c.c_int, c.c_int]
     lib.ears_set_plan.restype = c.c_int
+    lib.ears_profile_begin.argtypes = [c.c_int]
+    lib.ears_profile_begin.restype = c.c_int
+    lib.ears_profile_end.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.POINTER(c.c_int)]
+    lib.ears_profile_end.restype = c.c_int
     lib.ears_status_string.argtypes = [c.c_int]
     lib.ears_status_string.restype = c.c_char_p
     lib.ears_last_cuda_error.argtypes = []
@@ -206,6 +210,19 @@ def philox_device(ctr_key: torch.Tensor) -> torch.Tensor:
 
 def set_plan(loader: int = 0, parts_stats: int = 0, parts_final: int = 0) -> None:
     _check(load_library().ears_set_plan(loader, parts_stats, parts_final))
+
+
+def profile_begin(max_calls: int) -> None:
+    _check(load_library().ears_profile_begin(int(max_calls)))
+
+
+def profile_end(capacity: int):
+    """-> (stats_ms, final_ms): per-call device durations of the two kernels."""
+    a = (ctypes.c_float * capacity)()
+    b = (ctypes.c_float * capacity)()
+    n = ctypes.c_int(0)
+    _check(load_library().ears_profile_end(a, b, capacity, ctypes.byref(n)))
+    return list(a[:n.value]), list(b[:n.value])
 
 
 def version() -> int:

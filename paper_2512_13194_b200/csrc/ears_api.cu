@@ -8,6 +8,7 @@
 #include <map>
 #include <mutex>
 #include <utility>
+#include <vector>
 
 #include "ears_common.cuh"
 #include "ears_k1.cuh"
@@ -44,6 +45,12 @@ std::map<int, DeviceInfo> g_devices;
 struct Buffer { void* ptr = nullptr; size_t bytes = 0; };
 std::map<std::pair<int, void*>, Buffer> g_workspaces;  // (device, stream) -> scratch
 std::map<std::pair<int, void*>, Buffer> g_staging;     // (device, stream) -> host-entry staging
+
+struct Profile {
+    bool active = false;
+    int max_calls = 0;
+    std::vector<cudaEvent_t> events;  // 3 per timed call
+} g_profile;
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -139,6 +146,15 @@ int set_attrs() {
     return EARS_OK;
 }
 
+int profile_mark(cudaStream_t stream, bool timed) {
+    if (!timed) return EARS_OK;
+    cudaEvent_t ev;
+    EARS_CUDA(cudaEventCreate(&ev));
+    g_profile.events.push_back(ev);
+    EARS_CUDA(cudaEventRecord(ev, stream));
+    return EARS_OK;
+}
+
 template <typename E>
 int launch(const Params& p, int sms, cudaStream_t stream) {
     const long long units1 = (long long)p.B * (2 * p.K + 1) * p.plan.parts1;
@@ -146,11 +162,16 @@ int launch(const Params& p, int sms, cudaStream_t stream) {
     const long long cap = (long long)sms * kCtasPerSm;
     const int grid1 = (int)(units1 < cap ? units1 : cap);
     const int grid2 = (int)(units2 < cap ? units2 : cap);
+    const bool timed = g_profile.active && (int)g_profile.events.size() + 3 <= 3 * g_profile.max_calls;
+    int rc = profile_mark(stream, timed);
+    if (rc) return rc;
     k1_rowstats_decide<E, kStages1><<<grid1, kThreads, smem1<E>(), stream>>>(p);
     EARS_CUDA(cudaGetLastError());
+    rc = profile_mark(stream, timed);
+    if (rc) return rc;
     k2_final_token<E, kStages2><<<grid2, kThreads, smem2<E>(), stream>>>(p);
     EARS_CUDA(cudaGetLastError());
-    return EARS_OK;
+    return profile_mark(stream, timed);
 }
 
 int get_buffer(std::map<std::pair<int, void*>, Buffer>& pool, int dev, void* stream, size_t bytes, void** out) {
@@ -393,6 +414,37 @@ int ears_set_plan(int loader, int parts_stats, int parts_final) {
     g_override.parts1 = parts_stats;
     g_override.parts2 = parts_final;
     return EARS_OK;
+}
+
+int ears_profile_begin(int max_calls) {
+    if (max_calls < 1 || max_calls > (1 << 20)) return EARS_ERR_PARAM;
+    for (cudaEvent_t ev : g_profile.events) cudaEventDestroy(ev);
+    g_profile.events.clear();
+    g_profile.events.reserve((size_t)3 * max_calls);
+    g_profile.max_calls = max_calls;
+    g_profile.active = true;
+    return EARS_OK;
+}
+
+int ears_profile_end(float* stats_ms, float* final_ms, int capacity, int* n_calls) {
+    if (!stats_ms || !final_ms || !n_calls) return EARS_ERR_NULL;
+    g_profile.active = false;
+    const int calls = (int)(g_profile.events.size() / 3);
+    int rc = EARS_OK;
+    if (calls > 0) {
+        cudaError_t e = cudaEventSynchronize(g_profile.events[(size_t)3 * calls - 1]);
+        if (e != cudaSuccess) rc = cuda_fail(e, "cudaEventSynchronize");
+    }
+    int n = 0;
+    for (int i = 0; i < calls && i < capacity && rc == EARS_OK; ++i, ++n) {
+        cudaError_t e = cudaEventElapsedTime(&stats_ms[i], g_profile.events[3 * i], g_profile.events[3 * i + 1]);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&final_ms[i], g_profile.events[3 * i + 1], g_profile.events[3 * i + 2]);
+        if (e != cudaSuccess) rc = cuda_fail(e, "cudaEventElapsedTime");
+    }
+    for (cudaEvent_t ev : g_profile.events) cudaEventDestroy(ev);
+    g_profile.events.clear();
+    *n_calls = n;
+    return rc;
 }
 
 const char* ears_status_string(int status) {
