@@ -75,7 +75,7 @@ enum {
 
 enum { EARS_DTYPE_F32 = 0, EARS_DTYPE_BF16 = 1 };
 
-/* bits of the sticky device status word */
+/* bits of the device status word of a call */
 enum { EARS_DEV_INVALID_INPUT = 1, EARS_DEV_TIMEOUT = 2 };
 
 #define EARS_MAX_K 64
@@ -146,9 +146,9 @@ int ears_verify_host(int dtype, const void* target_logits, const void* draft_log
 size_t ears_workspace_bytes(int B, int K, int V);
 
 /*
- * Waits for `stream`, then returns and clears the sticky device status of the
- * library-owned workspace of (current device, stream): an OR of EARS_DEV_* bits,
- * or a negative EARS_ERR_* if the wait itself failed.
+ * Waits for `stream`, then returns the device status of the most recent call that
+ * used the library-owned workspace of (current device, stream): an OR of EARS_DEV_*
+ * bits (every call starts from 0), or a negative EARS_ERR_* if the wait itself failed.
  */
 int ears_last_device_status(void* stream);
 
