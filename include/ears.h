@@ -142,6 +142,47 @@ int ears_verify_host(int dtype, const void* target_logits, const void* draft_log
                      int64_t b_first, int32_t* out_accept_len, int32_t* out_tokens,
                      void* stream);
 
+/*
+ * Verification step for callers that must not allocate device memory.
+ * (The paper has no counterpart; this is a packaging variant of ears_verify_ex.)
+ *
+ * Some hosts of this library cannot call cudaMalloc at the moment they verify: code
+ * running while a CUDA graph is being captured on the thread, a serving loop that gave
+ * all device memory to its own pool at start-up and forbids later driver allocations,
+ * or a latency-critical thread that must never take the allocator's device-wide lock.
+ * ears_verify_ex allocates when it is given no workspace, and a caller workspace has
+ * to come from somewhere.  This entry point instead keeps its scratch in a fixed
+ * array of EARS_NOALLOC_SCRATCH_BYTES that is part of the library image: every GPU
+ * that loads the library holds those bytes until the process exits, whether or not
+ * this function is ever called.
+ *
+ * Arguments and results are those of ears_verify_ex without the optional outputs and
+ * without a workspace; inputs and outputs are still the caller's device buffers.
+ * The function calls no cudaMalloc, cudaFree or other allocating routine (keep the
+ * ears_profile_* timing hooks off around it: they create events).
+ *
+ *   - Shapes whose scratch need, ears_workspace_bytes(B,K,V), exceeds
+ *     EARS_NOALLOC_SCRATCH_BYTES are refused with EARS_ERR_WORKSPACE before anything
+ *     is enqueued (B=512, K=3, V=256000 needs about 2.2 MB).
+ *   - The first call on each device looks up the array's device address (and sets the
+ *     kernels' shared-memory attribute); make that first call outside any stream
+ *     capture.  The device must be current, as for every other entry point.
+ *   - All calls on a device share the one array.  It keeps the previous call's
+ *     contents; the counters that must start at zero are cleared at the start of every
+ *     call, on the call's stream.  Calls that can overlap on the GPU (different streams
+ *     without an ordering between them, or different host threads) race on it and
+ *     give wrong results: serialise them, or use ears_verify_ex with separate workspaces.
+ *   - out_device_status: optional DEVICE pointer to one int32; when not NULL the call's
+ *     status word (EARS_DEV_* bits, 0 = clean) is copied there on `stream` after the
+ *     kernels, for the caller to read once the stream has been waited for.
+ */
+#define EARS_NOALLOC_SCRATCH_BYTES (4u << 20)
+int ears_verify_noalloc(int dtype, const void* target_logits, const void* draft_logits,
+                        const int32_t* draft_tokens, int B, int K, int V,
+                        float temperature, float beta, uint64_t seed, uint64_t offset,
+                        int64_t b_first, int32_t* out_accept_len, int32_t* out_tokens,
+                        int32_t* out_device_status, void* stream);
+
 /* Upper bound of the scratch bytes a call with these sizes needs (either dtype). */
 size_t ears_workspace_bytes(int B, int K, int V);
 

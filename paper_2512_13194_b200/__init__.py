@@ -19,6 +19,7 @@ from .binding import (  # noqa: F401
     verify,
     verify_abi,
     verify_host,
+    verify_noalloc,
     version,
     workspace_bytes,
     workspace_device_status,

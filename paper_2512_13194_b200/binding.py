@@ -45,6 +45,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ears_verify_ex.restype = c.c_int
     lib.ears_verify_host.argtypes = [c.c_int] + common + [c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p]
     lib.ears_verify_host.restype = c.c_int
+    lib.ears_verify_noalloc.argtypes = [c.c_int] + common + [c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
+    lib.ears_verify_noalloc.restype = c.c_int
     lib.ears_workspace_bytes.argtypes = [c.c_int, c.c_int, c.c_int]
     lib.ears_workspace_bytes.restype = c.c_size_t
     lib.ears_last_device_status.argtypes = [c.c_void_p]
@@ -178,6 +180,37 @@ def verify_host(target_logits: torch.Tensor, draft_logits: torch.Tensor, draft_t
                               int(offset), int(b_first), acc.data_ptr(), tok.data_ptr(), _stream_ptr(stream))
     _check(rc)
     return acc, tok
+
+
+NOALLOC_SCRATCH_BYTES = 4 << 20
+
+
+def verify_noalloc(target_logits, draft_logits, draft_tokens, temperature, beta, seed, offset, *,
+                   out_accept_len: torch.Tensor, out_tokens: torch.Tensor, b_first: int = 0,
+                   out_device_status: Optional[torch.Tensor] = None, stream=None) -> None:
+    """ears_verify_noalloc: the step for callers that cannot allocate device memory.
+
+    Every buffer, outputs included, is the caller's (this wrapper creates no tensor); the
+    library's scratch is a fixed array inside the library.  Shapes needing more scratch than
+    NOALLOC_SCRATCH_BYTES raise EarsError(-5).  Calls that may overlap on the GPU share that
+    one array and race: keep them on one stream or otherwise ordered.
+    """
+    lib = load_library()
+    B, K, V = _shapes(target_logits, draft_logits, draft_tokens)
+    for a in (target_logits, draft_logits, draft_tokens, out_accept_len, out_tokens):
+        if not a.is_cuda or not a.is_contiguous():
+            raise ValueError("verify_noalloc takes contiguous CUDA tensors and converts nothing")
+    if draft_tokens.dtype != torch.int32 or out_accept_len.dtype != torch.int32 or out_tokens.dtype != torch.int32:
+        raise TypeError("token and output tensors must be int32")
+    if out_accept_len.numel() != B or tuple(out_tokens.shape) != (B, K + 1):
+        raise ValueError("outputs must be [B] and [B,K+1]")
+    with torch.cuda.device(target_logits.device):
+        rc = lib.ears_verify_noalloc(_dtype_code(target_logits), target_logits.data_ptr(), draft_logits.data_ptr(),
+                                     draft_tokens.data_ptr(), B, K, V, float(temperature), float(beta), int(seed),
+                                     int(offset), int(b_first), out_accept_len.data_ptr(), out_tokens.data_ptr(),
+                                     None if out_device_status is None else out_device_status.data_ptr(),
+                                     _stream_ptr(stream))
+    _check(rc)
 
 
 def workspace_bytes(B: int, K: int, V: int) -> int:

@@ -282,6 +282,25 @@ size_t workspace_bound(int B, int K, int V) {
     return best;
 }
 
+// Scratch of the allocation-free entry point.  Part of the library image: each GPU that
+// loads the library carries it.  In host code this name is only a handle for
+// cudaGetSymbolAddress; the kernels must be given the address that call returns.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[EARS_NOALLOC_SCRATCH_BYTES];
+std::map<int, void*> g_noalloc_ptr;  // device -> device address of g_noalloc_scratch
+
+int noalloc_scratch(int dev, void** out) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    auto it = g_noalloc_ptr.find(dev);
+    if (it == g_noalloc_ptr.end()) {
+        void* ptr = nullptr;
+        EARS_CUDA(cudaGetSymbolAddress(&ptr, g_noalloc_scratch));  // for the current device
+        if (!ptr || ((uintptr_t)ptr % 256)) return EARS_ERR_ALIGN;
+        it = g_noalloc_ptr.emplace(dev, ptr).first;
+    }
+    *out = it->second;
+    return EARS_OK;
+}
+
 __global__ void philox_kernel(const uint32_t* ctr_key, uint32_t* out, int n) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
@@ -370,6 +389,29 @@ int ears_verify_host(int dtype, const void* target_logits, const void* draft_log
     const int status = ears_last_device_status(stream_);
     if (status < 0) return status;
     return (status & EARS_DEV_TIMEOUT) ? EARS_ERR_TIMEOUT : EARS_OK;
+}
+
+int ears_verify_noalloc(int dtype, const void* target_logits, const void* draft_logits,
+                        const int32_t* draft_tokens, int B, int K, int V, float temperature, float beta,
+                        uint64_t seed, uint64_t offset, int64_t b_first, int32_t* out_accept_len,
+                        int32_t* out_tokens, int32_t* out_device_status, void* stream) {
+    if (!target_logits || !draft_logits || !draft_tokens || !out_accept_len || !out_tokens) return EARS_ERR_NULL;
+    int rc = check_shape(B, K, V);
+    if (rc) return rc;
+    if (workspace_bound(B, K, V) > (size_t)EARS_NOALLOC_SCRATCH_BYTES) return EARS_ERR_WORKSPACE;
+    int dev = 0;
+    EARS_CUDA(cudaGetDevice(&dev));
+    void* scratch = nullptr;
+    rc = noalloc_scratch(dev, &scratch);
+    if (rc) return rc;
+    rc = verify_impl(dtype, target_logits, draft_logits, draft_tokens, B, K, V, temperature, beta, seed, offset,
+                     b_first, out_accept_len, out_tokens, nullptr, nullptr, nullptr, nullptr, nullptr, scratch,
+                     (size_t)EARS_NOALLOC_SCRATCH_BYTES, stream);
+    if (rc) return rc;
+    if (out_device_status)  // the status word is heads[2] at the start of the scratch
+        EARS_CUDA(cudaMemcpyAsync(out_device_status, (const int*)scratch + 2, sizeof(int),
+                                  cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+    return EARS_OK;
 }
 
 size_t ears_workspace_bytes(int B, int K, int V) {
