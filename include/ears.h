@@ -205,23 +205,22 @@ int ears_philox_device(const uint32_t* ctr_key, uint32_t* out, int n, void* stre
 /*
  * Launch-plan override for tests (0 = automatic for every field):
  *   loader 1 = bulk-copy (TMA) loader where alignment allows, 2 = element-wise loader;
- *   parts_stats / parts_final = number of pieces each row is split into for the
- *   statistics kernel / the final-token kernel (clamped to what the row allows).
+ *   parts  = number of pieces each row is split into for the statistics pass (clamped
+ *   to what the row allows).
  * Results never depend on the plan except through floating-point summation order.
  */
-int ears_set_plan(int loader, int parts_stats, int parts_final);
+int ears_set_plan(int loader, int parts);
 
 /*
- * Per-kernel device timing for benchmarks.  After ears_profile_begin(max_calls) every
- * verification call (up to max_calls) records CUDA events on its stream before the
- * statistics kernel, between the two kernels and after the final-token kernel; nothing
- * synchronises.  ears_profile_end waits for the last recorded event, writes the
- * per-call durations in milliseconds (statistics kernel, final-token kernel) into the
- * two host arrays of `capacity` floats, stores the number of calls timed in *n_calls
- * and releases the events.  Not thread-safe against concurrent verification calls.
+ * Device timing of the kernel for benchmarks.  After ears_profile_begin(max_calls) every
+ * verification call (up to max_calls) records a CUDA event on its stream right before and
+ * right after its kernel; nothing synchronises.  ears_profile_end waits for the last
+ * recorded event, writes the per-call kernel durations in milliseconds into the host array
+ * of `capacity` floats, stores the number of calls timed in *n_calls and releases the
+ * events.  Not thread-safe against concurrent verification calls.
  */
 int ears_profile_begin(int max_calls);
-int ears_profile_end(float* stats_ms, float* final_ms, int capacity, int* n_calls);
+int ears_profile_end(float* kernel_ms, int capacity, int* n_calls);
 
 const char* ears_status_string(int status);
 const char* ears_last_cuda_error(void); /* text of the last failing CUDA call on this thread, or "" */

@@ -55,11 +55,11 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ears_workspace_device_status.restype = c.c_int
     lib.ears_philox_device.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_void_p]
     lib.ears_philox_device.restype = c.c_int
-    lib.ears_set_plan.argtypes = [c.c_int, c.c_int, c.c_int]
+    lib.ears_set_plan.argtypes = [c.c_int, c.c_int]
     lib.ears_set_plan.restype = c.c_int
     lib.ears_profile_begin.argtypes = [c.c_int]
     lib.ears_profile_begin.restype = c.c_int
-    lib.ears_profile_end.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.POINTER(c.c_int)]
+    lib.ears_profile_end.argtypes = [c.c_void_p, c.c_int, c.POINTER(c.c_int)]
     lib.ears_profile_end.restype = c.c_int
     lib.ears_status_string.argtypes = [c.c_int]
     lib.ears_status_string.restype = c.c_char_p
@@ -241,8 +241,8 @@ def philox_device(ctr_key: torch.Tensor) -> torch.Tensor:
     return out
 
 
-def set_plan(loader: int = 0, parts_stats: int = 0, parts_final: int = 0) -> None:
-    _check(load_library().ears_set_plan(loader, parts_stats, parts_final))
+def set_plan(loader: int = 0, parts: int = 0) -> None:
+    _check(load_library().ears_set_plan(loader, parts))
 
 
 def profile_begin(max_calls: int) -> None:
@@ -250,12 +250,11 @@ def profile_begin(max_calls: int) -> None:
 
 
 def profile_end(capacity: int):
-    """-> (stats_ms, final_ms): per-call device durations of the two kernels."""
+    """-> per-call device durations (ms) of the verification kernel."""
     a = (ctypes.c_float * capacity)()
-    b = (ctypes.c_float * capacity)()
     n = ctypes.c_int(0)
-    _check(load_library().ears_profile_end(a, b, capacity, ctypes.byref(n)))
-    return list(a[:n.value]), list(b[:n.value])
+    _check(load_library().ears_profile_end(a, capacity, ctypes.byref(n)))
+    return list(a[:n.value])
 
 
 def version() -> int:

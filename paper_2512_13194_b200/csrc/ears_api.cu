@@ -1,5 +1,5 @@
 // C ABI of the EARS verification step (see include/ears.h): argument checks,
-// launch plan, workspace management and the two kernel launches.
+// launch plan, workspace management and the kernel launch.
 #include "../../include/ears.h"
 
 #include <cmath>
@@ -11,17 +11,18 @@
 #include <vector>
 
 #include "ears_common.cuh"
-#include "ears_k1.cuh"
-#include "ears_k2.cuh"
+#include "ears_kernel.cuh"
 
 namespace {
 
 using namespace ears;
 
-constexpr int kStages1 = 6;  // 6 x 16 KB per CTA, two CTAs per SM
-constexpr int kStages2 = 3;  // 3 x 2 x 16 KB
+constexpr int kStages = 6;  // 6 x 16 KB per CTA, two CTAs per SM
 constexpr int kCtasPerSm = 2;
-constexpr int kUnitChunks = 16;  // 256 KB of one row per unit when there is plenty of work
+// 64 KB of one row per unit when there is plenty of work: small enough that the rows of a
+// sequence are still in L2 when its final token is drawn, large enough to amortise the
+// per-unit reduction and ticket.
+constexpr int kUnitChunks = 4;
 
 thread_local char g_cuda_error[256] = "";
 
@@ -35,7 +36,7 @@ int cuda_fail(cudaError_t e, const char* what) {
         if (e_ != cudaSuccess) return cuda_fail(e_, #call); \
     } while (0)
 
-struct PlanOverride { int loader = 0, parts1 = 0, parts2 = 0; };
+struct PlanOverride { int loader = 0, parts1 = 0; };
 PlanOverride g_override;
 std::mutex g_mutex;
 
@@ -49,7 +50,7 @@ std::map<std::pair<int, void*>, Buffer> g_staging;     // (device, stream) -> ho
 struct Profile {
     bool active = false;
     int max_calls = 0;
-    std::vector<cudaEvent_t> events;  // 3 per timed call
+    std::vector<cudaEvent_t> events;  // 2 per timed call
 } g_profile;
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -79,13 +80,12 @@ Plan make_plan(int B, int K, int V, int esize, bool aligned, int sms, const Plan
     const int chunks = (V + chunk_elems - 1) / chunk_elems;
     pl.use_tma = aligned && ov.loader != 2;
     split_rows((long long)B * (2 * K + 1), chunks, sms, ov.parts1, &pl.parts1, &pl.cpp1);
-    split_rows((long long)B, chunks, sms, ov.parts2, &pl.parts2, &pl.cpp2);
     pl.nseg = (V + kSegElems - 1) / kSegElems;
     return pl;
 }
 
 struct Layout {
-    size_t ticket1, ticket2, heads, counters_bytes;
+    size_t ticket1, heads, counters_bytes;
     size_t partial, rowstat, pt_tok, pd_tok, max_pt, cls, resid, segsum, total;
 };
 
@@ -95,7 +95,6 @@ Layout make_layout(int B, int K, int V, int parts1) {
     size_t o = 0;
     L.heads = o; o += 16;  // fixed place: the status word is heads[2] of any workspace
     L.ticket1 = o; o += (size_t)B * 4;
-    L.ticket2 = o; o += (size_t)B * 4;
     L.counters_bytes = o;
     o = align_up(o, 256);
     L.partial = o; o = align_up(o + rows * parts1 * sizeof(float2), 256);
@@ -132,17 +131,12 @@ int device_info(int dev, DeviceInfo** out) {
     return EARS_OK;
 }
 
-template <typename E>
-size_t smem1() { return sizeof(PipeSmem<kStages1, 1>) + 128; }
-template <typename E>
-size_t smem2() { return sizeof(PipeSmem<kStages2, 2>) + 128; }
+size_t smem_bytes() { return sizeof(PipeSmem<kStages>) + 128; }
 
 template <typename E>
 int set_attrs() {
-    EARS_CUDA(cudaFuncSetAttribute(k1_rowstats_decide<E, kStages1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   (int)smem1<E>()));
-    EARS_CUDA(cudaFuncSetAttribute(k2_final_token<E, kStages2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   (int)smem2<E>()));
+    EARS_CUDA(cudaFuncSetAttribute(ears_verify_kernel<E, kStages>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)smem_bytes()));
     return EARS_OK;
 }
 
@@ -157,19 +151,13 @@ int profile_mark(cudaStream_t stream, bool timed) {
 
 template <typename E>
 int launch(const Params& p, int sms, cudaStream_t stream) {
-    const long long units1 = (long long)p.B * (2 * p.K + 1) * p.plan.parts1;
-    const long long units2 = (long long)p.B * p.plan.parts2;
+    const long long units = (long long)p.B * (2 * p.K + 1) * p.plan.parts1;
     const long long cap = (long long)sms * kCtasPerSm;
-    const int grid1 = (int)(units1 < cap ? units1 : cap);
-    const int grid2 = (int)(units2 < cap ? units2 : cap);
-    const bool timed = g_profile.active && (int)g_profile.events.size() + 3 <= 3 * g_profile.max_calls;
+    const int grid = (int)(units < cap ? units : cap);
+    const bool timed = g_profile.active && (int)g_profile.events.size() + 2 <= 2 * g_profile.max_calls;
     int rc = profile_mark(stream, timed);
     if (rc) return rc;
-    k1_rowstats_decide<E, kStages1><<<grid1, kThreads, smem1<E>(), stream>>>(p);
-    EARS_CUDA(cudaGetLastError());
-    rc = profile_mark(stream, timed);
-    if (rc) return rc;
-    k2_final_token<E, kStages2><<<grid2, kThreads, smem2<E>(), stream>>>(p);
+    ears_verify_kernel<E, kStages><<<grid, kThreads, smem_bytes(), stream>>>(p);
     EARS_CUDA(cudaGetLastError());
     return profile_mark(stream, timed);
 }
@@ -254,7 +242,6 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
     p.cls = o_cls ? o_cls : (uint8_t*)(w + L.cls);
     p.resid = o_resid ? o_resid : (double*)(w + L.resid);
     p.ticket1 = (int*)(w + L.ticket1);
-    p.ticket2 = (int*)(w + L.ticket2);
     p.heads = (int*)(w + L.heads);
     p.partial = (float2*)(w + L.partial);
     p.rowstat = (float2*)(w + L.rowstat);
@@ -449,12 +436,11 @@ int ears_philox_device(const uint32_t* ctr_key, uint32_t* out, int n, void* stre
     return EARS_OK;
 }
 
-int ears_set_plan(int loader, int parts_stats, int parts_final) {
-    if (loader < 0 || loader > 2 || parts_stats < 0 || parts_final < 0) return EARS_ERR_PARAM;
+int ears_set_plan(int loader, int parts) {
+    if (loader < 0 || loader > 2 || parts < 0) return EARS_ERR_PARAM;
     std::lock_guard<std::mutex> lock(g_mutex);
     g_override.loader = loader;
-    g_override.parts1 = parts_stats;
-    g_override.parts2 = parts_final;
+    g_override.parts1 = parts;
     return EARS_OK;
 }
 
@@ -462,25 +448,24 @@ int ears_profile_begin(int max_calls) {
     if (max_calls < 1 || max_calls > (1 << 20)) return EARS_ERR_PARAM;
     for (cudaEvent_t ev : g_profile.events) cudaEventDestroy(ev);
     g_profile.events.clear();
-    g_profile.events.reserve((size_t)3 * max_calls);
+    g_profile.events.reserve((size_t)2 * max_calls);
     g_profile.max_calls = max_calls;
     g_profile.active = true;
     return EARS_OK;
 }
 
-int ears_profile_end(float* stats_ms, float* final_ms, int capacity, int* n_calls) {
-    if (!stats_ms || !final_ms || !n_calls) return EARS_ERR_NULL;
+int ears_profile_end(float* kernel_ms, int capacity, int* n_calls) {
+    if (!kernel_ms || !n_calls) return EARS_ERR_NULL;
     g_profile.active = false;
-    const int calls = (int)(g_profile.events.size() / 3);
+    const int calls = (int)(g_profile.events.size() / 2);
     int rc = EARS_OK;
     if (calls > 0) {
-        cudaError_t e = cudaEventSynchronize(g_profile.events[(size_t)3 * calls - 1]);
+        cudaError_t e = cudaEventSynchronize(g_profile.events[(size_t)2 * calls - 1]);
         if (e != cudaSuccess) rc = cuda_fail(e, "cudaEventSynchronize");
     }
     int n = 0;
     for (int i = 0; i < calls && i < capacity && rc == EARS_OK; ++i, ++n) {
-        cudaError_t e = cudaEventElapsedTime(&stats_ms[i], g_profile.events[3 * i], g_profile.events[3 * i + 1]);
-        if (e == cudaSuccess) e = cudaEventElapsedTime(&final_ms[i], g_profile.events[3 * i + 1], g_profile.events[3 * i + 2]);
+        cudaError_t e = cudaEventElapsedTime(&kernel_ms[i], g_profile.events[2 * i], g_profile.events[2 * i + 1]);
         if (e != cudaSuccess) rc = cuda_fail(e, "cudaEventElapsedTime");
     }
     for (cudaEvent_t ev : g_profile.events) cudaEventDestroy(ev);

@@ -1,4 +1,4 @@
-// Shapes, launch plan and workspace layout shared by the two kernels and the host API.
+// Shapes, launch plan and workspace layout shared by the kernel and the host API.
 #pragma once
 #include <cstddef>
 #include <cstdint>
@@ -8,9 +8,11 @@ namespace ears {
 
 constexpr int kConsumerWarps = 8;                    // warps that reduce the staged chunks
 constexpr int kConsumers = kConsumerWarps * 32;
-constexpr int kThreads = kConsumers + 32;            // + one loader warp
-constexpr int kChunkBytes = 16384;                   // bytes of one row staged per pipeline slot
-constexpr int kSegElems = 512;                       // elements per final-token segment sum
+constexpr int kLoaderWarp = kConsumerWarps;          // streams logits into shared memory
+constexpr int kEpilogueWarp = kConsumerWarps + 1;    // per-sequence decisions and the final pick
+constexpr int kThreads = kConsumers + 64;
+constexpr int kChunkBytes = 16384;                   // bytes staged per pipeline slot
+constexpr int kSegElems = 256;                       // elements per final-token segment sum
 constexpr double kEps = 1e-10;                       // division guard, Sec. 3.3 item 2
 constexpr double kTinyMass = 1e-300;                 // below this a residual is treated as empty
 
@@ -20,15 +22,13 @@ constexpr int kDevTimeout = 2;
 
 struct Plan {
     int use_tma;   // 1: bulk asynchronous copies, 0: element-wise loader
-    int parts1;    // pieces per row, statistics kernel
+    int parts1;    // pieces per row in the statistics pass
     int cpp1;      // chunks per piece
-    int parts2;    // pieces per row, final-token kernel
-    int cpp2;
     int nseg;      // segment sums per sequence
 };
 
-// Counter block at the start of the workspace, zeroed by one memset per call.
-//   ticket1[B] ticket2[B] head1 head2 status pad
+// Counter block at the start of the workspace, zeroed by one memset per call:
+//   heads[4] (queue head, unused, status, unused) then ticket1[B].
 struct Params {
     const void* t;        // target logits [B,K+1,V]
     const void* d;        // draft logits  [B,K,V]
@@ -47,8 +47,7 @@ struct Params {
     uint8_t* cls;         // [B,K]
     double* resid;        // [B]
     int* ticket1;         // [B] arrivals of statistics pieces
-    int* ticket2;         // [B] arrivals of final-token pieces
-    int* heads;           // [0] statistics queue, [1] final-token queue, [2] status
+    int* heads;           // [0] unit queue, [2] status
     float2* partial;      // [B*(2K+1)*parts1] (m, s) per row piece
     float2* rowstat;      // [B*(2K+1)] (m, Z) per row
     double* segsum;       // [B*nseg]

@@ -62,7 +62,7 @@ def test_bad_arguments_are_rejected_on_the_host():
     assert lib.ears_verify_ex(0, p, p, p, 1, 1, 4, 1.0, 0.1, 0, 0, 0, p, p, None, None, None, None, None,
                               p + 4, 1 << 20, None) == -4
     assert lib.ears_verify_host(0, None, p, p, 1, 1, 4, 1.0, 0.1, 0, 0, 0, p, p, None) == -1
-    assert lib.ears_set_plan(3, 0, 0) == -3 and lib.ears_set_plan(0, 0, 0) == 0
+    assert lib.ears_set_plan(3, 0) == -3 and lib.ears_set_plan(0, 0) == 0
     assert lib.ears_philox_device(None, None, -1, None) == -2
     assert lib.ears_philox_device(None, None, 0, None) == 0
 
