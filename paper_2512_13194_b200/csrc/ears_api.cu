@@ -4,6 +4,7 @@
 
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <mutex>
@@ -19,10 +20,9 @@ using namespace ears;
 
 constexpr int kStages = 6;  // 6 x 16 KB per CTA, two CTAs per SM
 constexpr int kCtasPerSm = 2;
-// 64 KB of one row per unit when there is plenty of work: small enough that the rows of a
-// sequence are still in L2 when its final token is drawn, large enough to amortise the
-// per-unit reduction and ticket.
-constexpr int kUnitChunks = 4;
+// 256 KB of one row per unit when there is plenty of work (smaller units cost more per-unit
+// bookkeeping than they gain in balance; measured on B=512, V=256000).
+constexpr int kUnitChunks = 16;
 
 thread_local char g_cuda_error[256] = "";
 
@@ -36,7 +36,7 @@ int cuda_fail(cudaError_t e, const char* what) {
         if (e_ != cudaSuccess) return cuda_fail(e_, #call); \
     } while (0)
 
-struct PlanOverride { int loader = 0, parts1 = 0; };
+struct PlanOverride { int loader = 0, parts1 = 0, streams = 0, claim = 0; };
 PlanOverride g_override;
 std::mutex g_mutex;
 
@@ -81,11 +81,24 @@ Plan make_plan(int B, int K, int V, int esize, bool aligned, int sms, const Plan
     pl.use_tma = aligned && ov.loader != 2;
     split_rows((long long)B * (2 * K + 1), chunks, sms, ov.parts1, &pl.parts1, &pl.cpp1);
     pl.nseg = (V + kSegElems - 1) / kSegElems;
+    // With many units per CTA one atomic on the queue head hands out several units (spaced a
+    // grid apart, so CTAs still sweep the rows in step); same-address atomics are slow.
+    const long long units = (long long)B * (2 * K + 1) * pl.parts1;
+    const long long ctas = (long long)sms * kCtasPerSm;
+    pl.claim = units >= 32 * ctas ? 4 : (units >= 8 * ctas ? 2 : 1);
+    if (ov.claim > 0) pl.claim = ov.claim;
+    // final-token pass: 64 KB of each row per piece, single chunks when there are few sequences
+    const int job_chunks = (long long)B * ((chunks + 3) / 4) >= ctas ? 4 : 1;
+    pl.job_elems = job_chunks * chunk_elems;
+    pl.parts2 = (V + pl.job_elems - 1) / pl.job_elems;
+    pl.streams = ov.streams > 0 ? ov.streams : 1;
+    if (pl.streams > B) pl.streams = B;
+    pl.seq_per_stream = (B + pl.streams - 1) / pl.streams;
     return pl;
 }
 
 struct Layout {
-    size_t ticket1, heads, counters_bytes;
+    size_t ticket1, ticket2, job_ctr, ticket_row, ready, heads, counters_bytes;
     size_t partial, rowstat, pt_tok, pd_tok, max_pt, cls, resid, segsum, total;
 };
 
@@ -95,6 +108,11 @@ Layout make_layout(int B, int K, int V, int parts1) {
     size_t o = 0;
     L.heads = o; o += 16;  // fixed place: the status word is heads[2] of any workspace
     L.ticket1 = o; o += (size_t)B * 4;
+    L.ticket2 = o; o += (size_t)B * 4;
+    L.job_ctr = o; o += (size_t)B * 4;
+    L.ticket_row = o; o += rows * 4;
+    o = align_up(o, 8);
+    L.ready = o; o += (size_t)B * 8;
     L.counters_bytes = o;
     o = align_up(o, 256);
     L.partial = o; o = align_up(o + rows * parts1 * sizeof(float2), 256);
@@ -104,7 +122,7 @@ Layout make_layout(int B, int K, int V, int parts1) {
     L.max_pt = o; o = align_up(o + (size_t)B * K * 8, 256);
     L.cls = o; o = align_up(o + (size_t)B * K, 256);
     L.resid = o; o = align_up(o + (size_t)B * 8, 256);
-    L.segsum = o; o = align_up(o + (size_t)B * ((V + kSegElems - 1) / kSegElems) * 8, 256);
+    L.segsum = o; o = align_up(o + (size_t)B * ((V + kSegElems - 1) / kSegElems) * 4, 256);
     L.total = o;
     return L;
 }
@@ -242,10 +260,14 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
     p.cls = o_cls ? o_cls : (uint8_t*)(w + L.cls);
     p.resid = o_resid ? o_resid : (double*)(w + L.resid);
     p.ticket1 = (int*)(w + L.ticket1);
+    p.ticket_row = (int*)(w + L.ticket_row);
+    p.ticket2 = (int*)(w + L.ticket2);
+    p.job_ctr = (int*)(w + L.job_ctr);
+    p.ready = (unsigned long long*)(w + L.ready);
     p.heads = (int*)(w + L.heads);
     p.partial = (float2*)(w + L.partial);
     p.rowstat = (float2*)(w + L.rowstat);
-    p.segsum = (double*)(w + L.segsum);
+    p.segsum = (float*)(w + L.segsum);
     p.plan = plan;
     return dtype == EARS_DTYPE_F32 ? launch<float>(p, di->sms, stream) : launch<uint16_t>(p, di->sms, stream);
 }
@@ -441,6 +463,10 @@ int ears_set_plan(int loader, int parts) {
     std::lock_guard<std::mutex> lock(g_mutex);
     g_override.loader = loader;
     g_override.parts1 = parts;
+    const char* e = getenv("EARS_STREAMS");
+    g_override.streams = e ? atoi(e) : 0;
+    e = getenv("EARS_CLAIM");
+    g_override.claim = e ? atoi(e) : 0;
     return EARS_OK;
 }
 

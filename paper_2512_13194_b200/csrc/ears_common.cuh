@@ -9,8 +9,9 @@ namespace ears {
 constexpr int kConsumerWarps = 8;                    // warps that reduce the staged chunks
 constexpr int kConsumers = kConsumerWarps * 32;
 constexpr int kLoaderWarp = kConsumerWarps;          // streams logits into shared memory
-constexpr int kEpilogueWarp = kConsumerWarps + 1;    // per-sequence decisions and the final pick
-constexpr int kThreads = kConsumers + 64;
+constexpr int kEpilogueWarp = kConsumerWarps + 1;    // counts finished pieces of rows
+constexpr int kSequenceWarp = kConsumerWarps + 2;    // per-sequence decisions and the final pick
+constexpr int kThreads = kConsumers + 96;
 constexpr int kChunkBytes = 16384;                   // bytes staged per pipeline slot
 constexpr int kSegElems = 256;                       // elements per final-token segment sum
 constexpr double kEps = 1e-10;                       // division guard, Sec. 3.3 item 2
@@ -24,11 +25,17 @@ struct Plan {
     int use_tma;   // 1: bulk asynchronous copies, 0: element-wise loader
     int parts1;    // pieces per row in the statistics pass
     int cpp1;      // chunks per piece
+    int claim;     // units a CTA takes from the queue per atomic (spaced one grid apart)
+    int streams;   // the batch is swept as this many interleaved runs of sequences
+    int seq_per_stream;
+    int parts2;    // pieces per row in the final-token pass
+    int job_elems; // elements of each row per piece of the final-token pass
     int nseg;      // segment sums per sequence
 };
 
 // Counter block at the start of the workspace, zeroed by one memset per call:
-//   heads[4] (queue head, unused, status, unused) then ticket1[B].
+//   heads[4] (unit queue head, finalised sequences, status, published sequences),
+//   ticket1[B], ticket2[B], job_ctr[B], ticket_row[B*(2K+1)], ready[B].
 struct Params {
     const void* t;        // target logits [B,K+1,V]
     const void* d;        // draft logits  [B,K,V]
@@ -46,11 +53,15 @@ struct Params {
     double* max_pt;       // [B,K]
     uint8_t* cls;         // [B,K]
     double* resid;        // [B]
-    int* ticket1;         // [B] arrivals of statistics pieces
-    int* heads;           // [0] unit queue, [2] status
+    int* ticket1;         // [B] rows of the sequence whose pieces are all in
+    int* ticket_row;      // [B*(2K+1)] pieces of the row that are in
+    int* ticket2;         // [B] final-token pieces of the sequence that are in
+    unsigned long long* ready;  // [B] published sequences: (b + 1) << 32 | n, 0 = not yet
+    int* job_ctr;         // [B] final-token pieces handed out, per published slot
+    int* heads;           // [0] unit queue, [1] finalised sequences, [2] status, [3] published sequences
     float2* partial;      // [B*(2K+1)*parts1] (m, s) per row piece
     float2* rowstat;      // [B*(2K+1)] (m, Z) per row
-    double* segsum;       // [B*nseg]
+    float* segsum;        // [B*nseg] segment sums of the final-token masses
     Plan plan;
 };
 

@@ -9,9 +9,9 @@
 //                  copies when the data is not 16-byte aligned);
 //   8 consumer     keep a running (max, sum exp2) per thread over the slots [softmax
 //   warps          statistics, Sec. 3.1], reduce them per unit and publish the piece;
-//                  the CTA that delivers the last piece of a sequence hands the
-//                  sequence to its epilogue warp;
-//   epilogue warp  merges the pieces, forms P_t(x), P_d(x), max P_t = 1/Z_t, draws U_k,
+//   epilogue warp  publishes the pieces and counts them with one atomic ticket per
+//                  sequence; for a sequence whose last piece it delivered it merges the
+//                  pieces, forms P_t(x), P_d(x), max P_t = 1/Z_t, draws U_k,
 //                  decides every position (Sec. 3.2 with the guards of Sec. 3.3 item 2),
 //                  scans for the first rejection (Sec. 3.1) and asks the loader for the
 //                  one or two rows the final token needs.  Those rows were streamed
@@ -29,7 +29,7 @@
 namespace ears {
 
 enum ChunkKind : int { kStats = 0, kBonus = 1, kResid = 2, kDrain = 3, kEnd = 4 };
-enum MsgKind : int { kMsgFinalize = 0, kMsgSelect = 1, kMsgDrain = 2, kMsgExit = 3, kMsgJob = 4, kMsgAck = 5 };
+enum MsgKind : int { kMsgPiece = 0, kMsgJobPiece = 1, kMsgDrain = 2, kMsgExit = 3, kMsgAck = 5, kMsgNone = 6, kMsgFinalize = 7, kMsgSelect = 8 };
 
 struct StageMeta {
     int kind;    // ChunkKind
@@ -40,13 +40,13 @@ struct StageMeta {
     int aux;     // accepted length n of the sequence (final-token rows)
 };
 
-struct Msg { int kind, a, b; };
+struct Msg { int kind, a, b, c; };
 
 // Single-producer single-consumer ring in shared memory.  One lane pushes, one lane pops.
 template <int CAP>
 struct Mailbox {
     volatile int head, tail;
-    volatile int slot[CAP][3];
+    volatile int slot[CAP][4];
 
     __device__ __forceinline__ void init() { head = 0; tail = 0; }
 
@@ -63,7 +63,7 @@ struct Mailbox {
             __nanosleep(40);
         }
         const int t = tail;
-        slot[t % CAP][0] = m.kind; slot[t % CAP][1] = m.a; slot[t % CAP][2] = m.b;
+        slot[t % CAP][0] = m.kind; slot[t % CAP][1] = m.a; slot[t % CAP][2] = m.b; slot[t % CAP][3] = m.c;
         __threadfence_block();
         tail = t + 1;
         return true;
@@ -72,11 +72,32 @@ struct Mailbox {
         const int h = head;
         if (h == tail) return false;
         __threadfence_block();
-        m.kind = slot[h % CAP][0]; m.a = slot[h % CAP][1]; m.b = slot[h % CAP][2];
+        m.kind = slot[h % CAP][0]; m.a = slot[h % CAP][1]; m.b = slot[h % CAP][2]; m.c = slot[h % CAP][3];
         __threadfence_block();
         head = h + 1;
         return true;
     }
+    // Waits for at least one message; returns how many (<= 32) are ready starting at *first,
+    // or -1 when the block is aborting or the time limit passed.  Called by one lane.
+    __device__ __forceinline__ int wait_batch(int* first, volatile int* abort_flag, unsigned long long limit_ns) {
+        unsigned long long t0 = 0;
+        for (unsigned spin = 0;; ++spin) {
+            const int h = head, n = tail - h;
+            if (n > 0) { *first = h; return n < 32 ? n : 32; }
+            if ((spin & 15u) == 15u) {
+                if (*abort_flag) return -1;
+                unsigned long long now = global_timer_ns();
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > limit_ns) { *abort_flag = 1; return -1; }
+            }
+            __nanosleep(64);
+        }
+    }
+    __device__ __forceinline__ Msg peek(int index) const {
+        return Msg{slot[index % CAP][0], slot[index % CAP][1], slot[index % CAP][2], slot[index % CAP][3]};
+    }
+    __device__ __forceinline__ void release(int new_head) { __threadfence_block(); head = new_head; }
+
     __device__ __forceinline__ bool pop(Msg& m, volatile int* abort_flag, unsigned long long limit_ns) {
         unsigned long long t0 = 0;
         for (unsigned spin = 0;; ++spin) {
@@ -93,11 +114,17 @@ struct Mailbox {
 };
 
 // consumer warp 0 -> epilogue warp
-constexpr int kEpiCap = 32;
-// epilogue warp -> loader warp.  The loader serves this ring before it pulls a new unit, and one
-// unit produces at most one entry, so at most kEpiCap + slots + 2 entries are ever outstanding:
-// the ring never fills and the epilogue warp never blocks on it.
-constexpr int kJobCap = 64;
+constexpr int kEpiCap = 64;
+// epilogue warp -> loader warp: carries only the acknowledgement of the drain marker
+constexpr int kJobCap = 4;
+// epilogue warp -> sequence warp
+constexpr int kSeqCap = 64;
+// Ends of units are handed to the epilogue warp through a ring of slots: each consumer warp
+// drops its (m, s) there and arrives on the slot's barrier, so no consumer ever waits for
+// another at the end of a unit.  Consumer warps are at most one pipeline ring apart, and
+// warp 0 holds back while kUnitGuard ends are unread, hence the slots cannot be overrun.
+constexpr int kUnitSlots = 16;
+constexpr int kUnitGuard = 8;
 constexpr unsigned long long kIdleLimitNs = 30000000000ull;  // an idle warp may wait for the whole kernel
 
 template <int STAGES>
@@ -105,13 +132,31 @@ struct PipeSmem {
     alignas(128) unsigned char buf[STAGES][kChunkBytes];
     alignas(8) uint64_t full[STAGES];
     uint64_t empty[STAGES];
-    uint64_t red[STAGES];
+    uint64_t unit_bar[kUnitSlots];
     StageMeta meta[STAGES];
-    float2 scratch[STAGES][kConsumerWarps];
+    float2 scratch[kUnitSlots][kConsumerWarps];
+    volatile int units_read;   // unit ends the epilogue warp has taken out of the slots
     Mailbox<kEpiCap> epi;
     Mailbox<kJobCap> jobs;
+    Mailbox<kSeqCap> seq;
     int abort_flag;
 };
+
+// Consumer warp 0, one lane: announce the end of a unit, holding back while too many are unread.
+template <int STAGES>
+__device__ __forceinline__ void push_unit_end(PipeSmem<STAGES>& sm, const Msg& m) {
+    unsigned long long t0 = 0;
+    for (unsigned spin = 0; m.c - sm.units_read >= kUnitGuard; ++spin) {
+        if ((spin & 15u) == 15u) {
+            if (sm.abort_flag) return;
+            const unsigned long long now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) { sm.abort_flag = 1; return; }
+        }
+        __nanosleep(40);
+    }
+    sm.epi.push(m, &sm.abort_flag, kWaitLimitNs);
+}
 
 // ---- loader helpers -----------------------------------------------------------
 template <int STAGES>
@@ -143,7 +188,7 @@ __device__ __forceinline__ void loader_drain(PipeSmem<STAGES>& sm, uint32_t issu
 // Publishes a slot: `nelem` elements from src0 (and, at the half-slot offset, from src1).
 template <typename E, int STAGES>
 __device__ __forceinline__ void loader_fill(PipeSmem<STAGES>& sm, int stage, const StageMeta& mt, bool use_tma,
-                                            const E* src0, const E* src1, int lane) {
+                                            const E* src0, const E* src1, int lane, uint64_t policy) {
     if (lane == 0) sm.meta[stage] = mt;
     const uint32_t bytes = (uint32_t)mt.nelem * (uint32_t)sizeof(E);
     if (use_tma) {
@@ -152,8 +197,8 @@ __device__ __forceinline__ void loader_fill(PipeSmem<STAGES>& sm, int stage, con
                 mbar_arrive(&sm.full[stage]);
             } else {
                 mbar_arrive_expect_tx(&sm.full[stage], src1 ? 2 * bytes : bytes);
-                bulk_load(sm.buf[stage], src0, bytes, &sm.full[stage]);
-                if (src1) bulk_load(sm.buf[stage] + kChunkBytes / 2, src1, bytes, &sm.full[stage]);
+                bulk_load_hint(sm.buf[stage], src0, bytes, &sm.full[stage], policy);
+                if (src1) bulk_load_hint(sm.buf[stage] + kChunkBytes / 2, src1, bytes, &sm.full[stage], policy);
             }
         }
     } else {
@@ -223,28 +268,28 @@ __device__ __forceinline__ void chunk_stats(const unsigned char* buf, int nelem,
 }
 
 struct RowNorm {
-    float mt, md;     // row maxima
-    double izt, izd;  // 1 / Z
+    float mt, md;          // row maxima
+    float rho_hi, rho_lo;  // Z_t / Z_d split in two floats (residual rows)
+    double izt;            // 1 / Z_t
 };
 
-// Mass of one vocabulary entry for the final draw: P_t(v), or max(0, P_t(v) - P_d(v)).
-// Explicit rounding intrinsics so that the streaming pass and the in-segment pass
-// produce identical bits.
-template <bool RESID>
-__device__ __forceinline__ double entry_mass(float xt, float xd, const RowNorm& rn, float c) {
-    const float et = ex2_approx(__fmul_rn(__fsub_rn(xt, rn.mt), c));
-    double r = __dmul_rn((double)et, rn.izt);
-    if (RESID) {
-        const float ed = ex2_approx(__fmul_rn(__fsub_rn(xd, rn.md), c));
-        r = fmax(__dsub_rn(r, __dmul_rn((double)ed, rn.izd)), 0.0);
-    }
-    return r;
+__device__ __forceinline__ RowNorm make_rownorm(float2 st, float2 sd) {
+    const double rho = (double)st.y / (double)sd.y;
+    const float hi = (float)rho;
+    return RowNorm{st.x, sd.x, hi, (float)(rho - (double)hi), 1.0 / (double)st.y};
 }
 
-__device__ __forceinline__ double warp_sum(double v) {
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-    return v;
+// Mass of one vocabulary entry for the final draw in units of 1/Z_t:
+// Z_t P_t(v), or Z_t max(0, P_t(v) - P_d(v)) = max(0, e_t - e_d Z_t/Z_d).  The common factor
+// cancels in the inverse-CDF draw.  fp32 with the ratio carried as hi + lo so that no
+// systematic rounding of Z_t/Z_d tilts the residual; explicit rounding intrinsics so that the
+// streaming pass and the in-segment pass produce identical bits.
+template <bool RESID>
+__device__ __forceinline__ float entry_mass(float xt, float xd, const RowNorm& rn, float c) {
+    const float et = ex2_approx(__fmul_rn(__fsub_rn(xt, rn.mt), c));
+    if (!RESID) return et;
+    const float ed = ex2_approx(__fmul_rn(__fsub_rn(xd, rn.md), c));
+    return fmaxf(__fmaf_rn(-ed, rn.rho_lo, __fmaf_rn(-ed, rn.rho_hi, et)), 0.0f);
 }
 
 __device__ __forceinline__ double warp_inclusive_scan(double v, int lane) {
@@ -256,15 +301,47 @@ __device__ __forceinline__ double warp_inclusive_scan(double v, int lane) {
     return v;
 }
 
-// fp64 sums of kSegElems-element segments of a staged chunk; warp w takes segments w, w+8, ...
+// Sums of kSegElems-element segments of a staged chunk; warp w takes segments w, w+8, ...
+// All fp32: fp64 arithmetic is far too slow on this part to sit in the streaming path.  A
+// segment sum carries ~1e-7 relative rounding error, i.e. at most ~1e-7 of probability even
+// for a segment holding most of the mass; the final pick re-reads the chosen segment.
 template <typename E, bool RESID>
 __device__ __forceinline__ void chunk_segments(const unsigned char* bt, const unsigned char* bd, int nelem,
-                                               int warp, int lane, const RowNorm& rn, float c, double* seg_out) {
+                                               int warp, int lane, const RowNorm& rn, float c, float* seg_out) {
     constexpr int N = Vec<E>::N;
     constexpr int VECS = kSegElems / (32 * N);  // 16-byte vectors per lane per segment
+    constexpr int FULL_ELEMS = (RESID ? kChunkBytes / 2 : kChunkBytes) / (int)sizeof(E);
+    constexpr int SEGS = FULL_ELEMS / kSegElems / kConsumerWarps;  // segments per warp in a full slot
+    if (nelem == FULL_ELEMS) {
+        // full slot: all of the warp's segments at once, so that their loads, exponentials and
+        // shuffle trees overlap instead of running one after the other
+        float acc[SEGS];
+#pragma unroll
+        for (int g = 0; g < SEGS; ++g) {
+            acc[g] = 0.0f;
+#pragma unroll
+            for (int j = 0; j < VECS; ++j) {
+                const int vec = (g * kConsumerWarps + warp) * (kSegElems / N) + j * 32 + lane;
+                float xt[N], xd[N];
+                Vec<E>::load(bt, vec, xt);
+                if (RESID) Vec<E>::load(bd, vec, xd);
+#pragma unroll
+                for (int i = 0; i < N; ++i) acc[g] += entry_mass<RESID>(xt[i], RESID ? xd[i] : 0.f, rn, c);
+            }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1)
+#pragma unroll
+            for (int g = 0; g < SEGS; ++g) acc[g] += __shfl_xor_sync(0xffffffffu, acc[g], off);
+        if (lane == 0) {
+#pragma unroll
+            for (int g = 0; g < SEGS; ++g) seg_out[g * kConsumerWarps + warp] = acc[g];
+        }
+        return;
+    }
     const int nseg = (nelem + kSegElems - 1) / kSegElems;
     for (int sgm = warp; sgm < nseg; sgm += kConsumerWarps) {
-        double acc = 0.0;
+        float acc = 0.0f;
 #pragma unroll
         for (int j = 0; j < VECS; ++j) {
             const int vec = sgm * (kSegElems / N) + j * 32 + lane;
@@ -273,11 +350,12 @@ __device__ __forceinline__ void chunk_segments(const unsigned char* bt, const un
             if (RESID) Vec<E>::load(bd, vec, xd);
 #pragma unroll
             for (int i = 0; i < N; ++i) {
-                const double r = entry_mass<RESID>(xt[i], RESID ? xd[i] : 0.f, rn, c);
+                const float r = entry_mass<RESID>(xt[i], RESID ? xd[i] : 0.f, rn, c);
                 if (vec * N + i < nelem) acc += r;
             }
         }
-        acc = warp_sum(acc);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
         if (lane == 0) seg_out[sgm] = acc;
     }
 }
@@ -357,7 +435,7 @@ __device__ int warp_sample_pt_slow(const E* row, int V, const RowNorm& rn, float
     const int per = (V + 31) / 32;
     const int v0 = min(V, lane * per), v1 = min(V, v0 + per);
     double loc = 0.0;
-    for (int v = v0; v < v1; ++v) loc += entry_mass<false>(load_logit(row + v), 0.f, rn, c);
+    for (int v = v0; v < v1; ++v) loc += (double)entry_mass<false>(load_logit(row + v), 0.f, rn, c);
     const double inc = warp_inclusive_scan(loc, lane);
     const double S = __shfl_sync(0xffffffffu, inc, 31);
     const double target = u * S;
@@ -369,7 +447,7 @@ __device__ int warp_sample_pt_slow(const E* row, int V, const RowNorm& rn, float
         double cum = inc - loc;
         int lastpos = -1;
         for (int v = v0; v < v1; ++v) {
-            const double r = entry_mass<false>(load_logit(row + v), 0.f, rn, c);
+            const double r = (double)entry_mass<false>(load_logit(row + v), 0.f, rn, c);
             if (r > 0.0) lastpos = v;
             cum += r;
             if (target < cum && r > 0.0) { tok = v; break; }
@@ -391,20 +469,26 @@ __device__ void select_token(const Params& p, int b, int n, int lane) {
     const E* drow = reinterpret_cast<const E*>(p.d) + (size_t)draft_row(b, resid ? n : 0, K) * V;
     const float2 st = __ldcg(&p.rowstat[(size_t)b * R + (resid ? 2 * n : 2 * K)]);
     const float2 sd = resid ? __ldcg(&p.rowstat[(size_t)b * R + 2 * n + 1]) : make_float2(0.f, 1.f);
-    const RowNorm rn{st.x, sd.x, 1.0 / (double)st.y, 1.0 / (double)sd.y};
-    const double* ss = p.segsum + (size_t)b * nseg;
+    const RowNorm rn = make_rownorm(st, sd);
+    const float* ss = p.segsum + (size_t)b * nseg;
     const double u = uniform_final(p.seed, p.offset, (uint32_t)(p.b_first + b), (uint32_t)K);
 
     // level 1: which segment
     const int per = (nseg + 31) / 32;
     const int g0 = min(nseg, lane * per), g1 = min(nseg, g0 + per);
     double loc = 0.0;
-    for (int g = g0; g < g1; ++g) loc += __ldcg(ss + g);
+    for (int g = g0; g < g1; g += 8) {  // loads first, then the adds: eight reads in flight
+        float v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = g + i < g1 ? __ldcg(ss + g + i) : 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) loc += (double)v[i];
+    }
     const double inc = warp_inclusive_scan(loc, lane);
     const double S = __shfl_sync(0xffffffffu, inc, 31);
     int tok;
     double S_used = S;
-    if (!(S >= kTinyMass)) {
+    if (!(S * rn.izt >= kTinyMass)) {
         // a rejection implies residual mass; if rounding erased it, draw from P_t instead
         tok = warp_sample_pt_slow<E>(trow, V, rn, p.c, u, lane, &S_used);
     } else {
@@ -417,12 +501,24 @@ __device__ void select_token(const Params& p, int b, int n, int lane) {
         int seg = -1, lastseg = gl0;
         double before = excl_L, before_last = excl_L;
         {
-            double cum = excl_L;
-            for (int g = gl0; g < gl1; ++g) {  // every lane walks the same few sums
-                const double v = __ldcg(ss + g);
-                if (v > 0.0) { lastseg = g; before_last = cum; }
-                if (seg < 0 && v > 0.0 && target < cum + v) { seg = g; before = cum; }
-                cum += v;
+            double run = excl_L;
+            for (int gb = gl0; gb < gl1 && seg < 0; gb += 32) {  // lane L's block, 32 sums at a time
+                const int g = gb + lane;
+                const double v = g < gl1 ? (double)__ldcg(ss + g) : 0.0;
+                const double incl = warp_inclusive_scan(v, lane);
+                const unsigned h = __ballot_sync(0xffffffffu, v > 0.0 && target < run + incl);
+                const unsigned ps = __ballot_sync(0xffffffffu, v > 0.0);
+                if (ps) {
+                    const int ll = 31 - __clz(ps);
+                    lastseg = gb + ll;
+                    before_last = run + __shfl_sync(0xffffffffu, incl - v, ll);
+                }
+                if (h) {
+                    const int l1 = __ffs(h) - 1;
+                    seg = gb + l1;
+                    before = run + __shfl_sync(0xffffffffu, incl - v, l1);
+                }
+                run += __shfl_sync(0xffffffffu, incl, 31);
             }
         }
         if (seg < 0) { seg = lastseg; before = before_last; }
@@ -443,7 +539,7 @@ __device__ void select_token(const Params& p, int b, int n, int lane) {
                 if (e < V) {
                     const float xt = load_logit(trow + e);
                     const float xd = resid ? load_logit(drow + e) : 0.f;
-                    r[i] = resid ? entry_mass<true>(xt, xd, rn, p.c) : entry_mass<false>(xt, 0.f, rn, p.c);
+                    r[i] = (double)(resid ? entry_mass<true>(xt, xd, rn, p.c) : entry_mass<false>(xt, 0.f, rn, p.c));
                 }
                 if (r[i] > 0.0) mylast = e;
                 mine += r[i];
@@ -477,7 +573,7 @@ __device__ void select_token(const Params& p, int b, int n, int lane) {
     }
     if (lane == 0) {
         p.out_tok[(size_t)b * (K + 1) + n] = tok;
-        p.resid[b] = S_used;
+        p.resid[b] = S_used * rn.izt;
     }
 }
 
@@ -491,7 +587,9 @@ __global__ void __launch_bounds__(kThreads, 2) ears_verify_kernel(const Params p
     const int K = p.K, R = 2 * K + 1, V = p.V, P = p.plan.parts1, cpp = p.plan.cpp1, nseg = p.plan.nseg;
     const bool use_tma = p.plan.use_tma != 0;
     const int chunks_per_row = (V + CHUNK_ELEMS - 1) / CHUNK_ELEMS;
-    const long long total_units = (long long)p.B * R * P;
+    const long long units_per_stream = (long long)p.plan.seq_per_stream * R * P;
+    const long long total_units = units_per_stream * p.plan.streams;  // order space; holes are skipped
+    const long long real_units = (long long)p.B * R * P;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const E* tbase = reinterpret_cast<const E*>(p.t);
     const E* dbase = reinterpret_cast<const E*>(p.d);
@@ -500,10 +598,12 @@ __global__ void __launch_bounds__(kThreads, 2) ears_verify_kernel(const Params p
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(&sm.full[s], use_tma ? 1u : 32u);
             mbar_init(&sm.empty[s], kConsumerWarps);
-            mbar_init(&sm.red[s], kConsumerWarps);
         }
+        for (int s = 0; s < kUnitSlots; ++s) mbar_init(&sm.unit_bar[s], kConsumerWarps);
+        sm.units_read = 0;
         sm.epi.init();
         sm.jobs.init();
+        sm.seq.init();
         sm.abort_flag = 0;
         mbar_init_fence();
     }
@@ -513,76 +613,239 @@ __global__ void __launch_bounds__(kThreads, 2) ears_verify_kernel(const Params p
         // =============================== loader warp
         uint32_t q = 0;
         bool ok = true, stats_done = false, acked = false;
-        while (ok && !acked) {
-            // 1. rows for a final token come first: they are hot in L2 right now
-            Msg job{-1, 0, 0};
-            int have = 0;
-            if (lane == 0) {
-                if (stats_done) have = sm.jobs.pop(job, &sm.abort_flag, kIdleLimitNs) ? 1 : -1;
-                else have = sm.jobs.try_pop(job) ? 1 : 0;
+        // The queue index of the next unit is fetched one unit ahead (lane 0 holds it) so that the
+        // round trip of the atomic overlaps with streaming the current unit.
+        // One claim covers `claim` units spaced one grid apart.
+        const int claim = p.plan.claim;
+        const long long G = gridDim.x;
+        long long u_ahead = 0;        // lane 0: next claim ticket
+        long long tk = -1;            // current claim ticket
+        int ci = 0;                   // units of the current claim already taken
+        if (lane == 0) u_ahead = atomicAdd(&p.heads[0], 1);
+        // First pass over a row: ask L2 to keep it (one or two rows of the sequence are read again
+        // within microseconds); second pass: the line can go.
+        const uint64_t pol_keep = l2_policy_evict_last();
+        const uint64_t pol_last_use = l2_policy_evict_first();
+        const int P2 = p.plan.parts2;
+        unsigned long long wait_t0 = 0;
+        int cursor = 0;        // first published slot that may still have pieces
+        bool again = false;    // the last look at the published slots found pieces left
+        bool all_final = false;  // every sequence of the batch has been finalised
+        int jb = -1, jn = 0, jpart = 0;  // final-token piece claimed for the next round
+        bool piece_last = false;         // the previous round served a final-token piece
+        while (ok) {
+            // Published sequences form a global queue of (sequence, piece) served by every CTA in order:
+            // each lane looks at one of the next 32 published slots; the first slot with pieces
+            // left is tried with one atomic (an overshoot only means someone else was quicker).
+            // A unit this CTA already holds a ticket for must not wait behind a long run of pieces
+            // (its sequence could not finish): pieces and units alternate while both exist.
+            jb = -1;
+            if (!(piece_last && !stats_done)) {
+                const int slot = cursor + lane;
+                unsigned long long e = 0;
+                int taken = P2;
+                if (slot < p.B) {
+                    e = *reinterpret_cast<volatile unsigned long long*>(&p.ready[slot]);
+                    taken = *reinterpret_cast<volatile int*>(&p.job_ctr[slot]);
+                }
+                const unsigned open = __ballot_sync(0xffffffffu, e != 0 && taken < P2);
+                const unsigned done = __ballot_sync(0xffffffffu, e != 0 && taken >= P2);
+                cursor += done == 0xffffffffu ? 32 : __ffs(~done) - 1;    // skip leading exhausted slots
+                again = open != 0;
+                if (open) {
+                    const int L = __ffs(open) - 1;
+                    int piece = P2;
+                    if (lane == L) piece = atomicAdd(&p.job_ctr[slot], 1);
+                    piece = __shfl_sync(0xffffffffu, piece, L);
+                    if (piece < P2) {
+                        const unsigned long long el = __shfl_sync(0xffffffffu, e, L);
+                        jb = (int)(el >> 32) - 1; jn = (int)(unsigned)el; jpart = piece;
+                    }
+                }
             }
-            have = __shfl_sync(0xffffffffu, have, 0);
-            if (have < 0) { ok = false; break; }
-            if (have > 0) {
-                job.kind = __shfl_sync(0xffffffffu, job.kind, 0);
-                job.a = __shfl_sync(0xffffffffu, job.a, 0);
-                job.b = __shfl_sync(0xffffffffu, job.b, 0);
-                if (job.kind == kMsgAck) { acked = true; break; }
-                const int b = job.a, n = job.b;
+            piece_last = jb >= 0;
+            if (jb >= 0) {
+                // 1. rows for a final token come first: they are hot in L2 right now
+                __threadfence();
+                const int b = jb, n = jn;
                 const bool resid = n < K;
                 const int step = resid ? CHUNK_ELEMS / 2 : CHUNK_ELEMS;
                 const E* trow = tbase + (size_t)target_row(b, n, K) * V;
                 const E* drow = resid ? dbase + (size_t)draft_row(b, n, K) * V : nullptr;
-                for (int e0 = 0; e0 < V; e0 += step, ++q) {
+                const int e_begin = jpart * p.plan.job_elems;
+                const int e_end = min(V, e_begin + p.plan.job_elems);
+                for (int e0 = e_begin; e0 < e_end; e0 += step, ++q) {
                     ok = loader_acquire(sm, q, lane);
                     if (!ok) break;
-                    const int ne = min(step, V - e0);
-                    const StageMeta mt{resid ? kResid : kBonus, b, ne, (e0 == 0 ? 1 : 0) | (e0 + step >= V ? 2 : 0), e0, n};
-                    loader_fill<E>(sm, q % STAGES, mt, use_tma, trow + e0, resid ? drow + e0 : nullptr, lane);
+                    const int ne = min(step, e_end - e0);
+                    const StageMeta mt{resid ? kResid : kBonus, b, ne, (e0 == e_begin ? 1 : 0) | (e0 + step >= e_end ? 2 : 0), e0, n};
+                    loader_fill<E>(sm, q % STAGES, mt, use_tma, trow + e0, resid ? drow + e0 : nullptr, lane, pol_last_use);
                 }
-                continue;
-            }
-            // 2. next piece of a row for the statistics pass
-            long long u = 0;
-            if (lane == 0) u = atomicAdd(&p.heads[0], 1);
-            u = __shfl_sync(0xffffffffu, u, 0);
-            if (sm.abort_flag) { ok = false; break; }
-            if (u >= total_units) {
-                // nothing left to pull: tell the consumers, then serve final-token rows until acknowledged
-                ok = loader_acquire(sm, q, lane);
                 if (!ok) break;
-                loader_fill<E>(sm, q % STAGES, StageMeta{kDrain, 0, 0, 0, 0, 0}, use_tma, nullptr, nullptr, lane);
-                ++q;
-                stats_done = true;
-                continue;
-            }
-            const int b = (int)(u / (R * P));
-            const int rem = (int)(u % (R * P));
-            const int ridx = rem / P, part = rem % P;
-            const E* row = (ridx == 2 * K) ? tbase + (size_t)target_row(b, K, K) * V
-                                           : ((ridx & 1) ? dbase + (size_t)draft_row(b, ridx >> 1, K) * V
-                                                         : tbase + (size_t)target_row(b, ridx >> 1, K) * V);
-            const int ch0 = part * cpp;
-            const int ch1 = min(chunks_per_row, ch0 + cpp);
-            for (int ch = ch0; ch < ch1; ++ch, ++q) {
-                ok = loader_acquire(sm, q, lane);
-                if (!ok) break;
-                const int e0 = ch * CHUNK_ELEMS;
-                const StageMeta mt{kStats, (int)u, min(CHUNK_ELEMS, V - e0), (ch == ch0 ? 1 : 0) | (ch == ch1 - 1 ? 2 : 0), e0, 0};
-                loader_fill<E>(sm, q % STAGES, mt, use_tma, row + e0, nullptr, lane);
+            } else if (!stats_done) {
+                // 2. next piece of a row for the statistics pass
+                if (sm.abort_flag) { ok = false; break; }
+                if (tk < 0 || ci == claim) {
+                    tk = __shfl_sync(0xffffffffu, u_ahead, 0);
+                    ci = 0;
+                    if (lane == 0 && (tk / G) * claim * G < total_units) u_ahead = atomicAdd(&p.heads[0], 1);
+                }
+                const long long j = ((tk / G) * claim + ci) * G + tk % G;  // position in the sweep order
+                ++ci;
+                // interleaved runs: consecutive positions visit different parts of the batch
+                const long long u = (j % p.plan.streams) * units_per_stream + j / p.plan.streams;
+                if (j >= total_units) {
+                    if ((tk / G) * claim * G + tk % G >= total_units) {
+                        // nothing left to pull: tell the consumers; final-token rows are served until
+                        // this CTA's epilogue warp has acknowledged
+                        ok = loader_acquire(sm, q, lane);
+                        if (!ok) break;
+                        loader_fill<E>(sm, q % STAGES, StageMeta{kDrain, 0, 0, 0, 0, 0}, use_tma, (const E*)nullptr, (const E*)nullptr, lane, pol_keep);
+                        ++q;
+                        stats_done = true;
+                    }  // else: a hole in the last sweep
+                } else if (u < real_units) {  // else: a hole in the last run
+                    const int b = (int)(u / (R * P));
+                    const int rem = (int)(u % (R * P));
+                    const int ridx = rem / P, part = rem % P;
+                    const E* row = (ridx == 2 * K) ? tbase + (size_t)target_row(b, K, K) * V
+                                                   : ((ridx & 1) ? dbase + (size_t)draft_row(b, ridx >> 1, K) * V
+                                                                 : tbase + (size_t)target_row(b, ridx >> 1, K) * V);
+                    const int ch0 = part * cpp;
+                    const int ch1 = min(chunks_per_row, ch0 + cpp);
+                    for (int ch = ch0; ch < ch1; ++ch, ++q) {
+                        ok = loader_acquire(sm, q, lane);
+                        if (!ok) break;
+                        const int e0 = ch * CHUNK_ELEMS;
+                        const StageMeta mt{kStats, (int)u, min(CHUNK_ELEMS, V - e0), (ch == ch0 ? 1 : 0) | (ch == ch1 - 1 ? 2 : 0), e0, 0};
+                        // the extra target row is the likeliest to be read again (every draft accepted)
+                        loader_fill<E>(sm, q % STAGES, mt, use_tma, row + e0, nullptr, lane, ridx == 2 * K ? pol_keep : pol_last_use);
+                    }
+                    if (!ok) break;
+                }
+            } else {
+                // 3. No units left.  Stay and help with final-token pieces until every sequence of the
+                //    batch has been finalised (by whichever CTA) and no piece is left to claim:
+                //    leaving earlier would let the last sequences fall to very few CTAs.  The wait
+                //    cannot deadlock: a sequence is finalised by CTAs that already hold its units,
+                //    and those never wait for anyone.  It is bounded like every other wait.
+                if (acked && !again) {
+                    if (all_final) break;   // seen before the look above, so that look was complete
+                    int fin = 0;
+                    if (lane == 0) {
+                        fin = *reinterpret_cast<volatile int*>(&p.heads[1]) >= p.B ? 1 : 0;
+                        if (!fin) {
+                            if (sm.abort_flag) fin = -1;
+                            const unsigned long long now = global_timer_ns();
+                            if (wait_t0 == 0) wait_t0 = now;
+                            else if (now - wait_t0 > kIdleLimitNs) { sm.abort_flag = 1; fin = -1; }
+                            __nanosleep(200);
+                        }
+                    }
+                    fin = __shfl_sync(0xffffffffu, fin, 0);
+                    if (fin < 0) { ok = false; break; }
+                    if (fin > 0) { all_final = true; __threadfence(); }
+                }
+                if (!acked) {
+                    int st = 0;
+                    if (lane == 0) {
+                        Msg m{kMsgNone, 0, 0, 0};
+                        if (sm.jobs.try_pop(m)) st = 1;
+                        else if (sm.abort_flag) st = -1;
+                        else {
+                            const unsigned long long now = global_timer_ns();
+                            if (wait_t0 == 0) wait_t0 = now;
+                            else if (now - wait_t0 > kIdleLimitNs) { sm.abort_flag = 1; st = -1; }
+                            __nanosleep(100);
+                        }
+                    }
+                    st = __shfl_sync(0xffffffffu, st, 0);
+                    if (st < 0) { ok = false; break; }
+                    if (st > 0) acked = true;
+                }
             }
         }
         if (ok && loader_acquire(sm, q, lane)) {
-            loader_fill<E>(sm, q % STAGES, StageMeta{kEnd, 0, 0, 0, 0, 0}, use_tma, nullptr, nullptr, lane);
+            loader_fill<E>(sm, q % STAGES, StageMeta{kEnd, 0, 0, 0, 0, 0}, use_tma, (const E*)nullptr, (const E*)nullptr, lane, pol_keep);
         } else if (use_tma && lane == 0) {
             loader_drain(sm, q);
         }
     } else if (warp == kEpilogueWarp) {
         // =============================== epilogue warp
+        // Takes up to 32 messages at a time.  Pieces are published in parallel (one lane each:
+        // store, fence, ticket); what needs the whole warp then runs in message order.
+        bool running = true;
+        while (running) {
+            int first = 0, cnt = 0;
+            if (lane == 0) cnt = sm.epi.wait_batch(&first, &sm.abort_flag, kIdleLimitNs);
+            cnt = __shfl_sync(0xffffffffu, cnt, 0);
+            first = __shfl_sync(0xffffffffu, first, 0);
+            if (cnt < 0) break;
+            __threadfence_block();
+            Msg m{kMsgNone, 0, 0, 0};
+            if (lane < cnt) m = sm.epi.peek(first + lane);
+            __syncwarp();
+            if (lane == 0) sm.epi.release(first + cnt);
+            int last_b = -1;
+            // every piece message names a unit slot: wait until all eight consumer warps are through
+            bool slot_ok = true;
+            int top = -1;
+            if (m.kind == kMsgJobPiece || m.kind == kMsgPiece) {
+                slot_ok = mbar_wait(&sm.unit_bar[m.c % kUnitSlots], (m.c / kUnitSlots) & 1, &sm.abort_flag);
+                top = m.c;
+            }
+            float pm = -INFINITY, ps = 0.f;
+            if (m.kind == kMsgPiece && slot_ok) {
+                for (int w = 0; w < kConsumerWarps; ++w) {
+                    const float2 v = sm.scratch[m.c % kUnitSlots][w];
+                    merge_ms(pm, ps, v.x, v.y, p.c);
+                }
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) top = max(top, __shfl_xor_sync(0xffffffffu, top, off));
+            __syncwarp();
+            if (lane == 0 && top >= 0) { __threadfence_block(); sm.units_read = top + 1; }
+            if (m.kind == kMsgJobPiece && slot_ok) {
+                __threadfence();
+                if (atomicAdd(&p.ticket2[m.a], 1) == p.plan.parts2 - 1) last_b = m.a;  // all masses summed
+            }
+            if (m.kind == kMsgPiece && slot_ok) {
+                const int b = m.a / (R * P);
+                const int rem = m.a % (R * P);
+                p.partial[((size_t)b * R + rem / P) * P + rem % P] = make_float2(pm, ps);
+                // two-level count (row, then sequence) spreads the atomics over many addresses
+                __threadfence();
+                bool row_done = true;
+                if (P > 1) {
+                    row_done = atomicAdd(&p.ticket_row[(size_t)b * R + rem / P], 1) == P - 1;
+                    if (row_done) __threadfence();
+                }
+                if (row_done && atomicAdd(&p.ticket1[b], 1) == R - 1) last_b = b;  // last row of the sequence
+            }
+            // what needs a whole warp (decisions, final pick) goes to the sequence warp, in order
+            for (int i = 0; i < cnt && running; ++i) {
+                const int kind = __shfl_sync(0xffffffffu, m.kind, i);
+                const int a = __shfl_sync(0xffffffffu, m.a, i);
+                const int bb = __shfl_sync(0xffffffffu, m.b, i);
+                const int lb = __shfl_sync(0xffffffffu, last_b, i);
+                Msg fwd{kMsgNone, 0, 0, 0};
+                if (kind == kMsgPiece && lb >= 0) fwd = Msg{kMsgFinalize, lb, 0, 0};
+                else if (kind == kMsgJobPiece && lb >= 0) fwd = Msg{kMsgSelect, a, bb, 0};
+                else if (kind == kMsgDrain || kind == kMsgExit) fwd = Msg{kind, 0, 0, 0};
+                if (fwd.kind != kMsgNone) {
+                    int pushed = 1;
+                    if (lane == 0) pushed = sm.seq.push(fwd, &sm.abort_flag, kWaitLimitNs) ? 1 : 0;
+                    if (!__shfl_sync(0xffffffffu, pushed, 0)) running = false;
+                }
+                if (kind == kMsgExit) running = false;
+            }
+        }
+    } else if (warp == kSequenceWarp) {
+        // =============================== sequence warp: per-sequence decisions and the final pick
         for (;;) {
-            Msg m{kMsgExit, 0, 0};
+            Msg m{kMsgExit, 0, 0, 0};
             int got = 0;
-            if (lane == 0) got = sm.epi.pop(m, &sm.abort_flag, kIdleLimitNs) ? 1 : 0;
+            if (lane == 0) got = sm.seq.pop(m, &sm.abort_flag, kIdleLimitNs) ? 1 : 0;
             got = __shfl_sync(0xffffffffu, got, 0);
             if (!got) break;
             m.kind = __shfl_sync(0xffffffffu, m.kind, 0);
@@ -593,18 +856,26 @@ __global__ void __launch_bounds__(kThreads, 2) ears_verify_kernel(const Params p
                 __threadfence();
                 const int n = finalize_sequence<E>(p, m.a, lane);
                 if (n >= 0) {
-                    __threadfence();  // row statistics must be visible to the consumers of the job
+                    // publish the sequence for the final-token pass; its row statistics first
+                    __threadfence();
                     __syncwarp();
-                    int pushed = 1;
-                    if (lane == 0) pushed = sm.jobs.push(Msg{kMsgJob, m.a, n}, &sm.abort_flag, kWaitLimitNs) ? 1 : 0;
-                    if (!__shfl_sync(0xffffffffu, pushed, 0)) break;
+                    if (lane == 0) {
+                        const int slot = atomicAdd(&p.heads[3], 1);
+                        *reinterpret_cast<volatile unsigned long long*>(&p.ready[slot]) =
+                            ((unsigned long long)(m.a + 1) << 32) | (unsigned)n;
+                    }
+                }
+                if (lane == 0) {  // finalised (valid or not): lets idle CTAs know when to leave
+                    __threadfence();
+                    atomicAdd(&p.heads[1], 1);
                 }
             } else if (m.kind == kMsgSelect) {
                 __threadfence();
                 select_token<E>(p, m.a, m.b, lane);
             } else if (m.kind == kMsgDrain) {
+                // everything this CTA finalised is published by now
                 int pushed = 1;
-                if (lane == 0) pushed = sm.jobs.push(Msg{kMsgAck, 0, 0}, &sm.abort_flag, kWaitLimitNs) ? 1 : 0;
+                if (lane == 0) pushed = sm.jobs.push(Msg{kMsgAck, 0, 0, 0}, &sm.abort_flag, kWaitLimitNs) ? 1 : 0;
                 if (!__shfl_sync(0xffffffffu, pushed, 0)) break;
             }
         }
@@ -613,18 +884,18 @@ __global__ void __launch_bounds__(kThreads, 2) ears_verify_kernel(const Params p
         const int tid = threadIdx.x;
         float m_run = -INFINITY;
         float s[4] = {0.f, 0.f, 0.f, 0.f};
-        uint32_t red_phase = 0;
-        RowNorm rn{0.f, 0.f, 0.0, 0.0};
+        int unit_ends = 0;   // ends of units and pieces seen so far (same in every consumer warp)
+        RowNorm rn{0.f, 0.f, 0.f, 0.f, 0.0};
         for (uint32_t q = 0;; ++q) {
             const int stage = q % STAGES;
             if (!mbar_wait(&sm.full[stage], (q / STAGES) & 1u, &sm.abort_flag)) break;
             const StageMeta mt = sm.meta[stage];
             if (mt.kind == kEnd) {
-                if (warp == 0 && lane == 0) sm.epi.push(Msg{kMsgExit, 0, 0}, &sm.abort_flag, kWaitLimitNs);
+                if (warp == 0 && lane == 0) sm.epi.push(Msg{kMsgExit, 0, 0, 0}, &sm.abort_flag, kWaitLimitNs);
                 break;
             }
             if (mt.kind == kDrain) {
-                if (warp == 0 && lane == 0) sm.epi.push(Msg{kMsgDrain, 0, 0}, &sm.abort_flag, kWaitLimitNs);
+                if (warp == 0 && lane == 0) sm.epi.push(Msg{kMsgDrain, 0, 0, 0}, &sm.abort_flag, kWaitLimitNs);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sm.empty[stage]);
                 continue;
@@ -646,57 +917,36 @@ __global__ void __launch_bounds__(kThreads, 2) ears_verify_kernel(const Params p
                     merge_ms(m, sum, m2, s2, p.c);
                 }
                 if (lane == 0) {
-                    sm.scratch[stage][warp] = make_float2(m, sum);
-                    mbar_arrive(&sm.red[stage]);
+                    const int us = unit_ends % kUnitSlots;
+                    sm.scratch[us][warp] = make_float2(m, sum);
+                    mbar_arrive(&sm.unit_bar[us]);
+                    if (warp == 0) push_unit_end(sm, Msg{kMsgPiece, mt.id, 0, unit_ends});
+                    mbar_arrive(&sm.empty[stage]);
                 }
-                if (warp == 0) {
-                    const uint32_t ph = (red_phase >> stage) & 1u;
-                    red_phase ^= 1u << stage;
-                    const bool ok = mbar_wait(&sm.red[stage], ph, &sm.abort_flag);
-                    float2 v = lane < kConsumerWarps ? sm.scratch[stage][lane] : make_float2(-INFINITY, 0.f);
-                    m = v.x; sum = v.y;
-#pragma unroll
-                    for (int off = kConsumerWarps / 2; off > 0; off >>= 1) {
-                        float m2 = __shfl_xor_sync(0xffffffffu, m, off);
-                        float s2 = __shfl_xor_sync(0xffffffffu, sum, off);
-                        merge_ms(m, sum, m2, s2, p.c);
-                    }
-                    if (lane == 0 && ok) {
-                        const int b = mt.id / (R * P);
-                        const int rem = mt.id % (R * P);
-                        p.partial[((size_t)b * R + rem / P) * P + rem % P] = make_float2(m, sum);
-                        __threadfence();
-                        if (atomicAdd(&p.ticket1[b], 1) == R * P - 1)  // last piece of the sequence
-                            sm.epi.push(Msg{kMsgFinalize, b, 0}, &sm.abort_flag, kWaitLimitNs);
-                    }
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sm.empty[stage]);
+                ++unit_ends;
                 continue;
             }
-            // rows of a final token: fp64 segment sums of the masses
+            // rows of a final token: segment sums of the masses
             const int b = mt.id, n = mt.aux;
             const bool resid = mt.kind == kResid;
             if (mt.flags & 1) {
                 const float2 st = __ldcg(&p.rowstat[(size_t)b * R + (resid ? 2 * n : 2 * K)]);
                 const float2 sd = resid ? __ldcg(&p.rowstat[(size_t)b * R + 2 * n + 1]) : make_float2(0.f, 1.f);
-                rn = RowNorm{st.x, sd.x, 1.0 / (double)st.y, 1.0 / (double)sd.y};
+                rn = make_rownorm(st, sd);
             }
-            double* seg_out = p.segsum + (size_t)b * nseg + mt.elem0 / kSegElems;
+            float* seg_out = p.segsum + (size_t)b * nseg + mt.elem0 / kSegElems;
             if (resid) chunk_segments<E, true>(sm.buf[stage], sm.buf[stage] + kChunkBytes / 2, mt.nelem, warp, lane, rn, p.c, seg_out);
             else chunk_segments<E, false>(sm.buf[stage], sm.buf[stage], mt.nelem, warp, lane, rn, p.c, seg_out);
             if (mt.flags & 2) {
-                // last chunk of the row(s): publish the sums, then hand the pick to the epilogue warp
+                // last chunk of the piece: publish the sums; the epilogue warp counts the piece once
+                // all warps are through and, when it is the sequence's last, picks the token
+                __syncwarp();
                 if (lane == 0) {
                     __threadfence();
-                    mbar_arrive(&sm.red[stage]);
+                    mbar_arrive(&sm.unit_bar[unit_ends % kUnitSlots]);
+                    if (warp == 0) push_unit_end(sm, Msg{kMsgJobPiece, b, n, unit_ends});
                 }
-                if (warp == 0) {
-                    const uint32_t ph = (red_phase >> stage) & 1u;
-                    red_phase ^= 1u << stage;
-                    const bool ok = mbar_wait(&sm.red[stage], ph, &sm.abort_flag);
-                    if (lane == 0 && ok) sm.epi.push(Msg{kMsgSelect, b, n}, &sm.abort_flag, kWaitLimitNs);
-                }
+                ++unit_ends;
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.empty[stage]);
