@@ -18,8 +18,6 @@ namespace {
 
 using namespace ears;
 
-constexpr int kStages = 6;  // 6 x 16 KB per CTA, two CTAs per SM
-constexpr int kCtasPerSm = 2;
 // 256 KB of one row per unit when there is plenty of work (smaller units cost more per-unit
 // bookkeeping than they gain in balance; measured on B=512, V=256000).
 constexpr int kUnitChunks = 16;
@@ -99,7 +97,7 @@ Plan make_plan(int B, int K, int V, int esize, bool aligned, int sms, const Plan
 
 struct Layout {
     size_t ticket1, ticket2, job_ctr, ticket_row, ready, heads, counters_bytes;
-    size_t partial, rowstat, pt_tok, pd_tok, max_pt, cls, resid, segsum, total;
+    size_t partial, rowstat, pt_tok, pd_tok, max_pt, cls, resid, segsum, bonus_seg, total;
 };
 
 Layout make_layout(int B, int K, int V, int parts1) {
@@ -123,6 +121,8 @@ Layout make_layout(int B, int K, int V, int parts1) {
     L.cls = o; o = align_up(o + (size_t)B * K, 256);
     L.resid = o; o = align_up(o + (size_t)B * 8, 256);
     L.segsum = o; o = align_up(o + (size_t)B * ((V + kSegElems - 1) / kSegElems) * 4, 256);
+    // the extra row's per-warp chunk sums; 2-byte elements give the fewest chunks, 4-byte the most
+    L.bonus_seg = o; o = align_up(o + (size_t)B * ((V + kChunkBytes / 4 - 1) / (kChunkBytes / 4)) * kConsumerWarps * sizeof(float2), 256);
     L.total = o;
     return L;
 }
@@ -268,6 +268,7 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
     p.partial = (float2*)(w + L.partial);
     p.rowstat = (float2*)(w + L.rowstat);
     p.segsum = (float*)(w + L.segsum);
+    p.bonus_seg = (float2*)(w + L.bonus_seg);
     p.plan = plan;
     return dtype == EARS_DTYPE_F32 ? launch<float>(p, di->sms, stream) : launch<uint16_t>(p, di->sms, stream);
 }

@@ -6,7 +6,18 @@
 
 namespace ears {
 
-constexpr int kConsumerWarps = 8;                    // warps that reduce the staged chunks
+#ifndef EARS_CONSUMER_WARPS
+#define EARS_CONSUMER_WARPS 8
+#endif
+#ifndef EARS_CTAS_PER_SM
+#define EARS_CTAS_PER_SM 2
+#endif
+#ifndef EARS_STAGES
+#define EARS_STAGES 6
+#endif
+constexpr int kConsumerWarps = EARS_CONSUMER_WARPS;  // warps that reduce the staged chunks
+constexpr int kCtasPerSm = EARS_CTAS_PER_SM;
+constexpr int kStages = EARS_STAGES;                 // 16 KB slots in a CTA's ring
 constexpr int kConsumers = kConsumerWarps * 32;
 constexpr int kLoaderWarp = kConsumerWarps;          // streams logits into shared memory
 constexpr int kEpilogueWarp = kConsumerWarps + 1;    // counts finished pieces of rows
@@ -61,7 +72,8 @@ struct Params {
     int* heads;           // [0] unit queue, [1] finalised sequences, [2] status, [3] published sequences
     float2* partial;      // [B*(2K+1)*parts1] (m, s) per row piece
     float2* rowstat;      // [B*(2K+1)] (m, Z) per row
-    float* segsum;        // [B*nseg] segment sums of the final-token masses
+    float* segsum;        // [B*nseg] segment sums of the final-token masses (second pass)
+    float2* bonus_seg;    // [B*chunks*8] (sum, reference max) per chunk and consumer warp of the extra row
     Plan plan;
 };
 

@@ -90,7 +90,7 @@ struct Mailbox {
                 if (t0 == 0) t0 = now;
                 else if (now - t0 > limit_ns) { *abort_flag = 1; return -1; }
             }
-            __nanosleep(64);
+            __nanosleep(spin < 4 ? 100 : 400);  // idle warps must not eat the consumers' issue slots
         }
     }
     __device__ __forceinline__ Msg peek(int index) const {
@@ -108,7 +108,7 @@ struct Mailbox {
                 if (t0 == 0) t0 = now;
                 else if (now - t0 > limit_ns) { *abort_flag = 1; return false; }
             }
-            __nanosleep(64);
+            __nanosleep(spin < 4 ? 200 : 1000);
         }
     }
 };
@@ -197,8 +197,13 @@ __device__ __forceinline__ void loader_fill(PipeSmem<STAGES>& sm, int stage, con
                 mbar_arrive(&sm.full[stage]);
             } else {
                 mbar_arrive_expect_tx(&sm.full[stage], src1 ? 2 * bytes : bytes);
-                bulk_load_hint(sm.buf[stage], src0, bytes, &sm.full[stage], policy);
-                if (src1) bulk_load_hint(sm.buf[stage] + kChunkBytes / 2, src1, bytes, &sm.full[stage], policy);
+                if (policy) {
+                    bulk_load_hint(sm.buf[stage], src0, bytes, &sm.full[stage], policy);
+                    if (src1) bulk_load_hint(sm.buf[stage] + kChunkBytes / 2, src1, bytes, &sm.full[stage], policy);
+                } else {
+                    bulk_load(sm.buf[stage], src0, bytes, &sm.full[stage]);
+                    if (src1) bulk_load(sm.buf[stage] + kChunkBytes / 2, src1, bytes, &sm.full[stage]);
+                }
             }
         }
     } else {
@@ -234,37 +239,59 @@ __device__ __forceinline__ float load_logit(const uint16_t* p) { return bf16_bit
 
 // Running (m, s) of one thread over its share of a staged chunk:
 // s = sum exp2((l - m) * c), m = running maximum; s is rescaled when m grows.
-template <typename E>
-__device__ __forceinline__ void chunk_stats(const unsigned char* buf, int nelem, int tid, float c,
-                                            float& m_run, float (&s)[4]) {
+// Warp w owns the w-th eighth of the slot (contiguous), lane-interleaved in 16-byte vectors.
+//
+// BONUS (the extra target row K): the maximum is kept warp-uniform and the warp also emits
+// (sum, reference maximum) of its eighth of the chunk.  If every draft token turns out to be
+// accepted, the final token is drawn from exactly these sums and the row is not read again.
+template <typename E, bool BONUS>
+__device__ __forceinline__ void chunk_stats(const unsigned char* buf, int nelem, int warp, int lane, float c,
+                                            float& m_run, float (&s)[4], float2* warp_chunk_out) {
     constexpr int N = Vec<E>::N;
     constexpr int VECS = kChunkBytes / 16 / kConsumers;  // 16-byte vectors per thread per chunk
     constexpr int CHUNK_ELEMS = kChunkBytes / (int)sizeof(E);
     float x[VECS][N];
 #pragma unroll
-    for (int j = 0; j < VECS; ++j) Vec<E>::load(buf, j * kConsumers + tid, x[j]);
+    for (int j = 0; j < VECS; ++j) Vec<E>::load(buf, (warp * VECS + j) * 32 + lane, x[j]);
     if (nelem < CHUNK_ELEMS) {  // ragged last chunk of a row: mask what lies beyond it
 #pragma unroll
         for (int j = 0; j < VECS; ++j)
 #pragma unroll
             for (int i = 0; i < N; ++i)
-                if ((j * kConsumers + tid) * N + i >= nelem) x[j][i] = -INFINITY;
+                if (((warp * VECS + j) * 32 + lane) * N + i >= nelem) x[j][i] = -INFINITY;
     }
     float cm = -INFINITY;
 #pragma unroll
     for (int j = 0; j < VECS; ++j)
 #pragma unroll
         for (int i = 0; i < N; ++i) cm = fmaxf(cm, x[j][i]);
+    if (BONUS) {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, off));
+    }
     if (cm > m_run) {
         float sc = ex2_approx((m_run - cm) * c);  // m_run = -inf gives 0
         s[0] *= sc; s[1] *= sc; s[2] *= sc; s[3] *= sc;
         m_run = cm;
     }
     const float mu = (m_run == -INFINITY) ? 0.0f : m_run;
+    if (!BONUS) {
 #pragma unroll
-    for (int j = 0; j < VECS; ++j)
+        for (int j = 0; j < VECS; ++j)
 #pragma unroll
-        for (int i = 0; i < N; ++i) s[(j * N + i) & 3] += ex2_approx(__fmul_rn(__fsub_rn(x[j][i], mu), c));
+            for (int i = 0; i < N; ++i) s[(j * N + i) & 3] += ex2_approx(__fmul_rn(__fsub_rn(x[j][i], mu), c));
+    } else {
+        float cs[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int j = 0; j < VECS; ++j)
+#pragma unroll
+            for (int i = 0; i < N; ++i) cs[(j * N + i) & 3] += ex2_approx(__fmul_rn(__fsub_rn(x[j][i], mu), c));
+        s[0] += cs[0]; s[1] += cs[1]; s[2] += cs[2]; s[3] += cs[3];
+        float tot = (cs[0] + cs[1]) + (cs[2] + cs[3]);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, off);
+        if (lane == 0) *warp_chunk_out = make_float2(tot, m_run);   // m_run is warp-uniform here
+    }
 }
 
 struct RowNorm {
@@ -312,10 +339,10 @@ __device__ __forceinline__ void chunk_segments(const unsigned char* bt, const un
     constexpr int VECS = kSegElems / (32 * N);  // 16-byte vectors per lane per segment
     constexpr int FULL_ELEMS = (RESID ? kChunkBytes / 2 : kChunkBytes) / (int)sizeof(E);
     constexpr int SEGS = FULL_ELEMS / kSegElems / kConsumerWarps;  // segments per warp in a full slot
-    if (nelem == FULL_ELEMS) {
+    if (SEGS >= 1 && nelem == FULL_ELEMS) {
         // full slot: all of the warp's segments at once, so that their loads, exponentials and
         // shuffle trees overlap instead of running one after the other
-        float acc[SEGS];
+        float acc[SEGS > 0 ? SEGS : 1];
 #pragma unroll
         for (int g = 0; g < SEGS; ++g) {
             acc[g] = 0.0f;
@@ -458,11 +485,116 @@ __device__ int warp_sample_pt_slow(const E* row, int V, const RowNorm& rn, float
     return __shfl_sync(0xffffffffu, tok, L);
 }
 
-// Inverse-CDF pick for sequence b (accepted length n) from its segment sums:
-// token = smallest j with u*S < C_j.  Level 1 finds the segment, level 2 re-reads its
-// kSegElems entries and finishes inside the warp.
+// Last level of the inverse-CDF pick: entries [base, base + count) of the row(s) are read again,
+// their masses recomputed (same bits as in the streaming pass) and scanned in fp64 for the
+// smallest j with tin < running sum.  If rounding hides the crossing, the last entry with
+// positive mass is taken.  One warp; returns the token (or -1 if the range has no mass).
+template <typename E>
+__device__ int pick_in_range(const E* trow, const E* drow, bool resid, const RowNorm& rn, float c,
+                             int base, int count, double tin, int V, int lane) {
+    constexpr int N = Vec<E>::N;
+    double run = 0.0;
+    int found = -1, lastpos = -1;
+    for (int j0 = 0; j0 < count && found < 0; j0 += 32 * N) {
+        const int e0 = base + j0 + lane * N;
+        double r[N], mine = 0.0;
+        int mylast = -1;
+#pragma unroll
+        for (int i = 0; i < N; ++i) {
+            const int e = e0 + i;
+            r[i] = 0.0;
+            if (e < V && e < base + count) {
+                const float xt = load_logit(trow + e);
+                const float xd = resid ? load_logit(drow + e) : 0.f;
+                r[i] = (double)(resid ? entry_mass<true>(xt, xd, rn, c) : entry_mass<false>(xt, 0.f, rn, c));
+            }
+            if (r[i] > 0.0) mylast = e;
+            mine += r[i];
+        }
+        const double incl = warp_inclusive_scan(mine, lane);
+        const unsigned h = __ballot_sync(0xffffffffu, tin < run + incl && mine > 0.0);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) mylast = max(mylast, __shfl_xor_sync(0xffffffffu, mylast, off));
+        if (h) {
+            const int Lh = __ffs(h) - 1;
+            int t_here = -1;
+            if (lane == Lh) {
+                double cum = run + (incl - mine);
+                int lp = -1;
+#pragma unroll
+                for (int i = 0; i < N; ++i) {
+                    cum += r[i];
+                    if (r[i] > 0.0) lp = e0 + i;
+                    if (t_here < 0 && r[i] > 0.0 && tin < cum) t_here = e0 + i;
+                }
+                if (t_here < 0) t_here = lp;
+            }
+            found = __shfl_sync(0xffffffffu, t_here, Lh);
+        } else {
+            lastpos = max(lastpos, mylast);
+            run += __shfl_sync(0xffffffffu, incl, 31);
+        }
+    }
+    return found >= 0 ? found : lastpos;
+}
+
+// First level: `count` non-negative sums, value(i) for i in [0, count), evaluated by the
+// caller-supplied functor (fp64).  Finds the first index whose running sum exceeds u * S and
+// returns it with the running sum before it; S is the total.  One warp, lanes own contiguous
+// blocks; loads are batched so that a block costs a few memory round trips, not one per entry.
+template <typename F>
+__device__ int pick_block(F value, int count, double u, int lane, double* S_out, double* before_out) {
+    const int per = (count + 31) / 32;
+    const int g0 = min(count, lane * per), g1 = min(count, g0 + per);
+    double loc = 0.0;
+    for (int g = g0; g < g1; g += 8) {
+        double v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = g + i < g1 ? value(g + i) : 0.0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) loc += v[i];
+    }
+    const double inc = warp_inclusive_scan(loc, lane);
+    const double S = __shfl_sync(0xffffffffu, inc, 31);
+    *S_out = S;
+    if (!(S > 0.0)) { *before_out = 0.0; return -1; }
+    const double target = u * S;
+    const unsigned hit = __ballot_sync(0xffffffffu, target < inc && loc > 0.0);
+    const unsigned pos = __ballot_sync(0xffffffffu, loc > 0.0);
+    const int L = hit ? __ffs(hit) - 1 : 31 - __clz(pos);
+    const double excl_L = __shfl_sync(0xffffffffu, inc - loc, L);
+    const int gl0 = __shfl_sync(0xffffffffu, g0, L), gl1 = __shfl_sync(0xffffffffu, g1, L);
+    int seg = -1, lastseg = gl0;
+    double before = excl_L, before_last = excl_L, run = excl_L;
+    for (int gb = gl0; gb < gl1 && seg < 0; gb += 32) {  // lane L's block, 32 sums at a time
+        const int g = gb + lane;
+        const double v = g < gl1 ? value(g) : 0.0;
+        const double incl = warp_inclusive_scan(v, lane);
+        const unsigned h = __ballot_sync(0xffffffffu, v > 0.0 && target < run + incl);
+        const unsigned ps = __ballot_sync(0xffffffffu, v > 0.0);
+        if (ps) {
+            const int ll = 31 - __clz(ps);
+            lastseg = gb + ll;
+            before_last = run + __shfl_sync(0xffffffffu, incl - v, ll);
+        }
+        if (h) {
+            const int l1 = __ffs(h) - 1;
+            seg = gb + l1;
+            before = run + __shfl_sync(0xffffffffu, incl - v, l1);
+        }
+        run += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (seg < 0) { seg = lastseg; before = before_last; }
+    *before_out = before;
+    return seg;
+}
+
+// Final token of sequence b (accepted length n): token = smallest j with u*S < C_j over the
+// masses of the row(s).  The sums come from the second pass (n < K: residual) or, when every
+// draft was accepted, from what the statistics pass left behind for the extra target row.
 template <typename E>
 __device__ void select_token(const Params& p, int b, int n, int lane) {
+    constexpr int CHUNK_ELEMS = kChunkBytes / (int)sizeof(E);
     const int K = p.K, V = p.V, R = 2 * K + 1, nseg = p.plan.nseg;
     const bool resid = n < K;
     const E* trow = reinterpret_cast<const E*>(p.t) + (size_t)target_row(b, n, K) * V;
@@ -470,106 +602,31 @@ __device__ void select_token(const Params& p, int b, int n, int lane) {
     const float2 st = __ldcg(&p.rowstat[(size_t)b * R + (resid ? 2 * n : 2 * K)]);
     const float2 sd = resid ? __ldcg(&p.rowstat[(size_t)b * R + 2 * n + 1]) : make_float2(0.f, 1.f);
     const RowNorm rn = make_rownorm(st, sd);
-    const float* ss = p.segsum + (size_t)b * nseg;
     const double u = uniform_final(p.seed, p.offset, (uint32_t)(p.b_first + b), (uint32_t)K);
-
-    // level 1: which segment
-    const int per = (nseg + 31) / 32;
-    const int g0 = min(nseg, lane * per), g1 = min(nseg, g0 + per);
-    double loc = 0.0;
-    for (int g = g0; g < g1; g += 8) {  // loads first, then the adds: eight reads in flight
-        float v[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) v[i] = g + i < g1 ? __ldcg(ss + g + i) : 0.f;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) loc += (double)v[i];
+    double S = 0.0, before = 0.0;
+    int seg, seg_elems;
+    if (resid) {
+        const float* ss = p.segsum + (size_t)b * nseg;
+        seg = pick_block([ss](int g) { return (double)__ldcg(ss + g); }, nseg, u, lane, &S, &before);
+        seg_elems = kSegElems;
+    } else {
+        // one entry per (chunk, consumer warp) of the extra row: (sum, reference maximum)
+        const int chunks = (V + CHUNK_ELEMS - 1) / CHUNK_ELEMS;
+        const float2* bs = p.bonus_seg + (size_t)b * chunks * kConsumerWarps;
+        const float m = rn.mt, c = p.c;
+        seg = pick_block([bs, m, c](int g) {
+                  const float2 e = __ldcg(bs + g);
+                  return (double)(e.x * ex2_approx((e.y - m) * c));   // bring the sum to the row's maximum
+              }, chunks * kConsumerWarps, u, lane, &S, &before);
+        seg_elems = CHUNK_ELEMS / kConsumerWarps;
     }
-    const double inc = warp_inclusive_scan(loc, lane);
-    const double S = __shfl_sync(0xffffffffu, inc, 31);
     int tok;
     double S_used = S;
-    if (!(S * rn.izt >= kTinyMass)) {
+    if (seg < 0 || !(S * rn.izt >= kTinyMass)) {
         // a rejection implies residual mass; if rounding erased it, draw from P_t instead
         tok = warp_sample_pt_slow<E>(trow, V, rn, p.c, u, lane, &S_used);
     } else {
-        const double target = u * S;
-        const unsigned hit = __ballot_sync(0xffffffffu, target < inc && loc > 0.0);
-        const unsigned pos = __ballot_sync(0xffffffffu, loc > 0.0);
-        const int L = hit ? __ffs(hit) - 1 : 31 - __clz(pos);
-        const double excl_L = __shfl_sync(0xffffffffu, inc - loc, L);
-        const int gl0 = __shfl_sync(0xffffffffu, g0, L), gl1 = __shfl_sync(0xffffffffu, g1, L);
-        int seg = -1, lastseg = gl0;
-        double before = excl_L, before_last = excl_L;
-        {
-            double run = excl_L;
-            for (int gb = gl0; gb < gl1 && seg < 0; gb += 32) {  // lane L's block, 32 sums at a time
-                const int g = gb + lane;
-                const double v = g < gl1 ? (double)__ldcg(ss + g) : 0.0;
-                const double incl = warp_inclusive_scan(v, lane);
-                const unsigned h = __ballot_sync(0xffffffffu, v > 0.0 && target < run + incl);
-                const unsigned ps = __ballot_sync(0xffffffffu, v > 0.0);
-                if (ps) {
-                    const int ll = 31 - __clz(ps);
-                    lastseg = gb + ll;
-                    before_last = run + __shfl_sync(0xffffffffu, incl - v, ll);
-                }
-                if (h) {
-                    const int l1 = __ffs(h) - 1;
-                    seg = gb + l1;
-                    before = run + __shfl_sync(0xffffffffu, incl - v, l1);
-                }
-                run += __shfl_sync(0xffffffffu, incl, 31);
-            }
-        }
-        if (seg < 0) { seg = lastseg; before = before_last; }
-        // level 2: which element of the segment
-        const double tin = target - before;
-        constexpr int N = Vec<E>::N;
-        const int base = seg * kSegElems;
-        double run = 0.0;
-        int found = -1, lastpos = -1;
-        for (int j = 0; j < kSegElems / (32 * N) && found < 0; ++j) {
-            const int e0 = base + (j * 32 + lane) * N;
-            double r[N], mine = 0.0;
-            int mylast = -1;
-#pragma unroll
-            for (int i = 0; i < N; ++i) {
-                const int e = e0 + i;
-                r[i] = 0.0;
-                if (e < V) {
-                    const float xt = load_logit(trow + e);
-                    const float xd = resid ? load_logit(drow + e) : 0.f;
-                    r[i] = (double)(resid ? entry_mass<true>(xt, xd, rn, p.c) : entry_mass<false>(xt, 0.f, rn, p.c));
-                }
-                if (r[i] > 0.0) mylast = e;
-                mine += r[i];
-            }
-            const double incl = warp_inclusive_scan(mine, lane);
-            const unsigned h = __ballot_sync(0xffffffffu, tin < run + incl && mine > 0.0);
-            // remember the last positive entry seen so far (fallback if rounding hides the hit)
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) mylast = max(mylast, __shfl_xor_sync(0xffffffffu, mylast, off));
-            if (h) {
-                const int Lh = __ffs(h) - 1;
-                int t_here = -1;
-                if (lane == Lh) {
-                    double cum = run + (incl - mine);
-                    int lp = -1;
-#pragma unroll
-                    for (int i = 0; i < N; ++i) {
-                        cum += r[i];
-                        if (r[i] > 0.0) lp = e0 + i;
-                        if (t_here < 0 && r[i] > 0.0 && tin < cum) t_here = e0 + i;
-                    }
-                    if (t_here < 0) t_here = lp;
-                }
-                found = __shfl_sync(0xffffffffu, t_here, Lh);
-            } else {
-                lastpos = max(lastpos, mylast);
-                run += __shfl_sync(0xffffffffu, incl, 31);
-            }
-        }
-        tok = found >= 0 ? found : lastpos;
+        tok = pick_in_range<E>(trow, drow, resid, rn, p.c, seg * seg_elems, seg_elems, u * S - before, V, lane);
     }
     if (lane == 0) {
         p.out_tok[(size_t)b * (K + 1) + n] = tok;
@@ -579,7 +636,7 @@ __device__ void select_token(const Params& p, int b, int n, int lane) {
 
 // ---- the kernel -------------------------------------------------------------------
 template <typename E, int STAGES>
-__global__ void __launch_bounds__(kThreads, 2) ears_verify_kernel(const Params p) {
+__global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const Params p) {
     extern __shared__ unsigned char smem_raw[];
     using Smem = PipeSmem<STAGES>;
     Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
@@ -622,9 +679,9 @@ __global__ void __launch_bounds__(kThreads, 2) ears_verify_kernel(const Params p
         long long tk = -1;            // current claim ticket
         int ci = 0;                   // units of the current claim already taken
         if (lane == 0) u_ahead = atomicAdd(&p.heads[0], 1);
-        // First pass over a row: ask L2 to keep it (one or two rows of the sequence are read again
-        // within microseconds); second pass: the line can go.
-        const uint64_t pol_keep = l2_policy_evict_last();
+        // L2 hints: lines that will not be read again may go first; rows that may be read again
+        // by the second pass get the default policy (0 = no hint).
+        const uint64_t pol_keep = 0;
         const uint64_t pol_last_use = l2_policy_evict_first();
         const int P2 = p.plan.parts2;
         unsigned long long wait_t0 = 0;
@@ -717,9 +774,10 @@ __global__ void __launch_bounds__(kThreads, 2) ears_verify_kernel(const Params p
                         ok = loader_acquire(sm, q, lane);
                         if (!ok) break;
                         const int e0 = ch * CHUNK_ELEMS;
-                        const StageMeta mt{kStats, (int)u, min(CHUNK_ELEMS, V - e0), (ch == ch0 ? 1 : 0) | (ch == ch1 - 1 ? 2 : 0), e0, 0};
-                        // the extra target row is the likeliest to be read again (every draft accepted)
-                        loader_fill<E>(sm, q % STAGES, mt, use_tma, row + e0, nullptr, lane, ridx == 2 * K ? pol_keep : pol_last_use);
+                        const StageMeta mt{kStats, (int)u, min(CHUNK_ELEMS, V - e0), (ch == ch0 ? 1 : 0) | (ch == ch1 - 1 ? 2 : 0), e0, ridx == 2 * K ? 1 : 0};
+                        // the extra target row is never streamed again (its sums are kept); the other
+                        // rows may be, if their position turns out to be the first rejection
+                        loader_fill<E>(sm, q % STAGES, mt, use_tma, row + e0, nullptr, lane, ridx == 2 * K ? pol_last_use : pol_keep);
                     }
                     if (!ok) break;
                 }
@@ -855,7 +913,12 @@ __global__ void __launch_bounds__(kThreads, 2) ears_verify_kernel(const Params p
             if (m.kind == kMsgFinalize) {
                 __threadfence();
                 const int n = finalize_sequence<E>(p, m.a, lane);
-                if (n >= 0) {
+                if (n == K) {
+                    // every draft accepted: the sums of the extra row are already there
+                    __threadfence();
+                    __syncwarp();
+                    select_token<E>(p, m.a, n, lane);
+                } else if (n >= 0) {
                     // publish the sequence for the final-token pass; its row statistics first
                     __threadfence();
                     __syncwarp();
@@ -881,7 +944,6 @@ __global__ void __launch_bounds__(kThreads, 2) ears_verify_kernel(const Params p
         }
     } else {
         // =============================== consumer warps
-        const int tid = threadIdx.x;
         float m_run = -INFINITY;
         float s[4] = {0.f, 0.f, 0.f, 0.f};
         int unit_ends = 0;   // ends of units and pieces seen so far (same in every consumer warp)
@@ -902,7 +964,12 @@ __global__ void __launch_bounds__(kThreads, 2) ears_verify_kernel(const Params p
             }
             if (mt.kind == kStats) {
                 if (mt.flags & 1) { m_run = -INFINITY; s[0] = s[1] = s[2] = s[3] = 0.f; }
-                chunk_stats<E>(sm.buf[stage], mt.nelem, tid, p.c, m_run, s);
+                if (mt.aux) {  // a piece of the extra target row
+                    float2* out = p.bonus_seg + ((size_t)(mt.id / (R * P)) * chunks_per_row + mt.elem0 / CHUNK_ELEMS) * kConsumerWarps + warp;
+                    chunk_stats<E, true>(sm.buf[stage], mt.nelem, warp, lane, p.c, m_run, s, out);
+                } else {
+                    chunk_stats<E, false>(sm.buf[stage], mt.nelem, warp, lane, p.c, m_run, s, nullptr);
+                }
                 if (!(mt.flags & 2)) {
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&sm.empty[stage]);
