@@ -95,10 +95,14 @@ def physical_gpu_index(local_index: int) -> int:
     return local_index
 
 
-def resample_bytes(accept_len, K: int, V: int, esize: int) -> int:
-    """Bytes of the rows the final-token pass reads: two rows after a rejection, one for a bonus."""
+def final_token_bytes(accept_len, K: int, V: int, esize: int):
+    """-> (formula, read_again).  formula: the workload's byte count for the final token (two rows
+    after a rejection, one row for a bonus token).  read_again: what the kernel really streams a
+    second time (only the two rows of a rejected position; the bonus row's sums are kept from the
+    first pass), mostly out of L2."""
     n = accept_len[accept_len >= 0]
-    return int(((n < K).sum().item() * 2 + (n >= K).sum().item()) * V * esize)
+    rej, acc = (n < K).sum().item(), (n >= K).sum().item()
+    return int((rej * 2 + acc) * V * esize), int(rej * 2 * V * esize)
 
 
 def run_ours(args):
@@ -172,8 +176,8 @@ def run_ours(args):
     value = rows_total / (ms_step * 1e-3)
 
     logits_bytes = w.logit_bytes
-    rs_bytes = resample_bytes(acc, K, V, esize)
-    step_bytes = logits_bytes + rs_bytes
+    rs_formula, rs_again = final_token_bytes(acc, K, V, esize)
+    step_bytes = logits_bytes + rs_formula
     k_avg = statistics.fmean(kernel_ms)
     peak, peak_kind = measured_peak()
     # algorithmic HBM bytes of the kernel: every logit once.  The rows of the final token are a second
@@ -218,8 +222,9 @@ def run_ours(args):
                        "l2": "inputs (3.67 GB at the default workload) exceed L2; no flush needed"
                              if logits_bytes > 512e6 else "inputs fit L2: warm-cache number",
                        "mean_accept_len": float(acc.float().mean().item())},
-            "hbm_gbs_step": step_bytes / (ms_step * 1e-3) / 1e9,
-            "bytes_per_step": {"logits": logits_bytes, "final_token_rows": rs_bytes},
+            "gbs_step_formula": step_bytes / (ms_step * 1e-3) / 1e9,
+            "bytes_per_step": {"logits": logits_bytes, "final_token_rows_formula": rs_formula,
+                               "final_token_rows_streamed_again": rs_again},
             "kernel_ms": {"ears_verify_kernel": k_avg},
             "roofline": {"bound": "hbm", "kernel": "ears_verify_kernel", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",

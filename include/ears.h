@@ -163,7 +163,7 @@ int ears_verify_host(int dtype, const void* target_logits, const void* draft_log
  *
  *   - Shapes whose scratch need, ears_workspace_bytes(B,K,V), exceeds
  *     EARS_NOALLOC_SCRATCH_BYTES are refused with EARS_ERR_WORKSPACE before anything
- *     is enqueued (B=512, K=3, V=256000 needs about 2.2 MB).
+ *     is enqueued (B=512, K=3, V=256000 needs about 4.2 MB).
  *   - The first call on each device looks up the array's device address (and sets the
  *     kernels' shared-memory attribute); make that first call outside any stream
  *     capture.  The device must be current, as for every other entry point.
@@ -176,7 +176,7 @@ int ears_verify_host(int dtype, const void* target_logits, const void* draft_log
  *     status word (EARS_DEV_* bits, 0 = clean) is copied there on `stream` after the
  *     kernels, for the caller to read once the stream has been waited for.
  */
-#define EARS_NOALLOC_SCRATCH_BYTES (4u << 20)
+#define EARS_NOALLOC_SCRATCH_BYTES (8u << 20)
 int ears_verify_noalloc(int dtype, const void* target_logits, const void* draft_logits,
                         const int32_t* draft_tokens, int B, int K, int V,
                         float temperature, float beta, uint64_t seed, uint64_t offset,

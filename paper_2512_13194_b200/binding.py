@@ -182,7 +182,7 @@ def verify_host(target_logits: torch.Tensor, draft_logits: torch.Tensor, draft_t
     return acc, tok
 
 
-NOALLOC_SCRATCH_BYTES = 4 << 20
+NOALLOC_SCRATCH_BYTES = 8 << 20
 
 
 def verify_noalloc(target_logits, draft_logits, draft_tokens, temperature, beta, seed, offset, *,

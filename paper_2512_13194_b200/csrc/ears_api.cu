@@ -4,7 +4,6 @@
 
 #include <cmath>
 #include <cstdio>
-#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <mutex>
@@ -34,7 +33,7 @@ int cuda_fail(cudaError_t e, const char* what) {
         if (e_ != cudaSuccess) return cuda_fail(e_, #call); \
     } while (0)
 
-struct PlanOverride { int loader = 0, parts1 = 0, streams = 0, claim = 0; };
+struct PlanOverride { int loader = 0, parts1 = 0; };
 PlanOverride g_override;
 std::mutex g_mutex;
 
@@ -79,25 +78,17 @@ Plan make_plan(int B, int K, int V, int esize, bool aligned, int sms, const Plan
     pl.use_tma = aligned && ov.loader != 2;
     split_rows((long long)B * (2 * K + 1), chunks, sms, ov.parts1, &pl.parts1, &pl.cpp1);
     pl.nseg = (V + kSegElems - 1) / kSegElems;
-    // With many units per CTA one atomic on the queue head hands out several units (spaced a
-    // grid apart, so CTAs still sweep the rows in step); same-address atomics are slow.
-    const long long units = (long long)B * (2 * K + 1) * pl.parts1;
     const long long ctas = (long long)sms * kCtasPerSm;
-    pl.claim = units >= 32 * ctas ? 4 : (units >= 8 * ctas ? 2 : 1);
-    if (ov.claim > 0) pl.claim = ov.claim;
-    // final-token pass: 64 KB of each row per piece, single chunks when there are few sequences
+    // second pass (rejected positions): 64 KB of each row per piece, single chunks when there are few sequences
     const int job_chunks = (long long)B * ((chunks + 3) / 4) >= ctas ? 4 : 1;
     pl.job_elems = job_chunks * chunk_elems;
     pl.parts2 = (V + pl.job_elems - 1) / pl.job_elems;
-    pl.streams = ov.streams > 0 ? ov.streams : 1;
-    if (pl.streams > B) pl.streams = B;
-    pl.seq_per_stream = (B + pl.streams - 1) / pl.streams;
     return pl;
 }
 
 struct Layout {
     size_t ticket1, ticket2, job_ctr, ticket_row, ready, heads, counters_bytes;
-    size_t partial, rowstat, pt_tok, pd_tok, max_pt, cls, resid, segsum, bonus_seg, total;
+    size_t partial, rowstat, pt_tok, pd_tok, max_pt, cls, resid, seg, seg_stride, total;
 };
 
 Layout make_layout(int B, int K, int V, int parts1) {
@@ -120,9 +111,12 @@ Layout make_layout(int B, int K, int V, int parts1) {
     L.max_pt = o; o = align_up(o + (size_t)B * K * 8, 256);
     L.cls = o; o = align_up(o + (size_t)B * K, 256);
     L.resid = o; o = align_up(o + (size_t)B * 8, 256);
-    L.segsum = o; o = align_up(o + (size_t)B * ((V + kSegElems - 1) / kSegElems) * 4, 256);
-    // the extra row's per-warp chunk sums; 2-byte elements give the fewest chunks, 4-byte the most
-    L.bonus_seg = o; o = align_up(o + (size_t)B * ((V + kChunkBytes / 4 - 1) / (kChunkBytes / 4)) * kConsumerWarps * sizeof(float2), 256);
+    // per sequence: BonusSeg per (chunk, consumer warp) of the extra row, later reused for the
+    // second pass's segment sums; 4-byte elements give the most chunks
+    const size_t bonus_bytes = (size_t)((V + kChunkBytes / 4 - 1) / (kChunkBytes / 4)) * kConsumerWarps * sizeof(BonusSeg);
+    const size_t seg_bytes = (size_t)((V + kSegElems - 1) / kSegElems) * sizeof(double);
+    L.seg_stride = align_up(bonus_bytes > seg_bytes ? bonus_bytes : seg_bytes, 16);
+    L.seg = o; o = align_up(o + (size_t)B * L.seg_stride, 256);
     L.total = o;
     return L;
 }
@@ -267,8 +261,8 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
     p.heads = (int*)(w + L.heads);
     p.partial = (float2*)(w + L.partial);
     p.rowstat = (float2*)(w + L.rowstat);
-    p.segsum = (float*)(w + L.segsum);
-    p.bonus_seg = (float2*)(w + L.bonus_seg);
+    p.seg_base = (unsigned char*)(w + L.seg);
+    p.seg_stride = L.seg_stride;
     p.plan = plan;
     return dtype == EARS_DTYPE_F32 ? launch<float>(p, di->sms, stream) : launch<uint16_t>(p, di->sms, stream);
 }
@@ -464,10 +458,6 @@ int ears_set_plan(int loader, int parts) {
     std::lock_guard<std::mutex> lock(g_mutex);
     g_override.loader = loader;
     g_override.parts1 = parts;
-    const char* e = getenv("EARS_STREAMS");
-    g_override.streams = e ? atoi(e) : 0;
-    e = getenv("EARS_CLAIM");
-    g_override.claim = e ? atoi(e) : 0;
     return EARS_OK;
 }
 

@@ -32,13 +32,13 @@ constexpr double kTinyMass = 1e-300;                 // below this a residual is
 constexpr int kDevInvalidInput = 1;
 constexpr int kDevTimeout = 2;
 
+// Sum of exp2((l - ref) c) over one consumer warp's share of a chunk of the extra target row.
+struct BonusSeg { double sum; float ref; float pad; };
+
 struct Plan {
     int use_tma;   // 1: bulk asynchronous copies, 0: element-wise loader
     int parts1;    // pieces per row in the statistics pass
     int cpp1;      // chunks per piece
-    int claim;     // units a CTA takes from the queue per atomic (spaced one grid apart)
-    int streams;   // the batch is swept as this many interleaved runs of sequences
-    int seq_per_stream;
     int parts2;    // pieces per row in the final-token pass
     int job_elems; // elements of each row per piece of the final-token pass
     int nseg;      // segment sums per sequence
@@ -72,10 +72,16 @@ struct Params {
     int* heads;           // [0] unit queue, [1] finalised sequences, [2] status, [3] published sequences
     float2* partial;      // [B*(2K+1)*parts1] (m, s) per row piece
     float2* rowstat;      // [B*(2K+1)] (m, Z) per row
-    float* segsum;        // [B*nseg] segment sums of the final-token masses (second pass)
-    float2* bonus_seg;    // [B*chunks*8] (sum, reference max) per chunk and consumer warp of the extra row
+    // Per sequence one region of seg_stride bytes, used first for the extra row's BonusSeg
+    // entries [chunks*8] and, if a position is rejected, afterwards for the second pass's
+    // segment sums (double [nseg]); a sequence never needs both at once.
+    unsigned char* seg_base;
+    size_t seg_stride;
     Plan plan;
 };
+
+__host__ __device__ inline double* seg_sums(const Params& p, int b) { return reinterpret_cast<double*>(p.seg_base + (size_t)b * p.seg_stride); }
+__host__ __device__ inline BonusSeg* bonus_segs(const Params& p, int b) { return reinterpret_cast<BonusSeg*>(p.seg_base + (size_t)b * p.seg_stride); }
 
 // Row order inside a sequence: target k, draft k for k = 0..K-1, then the bonus
 // target row K.  ridx in [0, 2K].

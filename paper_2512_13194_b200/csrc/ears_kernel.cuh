@@ -1,26 +1,28 @@
 // The verification step as one persistent kernel.
 //
-// Work is cut into "units" (a piece of one logits row) that CTAs pull from an atomic
-// queue, sequence by sequence, so that the 2K+1 rows of a sequence stream through the
-// GPU at about the same time.  Inside a CTA:
+// Work is cut into "units" (a piece of one logits row) that CTAs pull from an atomic queue,
+// sequence by sequence.  Inside a CTA:
 //
-//   loader warp    pulls units and streams them into a ring of shared-memory slots with
-//                  1-D bulk asynchronous copies completing on mbarriers (element-wise
-//                  copies when the data is not 16-byte aligned);
-//   8 consumer     keep a running (max, sum exp2) per thread over the slots [softmax
-//   warps          statistics, Sec. 3.1], reduce them per unit and publish the piece;
-//   epilogue warp  publishes the pieces and counts them with one atomic ticket per
-//                  sequence; for a sequence whose last piece it delivered it merges the
-//                  pieces, forms P_t(x), P_d(x), max P_t = 1/Z_t, draws U_k,
-//                  decides every position (Sec. 3.2 with the guards of Sec. 3.3 item 2),
-//                  scans for the first rejection (Sec. 3.1) and asks the loader for the
-//                  one or two rows the final token needs.  Those rows were streamed
-//                  moments ago by this and neighbouring CTAs and are normally still in
-//                  L2, so the second pass costs little or no HBM traffic.  The consumers
-//                  turn them into fp64 segment sums of the masses; the epilogue warp then
-//                  picks the token by inverse CDF.
+//   loader warp     pulls units and streams them into a ring of shared-memory slots with 1-D
+//                   bulk asynchronous copies completing on mbarriers (element-wise copies when
+//                   the data is not 16-byte aligned); also serves the second pass (below);
+//   8 consumer      keep a running (max, sum exp2) per thread over the slots [softmax
+//   warps           statistics, Sec. 3.1] and reduce them per unit; for the extra target row K
+//                   they also leave per-warp chunk sums behind;
+//   epilogue warp   publishes the pieces of rows and counts them with atomic tickets (per row,
+//                   then per sequence), so that consumers never wait at the end of a unit;
+//   sequence warp   for a sequence whose last piece this CTA delivered: merges the pieces, forms
+//                   P_t(x), P_d(x), max P_t = 1/Z_t, draws U_k, decides every position (Sec. 3.2
+//                   with the guards of Sec. 3.3 item 2) and scans for the first rejection
+//                   (Sec. 3.1).  If every draft was accepted the bonus token is drawn at once
+//                   from the chunk sums of row K.  Otherwise the sequence is published for a
+//                   second pass over the two rows of the rejected position: all CTAs serve
+//                   those rows in pieces (they were streamed moments ago and are mostly still
+//                   in L2), consumers turn them into segment sums of max(0, P_t - P_d), and the
+//                   CTA that delivers the last piece picks the token by inverse CDF.
 //
-// No CTA ever waits for another CTA; all waits inside a CTA are bounded.
+// A CTA never waits for work another CTA has yet to start; the only cross-CTA wait is the idle
+// wait at the very end (see the loader), which cannot deadlock.  Every wait is bounded.
 #pragma once
 #include "ears_common.cuh"
 #include "ears_philox.cuh"
@@ -28,7 +30,7 @@
 
 namespace ears {
 
-enum ChunkKind : int { kStats = 0, kBonus = 1, kResid = 2, kDrain = 3, kEnd = 4 };
+enum ChunkKind : int { kStats = 0, kFinal = 1, kDrain = 3, kEnd = 4 };
 enum MsgKind : int { kMsgPiece = 0, kMsgJobPiece = 1, kMsgDrain = 2, kMsgExit = 3, kMsgAck = 5, kMsgNone = 6, kMsgFinalize = 7, kMsgSelect = 8 };
 
 struct StageMeta {
@@ -37,7 +39,7 @@ struct StageMeta {
     int nelem;   // valid elements per row in the slot
     int flags;   // bit 0: first chunk of the unit / row, bit 1: last chunk
     int elem0;   // index of the slot's first element within its row
-    int aux;     // accepted length n of the sequence (final-token rows)
+    int aux;     // statistics: 1 for the extra target row; final-token rows: position n
 };
 
 struct Msg { int kind, a, b, c; };
@@ -246,7 +248,7 @@ __device__ __forceinline__ float load_logit(const uint16_t* p) { return bf16_bit
 // accepted, the final token is drawn from exactly these sums and the row is not read again.
 template <typename E, bool BONUS>
 __device__ __forceinline__ void chunk_stats(const unsigned char* buf, int nelem, int warp, int lane, float c,
-                                            float& m_run, float (&s)[4], float2* warp_chunk_out) {
+                                            float& m_run, float (&s)[4], BonusSeg* warp_chunk_out) {
     constexpr int N = Vec<E>::N;
     constexpr int VECS = kChunkBytes / 16 / kConsumers;  // 16-byte vectors per thread per chunk
     constexpr int CHUNK_ELEMS = kChunkBytes / (int)sizeof(E);
@@ -287,10 +289,12 @@ __device__ __forceinline__ void chunk_stats(const unsigned char* buf, int nelem,
 #pragma unroll
             for (int i = 0; i < N; ++i) cs[(j * N + i) & 3] += ex2_approx(__fmul_rn(__fsub_rn(x[j][i], mu), c));
         s[0] += cs[0]; s[1] += cs[1]; s[2] += cs[2]; s[3] += cs[3];
-        float tot = (cs[0] + cs[1]) + (cs[2] + cs[3]);
+        // a lane's few terms add up in fp32; across lanes in fp64, so that the running sums of the
+        // final draw stay exact to ~1e-9 of the row's mass
+        double tot = (double)((cs[0] + cs[1]) + (cs[2] + cs[3]));
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, off);
-        if (lane == 0) *warp_chunk_out = make_float2(tot, m_run);   // m_run is warp-uniform here
+        if (lane == 0) *warp_chunk_out = BonusSeg{tot, m_run, 0.f};   // m_run is warp-uniform here
     }
 }
 
@@ -329,12 +333,10 @@ __device__ __forceinline__ double warp_inclusive_scan(double v, int lane) {
 }
 
 // Sums of kSegElems-element segments of a staged chunk; warp w takes segments w, w+8, ...
-// All fp32: fp64 arithmetic is far too slow on this part to sit in the streaming path.  A
-// segment sum carries ~1e-7 relative rounding error, i.e. at most ~1e-7 of probability even
-// for a segment holding most of the mass; the final pick re-reads the chosen segment.
+// A lane adds its few masses in fp32; lanes are added in fp64.
 template <typename E, bool RESID>
 __device__ __forceinline__ void chunk_segments(const unsigned char* bt, const unsigned char* bd, int nelem,
-                                               int warp, int lane, const RowNorm& rn, float c, float* seg_out) {
+                                               int warp, int lane, const RowNorm& rn, float c, double* seg_out) {
     constexpr int N = Vec<E>::N;
     constexpr int VECS = kSegElems / (32 * N);  // 16-byte vectors per lane per segment
     constexpr int FULL_ELEMS = (RESID ? kChunkBytes / 2 : kChunkBytes) / (int)sizeof(E);
@@ -342,10 +344,10 @@ __device__ __forceinline__ void chunk_segments(const unsigned char* bt, const un
     if (SEGS >= 1 && nelem == FULL_ELEMS) {
         // full slot: all of the warp's segments at once, so that their loads, exponentials and
         // shuffle trees overlap instead of running one after the other
-        float acc[SEGS > 0 ? SEGS : 1];
+        double acc[SEGS > 0 ? SEGS : 1];
 #pragma unroll
         for (int g = 0; g < SEGS; ++g) {
-            acc[g] = 0.0f;
+            float a = 0.0f;
 #pragma unroll
             for (int j = 0; j < VECS; ++j) {
                 const int vec = (g * kConsumerWarps + warp) * (kSegElems / N) + j * 32 + lane;
@@ -353,8 +355,9 @@ __device__ __forceinline__ void chunk_segments(const unsigned char* bt, const un
                 Vec<E>::load(bt, vec, xt);
                 if (RESID) Vec<E>::load(bd, vec, xd);
 #pragma unroll
-                for (int i = 0; i < N; ++i) acc[g] += entry_mass<RESID>(xt[i], RESID ? xd[i] : 0.f, rn, c);
+                for (int i = 0; i < N; ++i) a += entry_mass<RESID>(xt[i], RESID ? xd[i] : 0.f, rn, c);
             }
+            acc[g] = (double)a;
         }
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1)
@@ -368,7 +371,7 @@ __device__ __forceinline__ void chunk_segments(const unsigned char* bt, const un
     }
     const int nseg = (nelem + kSegElems - 1) / kSegElems;
     for (int sgm = warp; sgm < nseg; sgm += kConsumerWarps) {
-        float acc = 0.0f;
+        float a = 0.0f;
 #pragma unroll
         for (int j = 0; j < VECS; ++j) {
             const int vec = sgm * (kSegElems / N) + j * 32 + lane;
@@ -378,9 +381,10 @@ __device__ __forceinline__ void chunk_segments(const unsigned char* bt, const un
 #pragma unroll
             for (int i = 0; i < N; ++i) {
                 const float r = entry_mass<RESID>(xt[i], RESID ? xd[i] : 0.f, rn, c);
-                if (vec * N + i < nelem) acc += r;
+                if (vec * N + i < nelem) a += r;
             }
         }
+        double acc = (double)a;
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
         if (lane == 0) seg_out[sgm] = acc;
@@ -606,17 +610,19 @@ __device__ void select_token(const Params& p, int b, int n, int lane) {
     double S = 0.0, before = 0.0;
     int seg, seg_elems;
     if (resid) {
-        const float* ss = p.segsum + (size_t)b * nseg;
-        seg = pick_block([ss](int g) { return (double)__ldcg(ss + g); }, nseg, u, lane, &S, &before);
+        const double* ss = seg_sums(p, b);
+        seg = pick_block([ss](int g) { return __ldcg(ss + g); }, nseg, u, lane, &S, &before);
         seg_elems = kSegElems;
     } else {
         // one entry per (chunk, consumer warp) of the extra row: (sum, reference maximum)
         const int chunks = (V + CHUNK_ELEMS - 1) / CHUNK_ELEMS;
-        const float2* bs = p.bonus_seg + (size_t)b * chunks * kConsumerWarps;
-        const float m = rn.mt, c = p.c;
+        const BonusSeg* bs = bonus_segs(p, b);
+        const double m = (double)rn.mt, c = (double)p.c;
         seg = pick_block([bs, m, c](int g) {
-                  const float2 e = __ldcg(bs + g);
-                  return (double)(e.x * ex2_approx((e.y - m) * c));   // bring the sum to the row's maximum
+                  const double sum = __ldcg(&bs[g].sum);
+                  const float ref = __ldcg(&bs[g].ref);
+                  // bring the sum from its own reference maximum to the row's (fp64: no new error)
+                  return sum > 0.0 ? sum * exp2(((double)ref - m) * c) : 0.0;
               }, chunks * kConsumerWarps, u, lane, &S, &before);
         seg_elems = CHUNK_ELEMS / kConsumerWarps;
     }
@@ -644,9 +650,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
     const int K = p.K, R = 2 * K + 1, V = p.V, P = p.plan.parts1, cpp = p.plan.cpp1, nseg = p.plan.nseg;
     const bool use_tma = p.plan.use_tma != 0;
     const int chunks_per_row = (V + CHUNK_ELEMS - 1) / CHUNK_ELEMS;
-    const long long units_per_stream = (long long)p.plan.seq_per_stream * R * P;
-    const long long total_units = units_per_stream * p.plan.streams;  // order space; holes are skipped
-    const long long real_units = (long long)p.B * R * P;
+    const long long total_units = (long long)p.B * R * P;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const E* tbase = reinterpret_cast<const E*>(p.t);
     const E* dbase = reinterpret_cast<const E*>(p.d);
@@ -672,12 +676,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
         bool ok = true, stats_done = false, acked = false;
         // The queue index of the next unit is fetched one unit ahead (lane 0 holds it) so that the
         // round trip of the atomic overlaps with streaming the current unit.
-        // One claim covers `claim` units spaced one grid apart.
-        const int claim = p.plan.claim;
-        const long long G = gridDim.x;
-        long long u_ahead = 0;        // lane 0: next claim ticket
-        long long tk = -1;            // current claim ticket
-        int ci = 0;                   // units of the current claim already taken
+        long long u_ahead = 0;
         if (lane == 0) u_ahead = atomicAdd(&p.heads[0], 1);
         // L2 hints: lines that will not be read again may go first; rows that may be read again
         // by the second pass get the default policy (0 = no hint).
@@ -724,44 +723,34 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
             if (jb >= 0) {
                 // 1. rows for a final token come first: they are hot in L2 right now
                 __threadfence();
-                const int b = jb, n = jn;
-                const bool resid = n < K;
-                const int step = resid ? CHUNK_ELEMS / 2 : CHUNK_ELEMS;
+                const int b = jb, n = jn;          // n < K: the first rejected position
+                const int step = CHUNK_ELEMS / 2;  // half a slot of each of the two rows
                 const E* trow = tbase + (size_t)target_row(b, n, K) * V;
-                const E* drow = resid ? dbase + (size_t)draft_row(b, n, K) * V : nullptr;
+                const E* drow = dbase + (size_t)draft_row(b, n, K) * V;
                 const int e_begin = jpart * p.plan.job_elems;
                 const int e_end = min(V, e_begin + p.plan.job_elems);
                 for (int e0 = e_begin; e0 < e_end; e0 += step, ++q) {
                     ok = loader_acquire(sm, q, lane);
                     if (!ok) break;
                     const int ne = min(step, e_end - e0);
-                    const StageMeta mt{resid ? kResid : kBonus, b, ne, (e0 == e_begin ? 1 : 0) | (e0 + step >= e_end ? 2 : 0), e0, n};
-                    loader_fill<E>(sm, q % STAGES, mt, use_tma, trow + e0, resid ? drow + e0 : nullptr, lane, pol_last_use);
+                    const StageMeta mt{kFinal, b, ne, (e0 == e_begin ? 1 : 0) | (e0 + step >= e_end ? 2 : 0), e0, n};
+                    loader_fill<E>(sm, q % STAGES, mt, use_tma, trow + e0, drow + e0, lane, pol_last_use);
                 }
                 if (!ok) break;
             } else if (!stats_done) {
                 // 2. next piece of a row for the statistics pass
                 if (sm.abort_flag) { ok = false; break; }
-                if (tk < 0 || ci == claim) {
-                    tk = __shfl_sync(0xffffffffu, u_ahead, 0);
-                    ci = 0;
-                    if (lane == 0 && (tk / G) * claim * G < total_units) u_ahead = atomicAdd(&p.heads[0], 1);
-                }
-                const long long j = ((tk / G) * claim + ci) * G + tk % G;  // position in the sweep order
-                ++ci;
-                // interleaved runs: consecutive positions visit different parts of the batch
-                const long long u = (j % p.plan.streams) * units_per_stream + j / p.plan.streams;
-                if (j >= total_units) {
-                    if ((tk / G) * claim * G + tk % G >= total_units) {
-                        // nothing left to pull: tell the consumers; final-token rows are served until
-                        // this CTA's epilogue warp has acknowledged
-                        ok = loader_acquire(sm, q, lane);
-                        if (!ok) break;
-                        loader_fill<E>(sm, q % STAGES, StageMeta{kDrain, 0, 0, 0, 0, 0}, use_tma, (const E*)nullptr, (const E*)nullptr, lane, pol_keep);
-                        ++q;
-                        stats_done = true;
-                    }  // else: a hole in the last sweep
-                } else if (u < real_units) {  // else: a hole in the last run
+                const long long u = __shfl_sync(0xffffffffu, u_ahead, 0);
+                if (u >= total_units) {
+                    // nothing left to pull: tell the consumers; final-token rows are served until
+                    // this CTA's sequence warp has acknowledged
+                    ok = loader_acquire(sm, q, lane);
+                    if (!ok) break;
+                    loader_fill<E>(sm, q % STAGES, StageMeta{kDrain, 0, 0, 0, 0, 0}, use_tma, (const E*)nullptr, (const E*)nullptr, lane, pol_keep);
+                    ++q;
+                    stats_done = true;
+                } else {
+                    if (lane == 0) u_ahead = atomicAdd(&p.heads[0], 1);
                     const int b = (int)(u / (R * P));
                     const int rem = (int)(u % (R * P));
                     const int ridx = rem / P, part = rem % P;
@@ -965,7 +954,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
             if (mt.kind == kStats) {
                 if (mt.flags & 1) { m_run = -INFINITY; s[0] = s[1] = s[2] = s[3] = 0.f; }
                 if (mt.aux) {  // a piece of the extra target row
-                    float2* out = p.bonus_seg + ((size_t)(mt.id / (R * P)) * chunks_per_row + mt.elem0 / CHUNK_ELEMS) * kConsumerWarps + warp;
+                    BonusSeg* out = bonus_segs(p, mt.id / (R * P)) + (size_t)(mt.elem0 / CHUNK_ELEMS) * kConsumerWarps + warp;
                     chunk_stats<E, true>(sm.buf[stage], mt.nelem, warp, lane, p.c, m_run, s, out);
                 } else {
                     chunk_stats<E, false>(sm.buf[stage], mt.nelem, warp, lane, p.c, m_run, s, nullptr);
@@ -993,17 +982,15 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
                 ++unit_ends;
                 continue;
             }
-            // rows of a final token: segment sums of the masses
+            // the two rows of a rejected position: segment sums of max(0, P_t - P_d)
             const int b = mt.id, n = mt.aux;
-            const bool resid = mt.kind == kResid;
             if (mt.flags & 1) {
-                const float2 st = __ldcg(&p.rowstat[(size_t)b * R + (resid ? 2 * n : 2 * K)]);
-                const float2 sd = resid ? __ldcg(&p.rowstat[(size_t)b * R + 2 * n + 1]) : make_float2(0.f, 1.f);
+                const float2 st = __ldcg(&p.rowstat[(size_t)b * R + 2 * n]);
+                const float2 sd = __ldcg(&p.rowstat[(size_t)b * R + 2 * n + 1]);
                 rn = make_rownorm(st, sd);
             }
-            float* seg_out = p.segsum + (size_t)b * nseg + mt.elem0 / kSegElems;
-            if (resid) chunk_segments<E, true>(sm.buf[stage], sm.buf[stage] + kChunkBytes / 2, mt.nelem, warp, lane, rn, p.c, seg_out);
-            else chunk_segments<E, false>(sm.buf[stage], sm.buf[stage], mt.nelem, warp, lane, rn, p.c, seg_out);
+            double* seg_out = seg_sums(p, b) + mt.elem0 / kSegElems;
+            chunk_segments<E, true>(sm.buf[stage], sm.buf[stage] + kChunkBytes / 2, mt.nelem, warp, lane, rn, p.c, seg_out);
             if (mt.flags & 2) {
                 // last chunk of the piece: publish the sums; the epilogue warp counts the piece once
                 // all warps are through and, when it is the sequence's last, picks the token

@@ -1,0 +1,48 @@
+"""Long parity run (not collected by pytest): accumulates GPU-vs-oracle comparisons over many
+verification steps of one workload and prints the disagreement counts.
+
+    python tests/soak_parity.py <workload 1..5> <rows to cover> [beta]
+
+Near-tie disagreements (explained by the oracle's margins) must stay below 1e-4 of rows; anything
+unexplained is a failure.
+"""
+import os
+import sys
+
+import numpy as np
+import torch
+
+sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
+import oracle  # noqa: E402
+import paper_2512_13194_b200 as ears  # noqa: E402
+from paper_2512_13194_b200 import synth  # noqa: E402
+from parity import Tally, compare  # noqa: E402
+
+
+def main():
+    idx, want_rows = int(sys.argv[1]), int(float(sys.argv[2]))
+    w = synth.workload(idx)
+    beta = float(sys.argv[3]) if len(sys.argv) > 3 else w.beta
+    t, d, x = synth.make_inputs(w, "cuda:0")
+    th, dh, xh = t.cpu(), d.cpu(), x.cpu()
+    tally, offset = Tally(), 0
+    threads = min(oracle.max_threads(), len(os.sched_getaffinity(0)))
+    while tally.rows < want_rows:
+        acc, tok, st = ears.verify(t, d, x, w.temperature, beta, w.verify_seed, offset, stats=True)
+        torch.cuda.synchronize()
+        ora = oracle.verify(th, dh, xh, w.temperature, beta, seed=w.verify_seed, offset=offset, nthreads=threads)
+        tally.merge(compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, w.K, {k: v.cpu().numpy() for k, v in st.items()}))
+        offset += 1
+    print(f"{w.name} beta={beta}: steps={offset} rows={tally.rows} sequences={tally.sequences} "
+          f"explained decisions={tally.explained_decisions} tokens={tally.explained_tokens} "
+          f"({tally.explained / tally.rows:.2e} of rows) unexplained={len(tally.unexplained)} "
+          f"flagged decisions={tally.flagged_decisions} tokens={tally.flagged_tokens} "
+          f"max rel prob err={tally.max_rel_prob_err:.2e}")
+    if tally.unexplained:
+        print("UNEXPLAINED:", tally.unexplained[:5])
+        sys.exit(1)
+
+
+if __name__ == "__main__":
+    main()
