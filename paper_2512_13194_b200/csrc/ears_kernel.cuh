@@ -647,7 +647,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
     using Smem = PipeSmem<STAGES>;
     Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     constexpr int CHUNK_ELEMS = kChunkBytes / (int)sizeof(E);
-    const int K = p.K, R = 2 * K + 1, V = p.V, P = p.plan.parts1, cpp = p.plan.cpp1, nseg = p.plan.nseg;
+    const int K = p.K, R = 2 * K + 1, V = p.V, P = p.plan.parts1, cpp = p.plan.cpp1;
     const bool use_tma = p.plan.use_tma != 0;
     const int chunks_per_row = (V + CHUNK_ELEMS - 1) / CHUNK_ELEMS;
     const long long total_units = (long long)p.B * R * P;
@@ -853,21 +853,16 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
             __syncwarp();
             if (lane == 0 && top >= 0) { __threadfence_block(); sm.units_read = top + 1; }
             if (m.kind == kMsgJobPiece && slot_ok) {
-                __threadfence();
-                if (atomicAdd(&p.ticket2[m.a], 1) == p.plan.parts2 - 1) last_b = m.a;  // all masses summed
+                if (ticket_add(&p.ticket2[m.a]) == p.plan.parts2 - 1) last_b = m.a;  // all masses summed
             }
             if (m.kind == kMsgPiece && slot_ok) {
                 const int b = m.a / (R * P);
                 const int rem = m.a % (R * P);
                 p.partial[((size_t)b * R + rem / P) * P + rem % P] = make_float2(pm, ps);
                 // two-level count (row, then sequence) spreads the atomics over many addresses
-                __threadfence();
                 bool row_done = true;
-                if (P > 1) {
-                    row_done = atomicAdd(&p.ticket_row[(size_t)b * R + rem / P], 1) == P - 1;
-                    if (row_done) __threadfence();
-                }
-                if (row_done && atomicAdd(&p.ticket1[b], 1) == R - 1) last_b = b;  // last row of the sequence
+                if (P > 1) row_done = ticket_add(&p.ticket_row[(size_t)b * R + rem / P]) == P - 1;
+                if (row_done && ticket_add(&p.ticket1[b]) == R - 1) last_b = b;  // last row of the sequence
             }
             // what needs a whole warp (decisions, final pick) goes to the sequence warp, in order
             for (int i = 0; i < cnt && running; ++i) {

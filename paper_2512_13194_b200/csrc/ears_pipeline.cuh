@@ -99,6 +99,15 @@ __device__ __forceinline__ uint64_t l2_policy_evict_first() {
     return pol;
 }
 
+// Counts an arrival with release + acquire semantics at device scope in the atomic itself:
+// what this thread wrote (or observed) before is visible to whoever sees the count, and what
+// earlier arrivals published is visible to this thread afterwards.  One round trip, no fence.
+__device__ __forceinline__ int ticket_add(int* addr) {
+    int old;
+    asm volatile("atom.add.acq_rel.gpu.s32 %0, [%1], 1;" : "=r"(old) : "l"(addr) : "memory");
+    return old;
+}
+
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
