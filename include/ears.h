@@ -197,6 +197,15 @@ int ears_last_device_status(void* stream);
 int ears_workspace_device_status(void* workspace, void* stream);
 
 /*
+ * Self-test of the kernels' bounded waits (every device-side wait in this library gives up
+ * after a time limit, sets EARS_DEV_TIMEOUT and lets the kernel return; nothing can hang
+ * the GPU).  Launches a tiny kernel that waits limit_ms (1..2000) on a barrier no thread ever
+ * completes, waits for it and returns EARS_ERR_TIMEOUT when the wait gave up as designed
+ * (EARS_OK would mean the limit did not work).  The context stays usable.
+ */
+int ears_selftest_bounded_wait(int limit_ms, void* stream);
+
+/*
  * Test hook for the device random stream: out[i, 0:4] = Philox4x32-10 of counter
  * ctr_key[i, 0:4] and key ctr_key[i, 4:6]; both device pointers, n >= 0.
  */

@@ -14,6 +14,7 @@ from .binding import (  # noqa: F401
     philox_device,
     profile_begin,
     profile_end,
+    selftest_bounded_wait,
     set_plan,
     shutdown,
     verify,

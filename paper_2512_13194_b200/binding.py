@@ -53,6 +53,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ears_last_device_status.restype = c.c_int
     lib.ears_workspace_device_status.argtypes = [c.c_void_p, c.c_void_p]
     lib.ears_workspace_device_status.restype = c.c_int
+    lib.ears_selftest_bounded_wait.argtypes = [c.c_int, c.c_void_p]
+    lib.ears_selftest_bounded_wait.restype = c.c_int
     lib.ears_philox_device.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_void_p]
     lib.ears_philox_device.restype = c.c_int
     lib.ears_set_plan.argtypes = [c.c_int, c.c_int]
@@ -229,6 +231,11 @@ def workspace_device_status(workspace: torch.Tensor, stream=None) -> int:
     if rc < 0:
         _check(rc)
     return rc
+
+
+def selftest_bounded_wait(limit_ms: int = 50, stream=None) -> int:
+    """Runs the bounded-wait self-test; returns the raw status (-7 = the wait gave up as designed)."""
+    return int(load_library().ears_selftest_bounded_wait(int(limit_ms), _stream_ptr(stream)))
 
 
 def philox_device(ctr_key: torch.Tensor) -> torch.Tensor:

@@ -67,6 +67,9 @@ void split_rows(long long items, int chunks, int sms, int forced_parts, int* par
         c = (chunks + fp - 1) / fp;
     }
     if (c > chunks) c = chunks;
+    // equal pieces: 19 chunks in 2 pieces are 10 + 9, not 16 + 3
+    const int n = (chunks + c - 1) / c;
+    c = (chunks + n - 1) / n;
     *cpp = c;
     *parts = (chunks + c - 1) / c;
 }
@@ -305,6 +308,23 @@ int noalloc_scratch(int dev, void** out) {
     return EARS_OK;
 }
 
+// Self-test of the bounded wait: a barrier nobody ever arrives at.  The wait must give up after
+// the limit, raise the abort flag and let the kernel return normally with the timeout bit set.
+static __device__ int g_selftest_status;
+
+__global__ void bounded_wait_kernel(unsigned long long limit_ns) {
+    __shared__ alignas(8) uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_flag = 0;
+        mbar_init_fence();
+    }
+    __syncthreads();
+    const bool ok = mbar_wait(&bar, 0, &abort_flag, limit_ns);   // every thread waits; all give up
+    if (!ok && threadIdx.x == 0) atomicOr(&g_selftest_status, kDevTimeout);
+}
+
 __global__ void philox_kernel(const uint32_t* ctr_key, uint32_t* out, int n) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
@@ -442,6 +462,18 @@ int ears_last_device_status(void* stream_) {
 int ears_workspace_device_status(void* workspace, void* stream_) {
     if (!workspace) return EARS_ERR_NULL;
     return read_status((int*)workspace, (cudaStream_t)stream_);
+}
+
+int ears_selftest_bounded_wait(int limit_ms, void* stream_) {
+    if (limit_ms < 1 || limit_ms > 2000) return EARS_ERR_PARAM;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    int seen = 0;
+    EARS_CUDA(cudaMemcpyToSymbolAsync(g_selftest_status, &seen, sizeof(int), 0, cudaMemcpyHostToDevice, stream));
+    bounded_wait_kernel<<<1, 64, 0, stream>>>((unsigned long long)limit_ms * 1000000ull);
+    EARS_CUDA(cudaGetLastError());
+    EARS_CUDA(cudaMemcpyFromSymbolAsync(&seen, g_selftest_status, sizeof(int), 0, cudaMemcpyDeviceToHost, stream));
+    EARS_CUDA(cudaStreamSynchronize(stream));
+    return (seen & EARS_DEV_TIMEOUT) ? EARS_ERR_TIMEOUT : EARS_OK;
 }
 
 int ears_philox_device(const uint32_t* ctr_key, uint32_t* out, int n, void* stream) {

@@ -197,3 +197,55 @@ def test_repeated_calls_are_reproducible(ears):
         assert torch.equal(again[0], first[0]) and torch.equal(again[1], first[1])
     other = ears.verify(tg, dg, xg, 1.0, 0.1, 1, 2)
     assert not torch.equal(other[1], first[1])
+
+
+@pytest.mark.parametrize("B,K,V,dtype,T,beta", [
+    (3, 64, 2051, "bf16", 1.0, 0.3),        # longest draft, unaligned rows, many rows per sequence
+    (5000, 1, 96, "fp32", 0.9, 0.1),        # many tiny sequences: tickets and the publish queue under load
+    (9, 2, 70000, "bf16", 1.0, 0.0),        # beta = 0 with a poor draft: nearly every sequence is rejected
+    (9, 2, 70000, "fp32", 1.4, 50.0),       # huge tolerance: everything accepted, bonus path only
+    (40, 3, 16384, "fp32", 1.0, 0.2),       # V an exact multiple of the slot size (no ragged chunk)
+    (40, 3, 16385, "bf16", 1.0, 0.2),       # one element past it, unaligned
+])
+def test_parity_extremes(ears, B, K, V, dtype, T, beta):
+    w, t, d, x = synth.tiny_inputs(B, K, V, dtype, seed=300 + K, noise=2.5 if beta == 0.0 else 0.5, temperature=T)
+    tally = Tally()
+    for offset in range(2):
+        tl, acc, tok, ora = run_both(ears, w, t, d, x, T, beta, seed=11, offset=offset)
+        tally.merge(tl)
+    assert_parity(tally, max_explained=max(1, int(np.ceil(1e-4 * tally.rows))))
+    if beta == 0.0:
+        assert (ora.accept_len < K).mean() > 0.5
+    if beta == 50.0:
+        assert (ora.accept_len == K).all()
+
+
+def test_alternating_shapes_share_one_workspace(ears):
+    """Back-to-back calls of different shapes on one stream reuse (and regrow) the library's
+    workspace; counters of an earlier call must never leak into the next."""
+    dev = "cuda:0"
+    cases = [synth.tiny_inputs(4, 3, 30000, "fp32", seed=71), synth.tiny_inputs(64, 2, 900, "bf16", seed=72),
+             synth.tiny_inputs(2, 5, 130000, "bf16", seed=73)]
+    gpu = [(w, t.to(dev), d.to(dev), x.to(dev)) for w, t, d, x in cases]
+    first = [ears.verify(t, d, x, 1.0, 0.1, 2, 0) for _, t, d, x in gpu]
+    for rep in range(3):
+        for i in (2, 0, 1, 1, 0, 2):
+            _, t, d, x = gpu[i]
+            a, k = ears.verify(t, d, x, 1.0, 0.1, 2, 0)
+            assert torch.equal(a, first[i][0]) and torch.equal(k, first[i][1])
+    assert ears.last_device_status() == 0
+
+
+def test_bounded_wait_gives_up_and_context_survives(ears):
+    """A device-side wait that can never complete returns after its limit with the timeout status
+    (no trap, no hang), and the same context keeps working."""
+    import time
+    t0 = time.perf_counter()
+    rc = ears.selftest_bounded_wait(50)
+    dt = time.perf_counter() - t0
+    assert rc == -7                      # EARS_ERR_TIMEOUT: the wait gave up as designed
+    assert 0.04 < dt < 1.5
+    w, t, d, x = synth.tiny_inputs(3, 2, 5000, "fp32", seed=5)
+    tl, *_ = run_both(ears, w, t, d, x, 1.0, 0.1)
+    assert_parity(tl, max_explained=0)
+    assert ears.load_library().ears_selftest_bounded_wait(0, None) == -3
