@@ -299,6 +299,72 @@ def run_reference(args):
     }), flush=True)
 
 
+def run_table(args):
+    """All five workloads (with the sweep of workload 2) on one GPU: a markdown table of device
+    times (cold = L2 flushed before every step, warm = back to back), throughput against the HBM
+    roofline, oracle times on the host and the GPU-vs-oracle comparison.  Not the benchmark line."""
+    import numpy as np
+    import torch
+
+    import oracle
+    import paper_2512_13194_b200 as ears
+    from paper_2512_13194_b200 import synth
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from parity import Tally, compare
+
+    torch.cuda.set_device(0)
+    ears.load_library()
+    peak, peak_kind = measured_peak()
+    cores = min(oracle.max_threads(), len(os.sched_getaffinity(0)))
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")   # > 4 x L2
+    stream = torch.cuda.current_stream()
+
+    def timed(fn, n, cold):
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+        for a, b in ev:
+            if cold:
+                flush.zero_()
+            a.record(stream)
+            fn()
+            b.record(stream)
+        torch.cuda.synchronize()
+        return statistics.median(a.elapsed_time(b) for a, b in ev) * 1e3   # us
+
+    print(f"| cfg | B | K | V | dtype | T | beta | mean accept_len | GPU us/step (cold / warm L2) | rows/s (cold) | "
+          f"GB/s logits (cold) | % of {peak:.0f} ({peak_kind}) | % of 8000 | oracle s (1 thread) | "
+          f"oracle s ({cores} threads) | disagreements / rows (explained / unexplained) | max rel. prob. error |")
+    print("|" + "---|" * 17)
+    for idx in range(1, 6):
+        w = synth.workload(idx)
+        for T in (w.temperatures or (w.temperature,)):
+            t, d, x = synth.make_inputs(w, "cuda:0", temperature=T)
+            th, dh, xh = t.cpu(), d.cpu(), x.cpu()
+            for beta in (w.betas or (w.beta,)):
+                run = lambda off=0: ears.verify(t, d, x, T, beta, w.verify_seed, off)
+                for i in range(5):
+                    run(i)
+                n = 30 if idx == 5 else 100
+                cold, warm = timed(run, n, True), timed(run, n, False)
+                acc, tok, st = ears.verify(t, d, x, T, beta, w.verify_seed, 7, stats=True)
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                ora = oracle.verify(th, dh, xh, T, beta, seed=w.verify_seed, offset=7, nthreads=cores)
+                o_n = time.perf_counter() - t0
+                if idx < 5 or args.table_full:
+                    t0 = time.perf_counter()
+                    oracle.verify(th, dh, xh, T, beta, seed=w.verify_seed, offset=7, nthreads=1)
+                    o_1 = f"{time.perf_counter() - t0:.3f}"
+                else:
+                    o_1 = f"~{o_n * cores:.1f} (threads x wall)"
+                tl = compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, w.K, {k: v.cpu().numpy() for k, v in st.items()})
+                gbs = w.logit_bytes / (cold * 1e-6) / 1e9
+                print(f"| {idx} | {w.B} | {w.K} | {w.V} | {w.dtype} | {T} | {beta} | {float(ora.accept_len.mean()):.2f} | "
+                      f"{cold:.1f} / {warm:.1f} | {w.rows / (cold * 1e-6):.3g} | {gbs:.0f} | {100 * gbs / peak:.1f} | "
+                      f"{100 * gbs / DATASHEET_HBM_GBS:.1f} | {o_1} | {o_n:.3f} | {tl.explained + len(tl.unexplained)} / {tl.rows} "
+                      f"({tl.explained} / {len(tl.unexplained)}) | {tl.max_rel_prob_err:.1e} |", flush=True)
+            del t, d, x
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -310,8 +376,12 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-sample", type=int, default=512, help="sequences given to the CPU baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--table", action="store_true", help="print the five-workload results table instead")
+    ap.add_argument("--table-full", action="store_true", help="also time the 1-thread oracle on workload 5")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.table:
+        run_table(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

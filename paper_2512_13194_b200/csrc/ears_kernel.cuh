@@ -92,7 +92,7 @@ struct Mailbox {
                 if (t0 == 0) t0 = now;
                 else if (now - t0 > limit_ns) { *abort_flag = 1; return -1; }
             }
-            __nanosleep(spin < 4 ? 100 : 400);  // idle warps must not eat the consumers' issue slots
+            __nanosleep(50);
         }
     }
     __device__ __forceinline__ Msg peek(int index) const {
@@ -110,7 +110,7 @@ struct Mailbox {
                 if (t0 == 0) t0 = now;
                 else if (now - t0 > limit_ns) { *abort_flag = 1; return false; }
             }
-            __nanosleep(spin < 4 ? 200 : 1000);
+            __nanosleep(50);
         }
     }
 };
@@ -492,28 +492,39 @@ __device__ int warp_sample_pt_slow(const E* row, int V, const RowNorm& rn, float
 // Last level of the inverse-CDF pick: entries [base, base + count) of the row(s) are read again,
 // their masses recomputed (same bits as in the streaming pass) and scanned in fp64 for the
 // smallest j with tin < running sum.  If rounding hides the crossing, the last entry with
-// positive mass is taken.  One warp; returns the token (or -1 if the range has no mass).
+// positive mass is taken.  One warp; count <= 128 * N entries, all loaded up front so that the
+// pick costs one memory round trip; returns the token (or -1 if the range has no mass).
 template <typename E>
 __device__ int pick_in_range(const E* trow, const E* drow, bool resid, const RowNorm& rn, float c,
                              int base, int count, double tin, int V, int lane) {
     constexpr int N = Vec<E>::N;
+    constexpr int ROUNDS = 4;  // 4 x 32 lanes x N entries cover the largest range (an eighth of a slot)
+    float mass[ROUNDS][N];
+#pragma unroll
+    for (int j = 0; j < ROUNDS; ++j)
+#pragma unroll
+        for (int i = 0; i < N; ++i) {
+            const int k = (j * 32 + lane) * N + i;
+            float xt = -INFINITY, xd = -INFINITY;
+            const bool valid = k < count && base + k < V;
+            if (valid) {
+                xt = load_logit(trow + base + k);
+                if (resid) xd = load_logit(drow + base + k);
+            }
+            mass[j][i] = !valid ? 0.f : (resid ? entry_mass<true>(xt, xd, rn, c) : entry_mass<false>(xt, 0.f, rn, c));
+        }
     double run = 0.0;
     int found = -1, lastpos = -1;
-    for (int j0 = 0; j0 < count && found < 0; j0 += 32 * N) {
-        const int e0 = base + j0 + lane * N;
-        double r[N], mine = 0.0;
+#pragma unroll
+    for (int j = 0; j < ROUNDS; ++j) {
+        if (found >= 0 || j * 32 * N >= count) break;
+        const int e0 = base + (j * 32 + lane) * N;
+        double mine = 0.0;
         int mylast = -1;
 #pragma unroll
         for (int i = 0; i < N; ++i) {
-            const int e = e0 + i;
-            r[i] = 0.0;
-            if (e < V && e < base + count) {
-                const float xt = load_logit(trow + e);
-                const float xd = resid ? load_logit(drow + e) : 0.f;
-                r[i] = (double)(resid ? entry_mass<true>(xt, xd, rn, c) : entry_mass<false>(xt, 0.f, rn, c));
-            }
-            if (r[i] > 0.0) mylast = e;
-            mine += r[i];
+            if (mass[j][i] > 0.f) mylast = e0 + i;
+            mine += (double)mass[j][i];
         }
         const double incl = warp_inclusive_scan(mine, lane);
         const unsigned h = __ballot_sync(0xffffffffu, tin < run + incl && mine > 0.0);
@@ -527,9 +538,9 @@ __device__ int pick_in_range(const E* trow, const E* drow, bool resid, const Row
                 int lp = -1;
 #pragma unroll
                 for (int i = 0; i < N; ++i) {
-                    cum += r[i];
-                    if (r[i] > 0.0) lp = e0 + i;
-                    if (t_here < 0 && r[i] > 0.0 && tin < cum) t_here = e0 + i;
+                    cum += (double)mass[j][i];
+                    if (mass[j][i] > 0.f) lp = e0 + i;
+                    if (t_here < 0 && mass[j][i] > 0.f && tin < cum) t_here = e0 + i;
                 }
                 if (t_here < 0) t_here = lp;
             }
@@ -786,7 +797,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
                             const unsigned long long now = global_timer_ns();
                             if (wait_t0 == 0) wait_t0 = now;
                             else if (now - wait_t0 > kIdleLimitNs) { sm.abort_flag = 1; fin = -1; }
-                            __nanosleep(200);
+                            __nanosleep(50);
                         }
                     }
                     fin = __shfl_sync(0xffffffffu, fin, 0);
