@@ -31,6 +31,10 @@ METRIC = "verify rows/s"
 UNIT = "rows/s"
 DATASHEET_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of ears_verify_kernel<float,6> from one ncu capture on
+# a 96-sequence batch of the default workload (690.71 MB + 4.45 MB), per sequence.  The traffic grows
+# in proportion to the number of sequences; set to None whenever the kernel changes after a capture.
+NCU_DRAM_BYTES_PER_SEQUENCE = (690710272 + 4452608) / 96
 
 
 def measured_peak():
@@ -225,11 +229,13 @@ def run_ours(args):
             "gbs_step_formula": step_bytes / (ms_step * 1e-3) / 1e9,
             "bytes_per_step": {"logits": logits_bytes, "final_token_rows_formula": rs_formula,
                                "final_token_rows_streamed_again": rs_again},
-            "kernel_ms": {"ears_verify_kernel": k_avg},
+            "kernel_ms": {"ears_verify_kernel": k_avg, "median": statistics.median(kernel_ms), "min": min(kernel_ms)},
             "roofline": {"bound": "hbm", "kernel": "ears_verify_kernel", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                          "frac_of_datasheet_8000": achieved / DATASHEET_HBM_GBS,
-                         "traffic": None},
+                         "traffic": (NCU_DRAM_BYTES_PER_SEQUENCE * w.B
+                                     if NCU_DRAM_BYTES_PER_SEQUENCE and args.workload == 5 else None),
+                         "traffic_note": "ncu DRAM read+write bytes of a 96-sequence capture scaled by sequences"},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps},
             "gpu_launches": args.steps,

@@ -206,6 +206,7 @@ def test_repeated_calls_are_reproducible(ears):
     (9, 2, 70000, "fp32", 1.4, 50.0),       # huge tolerance: everything accepted, bonus path only
     (40, 3, 16384, "fp32", 1.0, 0.2),       # V an exact multiple of the slot size (no ragged chunk)
     (40, 3, 16385, "bf16", 1.0, 0.2),       # one element past it, unaligned
+    (2, 1, 1000003, "fp32", 1.0, 0.05),     # a vocabulary of a million, unaligned: hundreds of chunks per row
 ])
 def test_parity_extremes(ears, B, K, V, dtype, T, beta):
     w, t, d, x = synth.tiny_inputs(B, K, V, dtype, seed=300 + K, noise=2.5 if beta == 0.0 else 0.5, temperature=T)
