@@ -90,7 +90,7 @@ Plan make_plan(int B, int K, int V, int esize, bool aligned, int sms, const Plan
 }
 
 struct Layout {
-    size_t ticket1, ticket2, job_ctr, ticket_row, ready, heads, counters_bytes;
+    size_t ticket1, ticket2, job_ctr, ticket_row, ready, heads, wq, counters_bytes;
     size_t partial, rowstat, pt_tok, pd_tok, max_pt, cls, resid, seg, seg_stride, total;
 };
 
@@ -98,7 +98,8 @@ Layout make_layout(int B, int K, int V, int parts1) {
     Layout L;
     const size_t rows = (size_t)B * (2 * K + 1);
     size_t o = 0;
-    L.heads = o; o += 16;  // fixed place: the status word is heads[2] of any workspace
+    L.heads = o; o += 32;  // fixed place: the status word is heads[2] of any workspace
+    L.wq = o; o += (size_t)B * 16;
     L.ticket1 = o; o += (size_t)B * 4;
     L.ticket2 = o; o += (size_t)B * 4;
     L.job_ctr = o; o += (size_t)B * 4;
@@ -262,6 +263,7 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
     p.job_ctr = (int*)(w + L.job_ctr);
     p.ready = (unsigned long long*)(w + L.ready);
     p.heads = (int*)(w + L.heads);
+    p.wq = (unsigned long long*)(w + L.wq);
     p.partial = (float2*)(w + L.partial);
     p.rowstat = (float2*)(w + L.rowstat);
     p.seg_base = (unsigned char*)(w + L.seg);

@@ -45,7 +45,8 @@ struct Plan {
 };
 
 // Counter block at the start of the workspace, zeroed by one memset per call:
-//   heads[4] (unit queue head, finalised sequences, status, published sequences),
+//   heads[8] (unit queue head, finalised sequences, status, published sequences,
+//   sequence-work queue tail and head), wq[2B],
 //   ticket1[B], ticket2[B], job_ctr[B], ticket_row[B*(2K+1)], ready[B].
 struct Params {
     const void* t;        // target logits [B,K+1,V]
@@ -69,7 +70,9 @@ struct Params {
     int* ticket2;         // [B] final-token pieces of the sequence that are in
     unsigned long long* ready;  // [B] published sequences: (b + 1) << 32 | n, 0 = not yet
     int* job_ctr;         // [B] final-token pieces handed out, per published slot
-    int* heads;           // [0] unit queue, [1] finalised sequences, [2] status, [3] published sequences
+    int* heads;           // [0] unit queue, [1] finalised sequences, [2] status, [3] published sequences,
+                          // [4] / [5] tail / head of the sequence-work queue
+    unsigned long long* wq;  // [2B] sequence work: bit 63 valid, bits 32..62 sequence, low word n or ~0 (decide)
     float2* partial;      // [B*(2K+1)*parts1] (m, s) per row piece
     float2* rowstat;      // [B*(2K+1)] (m, Z) per row
     // Per sequence one region of seg_stride bytes, used first for the extra row's BonusSeg

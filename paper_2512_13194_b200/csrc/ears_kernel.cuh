@@ -30,8 +30,8 @@
 
 namespace ears {
 
-enum ChunkKind : int { kStats = 0, kFinal = 1, kDrain = 3, kEnd = 4 };
-enum MsgKind : int { kMsgPiece = 0, kMsgJobPiece = 1, kMsgDrain = 2, kMsgExit = 3, kMsgAck = 5, kMsgNone = 6, kMsgFinalize = 7, kMsgSelect = 8 };
+enum ChunkKind : int { kStats = 0, kFinal = 1, kEnd = 4 };
+enum MsgKind : int { kMsgPiece = 0, kMsgJobPiece = 1, kMsgExit = 3, kMsgNone = 6 };
 
 struct StageMeta {
     int kind;    // ChunkKind
@@ -117,10 +117,8 @@ struct Mailbox {
 
 // consumer warp 0 -> epilogue warp
 constexpr int kEpiCap = 64;
-// epilogue warp -> loader warp: carries only the acknowledgement of the drain marker
-constexpr int kJobCap = 4;
-// epilogue warp -> sequence warp
-constexpr int kSeqCap = 64;
+// epilogue warp -> sequence warp: only the exit message
+constexpr int kSeqCap = 4;
 // Ends of units are handed to the epilogue warp through a ring of slots: each consumer warp
 // drops its (m, s) there and arrives on the slot's barrier, so no consumer ever waits for
 // another at the end of a unit.  Consumer warps are at most one pipeline ring apart, and
@@ -139,7 +137,6 @@ struct PipeSmem {
     float2 scratch[kUnitSlots][kConsumerWarps];
     volatile int units_read;   // unit ends the epilogue warp has taken out of the slots
     Mailbox<kEpiCap> epi;
-    Mailbox<kJobCap> jobs;
     Mailbox<kSeqCap> seq;
     int abort_flag;
 };
@@ -674,7 +671,6 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
         for (int s = 0; s < kUnitSlots; ++s) mbar_init(&sm.unit_bar[s], kConsumerWarps);
         sm.units_read = 0;
         sm.epi.init();
-        sm.jobs.init();
         sm.seq.init();
         sm.abort_flag = 0;
         mbar_init_fence();
@@ -684,7 +680,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
     if (warp == kLoaderWarp) {
         // =============================== loader warp
         uint32_t q = 0;
-        bool ok = true, stats_done = false, acked = false;
+        bool ok = true, stats_done = false;
         // The queue index of the next unit is fetched one unit ahead (lane 0 holds it) so that the
         // round trip of the atomic overlaps with streaming the current unit.
         long long u_ahead = 0;
@@ -753,13 +749,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
                 if (sm.abort_flag) { ok = false; break; }
                 const long long u = __shfl_sync(0xffffffffu, u_ahead, 0);
                 if (u >= total_units) {
-                    // nothing left to pull: tell the consumers; final-token rows are served until
-                    // this CTA's sequence warp has acknowledged
-                    ok = loader_acquire(sm, q, lane);
-                    if (!ok) break;
-                    loader_fill<E>(sm, q % STAGES, StageMeta{kDrain, 0, 0, 0, 0, 0}, use_tma, (const E*)nullptr, (const E*)nullptr, lane, pol_keep);
-                    ++q;
-                    stats_done = true;
+                    stats_done = true;   // nothing left to pull
                 } else {
                     if (lane == 0) u_ahead = atomicAdd(&p.heads[0], 1);
                     const int b = (int)(u / (R * P));
@@ -787,7 +777,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
                 //    leaving earlier would let the last sequences fall to very few CTAs.  The wait
                 //    cannot deadlock: a sequence is finalised by CTAs that already hold its units,
                 //    and those never wait for anyone.  It is bounded like every other wait.
-                if (acked && !again) {
+                if (!again) {
                     if (all_final) break;   // seen before the look above, so that look was complete
                     int fin = 0;
                     if (lane == 0) {
@@ -803,23 +793,6 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
                     fin = __shfl_sync(0xffffffffu, fin, 0);
                     if (fin < 0) { ok = false; break; }
                     if (fin > 0) { all_final = true; __threadfence(); }
-                }
-                if (!acked) {
-                    int st = 0;
-                    if (lane == 0) {
-                        Msg m{kMsgNone, 0, 0, 0};
-                        if (sm.jobs.try_pop(m)) st = 1;
-                        else if (sm.abort_flag) st = -1;
-                        else {
-                            const unsigned long long now = global_timer_ns();
-                            if (wait_t0 == 0) wait_t0 = now;
-                            else if (now - wait_t0 > kIdleLimitNs) { sm.abort_flag = 1; st = -1; }
-                            __nanosleep(100);
-                        }
-                    }
-                    st = __shfl_sync(0xffffffffu, st, 0);
-                    if (st < 0) { ok = false; break; }
-                    if (st > 0) acked = true;
                 }
             }
         }
@@ -875,66 +848,98 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
                 if (P > 1) row_done = ticket_add(&p.ticket_row[(size_t)b * R + rem / P]) == P - 1;
                 if (row_done && ticket_add(&p.ticket1[b]) == R - 1) last_b = b;  // last row of the sequence
             }
-            // what needs a whole warp (decisions, final pick) goes to the sequence warp, in order
+            // What needs a whole warp (decisions, final pick) goes to a global queue served by the
+            // sequence warps of all CTAs: the CTA that happens to deliver the last piece of many
+            // sequences (typically a slow one) must not also do all their epilogues.
             for (int i = 0; i < cnt && running; ++i) {
                 const int kind = __shfl_sync(0xffffffffu, m.kind, i);
                 const int a = __shfl_sync(0xffffffffu, m.a, i);
                 const int bb = __shfl_sync(0xffffffffu, m.b, i);
                 const int lb = __shfl_sync(0xffffffffu, last_b, i);
-                Msg fwd{kMsgNone, 0, 0, 0};
-                if (kind == kMsgPiece && lb >= 0) fwd = Msg{kMsgFinalize, lb, 0, 0};
-                else if (kind == kMsgJobPiece && lb >= 0) fwd = Msg{kMsgSelect, a, bb, 0};
-                else if (kind == kMsgDrain || kind == kMsgExit) fwd = Msg{kind, 0, 0, 0};
-                if (fwd.kind != kMsgNone) {
-                    int pushed = 1;
-                    if (lane == 0) pushed = sm.seq.push(fwd, &sm.abort_flag, kWaitLimitNs) ? 1 : 0;
-                    if (!__shfl_sync(0xffffffffu, pushed, 0)) running = false;
+                if ((kind == kMsgPiece || kind == kMsgJobPiece) && lb >= 0 && lane == 0) {
+                    const unsigned long long item = (1ull << 63) | ((unsigned long long)lb << 32) |
+                                                    (kind == kMsgPiece ? 0xffffffffull : (unsigned long long)(unsigned)bb);
+                    __threadfence();  // everything counted so far is visible before the item is
+                    const int slot = atomicAdd(&p.heads[4], 1);
+                    *reinterpret_cast<volatile unsigned long long*>(&p.wq[slot]) = item;
                 }
-                if (kind == kMsgExit) running = false;
+                if (kind == kMsgExit) {
+                    int pushed = 1;
+                    if (lane == 0) pushed = sm.seq.push(Msg{kMsgExit, 0, 0, 0}, &sm.abort_flag, kWaitLimitNs) ? 1 : 0;
+                    (void)__shfl_sync(0xffffffffu, pushed, 0);
+                    running = false;
+                }
             }
         }
     } else if (warp == kSequenceWarp) {
         // =============================== sequence warp: per-sequence decisions and the final pick
+        // Serves the global queue of sequence work (any CTA's sequences).  Leaves when its own
+        // CTA has wound down and nothing can be claimed: whatever a CTA's epilogue warp published
+        // was published before that CTA's exit message, so the publisher's own sequence warp at
+        // the latest picks it up.
+        bool exiting = false;
+        unsigned long long idle_t0 = 0;
         for (;;) {
-            Msg m{kMsgExit, 0, 0, 0};
-            int got = 0;
-            if (lane == 0) got = sm.seq.pop(m, &sm.abort_flag, kIdleLimitNs) ? 1 : 0;
-            got = __shfl_sync(0xffffffffu, got, 0);
-            if (!got) break;
-            m.kind = __shfl_sync(0xffffffffu, m.kind, 0);
-            m.a = __shfl_sync(0xffffffffu, m.a, 0);
-            m.b = __shfl_sync(0xffffffffu, m.b, 0);
-            if (m.kind == kMsgExit) break;
-            if (m.kind == kMsgFinalize) {
-                __threadfence();
-                const int n = finalize_sequence<E>(p, m.a, lane);
+            int kind = -1, b = 0, n = 0;   // kind 0: decide the sequence, 1: final pick after the second pass
+            if (lane == 0) {
+                Msg m{kMsgNone, 0, 0, 0};
+                if (!exiting && sm.seq.try_pop(m) && m.kind == kMsgExit) kind = 2;
+                if (kind < 0) {
+                    for (int tries = 0; tries < 64; ++tries) {
+                        const int h = *reinterpret_cast<volatile int*>(&p.heads[5]);
+                        if (h >= 2 * p.B) break;
+                        const unsigned long long e = *reinterpret_cast<volatile unsigned long long*>(&p.wq[h]);
+                        if (e == 0) break;                               // nothing published there (yet)
+                        if (atomicCAS(&p.heads[5], h, h + 1) == h) {
+                            b = (int)((e >> 32) & 0x7fffffffu);
+                            n = (int)(unsigned)e;
+                            kind = (unsigned)e == 0xffffffffu ? 0 : 1;
+                            break;
+                        }
+                    }
+                }
+                if (kind < 0 && sm.abort_flag) kind = 3;
+            }
+            kind = __shfl_sync(0xffffffffu, kind, 0);
+            if (kind == 3) break;
+            if (kind == 2) { exiting = true; continue; }
+            if (kind < 0) {
+                if (exiting) break;
+                if (lane == 0) {
+                    const unsigned long long now = global_timer_ns();
+                    if (idle_t0 == 0) idle_t0 = now;
+                    else if (now - idle_t0 > kIdleLimitNs) sm.abort_flag = 1;
+                    __nanosleep(300);
+                }
+                continue;
+            }
+            b = __shfl_sync(0xffffffffu, b, 0);
+            n = __shfl_sync(0xffffffffu, n, 0);
+            idle_t0 = 0;
+            __threadfence();
+            if (kind == 0) {
+                n = finalize_sequence<E>(p, b, lane);
                 if (n == K) {
                     // every draft accepted: the sums of the extra row are already there
                     __threadfence();
                     __syncwarp();
-                    select_token<E>(p, m.a, n, lane);
+                    select_token<E>(p, b, n, lane);
                 } else if (n >= 0) {
-                    // publish the sequence for the final-token pass; its row statistics first
+                    // publish the sequence for the second pass; its row statistics first
                     __threadfence();
                     __syncwarp();
                     if (lane == 0) {
                         const int slot = atomicAdd(&p.heads[3], 1);
                         *reinterpret_cast<volatile unsigned long long*>(&p.ready[slot]) =
-                            ((unsigned long long)(m.a + 1) << 32) | (unsigned)n;
+                            ((unsigned long long)(b + 1) << 32) | (unsigned)n;
                     }
                 }
                 if (lane == 0) {  // finalised (valid or not): lets idle CTAs know when to leave
                     __threadfence();
                     atomicAdd(&p.heads[1], 1);
                 }
-            } else if (m.kind == kMsgSelect) {
-                __threadfence();
-                select_token<E>(p, m.a, m.b, lane);
-            } else if (m.kind == kMsgDrain) {
-                // everything this CTA finalised is published by now
-                int pushed = 1;
-                if (lane == 0) pushed = sm.jobs.push(Msg{kMsgAck, 0, 0, 0}, &sm.abort_flag, kWaitLimitNs) ? 1 : 0;
-                if (!__shfl_sync(0xffffffffu, pushed, 0)) break;
+            } else {
+                select_token<E>(p, b, n, lane);
             }
         }
     } else {
@@ -950,12 +955,6 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
             if (mt.kind == kEnd) {
                 if (warp == 0 && lane == 0) sm.epi.push(Msg{kMsgExit, 0, 0, 0}, &sm.abort_flag, kWaitLimitNs);
                 break;
-            }
-            if (mt.kind == kDrain) {
-                if (warp == 0 && lane == 0) sm.epi.push(Msg{kMsgDrain, 0, 0, 0}, &sm.abort_flag, kWaitLimitNs);
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sm.empty[stage]);
-                continue;
             }
             if (mt.kind == kStats) {
                 if (mt.flags & 1) { m_run = -INFINITY; s[0] = s[1] = s[2] = s[3] = 0.f; }
