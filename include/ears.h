@@ -221,6 +221,28 @@ int ears_philox_device(const uint32_t* ctr_key, uint32_t* out, int n, void* stre
 int ears_set_plan(int loader, int parts);
 
 /*
+ * Choice between the two kernels, for tests and measurements (0 = automatic for both fields):
+ *   path 1 = streaming kernel (rows pass through a ring of shared-memory slots; the rows of a
+ *            rejected position are read a second time), 2 = resident kernel (the two rows of a
+ *            position stay in the shared memory of a thread-block cluster; every logit is read
+ *            once).  Forcing path 2 on a shape whose rows do not fit a cluster makes the
+ *            verification calls return EARS_ERR_SHAPE.  A non-zero `parts` of ears_set_plan
+ *            also selects the streaming kernel.
+ *   cluster = CTAs per cluster of the resident kernel: 1, 2, 4, 8 or 16.
+ * Both kernels implement the same step (Sec. 3.1-3.3); results differ only through
+ * floating-point summation order.
+ */
+int ears_set_path(int path, int cluster);
+
+/*
+ * Writes a one-line description of the launch plan a verification call with these sizes
+ * would use on the current device (which kernel, cluster size and slices or pieces per row,
+ * how many CTAs) into the HOST buffer `out` of `out_bytes` bytes (NUL-terminated, truncated
+ * if short).  Launches nothing.
+ */
+int ears_describe_plan(int dtype, int B, int K, int V, char* out, size_t out_bytes);
+
+/*
  * Device timing of the kernel for benchmarks.  After ears_profile_begin(max_calls) every
  * verification call (up to max_calls) records a CUDA event on its stream right before and
  * right after its kernel; nothing synchronises.  ears_profile_end waits for the last

@@ -9,12 +9,14 @@ from .binding import (  # noqa: F401
     DEV_INVALID_INPUT,
     DEV_TIMEOUT,
     EarsError,
+    describe_plan,
     last_device_status,
     load_library,
     philox_device,
     profile_begin,
     profile_end,
     selftest_bounded_wait,
+    set_path,
     set_plan,
     shutdown,
     verify,

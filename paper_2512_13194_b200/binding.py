@@ -59,6 +59,10 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ears_philox_device.restype = c.c_int
     lib.ears_set_plan.argtypes = [c.c_int, c.c_int]
     lib.ears_set_plan.restype = c.c_int
+    lib.ears_set_path.argtypes = [c.c_int, c.c_int]
+    lib.ears_set_path.restype = c.c_int
+    lib.ears_describe_plan.argtypes = [c.c_int, c.c_int, c.c_int, c.c_int, c.c_char_p, c.c_size_t]
+    lib.ears_describe_plan.restype = c.c_int
     lib.ears_profile_begin.argtypes = [c.c_int]
     lib.ears_profile_begin.restype = c.c_int
     lib.ears_profile_end.argtypes = [c.c_void_p, c.c_int, c.POINTER(c.c_int)]
@@ -250,6 +254,18 @@ def philox_device(ctr_key: torch.Tensor) -> torch.Tensor:
 
 def set_plan(loader: int = 0, parts: int = 0) -> None:
     _check(load_library().ears_set_plan(loader, parts))
+
+
+def set_path(path: int = 0, cluster: int = 0) -> None:
+    """0 = automatic; path 1 streaming kernel, 2 resident (cluster) kernel; cluster = CTAs per cluster."""
+    _check(load_library().ears_set_path(path, cluster))
+
+
+def describe_plan(dtype: str, B: int, K: int, V: int) -> str:
+    """The launch plan a call with these sizes would use on the current device ("fp32" or "bf16")."""
+    buf = ctypes.create_string_buffer(256)
+    _check(load_library().ears_describe_plan(0 if dtype == "fp32" else 1, B, K, V, buf, len(buf)))
+    return buf.value.decode()
 
 
 def profile_begin(max_calls: int) -> None:

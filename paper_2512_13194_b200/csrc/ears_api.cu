@@ -12,6 +12,7 @@
 
 #include "ears_common.cuh"
 #include "ears_kernel.cuh"
+#include "ears_resident.cuh"
 
 namespace {
 
@@ -33,11 +34,16 @@ int cuda_fail(cudaError_t e, const char* what) {
         if (e_ != cudaSuccess) return cuda_fail(e_, #call); \
     } while (0)
 
-struct PlanOverride { int loader = 0, parts1 = 0; };
+struct PlanOverride { int loader = 0, parts1 = 0, path = 0, cluster = 0; };
 PlanOverride g_override;
 std::mutex g_mutex;
 
-struct DeviceInfo { int sms = 0; bool attrs_set = false; };
+struct DeviceInfo {
+    int sms = 0;
+    bool attrs_set = false;
+    bool cluster16 = false;                        // clusters of 16 CTAs may be launched
+    std::map<std::pair<int, int>, int> clusters;   // (cluster size, shared memory, element size) -> co-resident clusters
+};
 std::map<int, DeviceInfo> g_devices;
 
 struct Buffer { void* ptr = nullptr; size_t bytes = 0; };
@@ -125,6 +131,54 @@ Layout make_layout(int B, int K, int V, int parts1) {
     return L;
 }
 
+// ---- the resident path: one position's rows held in the shared memory of a cluster ----
+struct RPlan { bool ok = false; int C = 0, slice = 0, buf_bytes = 0; size_t smem = 0; bool roomy = false; };
+
+size_t resident_smem(int buf_bytes) { return ((sizeof(RSmem) + 127) & ~size_t(127)) + 2 * (size_t)buf_bytes + 128; }
+
+// Three CTAs per SM (74 KB each) when the slices allow it, else two (113 KB each); a pair of
+// rows that does not fit a cluster that way goes to the streaming kernel.
+constexpr size_t kResidentSmem3 = 74 * 1024, kResidentSmem2 = 113 * 1024;
+
+RPlan make_rplan(int B, int K, int V, int esize, int sms, int max_cluster, int forced_cluster) {
+    RPlan best;
+    const long long items = (long long)B * (K + 1);
+    for (int pass = 0; pass < 2 && !best.ok; ++pass) {
+        const size_t cap = pass == 0 ? kResidentSmem3 : kResidentSmem2;
+        for (int C = 1; C <= max_cluster; C *= 2) {
+            if (forced_cluster > 0 && C != forced_cluster) continue;
+            const int slice = (int)align_up((size_t)((V + C - 1) / C), kSegElems);
+            const int buf = (int)align_up((size_t)slice * esize, kRSubBytes);
+            if (buf > kRMaxSub * kRSubBytes || resident_smem(buf) > cap) continue;
+            if (best.ok && items * best.C >= 2LL * sms) break;   // enough CTAs already: keep the slices large
+            best.ok = true; best.C = C; best.slice = slice; best.buf_bytes = buf; best.smem = resident_smem(buf);
+            best.roomy = pass == 0;
+        }
+    }
+    return best;
+}
+
+struct RLayout { size_t heads, ticket, counters_bytes, flag, cand, cand_mass, pt_tok, pd_tok, max_pt, cls, resid, total; };
+
+RLayout make_rlayout(int B, int K) {
+    RLayout L;
+    size_t o = 0;
+    L.heads = o; o += 32;   // the status word is heads[2] of any workspace
+    L.ticket = o; o += (size_t)B * 4;
+    L.counters_bytes = o;
+    o = align_up(o, 256);
+    L.flag = o; o = align_up(o + (size_t)B * (K + 1), 256);
+    L.cand = o; o = align_up(o + (size_t)B * (K + 1) * 4, 256);
+    L.cand_mass = o; o = align_up(o + (size_t)B * (K + 1) * 8, 256);
+    L.pt_tok = o; o = align_up(o + (size_t)B * K * 8, 256);
+    L.pd_tok = o; o = align_up(o + (size_t)B * K * 8, 256);
+    L.max_pt = o; o = align_up(o + (size_t)B * K * 8, 256);
+    L.cls = o; o = align_up(o + (size_t)B * K, 256);
+    L.resid = o; o = align_up(o + (size_t)B * 8, 256);
+    L.total = o;
+    return L;
+}
+
 int check_shape(int B, int K, int V) {
     if (B < 1 || K < 1 || V < 1) return EARS_ERR_SHAPE;
     if (K > EARS_MAX_K || V > (1 << 30)) return EARS_ERR_SHAPE;
@@ -149,13 +203,6 @@ int device_info(int dev, DeviceInfo** out) {
 
 size_t smem_bytes() { return sizeof(PipeSmem<kStages>) + 128; }
 
-template <typename E>
-int set_attrs() {
-    EARS_CUDA(cudaFuncSetAttribute(ears_verify_kernel<E, kStages>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   (int)smem_bytes()));
-    return EARS_OK;
-}
-
 int profile_mark(cudaStream_t stream, bool timed) {
     if (!timed) return EARS_OK;
     cudaEvent_t ev;
@@ -163,6 +210,73 @@ int profile_mark(cudaStream_t stream, bool timed) {
     g_profile.events.push_back(ev);
     EARS_CUDA(cudaEventRecord(ev, stream));
     return EARS_OK;
+}
+
+template <typename E>
+int set_attrs(bool* cluster16) {
+    EARS_CUDA(cudaFuncSetAttribute(ears_verify_kernel<E, kStages>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)smem_bytes()));
+    EARS_CUDA(cudaFuncSetAttribute(ears_resident_kernel<E>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)kResidentSmem2));
+    // several CTAs per SM only fit when the SM's memory is configured as shared memory
+    EARS_CUDA(cudaFuncSetAttribute(ears_resident_kernel<E>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                   (int)cudaSharedmemCarveoutMaxShared));
+    // clusters of more than 8 CTAs are an opt-in; without it the plans stop at 8
+    if (cudaFuncSetAttribute(ears_resident_kernel<E>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
+        (void)cudaGetLastError();
+        *cluster16 = false;
+    }
+    return EARS_OK;
+}
+
+// How many clusters of this shape the device can hold at once (cached per device).
+template <typename E>
+int resident_clusters(DeviceInfo* di, const RPlan& rp, int* out) {
+    const std::pair<int, int> key(rp.C * 8 + (int)sizeof(E), (int)rp.smem);
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        auto it = di->clusters.find(key);
+        if (it != di->clusters.end()) { *out = it->second; return EARS_OK; }
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(rp.C * di->sms), 1, 1);
+    cfg.blockDim = dim3(kRThreads, 1, 1);
+    cfg.dynamicSmemBytes = rp.smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)rp.C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, ears_resident_kernel<E>, &cfg) != cudaSuccess) {
+        (void)cudaGetLastError();
+        n = 0;
+    }
+    std::lock_guard<std::mutex> lock(g_mutex);
+    di->clusters[key] = n;
+    *out = n;
+    return EARS_OK;
+}
+
+template <typename E>
+int launch_resident(RParams& p, const RPlan& rp, int max_clusters, cudaStream_t stream) {
+    const long long items = (long long)p.B * (p.K + 1);
+    p.n_clusters = (int)(items < max_clusters ? items : max_clusters);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(p.n_clusters * rp.C), 1, 1);
+    cfg.blockDim = dim3(kRThreads, 1, 1);
+    cfg.dynamicSmemBytes = rp.smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)rp.C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const bool timed = g_profile.active && (int)g_profile.events.size() + 2 <= 2 * g_profile.max_calls;
+    int rc = profile_mark(stream, timed);
+    if (rc) return rc;
+    EARS_CUDA(cudaLaunchKernelEx(&cfg, ears_resident_kernel<E>, p));
+    return profile_mark(stream, timed);
 }
 
 template <typename E>
@@ -197,6 +311,46 @@ int get_buffer(std::map<std::pair<int, void*>, Buffer>& pool, int dev, void* str
     return EARS_OK;
 }
 
+// The resident plan for this shape, if its rows fit a cluster and the device can hold one.
+int choose_resident(int dtype, int B, int K, int V, DeviceInfo* di, const PlanOverride& ov, RPlan* rp, int* max_clusters) {
+    *rp = RPlan();
+    *max_clusters = 0;
+    if (ov.path == 1 || ov.parts1 != 0) return EARS_OK;
+    const int esize = dtype == EARS_DTYPE_F32 ? 4 : 2;
+    *rp = make_rplan(B, K, V, esize, di->sms, di->cluster16 ? kRMaxCluster : 8, ov.cluster);
+    if (rp->ok && ov.path == 0) {
+        // Holding rows in shared memory costs a few microseconds of latency per position that
+        // nothing else in that CTA can hide.  It wins when rows are short (a cluster of at most
+        // four CTAs holds a pair) and when there are few positions, where the streaming kernel's
+        // second pass and its queues dominate; long rows in large batches stream faster.
+        // Measured on B200 (B, K, V, dtype: us resident / streaming): 8,5,32000,bf16: 20 / 47;
+        // 4096,5,32000,bf16: 976 / 2624; 32,7,128256,bf16: 72 / 75; 128,4,152064,bf16: 195 / 148.
+        const long long items = (long long)B * (K + 1);
+        const long long limit = !rp->roomy ? 64 : (rp->C >= 8 ? 256 : (1LL << 62));
+        if (items > limit) rp->ok = false;
+    }
+    if (rp->ok) {
+        const int rc = dtype == EARS_DTYPE_F32 ? resident_clusters<float>(di, *rp, max_clusters)
+                                               : resident_clusters<uint16_t>(di, *rp, max_clusters);
+        if (rc) return rc;
+        if (*max_clusters < 1) rp->ok = false;
+    }
+    if (!rp->ok && ov.path == 2) return EARS_ERR_SHAPE;   // the forced path cannot take this shape
+    return EARS_OK;
+}
+
+int ensure_attrs(DeviceInfo* di) {
+    if (di->attrs_set) return EARS_OK;
+    bool c16 = true;
+    int rc = set_attrs<float>(&c16);
+    if (rc) return rc;
+    rc = set_attrs<uint16_t>(&c16);
+    if (rc) return rc;
+    di->cluster16 = c16;
+    di->attrs_set = true;
+    return EARS_OK;
+}
+
 int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B, int K, int V,
                 float temperature, float beta, uint64_t seed, uint64_t offset, int64_t b_first,
                 int32_t* out_len, int32_t* out_tok, double* o_pt, double* o_pd, double* o_max,
@@ -219,13 +373,8 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
     DeviceInfo* di = nullptr;
     rc = device_info(dev, &di);
     if (rc) return rc;
-    if (!di->attrs_set) {
-        rc = set_attrs<float>();
-        if (rc) return rc;
-        rc = set_attrs<uint16_t>();
-        if (rc) return rc;
-        di->attrs_set = true;
-    }
+    rc = ensure_attrs(di);
+    if (rc) return rc;
 
     const bool aligned = ((uintptr_t)t % 16 == 0) && ((uintptr_t)d % 16 == 0) && (((size_t)V * esize) % 16 == 0);
     PlanOverride ov;
@@ -233,6 +382,49 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
         std::lock_guard<std::mutex> lock(g_mutex);
         ov = g_override;
     }
+    const float c = (float)(1.4426950408889634 / (double)temperature);
+
+    // Rows small enough to stay in a cluster's shared memory take the resident path.
+    RPlan rp;
+    int max_clusters = 0;
+    rc = choose_resident(dtype, B, K, V, di, ov, &rp, &max_clusters);
+    if (rc) return rc;
+    if (rp.ok) {
+        const RLayout L = make_rlayout(B, K);
+        if (workspace) {
+            if (workspace_bytes < L.total) return EARS_ERR_WORKSPACE;
+        } else {
+            rc = get_buffer(g_workspaces, dev, stream_, L.total, &workspace);
+            if (rc) return rc;
+        }
+        char* w = (char*)workspace;
+        EARS_CUDA(cudaMemsetAsync(w, 0, L.counters_bytes, stream));
+        RParams p;
+        p.t = t; p.d = d; p.x = x;
+        p.B = B; p.K = K; p.V = V;
+        p.c = c;
+        p.T = (double)temperature;
+        p.beta = (double)beta;
+        p.seed = seed; p.offset = offset; p.b_first = b_first;
+        p.out_len = out_len; p.out_tok = out_tok;
+        p.pt_tok = o_pt ? o_pt : (double*)(w + L.pt_tok);
+        p.pd_tok = o_pd ? o_pd : (double*)(w + L.pd_tok);
+        p.max_pt = o_max ? o_max : (double*)(w + L.max_pt);
+        p.cls = o_cls ? o_cls : (uint8_t*)(w + L.cls);
+        p.resid = o_resid ? o_resid : (double*)(w + L.resid);
+        p.heads = (int*)(w + L.heads);
+        p.ticket = (int*)(w + L.ticket);
+        p.flag = (signed char*)(w + L.flag);
+        p.cand = (int32_t*)(w + L.cand);
+        p.cand_mass = (double*)(w + L.cand_mass);
+        p.C = rp.C; p.slice = rp.slice; p.buf_bytes = rp.buf_bytes;
+        p.use_tma = aligned && ov.loader != 2;
+        p.n_clusters = 0;
+        p.want_stats = (o_pt || o_pd || o_max || o_cls) ? 1 : 0;
+        return dtype == EARS_DTYPE_F32 ? launch_resident<float>(p, rp, max_clusters, stream)
+                                       : launch_resident<uint16_t>(p, rp, max_clusters, stream);
+    }
+
     const Plan plan = make_plan(B, K, V, esize, aligned, di->sms, ov);
     const Layout L = make_layout(B, K, V, plan.parts1);
     if (workspace) {
@@ -247,7 +439,7 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
     Params p;
     p.t = t; p.d = d; p.x = x;
     p.B = B; p.K = K; p.V = V;
-    p.c = (float)(1.4426950408889634 / (double)temperature);
+    p.c = c;
     p.T = (double)temperature;
     p.beta = (double)beta;
     p.seed = seed; p.offset = offset; p.b_first = b_first;
@@ -288,7 +480,8 @@ size_t workspace_bound(int B, int K, int V) {
             const size_t tot = make_layout(B, K, V, pl.parts1).total;
             if (tot > best) best = tot;
         }
-    return best;
+    const size_t res = make_rlayout(B, K).total;
+    return res > best ? res : best;
 }
 
 // Scratch of the allocation-free entry point.  Part of the library image: each GPU that
@@ -492,6 +685,53 @@ int ears_set_plan(int loader, int parts) {
     std::lock_guard<std::mutex> lock(g_mutex);
     g_override.loader = loader;
     g_override.parts1 = parts;
+    return EARS_OK;
+}
+
+int ears_describe_plan(int dtype, int B, int K, int V, char* out, size_t out_bytes) {
+    if (!out || out_bytes == 0) return EARS_ERR_NULL;
+    if (dtype != EARS_DTYPE_F32 && dtype != EARS_DTYPE_BF16) return EARS_ERR_PARAM;
+    int rc = check_shape(B, K, V);
+    if (rc) return rc;
+    int dev = 0;
+    EARS_CUDA(cudaGetDevice(&dev));
+    DeviceInfo* di = nullptr;
+    rc = device_info(dev, &di);
+    if (rc) return rc;
+    rc = ensure_attrs(di);
+    if (rc) return rc;
+    PlanOverride ov;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        ov = g_override;
+    }
+    RPlan rp;
+    int max_clusters = 0;
+    rc = choose_resident(dtype, B, K, V, di, ov, &rp, &max_clusters);
+    if (rc) return rc;
+    const int esize = dtype == EARS_DTYPE_F32 ? 4 : 2;
+    if (rp.ok) {
+        const long long items = (long long)B * (K + 1);
+        int per_sm = 0;
+        if (dtype == EARS_DTYPE_F32) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ears_resident_kernel<float>, kRThreads, rp.smem);
+        else cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ears_resident_kernel<uint16_t>, kRThreads, rp.smem);
+        snprintf(out, out_bytes, "resident: cluster=%d slice_elems=%d smem_bytes=%zu ctas_per_sm=%d clusters_resident=%d clusters_launched=%lld",
+                 rp.C, rp.slice, rp.smem, per_sm, max_clusters, items < max_clusters ? items : (long long)max_clusters);
+    } else {
+        const Plan pl = make_plan(B, K, V, esize, true, di->sms, ov);
+        const long long units = (long long)B * (2 * K + 1) * pl.parts1, cap = (long long)di->sms * kCtasPerSm;
+        snprintf(out, out_bytes, "streaming: pieces_per_row=%d chunks_per_piece=%d ctas=%lld second_pass_pieces=%d",
+                 pl.parts1, pl.cpp1, units < cap ? units : cap, pl.parts2);
+    }
+    return EARS_OK;
+}
+
+int ears_set_path(int path, int cluster) {
+    if (path < 0 || path > 2) return EARS_ERR_PARAM;
+    if (cluster != 0 && cluster != 1 && cluster != 2 && cluster != 4 && cluster != 8 && cluster != 16) return EARS_ERR_PARAM;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    g_override.path = path;
+    g_override.cluster = cluster;
     return EARS_OK;
 }
 

@@ -27,6 +27,7 @@
 #include "ears_common.cuh"
 #include "ears_philox.cuh"
 #include "ears_pipeline.cuh"
+#include "ears_math.cuh"
 
 namespace ears {
 
@@ -214,28 +215,6 @@ __device__ __forceinline__ void loader_fill(PipeSmem<STAGES>& sm, int stage, con
 }
 
 // ---- consumer arithmetic --------------------------------------------------------
-template <typename E> struct Vec;
-template <> struct Vec<float> {
-    static constexpr int N = 4;
-    __device__ static __forceinline__ void load(const unsigned char* buf, int vec_index, float (&x)[4]) {
-        float4 v = reinterpret_cast<const float4*>(buf)[vec_index];
-        x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
-    }
-};
-template <> struct Vec<uint16_t> {
-    static constexpr int N = 8;
-    __device__ static __forceinline__ void load(const unsigned char* buf, int vec_index, float (&x)[8]) {
-        uint4 v = reinterpret_cast<const uint4*>(buf)[vec_index];
-        x[0] = __uint_as_float(v.x << 16); x[1] = __uint_as_float(v.x & 0xffff0000u);
-        x[2] = __uint_as_float(v.y << 16); x[3] = __uint_as_float(v.y & 0xffff0000u);
-        x[4] = __uint_as_float(v.z << 16); x[5] = __uint_as_float(v.z & 0xffff0000u);
-        x[6] = __uint_as_float(v.w << 16); x[7] = __uint_as_float(v.w & 0xffff0000u);
-    }
-};
-
-__device__ __forceinline__ float load_logit(const float* p) { return __ldg(p); }
-__device__ __forceinline__ float load_logit(const uint16_t* p) { return bf16_bits_to_float(__ldg(p)); }
-
 // Running (m, s) of one thread over its share of a staged chunk:
 // s = sum exp2((l - m) * c), m = running maximum; s is rescaled when m grows.
 // Warp w owns the w-th eighth of the slot (contiguous), lane-interleaved in 16-byte vectors.
@@ -293,40 +272,6 @@ __device__ __forceinline__ void chunk_stats(const unsigned char* buf, int nelem,
         for (int off = 16; off > 0; off >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, off);
         if (lane == 0) *warp_chunk_out = BonusSeg{tot, m_run, 0.f};   // m_run is warp-uniform here
     }
-}
-
-struct RowNorm {
-    float mt, md;          // row maxima
-    float rho_hi, rho_lo;  // Z_t / Z_d split in two floats (residual rows)
-    double izt;            // 1 / Z_t
-};
-
-__device__ __forceinline__ RowNorm make_rownorm(float2 st, float2 sd) {
-    const double rho = (double)st.y / (double)sd.y;
-    const float hi = (float)rho;
-    return RowNorm{st.x, sd.x, hi, (float)(rho - (double)hi), 1.0 / (double)st.y};
-}
-
-// Mass of one vocabulary entry for the final draw in units of 1/Z_t:
-// Z_t P_t(v), or Z_t max(0, P_t(v) - P_d(v)) = max(0, e_t - e_d Z_t/Z_d).  The common factor
-// cancels in the inverse-CDF draw.  fp32 with the ratio carried as hi + lo so that no
-// systematic rounding of Z_t/Z_d tilts the residual; explicit rounding intrinsics so that the
-// streaming pass and the in-segment pass produce identical bits.
-template <bool RESID>
-__device__ __forceinline__ float entry_mass(float xt, float xd, const RowNorm& rn, float c) {
-    const float et = ex2_approx(__fmul_rn(__fsub_rn(xt, rn.mt), c));
-    if (!RESID) return et;
-    const float ed = ex2_approx(__fmul_rn(__fsub_rn(xd, rn.md), c));
-    return fmaxf(__fmaf_rn(-ed, rn.rho_lo, __fmaf_rn(-ed, rn.rho_hi, et)), 0.0f);
-}
-
-__device__ __forceinline__ double warp_inclusive_scan(double v, int lane) {
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        double t = __shfl_up_sync(0xffffffffu, v, off);
-        if (lane >= off) v += t;
-    }
-    return v;
 }
 
 // Sums of kSegElems-element segments of a staged chunk; warp w takes segments w, w+8, ...
@@ -405,7 +350,7 @@ __device__ int finalize_sequence(const Params& p, int b, int lane) {
             float2 v = __ldcg(pp + i);
             merge_ms(m, s, v.x, v.y, p.c);
         }
-        if (!(m > -INFINITY && m < INFINITY && s > 0.0f && s < INFINITY)) bad = true;  // NaN fails too
+        if (!rowstat_ok(m, s)) bad = true;
         p.rowstat[(size_t)b * R + r] = make_float2(m, s);
     }
     __syncwarp();
@@ -422,20 +367,14 @@ __device__ int finalize_sequence(const Params& p, int b, int lane) {
                 const float2 sd = __ldcg(&p.rowstat[(size_t)b * R + 2 * k + 1]);
                 const double lt = (double)load_logit(t + (size_t)target_row(b, k, K) * V + tok);
                 const double ld = (double)load_logit(d + (size_t)draft_row(b, k, K) * V + tok);
-                const double pt = exp((lt - (double)st.x) / p.T) / (double)st.y;
-                const double pd = exp((ld - (double)sd.x) / p.T) / (double)sd.y;
-                const double maxp = 1.0 / (double)st.y;                 // the largest term of Z is exp(0)
-                const double ratio = pt / fmax(pd, kEps);               // R_k with the division guard
-                const double tol = p.beta * (1.0 - maxp);               // Tolerance_k
                 const double U = uniform_accept(p.seed, p.offset, (uint32_t)(p.b_first + b), (uint32_t)k);
-                const double thr = fmax(U - tol, 0.0);                  // clamped threshold
-                const bool accept = ratio >= thr;
-                reject = !accept;
+                const Decision dc = decide_position(lt, ld, st, sd, p.T, p.beta, U);
+                reject = !dc.accept;
                 const size_t i = (size_t)b * K + k;
-                p.pt_tok[i] = pt;
-                p.pd_tok[i] = pd;
-                p.max_pt[i] = maxp;
-                p.cls[i] = ratio >= U ? 1 : (accept ? 2 : 0);
+                p.pt_tok[i] = dc.pt;
+                p.pd_tok[i] = dc.pd;
+                p.max_pt[i] = dc.maxp;
+                p.cls[i] = dc.cls;
             }
         }
         const unsigned rej = __ballot_sync(0xffffffffu, reject);
