@@ -32,9 +32,9 @@ UNIT = "rows/s"
 DATASHEET_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of ears_verify_kernel<float,6> from one ncu capture on
-# a 96-sequence batch of the default workload (690.71 MB + 4.45 MB), per sequence.  The traffic grows
+# a 96-sequence batch of the default workload (690.86 MB + 4.46 MB), per sequence.  The traffic grows
 # in proportion to the number of sequences; set to None whenever the kernel changes after a capture.
-NCU_DRAM_BYTES_PER_SEQUENCE = None  # kernel changed since the last capture (was (690710272 + 4452608) / 96)
+NCU_DRAM_BYTES_PER_SEQUENCE = (690858496 + 4463104) / 96
 
 
 def measured_peak():
@@ -183,6 +183,8 @@ def run_ours(args):
     rs_formula, rs_again = final_token_bytes(acc, K, V, esize)
     step_bytes = logits_bytes + rs_formula
     k_avg = statistics.fmean(kernel_ms)
+    plan = ears.describe_plan(w.dtype, w.B, K, V)
+    kernel_name = "ears_resident_kernel" if plan.startswith("resident") else "ears_verify_kernel"
     peak, peak_kind = measured_peak()
     # algorithmic HBM bytes of the kernel: every logit once.  The rows of the final token are a second
     # pass over bytes already counted (normally served by L2), so they are left out of the roofline.
@@ -225,12 +227,12 @@ def run_ours(args):
                        "temperature": w.temperature, "beta": w.beta, "parallelism": f"batch-shard x{world}",
                        "l2": "inputs (3.67 GB at the default workload) exceed L2; no flush needed"
                              if logits_bytes > 512e6 else "inputs fit L2: warm-cache number",
-                       "mean_accept_len": float(acc.float().mean().item())},
+                       "mean_accept_len": float(acc.float().mean().item()), "launch_plan": plan},
             "gbs_step_formula": step_bytes / (ms_step * 1e-3) / 1e9,
             "bytes_per_step": {"logits": logits_bytes, "final_token_rows_formula": rs_formula,
                                "final_token_rows_streamed_again": rs_again},
-            "kernel_ms": {"ears_verify_kernel": k_avg, "median": statistics.median(kernel_ms), "min": min(kernel_ms)},
-            "roofline": {"bound": "hbm", "kernel": "ears_verify_kernel", "achieved": achieved, "peak": peak,
+            "kernel_ms": {kernel_name: k_avg, "median": statistics.median(kernel_ms), "min": min(kernel_ms)},
+            "roofline": {"bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                          "frac_of_datasheet_8000": achieved / DATASHEET_HBM_GBS,
                          "traffic": (NCU_DRAM_BYTES_PER_SEQUENCE * w.B
