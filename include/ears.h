@@ -130,6 +130,29 @@ int ears_verify_ex(int dtype, const void* target_logits, const void* draft_logit
                    void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * ears_verify_ex with a temperature and a base tolerance per sequence.  Sec. 3.3 item 3 verifies
+ * all active sequences side by side and independently, and in a serving batch each request brings
+ * its own sampling temperature (Sec. 4.3 discusses its effect on the tolerance) and possibly its
+ * own beta (Sec. 3.2); the paper states both as scalars.
+ *   seq_temperature, seq_beta   DEVICE arrays [B] of float, either may be NULL.  Where given,
+ *               sequence b uses seq_temperature[b] / seq_beta[b] and the scalar argument of the
+ *               same name is ignored; where NULL the scalar applies to every sequence.
+ *   A value the scalar form would refuse (temperature not finite or <= 0, beta not finite or
+ *   < 0) cannot be seen by the host: it marks that one sequence invalid (out_accept_len = -1,
+ *   tokens -1, EARS_DEV_INVALID_INPUT), the others are unaffected.
+ * Everything else is as in ears_verify_ex.
+ */
+int ears_verify_var(int dtype, const void* target_logits, const void* draft_logits,
+                    const int32_t* draft_tokens, int B, int K, int V,
+                    float temperature, float beta,
+                    const float* seq_temperature, const float* seq_beta,
+                    uint64_t seed, uint64_t offset,
+                    int64_t b_first, int32_t* out_accept_len, int32_t* out_tokens,
+                    double* out_pt_tok, double* out_pd_tok, double* out_max_pt,
+                    uint8_t* out_class, double* out_resid_mass,
+                    void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Same step with HOST buffers: copies the inputs to library-owned device staging
  * buffers, runs the step, copies out_accept_len / out_tokens back and waits for
  * completion.  All pointers are host memory (pinned memory makes the copies

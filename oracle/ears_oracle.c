@@ -281,22 +281,25 @@ static void verify_one(const void* tl, const void* dl, int dtype, const int32_t*
  *   out_tokens [B,K+1] (n accepted draft tokens, then the resampled or bonus
  *   token, then -1).  Any diagnostic pointer may be NULL.
  * nthreads > 1 spreads sequences over OpenMP threads; results do not depend on it.
+ * seq_temperature, seq_beta: optional [B] arrays that replace the scalars per sequence.
  * Returns 0, -1 on bad arguments, -2 when out of memory.
  */
-int ears_oracle_verify(const void* target_logits, const void* draft_logits, int dtype,
-                       const int32_t* draft_tokens, int B, int K, int V,
-                       float temperature, float beta, uint64_t seed, uint64_t offset,
-                       int64_t b_first, double band,
-                       int32_t* out_accept_len, int32_t* out_tokens,
-                       double* pt_tok, double* pd_tok, double* max_pt, double* margin,
-                       uint8_t* cls, double* resid_mass, double* cdf_margin,
-                       int32_t* band_lo, int32_t* band_hi, int nthreads)
+int ears_oracle_verify_var(const void* target_logits, const void* draft_logits, int dtype,
+                           const int32_t* draft_tokens, int B, int K, int V,
+                           float temperature, float beta,
+                           const float* seq_temperature, const float* seq_beta,
+                           uint64_t seed, uint64_t offset,
+                           int64_t b_first, double band,
+                           int32_t* out_accept_len, int32_t* out_tokens,
+                           double* pt_tok, double* pd_tok, double* max_pt, double* margin,
+                           uint8_t* cls, double* resid_mass, double* cdf_margin,
+                           int32_t* band_lo, int32_t* band_hi, int nthreads)
 {
     if (!target_logits || !draft_logits || !draft_tokens || !out_accept_len || !out_tokens) return -1;
     if (B < 1 || K < 1 || V < 1 || (dtype != 0 && dtype != 1)) return -1;
-    if (!(temperature > 0.0f) || !isfinite(temperature) || !(beta >= 0.0f) || !isfinite(beta)) return -1;
+    if (!seq_temperature && (!(temperature > 0.0f) || !isfinite(temperature))) return -1;
+    if (!seq_beta && (!(beta >= 0.0f) || !isfinite(beta))) return -1;
     ears_oracle_diag dg = { pt_tok, pd_tok, max_pt, margin, cls, resid_mass, cdf_margin, band_lo, band_hi };
-    double T = (double)temperature, bt = (double)beta;
     if (nthreads < 1) nthreads = 1;
     int failed = 0;
 #ifdef _OPENMP
@@ -317,13 +320,38 @@ int ears_oracle_verify(const void* target_logits, const void* draft_logits, int 
 #pragma omp for schedule(dynamic, 1)
 #endif
         for (int b = 0; b < B; ++b) {
-            if (!failed)
-                verify_one(target_logits, draft_logits, dtype, draft_tokens, b, K, V, T, bt,
-                           seed, offset, b_first, band, out_accept_len, out_tokens, &dg, row, pt, pd);
+            if (failed) continue;
+            /* Every sequence is verified on its own [Sec. 3.3 item 3], so each may carry its own
+             * temperature [Sec. 4.3] and base tolerance beta [Sec. 3.2]; a value that the scalar
+             * form would refuse makes that one sequence invalid. */
+            float Tb = seq_temperature ? seq_temperature[b] : temperature;
+            float bb = seq_beta ? seq_beta[b] : beta;
+            if (!(Tb > 0.0f) || !isfinite(Tb) || !(bb >= 0.0f) || !isfinite(bb)) {
+                mark_invalid(b, K, out_accept_len, out_tokens);
+                continue;
+            }
+            verify_one(target_logits, draft_logits, dtype, draft_tokens, b, K, V, (double)Tb, (double)bb,
+                       seed, offset, b_first, band, out_accept_len, out_tokens, &dg, row, pt, pd);
         }
         free(row); free(pt); free(pd);
     }
     return failed ? -2 : 0;
+}
+
+/* The same with one temperature and one beta for the whole batch. */
+int ears_oracle_verify(const void* target_logits, const void* draft_logits, int dtype,
+                       const int32_t* draft_tokens, int B, int K, int V,
+                       float temperature, float beta, uint64_t seed, uint64_t offset,
+                       int64_t b_first, double band,
+                       int32_t* out_accept_len, int32_t* out_tokens,
+                       double* pt_tok, double* pd_tok, double* max_pt, double* margin,
+                       uint8_t* cls, double* resid_mass, double* cdf_margin,
+                       int32_t* band_lo, int32_t* band_hi, int nthreads)
+{
+    return ears_oracle_verify_var(target_logits, draft_logits, dtype, draft_tokens, B, K, V, temperature, beta,
+                                  NULL, NULL, seed, offset, b_first, band, out_accept_len, out_tokens,
+                                  pt_tok, pd_tok, max_pt, margin, cls, resid_mass, cdf_margin,
+                                  band_lo, band_hi, nthreads);
 }
 
 /* Softmax of one stored row, for tests that need the full distribution. */

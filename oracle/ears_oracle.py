@@ -52,6 +52,11 @@ def _load():
          c.c_float, c.c_float, c.c_uint64, c.c_uint64, c.c_int64, c.c_double]
         + [c.c_void_p] * 11 + [c.c_int])
     lib.ears_oracle_verify.restype = c.c_int
+    lib.ears_oracle_verify_var.argtypes = (
+        [c.c_void_p, c.c_void_p, c.c_int, c.c_void_p, c.c_int, c.c_int, c.c_int,
+         c.c_float, c.c_float, c.c_void_p, c.c_void_p, c.c_uint64, c.c_uint64, c.c_int64, c.c_double]
+        + [c.c_void_p] * 11 + [c.c_int])
+    lib.ears_oracle_verify_var.restype = c.c_int
     lib.ears_oracle_row_softmax.argtypes = [c.c_void_p, c.c_int, c.c_int64, c.c_int, c.c_float, c.c_void_p]
     lib.ears_oracle_row_softmax.restype = c.c_int
     lib.ears_oracle_max_threads.argtypes = []
@@ -159,7 +164,8 @@ class OracleResult:
 
 def verify(target_logits, draft_logits, draft_tokens, temperature: float, beta: float,
            seed: int = 0, offset: int = 0, b_first: int = 0, band: float = 1e-6,
-           nthreads: int = 1) -> OracleResult:
+           nthreads: int = 1, seq_temperature=None, seq_beta=None) -> OracleResult:
+    """seq_temperature / seq_beta: optional [B] float32 arrays replacing the scalars per sequence."""
     lib = _load()
     t, ct = _as_logits(target_logits)
     d, cd = _as_logits(draft_logits)
@@ -175,9 +181,14 @@ def verify(target_logits, draft_logits, draft_tokens, temperature: float, beta: 
     f = lambda *s: np.zeros(s, np.float64)
     res = OracleResult(acc, tok, f(B, K), f(B, K), f(B, K), f(B, K), np.zeros((B, K), np.uint8),
                        f(B), f(B), np.full(B, -1, np.int32), np.full(B, -1, np.int32))
-    rc = lib.ears_oracle_verify(
+    st = None if seq_temperature is None else np.ascontiguousarray(np.asarray(seq_temperature, dtype=np.float32))
+    sb = None if seq_beta is None else np.ascontiguousarray(np.asarray(seq_beta, dtype=np.float32))
+    if (st is not None and st.shape != (B,)) or (sb is not None and sb.shape != (B,)):
+        raise ValueError("per-sequence arrays must have shape [B]")
+    rc = lib.ears_oracle_verify_var(
         t.ctypes.data, d.ctypes.data, ct, x.ctypes.data, B, K, V,
-        float(temperature), float(beta), int(seed), int(offset), int(b_first), float(band),
+        float(temperature), float(beta), None if st is None else st.ctypes.data,
+        None if sb is None else sb.ctypes.data, int(seed), int(offset), int(b_first), float(band),
         acc.ctypes.data, tok.ctypes.data, res.pt_tok.ctypes.data, res.pd_tok.ctypes.data,
         res.max_pt.ctypes.data, res.margin.ctypes.data, res.cls.ctypes.data,
         res.resid_mass.ctypes.data, res.cdf_margin.ctypes.data,

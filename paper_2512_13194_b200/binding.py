@@ -43,6 +43,9 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ears_verify_ex.argtypes = ([c.c_int] + common + [c.c_int64] + [c.c_void_p] * 7
                                    + [c.c_void_p, c.c_size_t, c.c_void_p])
     lib.ears_verify_ex.restype = c.c_int
+    lib.ears_verify_var.argtypes = ([c.c_int] + common[:8] + [c.c_void_p, c.c_void_p] + common[8:] + [c.c_int64]
+                                    + [c.c_void_p] * 7 + [c.c_void_p, c.c_size_t, c.c_void_p])
+    lib.ears_verify_var.restype = c.c_int
     lib.ears_verify_host.argtypes = [c.c_int] + common + [c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p]
     lib.ears_verify_host.restype = c.c_int
     lib.ears_verify_noalloc.argtypes = [c.c_int] + common + [c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
@@ -115,11 +118,14 @@ def _stream_ptr(stream) -> int:
 
 def verify(target_logits: torch.Tensor, draft_logits: torch.Tensor, draft_tokens: torch.Tensor,
            temperature: float, beta: float, seed: int = 0, offset: int = 0, *, b_first: int = 0,
-           stats: bool = False, workspace: Optional[torch.Tensor] = None, stream=None):
+           stats: bool = False, workspace: Optional[torch.Tensor] = None, stream=None,
+           seq_temperature: Optional[torch.Tensor] = None, seq_beta: Optional[torch.Tensor] = None):
     """One EARS verification step on the current CUDA device.
 
     Returns (accept_len [B] int32, tokens [B,K+1] int32) and, with ``stats=True``, a dict with
     pt_tok, pd_tok, max_pt [B,K] float64, cls [B,K] uint8 and resid_mass [B] float64.
+    ``seq_temperature`` / ``seq_beta``: optional float32 CUDA tensors [B] that replace the scalar
+    for each sequence (ears_verify_var).
     The call is asynchronous on ``stream`` (default: torch's current stream).
     """
     lib = load_library()
@@ -143,9 +149,24 @@ def verify(target_logits: torch.Tensor, draft_logits: torch.Tensor, draft_tokens
                       resid_mass=torch.zeros(B, dtype=torch.float64, device=dev))
             ptrs = [st[k].data_ptr() for k in ("pt_tok", "pd_tok", "max_pt", "cls", "resid_mass")]
         ws_ptr, ws_bytes = (None, 0) if workspace is None else (workspace.data_ptr(), workspace.numel() * workspace.element_size())
-        rc = lib.ears_verify_ex(_dtype_code(t), t.data_ptr(), d.data_ptr(), x.data_ptr(), B, K, V,
-                                float(temperature), float(beta), int(seed), int(offset), int(b_first),
-                                acc.data_ptr(), tok.data_ptr(), *ptrs, ws_ptr, ws_bytes, _stream_ptr(stream))
+        if seq_temperature is None and seq_beta is None:
+            rc = lib.ears_verify_ex(_dtype_code(t), t.data_ptr(), d.data_ptr(), x.data_ptr(), B, K, V,
+                                    float(temperature), float(beta), int(seed), int(offset), int(b_first),
+                                    acc.data_ptr(), tok.data_ptr(), *ptrs, ws_ptr, ws_bytes, _stream_ptr(stream))
+        else:
+            arrs = []
+            for a in (seq_temperature, seq_beta):
+                if a is not None:
+                    if a.device != dev or a.dtype != torch.float32 or a.shape != (B,):
+                        raise ValueError("per-sequence arrays must be float32 CUDA tensors of shape [B]")
+                    a = a.contiguous()
+                arrs.append(a)
+            rc = lib.ears_verify_var(_dtype_code(t), t.data_ptr(), d.data_ptr(), x.data_ptr(), B, K, V,
+                                     float(temperature), float(beta),
+                                     None if arrs[0] is None else arrs[0].data_ptr(),
+                                     None if arrs[1] is None else arrs[1].data_ptr(),
+                                     int(seed), int(offset), int(b_first),
+                                     acc.data_ptr(), tok.data_ptr(), *ptrs, ws_ptr, ws_bytes, _stream_ptr(stream))
     _check(rc)
     return (acc, tok, st) if stats else (acc, tok)
 

@@ -352,15 +352,20 @@ int ensure_attrs(DeviceInfo* di) {
 }
 
 int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B, int K, int V,
-                float temperature, float beta, uint64_t seed, uint64_t offset, int64_t b_first,
+                float temperature, float beta, const float* seq_T, const float* seq_beta,
+                uint64_t seed, uint64_t offset, int64_t b_first,
                 int32_t* out_len, int32_t* out_tok, double* o_pt, double* o_pd, double* o_max,
                 uint8_t* o_cls, double* o_resid, void* workspace, size_t workspace_bytes, void* stream_) {
     if (!t || !d || !x || !out_len || !out_tok) return EARS_ERR_NULL;
     if (dtype != EARS_DTYPE_F32 && dtype != EARS_DTYPE_BF16) return EARS_ERR_PARAM;
     int rc = check_shape(B, K, V);
     if (rc) return rc;
+    // a per-sequence array replaces its scalar, which is then not looked at
+    if (seq_T) temperature = 1.0f;
+    if (seq_beta) beta = 0.0f;
     if (!(temperature > 0.0f) || !std::isfinite(temperature)) return EARS_ERR_PARAM;
     if (!(beta >= 0.0f) || !std::isfinite(beta)) return EARS_ERR_PARAM;
+    if (((uintptr_t)seq_T % 4) || ((uintptr_t)seq_beta % 4)) return EARS_ERR_ALIGN;
     if (b_first < 0 || (unsigned long long)b_first + (unsigned long long)B > 0xffffffffull) return EARS_ERR_PARAM;
     const int esize = dtype == EARS_DTYPE_F32 ? 4 : 2;
     if (((uintptr_t)t % esize) || ((uintptr_t)d % esize) || ((uintptr_t)x % 4)) return EARS_ERR_ALIGN;
@@ -405,6 +410,7 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
         p.c = c;
         p.T = (double)temperature;
         p.beta = (double)beta;
+        p.seq_T = seq_T; p.seq_beta = seq_beta;
         p.seed = seed; p.offset = offset; p.b_first = b_first;
         p.out_len = out_len; p.out_tok = out_tok;
         p.pt_tok = o_pt ? o_pt : (double*)(w + L.pt_tok);
@@ -442,6 +448,7 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
     p.c = c;
     p.T = (double)temperature;
     p.beta = (double)beta;
+    p.seq_T = seq_T; p.seq_beta = seq_beta;
     p.seed = seed; p.offset = offset; p.b_first = b_first;
     p.out_len = out_len; p.out_tok = out_tok;
     p.pt_tok = o_pt ? o_pt : (double*)(w + L.pt_tok);
@@ -548,16 +555,28 @@ int ears_verify_ex(int dtype, const void* target_logits, const void* draft_logit
                    int32_t* out_tokens, double* out_pt_tok, double* out_pd_tok, double* out_max_pt,
                    uint8_t* out_class, double* out_resid_mass, void* workspace, size_t workspace_bytes,
                    void* stream) {
-    return verify_impl(dtype, target_logits, draft_logits, draft_tokens, B, K, V, temperature, beta, seed,
-                       offset, b_first, out_accept_len, out_tokens, out_pt_tok, out_pd_tok, out_max_pt,
+    return verify_impl(dtype, target_logits, draft_logits, draft_tokens, B, K, V, temperature, beta, nullptr, nullptr,
+                       seed, offset, b_first, out_accept_len, out_tokens, out_pt_tok, out_pd_tok, out_max_pt,
                        out_class, out_resid_mass, workspace, workspace_bytes, stream);
+}
+
+int ears_verify_var(int dtype, const void* target_logits, const void* draft_logits,
+                    const int32_t* draft_tokens, int B, int K, int V, float temperature, float beta,
+                    const float* seq_temperature, const float* seq_beta,
+                    uint64_t seed, uint64_t offset, int64_t b_first, int32_t* out_accept_len,
+                    int32_t* out_tokens, double* out_pt_tok, double* out_pd_tok, double* out_max_pt,
+                    uint8_t* out_class, double* out_resid_mass, void* workspace, size_t workspace_bytes,
+                    void* stream) {
+    return verify_impl(dtype, target_logits, draft_logits, draft_tokens, B, K, V, temperature, beta,
+                       seq_temperature, seq_beta, seed, offset, b_first, out_accept_len, out_tokens, out_pt_tok,
+                       out_pd_tok, out_max_pt, out_class, out_resid_mass, workspace, workspace_bytes, stream);
 }
 
 int ears_verify_f32(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
                     int B, int K, int V, float temperature, float beta, uint64_t seed, uint64_t offset,
                     int32_t* out_accept_len, int32_t* out_tokens, void* stream) {
     return verify_impl(EARS_DTYPE_F32, target_logits, draft_logits, draft_tokens, B, K, V, temperature, beta,
-                       seed, offset, 0, out_accept_len, out_tokens, nullptr, nullptr, nullptr, nullptr, nullptr,
+                       nullptr, nullptr, seed, offset, 0, out_accept_len, out_tokens, nullptr, nullptr, nullptr, nullptr, nullptr,
                        nullptr, 0, stream);
 }
 
@@ -565,7 +584,7 @@ int ears_verify_bf16(const void* target_logits, const void* draft_logits, const 
                      int B, int K, int V, float temperature, float beta, uint64_t seed, uint64_t offset,
                      int32_t* out_accept_len, int32_t* out_tokens, void* stream) {
     return verify_impl(EARS_DTYPE_BF16, target_logits, draft_logits, draft_tokens, B, K, V, temperature, beta,
-                       seed, offset, 0, out_accept_len, out_tokens, nullptr, nullptr, nullptr, nullptr, nullptr,
+                       nullptr, nullptr, seed, offset, 0, out_accept_len, out_tokens, nullptr, nullptr, nullptr, nullptr, nullptr,
                        nullptr, 0, stream);
 }
 
@@ -599,8 +618,8 @@ int ears_verify_host(int dtype, const void* target_logits, const void* draft_log
     EARS_CUDA(cudaMemcpyAsync(s + o_t, target_logits, tb, cudaMemcpyHostToDevice, stream));
     EARS_CUDA(cudaMemcpyAsync(s + o_d, draft_logits, db, cudaMemcpyHostToDevice, stream));
     EARS_CUDA(cudaMemcpyAsync(s + o_x, draft_tokens, xb, cudaMemcpyHostToDevice, stream));
-    rc = verify_impl(dtype, s + o_t, s + o_d, (const int32_t*)(s + o_x), B, K, V, temperature, beta, seed, offset,
-                     b_first, (int32_t*)(s + o_l), (int32_t*)(s + o_o), nullptr, nullptr, nullptr, nullptr,
+    rc = verify_impl(dtype, s + o_t, s + o_d, (const int32_t*)(s + o_x), B, K, V, temperature, beta, nullptr, nullptr,
+                     seed, offset, b_first, (int32_t*)(s + o_l), (int32_t*)(s + o_o), nullptr, nullptr, nullptr, nullptr,
                      nullptr, nullptr, 0, stream_);
     if (rc) return rc;
     EARS_CUDA(cudaMemcpyAsync(out_accept_len, s + o_l, lb, cudaMemcpyDeviceToHost, stream));
@@ -623,8 +642,8 @@ int ears_verify_noalloc(int dtype, const void* target_logits, const void* draft_
     void* scratch = nullptr;
     rc = noalloc_scratch(dev, &scratch);
     if (rc) return rc;
-    rc = verify_impl(dtype, target_logits, draft_logits, draft_tokens, B, K, V, temperature, beta, seed, offset,
-                     b_first, out_accept_len, out_tokens, nullptr, nullptr, nullptr, nullptr, nullptr, scratch,
+    rc = verify_impl(dtype, target_logits, draft_logits, draft_tokens, B, K, V, temperature, beta, nullptr, nullptr,
+                     seed, offset, b_first, out_accept_len, out_tokens, nullptr, nullptr, nullptr, nullptr, nullptr, scratch,
                      (size_t)EARS_NOALLOC_SCRATCH_BYTES, stream);
     if (rc) return rc;
     if (out_device_status)  // the status word is heads[2] at the start of the scratch

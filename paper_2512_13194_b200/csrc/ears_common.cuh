@@ -56,6 +56,8 @@ struct Params {
     float c;              // log2(e) / temperature
     double T;             // temperature
     double beta;
+    const float* seq_T;   // [B] per-sequence temperature, or NULL (then T for all)
+    const float* seq_beta;  // [B] per-sequence beta, or NULL
     unsigned long long seed, offset;
     long long b_first;
     int32_t* out_len;     // [B]
@@ -82,6 +84,22 @@ struct Params {
     size_t seg_stride;
     Plan plan;
 };
+
+// Temperature and base tolerance of (local) sequence b: the per-sequence arrays where given,
+// else the call's scalars.  c = log2(e) / T is formed the way the host forms it for the scalar.
+template <class P> __device__ __forceinline__ double seq_temperature(const P& p, int b) {
+    return p.seq_T ? (double)__ldg(p.seq_T + b) : p.T;
+}
+template <class P> __device__ __forceinline__ double seq_beta(const P& p, int b) {
+    return p.seq_beta ? (double)__ldg(p.seq_beta + b) : p.beta;
+}
+template <class P> __device__ __forceinline__ float seq_c(const P& p, int b) {
+    return p.seq_T ? (float)(1.4426950408889634 / (double)__ldg(p.seq_T + b)) : p.c;
+}
+// What the host refuses in the scalar form makes a sequence invalid in the per-sequence form.
+__device__ __forceinline__ bool seq_params_ok(double T, double beta) {
+    return T > 0.0 && T < 1e300 && beta >= 0.0 && beta < 1e300;   // NaN fails every comparison
+}
 
 __host__ __device__ inline double* seg_sums(const Params& p, int b) { return reinterpret_cast<double*>(p.seg_base + (size_t)b * p.seg_stride); }
 __host__ __device__ inline BonusSeg* bonus_segs(const Params& p, int b) { return reinterpret_cast<BonusSeg*>(p.seg_base + (size_t)b * p.seg_stride); }

@@ -41,6 +41,7 @@ struct StageMeta {
     int flags;   // bit 0: first chunk of the unit / row, bit 1: last chunk
     int elem0;   // index of the slot's first element within its row
     int aux;     // statistics: 1 for the extra target row; final-token rows: position n
+    float c;     // log2(e) / temperature of the slot's sequence
 };
 
 struct Msg { int kind, a, b, c; };
@@ -342,13 +343,15 @@ __device__ int finalize_sequence(const Params& p, int b, int lane) {
     const int K = p.K, R = 2 * K + 1, V = p.V, P = p.plan.parts1;
     const E* t = reinterpret_cast<const E*>(p.t);
     const E* d = reinterpret_cast<const E*>(p.d);
-    bool bad = false;
+    const float cb = seq_c(p, b);
+    const double Tb = seq_temperature(p, b), betab = seq_beta(p, b);
+    bool bad = !seq_params_ok(Tb, betab);
     for (int r = lane; r < R; r += 32) {
         float m = -INFINITY, s = 0.0f;
         const float2* pp = p.partial + ((size_t)b * R + r) * P;
         for (int i = 0; i < P; ++i) {
             float2 v = __ldcg(pp + i);
-            merge_ms(m, s, v.x, v.y, p.c);
+            merge_ms(m, s, v.x, v.y, cb);
         }
         if (!rowstat_ok(m, s)) bad = true;
         p.rowstat[(size_t)b * R + r] = make_float2(m, s);
@@ -368,7 +371,7 @@ __device__ int finalize_sequence(const Params& p, int b, int lane) {
                 const double lt = (double)load_logit(t + (size_t)target_row(b, k, K) * V + tok);
                 const double ld = (double)load_logit(d + (size_t)draft_row(b, k, K) * V + tok);
                 const double U = uniform_accept(p.seed, p.offset, (uint32_t)(p.b_first + b), (uint32_t)k);
-                const Decision dc = decide_position(lt, ld, st, sd, p.T, p.beta, U);
+                const Decision dc = decide_position(lt, ld, st, sd, Tb, betab, U);
                 reject = !dc.accept;
                 const size_t i = (size_t)b * K + k;
                 p.pt_tok[i] = dc.pt;
@@ -547,6 +550,7 @@ template <typename E>
 __device__ void select_token(const Params& p, int b, int n, int lane) {
     constexpr int CHUNK_ELEMS = kChunkBytes / (int)sizeof(E);
     const int K = p.K, V = p.V, R = 2 * K + 1, nseg = p.plan.nseg;
+    const float cb = seq_c(p, b);
     const bool resid = n < K;
     const E* trow = reinterpret_cast<const E*>(p.t) + (size_t)target_row(b, n, K) * V;
     const E* drow = reinterpret_cast<const E*>(p.d) + (size_t)draft_row(b, resid ? n : 0, K) * V;
@@ -564,7 +568,7 @@ __device__ void select_token(const Params& p, int b, int n, int lane) {
         // one entry per (chunk, consumer warp) of the extra row: (sum, reference maximum)
         const int chunks = (V + CHUNK_ELEMS - 1) / CHUNK_ELEMS;
         const BonusSeg* bs = bonus_segs(p, b);
-        const double m = (double)rn.mt, c = (double)p.c;
+        const double m = (double)rn.mt, c = (double)cb;
         seg = pick_block([bs, m, c](int g) {
                   const double sum = __ldcg(&bs[g].sum);
                   const float ref = __ldcg(&bs[g].ref);
@@ -577,9 +581,9 @@ __device__ void select_token(const Params& p, int b, int n, int lane) {
     double S_used = S;
     if (seg < 0 || !(S * rn.izt >= kTinyMass)) {
         // a rejection implies residual mass; if rounding erased it, draw from P_t instead
-        tok = warp_sample_pt_slow<E>(trow, V, rn, p.c, u, lane, &S_used);
+        tok = warp_sample_pt_slow<E>(trow, V, rn, cb, u, lane, &S_used);
     } else {
-        tok = pick_in_range<E>(trow, drow, resid, rn, p.c, seg * seg_elems, seg_elems, u * S - before, V, lane);
+        tok = pick_in_range<E>(trow, drow, resid, rn, cb, seg * seg_elems, seg_elems, u * S - before, V, lane);
     }
     if (lane == 0) {
         p.out_tok[(size_t)b * (K + 1) + n] = tok;
@@ -673,13 +677,14 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
                 const int step = CHUNK_ELEMS / 2;  // half a slot of each of the two rows
                 const E* trow = tbase + (size_t)target_row(b, n, K) * V;
                 const E* drow = dbase + (size_t)draft_row(b, n, K) * V;
+                const float cj = seq_c(p, b);
                 const int e_begin = jpart * p.plan.job_elems;
                 const int e_end = min(V, e_begin + p.plan.job_elems);
                 for (int e0 = e_begin; e0 < e_end; e0 += step, ++q) {
                     ok = loader_acquire(sm, q, lane);
                     if (!ok) break;
                     const int ne = min(step, e_end - e0);
-                    const StageMeta mt{kFinal, b, ne, (e0 == e_begin ? 1 : 0) | (e0 + step >= e_end ? 2 : 0), e0, n};
+                    const StageMeta mt{kFinal, b, ne, (e0 == e_begin ? 1 : 0) | (e0 + step >= e_end ? 2 : 0), e0, n, cj};
                     loader_fill<E>(sm, q % STAGES, mt, use_tma, trow + e0, drow + e0, lane, pol_last_use);
                 }
                 if (!ok) break;
@@ -697,13 +702,14 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
                     const E* row = (ridx == 2 * K) ? tbase + (size_t)target_row(b, K, K) * V
                                                    : ((ridx & 1) ? dbase + (size_t)draft_row(b, ridx >> 1, K) * V
                                                                  : tbase + (size_t)target_row(b, ridx >> 1, K) * V);
+                    const float cu = seq_c(p, b);
                     const int ch0 = part * cpp;
                     const int ch1 = min(chunks_per_row, ch0 + cpp);
                     for (int ch = ch0; ch < ch1; ++ch, ++q) {
                         ok = loader_acquire(sm, q, lane);
                         if (!ok) break;
                         const int e0 = ch * CHUNK_ELEMS;
-                        const StageMeta mt{kStats, (int)u, min(CHUNK_ELEMS, V - e0), (ch == ch0 ? 1 : 0) | (ch == ch1 - 1 ? 2 : 0), e0, ridx == 2 * K ? 1 : 0};
+                        const StageMeta mt{kStats, (int)u, min(CHUNK_ELEMS, V - e0), (ch == ch0 ? 1 : 0) | (ch == ch1 - 1 ? 2 : 0), e0, ridx == 2 * K ? 1 : 0, cu};
                         // the extra target row is never streamed again (its sums are kept); the other
                         // rows may be, if their position turns out to be the first rejection
                         loader_fill<E>(sm, q % STAGES, mt, use_tma, row + e0, nullptr, lane, ridx == 2 * K ? pol_last_use : pol_keep);
@@ -736,7 +742,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
             }
         }
         if (ok && loader_acquire(sm, q, lane)) {
-            loader_fill<E>(sm, q % STAGES, StageMeta{kEnd, 0, 0, 0, 0, 0}, use_tma, (const E*)nullptr, (const E*)nullptr, lane, pol_keep);
+            loader_fill<E>(sm, q % STAGES, StageMeta{kEnd, 0, 0, 0, 0, 0, 0.f}, use_tma, (const E*)nullptr, (const E*)nullptr, lane, pol_keep);
         } else if (use_tma && lane == 0) {
             loader_drain(sm, q);
         }
@@ -766,9 +772,10 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
             }
             float pm = -INFINITY, ps = 0.f;
             if (m.kind == kMsgPiece && slot_ok) {
+                const float cu = seq_c(p, m.a / (R * P));
                 for (int w = 0; w < kConsumerWarps; ++w) {
                     const float2 v = sm.scratch[m.c % kUnitSlots][w];
-                    merge_ms(pm, ps, v.x, v.y, p.c);
+                    merge_ms(pm, ps, v.x, v.y, cu);
                 }
             }
 #pragma unroll
@@ -899,9 +906,9 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
                 if (mt.flags & 1) { m_run = -INFINITY; s[0] = s[1] = s[2] = s[3] = 0.f; }
                 if (mt.aux) {  // a piece of the extra target row
                     BonusSeg* out = bonus_segs(p, mt.id / (R * P)) + (size_t)(mt.elem0 / CHUNK_ELEMS) * kConsumerWarps + warp;
-                    chunk_stats<E, true>(sm.buf[stage], mt.nelem, warp, lane, p.c, m_run, s, out);
+                    chunk_stats<E, true>(sm.buf[stage], mt.nelem, warp, lane, mt.c, m_run, s, out);
                 } else {
-                    chunk_stats<E, false>(sm.buf[stage], mt.nelem, warp, lane, p.c, m_run, s, nullptr);
+                    chunk_stats<E, false>(sm.buf[stage], mt.nelem, warp, lane, mt.c, m_run, s, nullptr);
                 }
                 if (!(mt.flags & 2)) {
                     __syncwarp();
@@ -914,7 +921,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
                 for (int off = 16; off > 0; off >>= 1) {
                     float m2 = __shfl_xor_sync(0xffffffffu, m, off);
                     float s2 = __shfl_xor_sync(0xffffffffu, sum, off);
-                    merge_ms(m, sum, m2, s2, p.c);
+                    merge_ms(m, sum, m2, s2, mt.c);
                 }
                 if (lane == 0) {
                     const int us = unit_ends % kUnitSlots;
@@ -934,7 +941,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
                 rn = make_rownorm(st, sd);
             }
             double* seg_out = seg_sums(p, b) + mt.elem0 / kSegElems;
-            chunk_segments<E, true>(sm.buf[stage], sm.buf[stage] + kChunkBytes / 2, mt.nelem, warp, lane, rn, p.c, seg_out);
+            chunk_segments<E, true>(sm.buf[stage], sm.buf[stage] + kChunkBytes / 2, mt.nelem, warp, lane, rn, mt.c, seg_out);
             if (mt.flags & 2) {
                 // last chunk of the piece: publish the sums; the epilogue warp counts the piece once
                 // all warps are through and, when it is the sequence's last, picks the token

@@ -42,6 +42,8 @@ struct RParams {
     int B, K, V;
     float c;              // log2(e) / temperature
     double T, beta;
+    const float* seq_T;   // [B] per-sequence temperature, or NULL
+    const float* seq_beta;  // [B] per-sequence beta, or NULL
     unsigned long long seed, offset;
     long long b_first;
     int32_t* out_len;
@@ -379,6 +381,7 @@ __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RPara
     cluster_sync_all();
     while (have) {
         // ---- 1. statistics of the slices as the copies land
+        const float cb = seq_c(p, b);   // log2(e) / temperature of this sequence
         RowAcc at, ad;
         acc_open(at);
         acc_open(ad);
@@ -387,22 +390,22 @@ __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RPara
                 if (!mbar_wait(&sm.full[q], (full_phase >> q) & 1u, &sm.abort_flag)) failed = true;
             }
             if (failed) break;
-            stats_sub<E>(buf_t, q, n, tid, p.c, at);
-            if (pair) stats_sub<E>(buf_d, q, n, tid, p.c, ad);
+            stats_sub<E>(buf_t, q, n, tid, cb, at);
+            if (pair) stats_sub<E>(buf_d, q, n, tid, cb, ad);
         }
         if (use_tma) full_phase ^= issued;
         // (max, sum) of the warp's share: the maximum first (shuffles only), then one rescale per
         // thread and a sum -- a much shorter dependent chain than merging (m, s) pairs step by step
         const int par = round & 1;
         {
-            const float2 pt2 = acc_close(at, p.c), pd2 = acc_close(ad, p.c);
+            const float2 pt2 = acc_close(at, cb), pd2 = acc_close(ad, cb);
             float Mt = pt2.x, Md = pd2.x;
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) {
                 Mt = fmaxf(Mt, __shfl_xor_sync(0xffffffffu, Mt, off));
                 Md = fmaxf(Md, __shfl_xor_sync(0xffffffffu, Md, off));
             }
-            float St = rebase_sum(pt2.x, pt2.y, Mt, p.c), Sd = rebase_sum(pd2.x, pd2.y, Md, p.c);
+            float St = rebase_sum(pt2.x, pt2.y, Mt, cb), Sd = rebase_sum(pd2.x, pd2.y, Md, cb);
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) {
                 St += __shfl_xor_sync(0xffffffffu, St, off);
@@ -436,8 +439,8 @@ __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RPara
             float zt = 0.f, zd = 0.f;
             for (int i = lane; i < parts; i += 32) {
                 const float4 v = sm.xstat[par][i];
-                zt += rebase_sum(v.x, v.y, mt, p.c);
-                zd += rebase_sum(v.z, v.w, md, p.c);
+                zt += rebase_sum(v.x, v.y, mt, cb);
+                zd += rebase_sum(v.z, v.w, md, cb);
             }
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) {
@@ -445,8 +448,9 @@ __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RPara
                 zd += __shfl_xor_sync(0xffffffffu, zd, off);
             }
           if (lane == 0) {
+            const double Tb = seq_temperature(p, b), betab = seq_beta(p, b);
             int dec = 1;
-            if (!rowstat_ok(mt, zt) || (pair && (!rowstat_ok(md, zd) || !tok_ok))) dec = -1;
+            if (!rowstat_ok(mt, zt) || (pair && (!rowstat_ok(md, zd) || !tok_ok)) || !seq_params_ok(Tb, betab)) dec = -1;
             sm.rs_t = make_float2(mt, zt);
             sm.rs_d = pair ? make_float2(md, zd) : make_float2(0.f, 1.f);
             if (pair && dec >= 0) {
@@ -454,15 +458,15 @@ __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RPara
                 // band is some 25 times the fp32 error), in which case -- or when the caller wants
                 // the probabilities -- it is taken in fp64.  Either way every CTA of the cluster
                 // runs the same arithmetic on the same numbers.
-                const float pt32 = ex2_approx((lt - mt) * p.c) / zt;
-                const float pd32 = ex2_approx((ld - md) * p.c) / zd;
+                const float pt32 = ex2_approx((lt - mt) * cb) / zt;
+                const float pd32 = ex2_approx((ld - md) * cb) / zd;
                 const float ratio32 = pt32 / fmaxf(pd32, (float)kEps);
-                const float thr32 = fmaxf((float)U - (float)p.beta * (1.0f - 1.0f / zt), 0.0f);
+                const float thr32 = fmaxf((float)U - (float)betab * (1.0f - 1.0f / zt), 0.0f);
                 const float diff = ratio32 - thr32;
                 if (!p.want_stats && fabsf(diff) > 1e-4f * (ratio32 + thr32) + 1e-6f) {
                     dec = diff > 0.0f ? 1 : 0;
                 } else {
-                    const Decision dc = decide_position((double)lt, (double)ld, sm.rs_t, sm.rs_d, p.T, p.beta, U);
+                    const Decision dc = decide_position((double)lt, (double)ld, sm.rs_t, sm.rs_d, Tb, betab, U);
                     dec = dc.accept ? 1 : 0;
                     if (rank == 0 && p.want_stats) {
                         const size_t i = (size_t)b * K + j;
@@ -487,8 +491,8 @@ __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RPara
             const int nseg = (n + kSegElems - 1) / kSegElems;
             bool resid = pair;
             for (;;) {
-                if (resid) slice_segments<E, true>(buf_t, buf_d, n, warp, lane, rn, p.c, sm.segsum);
-                else slice_segments<E, false>(buf_t, buf_t, n, warp, lane, rn, p.c, sm.segsum);
+                if (resid) slice_segments<E, true>(buf_t, buf_d, n, warp, lane, rn, cb, sm.segsum);
+                else slice_segments<E, false>(buf_t, buf_t, n, warp, lane, rn, cb, sm.segsum);
                 __syncthreads();
                 const int mpar = mround & 1;
                 // warp 0: lanes own contiguous runs of segment sums
@@ -564,7 +568,7 @@ __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RPara
                     seg = __shfl_sync(0xffffffffu, seg, L);
                     before = __shfl_sync(0xffffffffu, before, L);
                     if (seg >= 0) {
-                        const int idx = pick_in_segment<E>(buf_t, resid ? buf_d : buf_t, resid, rn, p.c, seg * kSegElems,
+                        const int idx = pick_in_segment<E>(buf_t, resid ? buf_d : buf_t, resid, rn, cb, seg * kSegElems,
                                                            min(kSegElems, n - seg * kSegElems), tin - before, lane);
                         token = idx >= 0 ? e0 + idx : -1;
                     }

@@ -314,3 +314,51 @@ def test_bounded_wait_gives_up_and_context_survives(ears):
     tl, *_ = run_both(ears, w, t, d, x, 1.0, 0.1)
     assert_parity(tl, max_explained=0)
     assert ears.load_library().ears_selftest_bounded_wait(0, None) == -3
+
+
+@pytest.mark.parametrize("path,cluster", [(1, 0), (2, 0), (2, 4)])
+@pytest.mark.parametrize("B,K,V,dtype", [(12, 3, 9000, "fp32"), (9, 4, 20001, "bf16"), (300, 2, 700, "bf16")])
+def test_parity_per_sequence_temperature_and_beta(ears, forced_path, B, K, V, dtype, path, cluster):
+    """ears_verify_var: every sequence with its own temperature and beta, against the oracle run
+    with the same arrays; plus: equal entries reproduce the scalar call bit for bit, and an
+    unusable entry invalidates only its own sequence."""
+    forced_path(path, cluster)
+    dev = "cuda:0"
+    w, t, d, x = synth.tiny_inputs(B, K, V, dtype, seed=500 + K, noise=1.0)
+    rng = np.random.default_rng(B)
+    Ts = rng.uniform(0.5, 1.6, B).astype(np.float32)
+    betas = rng.choice(np.array([0.0, 0.1, 0.3, 1.0], np.float32), B)
+    tg, dg, xg = t.to(dev), d.to(dev), x.to(dev)
+    Tg, bg = torch.from_numpy(Ts).to(dev), torch.from_numpy(betas).to(dev)
+    tally = Tally()
+    for offset in range(2):
+        acc, tok, st = ears.verify(tg, dg, xg, 123.0, 456.0, 7, offset, b_first=3, stats=True, seq_temperature=Tg,
+                                   seq_beta=bg)
+        acc2, tok2 = ears.verify(tg, dg, xg, 123.0, 456.0, 7, offset, b_first=3, seq_temperature=Tg, seq_beta=bg)
+        torch.cuda.synchronize()
+        assert ears.last_device_status() == 0
+        assert torch.equal(acc, acc2) and torch.equal(tok, tok2)
+        ora = oracle.verify(t, d, x, 1.0, 0.0, seed=7, offset=offset, b_first=3, nthreads=8, seq_temperature=Ts,
+                            seq_beta=betas)
+        tally.merge(compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, K, {k: v.cpu().numpy() for k, v in st.items()}))
+    assert_parity(tally, max_explained=1)
+    assert tally.max_rel_prob_err < 1e-5
+    # equal entries == the scalar call
+    ref = ears.verify(tg, dg, xg, 0.9, 0.25, 7, 1)
+    same = ears.verify(tg, dg, xg, 5.0, 5.0, 7, 1, seq_temperature=torch.full((B,), 0.9, device=dev),
+                       seq_beta=torch.full((B,), 0.25, device=dev))
+    assert torch.equal(ref[0], same[0]) and torch.equal(ref[1], same[1])
+    only_T = ears.verify(tg, dg, xg, 5.0, 0.25, 7, 1, seq_temperature=torch.full((B,), 0.9, device=dev))
+    assert torch.equal(ref[0], only_T[0]) and torch.equal(ref[1], only_T[1])
+    # unusable entries
+    badT, badb = Ts.copy(), betas.copy()
+    badT[1] = 0.0
+    badT[4] = np.nan
+    badb[2] = -1.0
+    acc, tok = ears.verify(tg, dg, xg, 1.0, 0.0, 7, 0, b_first=3, seq_temperature=torch.from_numpy(badT).to(dev),
+                           seq_beta=torch.from_numpy(badb).to(dev))
+    torch.cuda.synchronize()
+    assert ears.last_device_status() & ears.DEV_INVALID_INPUT
+    ora = oracle.verify(t, d, x, 1.0, 0.0, seed=7, offset=0, b_first=3, nthreads=8, seq_temperature=badT, seq_beta=badb)
+    assert ora.accept_len[[1, 2, 4]].tolist() == [-1, -1, -1]
+    assert_parity(compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, K), max_explained=1)

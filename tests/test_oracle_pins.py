@@ -357,3 +357,44 @@ def test_invalid_sequences_are_marked_not_fatal():
         oracle.verify(t, d, x, 0.0, 0.1)
     with pytest.raises(ValueError):
         oracle.verify(t, d, x, 1.0, -0.1)
+
+
+# --------------------------------------------------------------------------- per-sequence temperature and beta
+def test_per_sequence_parameters_match_closed_forms_and_scalar_calls():
+    """Sec. 3.3 item 3 treats sequences independently, so each may carry its own temperature
+    (Sec. 4.3) and base tolerance (Sec. 3.2).  Pins: (i) probabilities of sequence b against a
+    library softmax at T_b; (ii) the whole result of sequence b against a scalar call on that
+    sequence alone with (T_b, beta_b) and the same global index; (iii) equal entries reproduce
+    the scalar call; (iv) a value the scalar form refuses invalidates only its own sequence."""
+    rng = np.random.default_rng(77)
+    B, K, V = 6, 3, 50
+    t = rng.normal(0, 2, (B, K + 1, V)).astype(np.float32)
+    d = (t[:, :K] + rng.normal(0, 0.8, (B, K, V))).astype(np.float32)
+    x = rng.integers(0, V, (B, K)).astype(np.int32)
+    Ts = np.array([0.5, 0.8, 1.0, 1.3, 2.0, 0.9], np.float32)
+    betas = np.array([0.0, 0.1, 0.3, 0.05, 1.0, 0.2], np.float32)
+    res = oracle.verify(t, d, x, 1.0, 0.1, seed=3, offset=9, b_first=4, seq_temperature=Ts, seq_beta=betas)
+    for b in range(B):
+        for k in range(K):
+            pt = sp_softmax(t[b, k].astype(np.float64) / float(Ts[b]))
+            pd = sp_softmax(d[b, k].astype(np.float64) / float(Ts[b]))
+            assert res.pt_tok[b, k] == pytest.approx(pt[x[b, k]], rel=1e-12)
+            assert res.pd_tok[b, k] == pytest.approx(pd[x[b, k]], rel=1e-12)
+            U = oracle.uniform_accept(3, 9, 4 + b, k)
+            thr = max(U - float(betas[b]) * (1.0 - pt.max()), 0.0)
+            assert res.margin[b, k] == pytest.approx(pt[x[b, k]] / max(pd[x[b, k]], EPS) - thr, abs=1e-12)
+        one = oracle.verify(t[b:b + 1], d[b:b + 1], x[b:b + 1], float(Ts[b]), float(betas[b]), seed=3, offset=9,
+                            b_first=4 + b)
+        assert one.accept_len[0] == res.accept_len[b]
+        assert np.array_equal(one.tokens[0], res.tokens[b])
+        assert one.resid_mass[0] == res.resid_mass[b]
+    same = oracle.verify(t, d, x, 7.0, 7.0, seed=3, offset=9, seq_temperature=np.full(B, 0.9, np.float32),
+                         seq_beta=np.full(B, 0.25, np.float32))
+    ref = oracle.verify(t, d, x, np.float32(0.9), 0.25, seed=3, offset=9)
+    assert np.array_equal(same.tokens, ref.tokens) and np.array_equal(same.margin, ref.margin)
+    bad_T = Ts.copy(); bad_T[2] = 0.0; bad_T[4] = np.nan
+    bad_b = betas.copy(); bad_b[1] = -0.5
+    bad = oracle.verify(t, d, x, 1.0, 0.1, seed=3, offset=9, b_first=4, seq_temperature=bad_T, seq_beta=bad_b)
+    assert bad.accept_len[[1, 2, 4]].tolist() == [-1, -1, -1] and (bad.tokens[[1, 2, 4]] == -1).all()
+    for b in (0, 3, 5):
+        assert bad.accept_len[b] == res.accept_len[b] and np.array_equal(bad.tokens[b], res.tokens[b])
