@@ -140,12 +140,22 @@ int ears_verify_ex(int dtype, const void* target_logits, const void* draft_logit
  *   A value the scalar form would refuse (temperature not finite or <= 0, beta not finite or
  *   < 0) cannot be seen by the host: it marks that one sequence invalid (out_accept_len = -1,
  *   tokens -1, EARS_DEV_INVALID_INPUT), the others are unaffected.
+ *   flags       0 or EARS_FLAG_STOP_AT_FIRST_REJECT.  Sec. 3.1: rejecting x_i discards every later
+ *               draft token.  With the flag, what lies after a sequence's first rejected position
+ *               (later rows and tokens, and the extra target row unless everything was accepted)
+ *               is not part of the step: it is not validated and the optional per-position
+ *               outputs are not written there; lengths and tokens are the same as without the
+ *               flag on valid data.  Where the resident kernel runs (see ears_set_path) those rows
+ *               are not even read -- a cluster then walks a sequence position by position -- which
+ *               saves their HBM traffic at the price of a longer chain per sequence; the
+ *               streaming kernel reads them anyway and ignores them.
  * Everything else is as in ears_verify_ex.
  */
+#define EARS_FLAG_STOP_AT_FIRST_REJECT 1u
 int ears_verify_var(int dtype, const void* target_logits, const void* draft_logits,
                     const int32_t* draft_tokens, int B, int K, int V,
                     float temperature, float beta,
-                    const float* seq_temperature, const float* seq_beta,
+                    const float* seq_temperature, const float* seq_beta, unsigned flags,
                     uint64_t seed, uint64_t offset,
                     int64_t b_first, int32_t* out_accept_len, int32_t* out_tokens,
                     double* out_pt_tok, double* out_pd_tok, double* out_max_pt,

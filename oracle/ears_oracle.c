@@ -194,7 +194,7 @@ static void mark_invalid(int b, int K, int32_t* out_accept_len, int32_t* out_tok
 }
 
 static void verify_one(const void* tl, const void* dl, int dtype, const int32_t* x,
-                       int b, int K, int V, double T, double beta,
+                       int b, int K, int V, double T, double beta, int stop_at_first_reject,
                        uint64_t seed, uint64_t offset, int64_t b_first, double band,
                        int32_t* out_accept_len, int32_t* out_tokens,
                        const ears_oracle_diag* dg,
@@ -231,9 +231,13 @@ static void verify_one(const void* tl, const void* dl, int dtype, const int32_t*
             if (dg->cls) dg->cls[i] = (uint8_t)cls;
         }
         if (!accept && n == K) n = k; /* first rejection; later positions are diagnostics only */
+        /* Sec. 3.1: a rejection discards every later draft token, so a caller may ask that their
+         * rows are not read at all (then they are neither validated nor reported) */
+        if (!accept && stop_at_first_reject) break;
     }
-    /* the bonus row is part of the step's input: validate it even when unused */
-    if (valid) {
+    /* the bonus row is part of the step's input: validate it even when unused
+     * (unless the caller asked to stop at the first rejection and there was one) */
+    if (valid && !(stop_at_first_reject && n < K)) {
         for (int v = 0; v < V; ++v) row[v] = logit_at(tl, dtype, ((int64_t)b * (K + 1) + K) * V + v);
         if (ears_oracle_softmax(row, V, T, pt, NULL, NULL)) valid = 0;
     }
@@ -282,12 +286,15 @@ static void verify_one(const void* tl, const void* dl, int dtype, const int32_t*
  *   token, then -1).  Any diagnostic pointer may be NULL.
  * nthreads > 1 spreads sequences over OpenMP threads; results do not depend on it.
  * seq_temperature, seq_beta: optional [B] arrays that replace the scalars per sequence.
+ * stop_at_first_reject != 0: rows and tokens after a sequence's first rejected position (and the
+ *   extra target row, unless everything was accepted) are not read: not validated, no diagnostics.
  * Returns 0, -1 on bad arguments, -2 when out of memory.
  */
 int ears_oracle_verify_var(const void* target_logits, const void* draft_logits, int dtype,
                            const int32_t* draft_tokens, int B, int K, int V,
                            float temperature, float beta,
                            const float* seq_temperature, const float* seq_beta,
+                           int stop_at_first_reject,
                            uint64_t seed, uint64_t offset,
                            int64_t b_first, double band,
                            int32_t* out_accept_len, int32_t* out_tokens,
@@ -331,7 +338,7 @@ int ears_oracle_verify_var(const void* target_logits, const void* draft_logits, 
                 continue;
             }
             verify_one(target_logits, draft_logits, dtype, draft_tokens, b, K, V, (double)Tb, (double)bb,
-                       seed, offset, b_first, band, out_accept_len, out_tokens, &dg, row, pt, pd);
+                       stop_at_first_reject, seed, offset, b_first, band, out_accept_len, out_tokens, &dg, row, pt, pd);
         }
         free(row); free(pt); free(pd);
     }
@@ -349,7 +356,7 @@ int ears_oracle_verify(const void* target_logits, const void* draft_logits, int 
                        int32_t* band_lo, int32_t* band_hi, int nthreads)
 {
     return ears_oracle_verify_var(target_logits, draft_logits, dtype, draft_tokens, B, K, V, temperature, beta,
-                                  NULL, NULL, seed, offset, b_first, band, out_accept_len, out_tokens,
+                                  NULL, NULL, 0, seed, offset, b_first, band, out_accept_len, out_tokens,
                                   pt_tok, pd_tok, max_pt, margin, cls, resid_mass, cdf_margin,
                                   band_lo, band_hi, nthreads);
 }

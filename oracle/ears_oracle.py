@@ -54,7 +54,7 @@ def _load():
     lib.ears_oracle_verify.restype = c.c_int
     lib.ears_oracle_verify_var.argtypes = (
         [c.c_void_p, c.c_void_p, c.c_int, c.c_void_p, c.c_int, c.c_int, c.c_int,
-         c.c_float, c.c_float, c.c_void_p, c.c_void_p, c.c_uint64, c.c_uint64, c.c_int64, c.c_double]
+         c.c_float, c.c_float, c.c_void_p, c.c_void_p, c.c_int, c.c_uint64, c.c_uint64, c.c_int64, c.c_double]
         + [c.c_void_p] * 11 + [c.c_int])
     lib.ears_oracle_verify_var.restype = c.c_int
     lib.ears_oracle_row_softmax.argtypes = [c.c_void_p, c.c_int, c.c_int64, c.c_int, c.c_float, c.c_void_p]
@@ -164,8 +164,10 @@ class OracleResult:
 
 def verify(target_logits, draft_logits, draft_tokens, temperature: float, beta: float,
            seed: int = 0, offset: int = 0, b_first: int = 0, band: float = 1e-6,
-           nthreads: int = 1, seq_temperature=None, seq_beta=None) -> OracleResult:
-    """seq_temperature / seq_beta: optional [B] float32 arrays replacing the scalars per sequence."""
+           nthreads: int = 1, seq_temperature=None, seq_beta=None,
+           stop_at_first_reject: bool = False) -> OracleResult:
+    """seq_temperature / seq_beta: optional [B] float32 arrays replacing the scalars per sequence.
+    stop_at_first_reject: rows after a sequence's first rejection are not read (nor validated)."""
     lib = _load()
     t, ct = _as_logits(target_logits)
     d, cd = _as_logits(draft_logits)
@@ -188,7 +190,8 @@ def verify(target_logits, draft_logits, draft_tokens, temperature: float, beta: 
     rc = lib.ears_oracle_verify_var(
         t.ctypes.data, d.ctypes.data, ct, x.ctypes.data, B, K, V,
         float(temperature), float(beta), None if st is None else st.ctypes.data,
-        None if sb is None else sb.ctypes.data, int(seed), int(offset), int(b_first), float(band),
+        None if sb is None else sb.ctypes.data, int(bool(stop_at_first_reject)),
+        int(seed), int(offset), int(b_first), float(band),
         acc.ctypes.data, tok.ctypes.data, res.pt_tok.ctypes.data, res.pd_tok.ctypes.data,
         res.max_pt.ctypes.data, res.margin.ctypes.data, res.cls.ctypes.data,
         res.resid_mass.ctypes.data, res.cdf_margin.ctypes.data,

@@ -43,7 +43,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ears_verify_ex.argtypes = ([c.c_int] + common + [c.c_int64] + [c.c_void_p] * 7
                                    + [c.c_void_p, c.c_size_t, c.c_void_p])
     lib.ears_verify_ex.restype = c.c_int
-    lib.ears_verify_var.argtypes = ([c.c_int] + common[:8] + [c.c_void_p, c.c_void_p] + common[8:] + [c.c_int64]
+    lib.ears_verify_var.argtypes = ([c.c_int] + common[:8] + [c.c_void_p, c.c_void_p, c.c_uint] + common[8:] + [c.c_int64]
                                     + [c.c_void_p] * 7 + [c.c_void_p, c.c_size_t, c.c_void_p])
     lib.ears_verify_var.restype = c.c_int
     lib.ears_verify_host.argtypes = [c.c_int] + common + [c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p]
@@ -119,13 +119,15 @@ def _stream_ptr(stream) -> int:
 def verify(target_logits: torch.Tensor, draft_logits: torch.Tensor, draft_tokens: torch.Tensor,
            temperature: float, beta: float, seed: int = 0, offset: int = 0, *, b_first: int = 0,
            stats: bool = False, workspace: Optional[torch.Tensor] = None, stream=None,
-           seq_temperature: Optional[torch.Tensor] = None, seq_beta: Optional[torch.Tensor] = None):
+           seq_temperature: Optional[torch.Tensor] = None, seq_beta: Optional[torch.Tensor] = None,
+           stop_at_first_reject: bool = False):
     """One EARS verification step on the current CUDA device.
 
     Returns (accept_len [B] int32, tokens [B,K+1] int32) and, with ``stats=True``, a dict with
     pt_tok, pd_tok, max_pt [B,K] float64, cls [B,K] uint8 and resid_mass [B] float64.
     ``seq_temperature`` / ``seq_beta``: optional float32 CUDA tensors [B] that replace the scalar
-    for each sequence (ears_verify_var).
+    for each sequence (ears_verify_var).  ``stop_at_first_reject``: rows after a sequence's first
+    rejection are not part of the step (EARS_FLAG_STOP_AT_FIRST_REJECT).
     The call is asynchronous on ``stream`` (default: torch's current stream).
     """
     lib = load_library()
@@ -149,7 +151,7 @@ def verify(target_logits: torch.Tensor, draft_logits: torch.Tensor, draft_tokens
                       resid_mass=torch.zeros(B, dtype=torch.float64, device=dev))
             ptrs = [st[k].data_ptr() for k in ("pt_tok", "pd_tok", "max_pt", "cls", "resid_mass")]
         ws_ptr, ws_bytes = (None, 0) if workspace is None else (workspace.data_ptr(), workspace.numel() * workspace.element_size())
-        if seq_temperature is None and seq_beta is None:
+        if seq_temperature is None and seq_beta is None and not stop_at_first_reject:
             rc = lib.ears_verify_ex(_dtype_code(t), t.data_ptr(), d.data_ptr(), x.data_ptr(), B, K, V,
                                     float(temperature), float(beta), int(seed), int(offset), int(b_first),
                                     acc.data_ptr(), tok.data_ptr(), *ptrs, ws_ptr, ws_bytes, _stream_ptr(stream))
@@ -165,6 +167,7 @@ def verify(target_logits: torch.Tensor, draft_logits: torch.Tensor, draft_tokens
                                      float(temperature), float(beta),
                                      None if arrs[0] is None else arrs[0].data_ptr(),
                                      None if arrs[1] is None else arrs[1].data_ptr(),
+                                     1 if stop_at_first_reject else 0,
                                      int(seed), int(offset), int(b_first),
                                      acc.data_ptr(), tok.data_ptr(), *ptrs, ws_ptr, ws_bytes, _stream_ptr(stream))
     _check(rc)

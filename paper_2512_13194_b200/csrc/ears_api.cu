@@ -46,7 +46,16 @@ struct DeviceInfo {
 };
 std::map<int, DeviceInfo> g_devices;
 
-struct Buffer { void* ptr = nullptr; size_t bytes = 0; };
+struct Buffer {
+    void* ptr = nullptr;
+    size_t bytes = 0;
+    // Library-owned workspaces carry two copies of the counter block.  A call uses one and its
+    // kernel zeroes the other for the next call of the same shape, which then needs no memset
+    // (and starts clean even if this call was cut short by a device-side timeout).
+    int clean_set = -1;            // copy that is known to be all zero, -1: none
+    unsigned long long sig = 0;    // kernel kind and sizes the copies were laid out for
+    void* status_word = nullptr;   // status word of the most recent call
+};
 std::map<std::pair<int, void*>, Buffer> g_workspaces;  // (device, stream) -> scratch
 std::map<std::pair<int, void*>, Buffer> g_staging;     // (device, stream) -> host-entry staging
 
@@ -214,7 +223,9 @@ int profile_mark(cudaStream_t stream, bool timed) {
 
 template <typename E>
 int set_attrs(bool* cluster16) {
-    EARS_CUDA(cudaFuncSetAttribute(ears_verify_kernel<E, kStages>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    EARS_CUDA(cudaFuncSetAttribute(ears_verify_kernel<E, kStages, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)smem_bytes()));
+    EARS_CUDA(cudaFuncSetAttribute(ears_verify_kernel<E, kStages, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)smem_bytes()));
     EARS_CUDA(cudaFuncSetAttribute(ears_resident_kernel<E>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)kResidentSmem2));
@@ -260,7 +271,7 @@ int resident_clusters(DeviceInfo* di, const RPlan& rp, int* out) {
 
 template <typename E>
 int launch_resident(RParams& p, const RPlan& rp, int max_clusters, cudaStream_t stream) {
-    const long long items = (long long)p.B * (p.K + 1);
+    const long long items = p.ordered ? (long long)p.B : (long long)p.B * (p.K + 1);
     p.n_clusters = (int)(items < max_clusters ? items : max_clusters);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(p.n_clusters * rp.C), 1, 1);
@@ -287,7 +298,8 @@ int launch(const Params& p, int sms, cudaStream_t stream) {
     const bool timed = g_profile.active && (int)g_profile.events.size() + 2 <= 2 * g_profile.max_calls;
     int rc = profile_mark(stream, timed);
     if (rc) return rc;
-    ears_verify_kernel<E, kStages><<<grid, kThreads, smem_bytes(), stream>>>(p);
+    if (p.seq_T) ears_verify_kernel<E, kStages, true><<<grid, kThreads, smem_bytes(), stream>>>(p);
+    else ears_verify_kernel<E, kStages, false><<<grid, kThreads, smem_bytes(), stream>>>(p);
     EARS_CUDA(cudaGetLastError());
     return profile_mark(stream, timed);
 }
@@ -306,8 +318,55 @@ int get_buffer(std::map<std::pair<int, void*>, Buffer>& pool, int dev, void* str
         const size_t want = align_up(bytes + bytes / 4, 1 << 20);
         EARS_CUDA(cudaMalloc(&b.ptr, want));
         b.bytes = want;
+        b.clean_set = -1;
+        b.status_word = nullptr;
     }
     *out = b.ptr;
+    return EARS_OK;
+}
+
+// A launch that failed has not cleared the other copy: the next call must start with a memset.
+void forget_clean_counters(int dev, void* stream_) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    auto it = g_workspaces.find(std::make_pair(dev, stream_));
+    if (it != g_workspaces.end()) it->second.clean_set = -1;
+}
+
+// Picks the counter block of a call on `stream`.  Caller-owned workspace: the block at its start,
+// cleared by a memset.  Library-owned: see Buffer.  *zero_ptr / *zero_words name the other copy,
+// which the kernel clears (0 words: nothing to clear).
+int pick_counters(void* caller_ws, int dev, void* stream_, int kind, size_t counters_bytes, size_t total,
+                  char** base, char** counters, int** zero_ptr, int* zero_words) {
+    cudaStream_t stream = (cudaStream_t)stream_;
+    const size_t cb = align_up(counters_bytes, 256);
+    if (caller_ws) {
+        *base = (char*)caller_ws;
+        *counters = *base;
+        *zero_ptr = nullptr;
+        *zero_words = 0;
+        EARS_CUDA(cudaMemsetAsync(*counters, 0, counters_bytes, stream));
+        return EARS_OK;
+    }
+    void* ws = nullptr;
+    const size_t main_bytes = align_up(total, 256);
+    int rc = get_buffer(g_workspaces, dev, stream_, main_bytes + cb, &ws);
+    if (rc) return rc;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    Buffer& b = g_workspaces[std::make_pair(dev, stream_)];
+    char* set[2] = {(char*)ws, (char*)ws + main_bytes};
+    const unsigned long long sig = ((unsigned long long)kind << 60) ^ ((unsigned long long)counters_bytes << 32) ^ (unsigned long long)total;
+    int use = b.clean_set;
+    if (use < 0 || b.sig != sig) {
+        use = 0;
+        EARS_CUDA(cudaMemsetAsync(set[0], 0, counters_bytes, stream));
+    }
+    b.sig = sig;
+    b.clean_set = 1 - use;          // the kernel of this call clears it
+    b.status_word = set[use] + 2 * sizeof(int);
+    *base = (char*)ws;
+    *counters = set[use];
+    *zero_ptr = (int*)set[1 - use];
+    *zero_words = (int)(cb / sizeof(int));
     return EARS_OK;
 }
 
@@ -352,12 +411,14 @@ int ensure_attrs(DeviceInfo* di) {
 }
 
 int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B, int K, int V,
-                float temperature, float beta, const float* seq_T, const float* seq_beta,
+                float temperature, float beta, const float* seq_T, const float* seq_beta, unsigned flags,
                 uint64_t seed, uint64_t offset, int64_t b_first,
                 int32_t* out_len, int32_t* out_tok, double* o_pt, double* o_pd, double* o_max,
                 uint8_t* o_cls, double* o_resid, void* workspace, size_t workspace_bytes, void* stream_) {
     if (!t || !d || !x || !out_len || !out_tok) return EARS_ERR_NULL;
     if (dtype != EARS_DTYPE_F32 && dtype != EARS_DTYPE_BF16) return EARS_ERR_PARAM;
+    if (flags & ~(unsigned)EARS_FLAG_STOP_AT_FIRST_REJECT) return EARS_ERR_PARAM;
+    const int stop_first = (flags & EARS_FLAG_STOP_AT_FIRST_REJECT) ? 1 : 0;
     int rc = check_shape(B, K, V);
     if (rc) return rc;
     // a per-sequence array replaces its scalar, which is then not looked at
@@ -396,15 +457,11 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
     if (rc) return rc;
     if (rp.ok) {
         const RLayout L = make_rlayout(B, K);
-        if (workspace) {
-            if (workspace_bytes < L.total) return EARS_ERR_WORKSPACE;
-        } else {
-            rc = get_buffer(g_workspaces, dev, stream_, L.total, &workspace);
-            if (rc) return rc;
-        }
-        char* w = (char*)workspace;
-        EARS_CUDA(cudaMemsetAsync(w, 0, L.counters_bytes, stream));
+        if (workspace && workspace_bytes < L.total) return EARS_ERR_WORKSPACE;
+        char *w = nullptr, *cw = nullptr;
         RParams p;
+        rc = pick_counters(workspace, dev, stream_, 2, L.counters_bytes, L.total, &w, &cw, &p.zero_ptr, &p.zero_words);
+        if (rc) return rc;
         p.t = t; p.d = d; p.x = x;
         p.B = B; p.K = K; p.V = V;
         p.c = c;
@@ -418,8 +475,8 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
         p.max_pt = o_max ? o_max : (double*)(w + L.max_pt);
         p.cls = o_cls ? o_cls : (uint8_t*)(w + L.cls);
         p.resid = o_resid ? o_resid : (double*)(w + L.resid);
-        p.heads = (int*)(w + L.heads);
-        p.ticket = (int*)(w + L.ticket);
+        p.heads = (int*)(cw + L.heads);
+        p.ticket = (int*)(cw + L.ticket);
         p.flag = (signed char*)(w + L.flag);
         p.cand = (int32_t*)(w + L.cand);
         p.cand_mass = (double*)(w + L.cand_mass);
@@ -427,22 +484,21 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
         p.use_tma = aligned && ov.loader != 2;
         p.n_clusters = 0;
         p.want_stats = (o_pt || o_pd || o_max || o_cls) ? 1 : 0;
-        return dtype == EARS_DTYPE_F32 ? launch_resident<float>(p, rp, max_clusters, stream)
-                                       : launch_resident<uint16_t>(p, rp, max_clusters, stream);
+        p.ordered = stop_first;
+        rc = dtype == EARS_DTYPE_F32 ? launch_resident<float>(p, rp, max_clusters, stream)
+                                     : launch_resident<uint16_t>(p, rp, max_clusters, stream);
+        if (rc && !workspace) forget_clean_counters(dev, stream_);
+        return rc;
     }
 
     const Plan plan = make_plan(B, K, V, esize, aligned, di->sms, ov);
     const Layout L = make_layout(B, K, V, plan.parts1);
-    if (workspace) {
-        if (workspace_bytes < L.total) return EARS_ERR_WORKSPACE;
-    } else {
-        rc = get_buffer(g_workspaces, dev, stream_, L.total, &workspace);
-        if (rc) return rc;
-    }
-    char* w = (char*)workspace;
-    EARS_CUDA(cudaMemsetAsync(w, 0, L.counters_bytes, stream));
-
+    if (workspace && workspace_bytes < L.total) return EARS_ERR_WORKSPACE;
+    char *w = nullptr, *cw = nullptr;
     Params p;
+    rc = pick_counters(workspace, dev, stream_, 1, L.counters_bytes, L.total, &w, &cw, &p.zero_ptr, &p.zero_words);
+    if (rc) return rc;
+
     p.t = t; p.d = d; p.x = x;
     p.B = B; p.K = K; p.V = V;
     p.c = c;
@@ -456,19 +512,22 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
     p.max_pt = o_max ? o_max : (double*)(w + L.max_pt);
     p.cls = o_cls ? o_cls : (uint8_t*)(w + L.cls);
     p.resid = o_resid ? o_resid : (double*)(w + L.resid);
-    p.ticket1 = (int*)(w + L.ticket1);
-    p.ticket_row = (int*)(w + L.ticket_row);
-    p.ticket2 = (int*)(w + L.ticket2);
-    p.job_ctr = (int*)(w + L.job_ctr);
-    p.ready = (unsigned long long*)(w + L.ready);
-    p.heads = (int*)(w + L.heads);
-    p.wq = (unsigned long long*)(w + L.wq);
+    p.ticket1 = (int*)(cw + L.ticket1);
+    p.ticket_row = (int*)(cw + L.ticket_row);
+    p.ticket2 = (int*)(cw + L.ticket2);
+    p.job_ctr = (int*)(cw + L.job_ctr);
+    p.ready = (unsigned long long*)(cw + L.ready);
+    p.heads = (int*)(cw + L.heads);
+    p.wq = (unsigned long long*)(cw + L.wq);
     p.partial = (float2*)(w + L.partial);
     p.rowstat = (float2*)(w + L.rowstat);
     p.seg_base = (unsigned char*)(w + L.seg);
     p.seg_stride = L.seg_stride;
+    p.stop_first = stop_first;
     p.plan = plan;
-    return dtype == EARS_DTYPE_F32 ? launch<float>(p, di->sms, stream) : launch<uint16_t>(p, di->sms, stream);
+    rc = dtype == EARS_DTYPE_F32 ? launch<float>(p, di->sms, stream) : launch<uint16_t>(p, di->sms, stream);
+    if (rc && !workspace) forget_clean_counters(dev, stream_);
+    return rc;
 }
 
 size_t workspace_bound(int B, int K, int V) {
@@ -555,20 +614,20 @@ int ears_verify_ex(int dtype, const void* target_logits, const void* draft_logit
                    int32_t* out_tokens, double* out_pt_tok, double* out_pd_tok, double* out_max_pt,
                    uint8_t* out_class, double* out_resid_mass, void* workspace, size_t workspace_bytes,
                    void* stream) {
-    return verify_impl(dtype, target_logits, draft_logits, draft_tokens, B, K, V, temperature, beta, nullptr, nullptr,
+    return verify_impl(dtype, target_logits, draft_logits, draft_tokens, B, K, V, temperature, beta, nullptr, nullptr, 0u,
                        seed, offset, b_first, out_accept_len, out_tokens, out_pt_tok, out_pd_tok, out_max_pt,
                        out_class, out_resid_mass, workspace, workspace_bytes, stream);
 }
 
 int ears_verify_var(int dtype, const void* target_logits, const void* draft_logits,
                     const int32_t* draft_tokens, int B, int K, int V, float temperature, float beta,
-                    const float* seq_temperature, const float* seq_beta,
+                    const float* seq_temperature, const float* seq_beta, unsigned flags,
                     uint64_t seed, uint64_t offset, int64_t b_first, int32_t* out_accept_len,
                     int32_t* out_tokens, double* out_pt_tok, double* out_pd_tok, double* out_max_pt,
                     uint8_t* out_class, double* out_resid_mass, void* workspace, size_t workspace_bytes,
                     void* stream) {
     return verify_impl(dtype, target_logits, draft_logits, draft_tokens, B, K, V, temperature, beta,
-                       seq_temperature, seq_beta, seed, offset, b_first, out_accept_len, out_tokens, out_pt_tok,
+                       seq_temperature, seq_beta, flags, seed, offset, b_first, out_accept_len, out_tokens, out_pt_tok,
                        out_pd_tok, out_max_pt, out_class, out_resid_mass, workspace, workspace_bytes, stream);
 }
 
@@ -576,7 +635,7 @@ int ears_verify_f32(const float* target_logits, const float* draft_logits, const
                     int B, int K, int V, float temperature, float beta, uint64_t seed, uint64_t offset,
                     int32_t* out_accept_len, int32_t* out_tokens, void* stream) {
     return verify_impl(EARS_DTYPE_F32, target_logits, draft_logits, draft_tokens, B, K, V, temperature, beta,
-                       nullptr, nullptr, seed, offset, 0, out_accept_len, out_tokens, nullptr, nullptr, nullptr, nullptr, nullptr,
+                       nullptr, nullptr, 0u, seed, offset, 0, out_accept_len, out_tokens, nullptr, nullptr, nullptr, nullptr, nullptr,
                        nullptr, 0, stream);
 }
 
@@ -584,7 +643,7 @@ int ears_verify_bf16(const void* target_logits, const void* draft_logits, const 
                      int B, int K, int V, float temperature, float beta, uint64_t seed, uint64_t offset,
                      int32_t* out_accept_len, int32_t* out_tokens, void* stream) {
     return verify_impl(EARS_DTYPE_BF16, target_logits, draft_logits, draft_tokens, B, K, V, temperature, beta,
-                       nullptr, nullptr, seed, offset, 0, out_accept_len, out_tokens, nullptr, nullptr, nullptr, nullptr, nullptr,
+                       nullptr, nullptr, 0u, seed, offset, 0, out_accept_len, out_tokens, nullptr, nullptr, nullptr, nullptr, nullptr,
                        nullptr, 0, stream);
 }
 
@@ -618,7 +677,7 @@ int ears_verify_host(int dtype, const void* target_logits, const void* draft_log
     EARS_CUDA(cudaMemcpyAsync(s + o_t, target_logits, tb, cudaMemcpyHostToDevice, stream));
     EARS_CUDA(cudaMemcpyAsync(s + o_d, draft_logits, db, cudaMemcpyHostToDevice, stream));
     EARS_CUDA(cudaMemcpyAsync(s + o_x, draft_tokens, xb, cudaMemcpyHostToDevice, stream));
-    rc = verify_impl(dtype, s + o_t, s + o_d, (const int32_t*)(s + o_x), B, K, V, temperature, beta, nullptr, nullptr,
+    rc = verify_impl(dtype, s + o_t, s + o_d, (const int32_t*)(s + o_x), B, K, V, temperature, beta, nullptr, nullptr, 0u,
                      seed, offset, b_first, (int32_t*)(s + o_l), (int32_t*)(s + o_o), nullptr, nullptr, nullptr, nullptr,
                      nullptr, nullptr, 0, stream_);
     if (rc) return rc;
@@ -642,7 +701,7 @@ int ears_verify_noalloc(int dtype, const void* target_logits, const void* draft_
     void* scratch = nullptr;
     rc = noalloc_scratch(dev, &scratch);
     if (rc) return rc;
-    rc = verify_impl(dtype, target_logits, draft_logits, draft_tokens, B, K, V, temperature, beta, nullptr, nullptr,
+    rc = verify_impl(dtype, target_logits, draft_logits, draft_tokens, B, K, V, temperature, beta, nullptr, nullptr, 0u,
                      seed, offset, b_first, out_accept_len, out_tokens, nullptr, nullptr, nullptr, nullptr, nullptr, scratch,
                      (size_t)EARS_NOALLOC_SCRATCH_BYTES, stream);
     if (rc) return rc;
@@ -660,17 +719,17 @@ size_t ears_workspace_bytes(int B, int K, int V) {
 int ears_last_device_status(void* stream_) {
     int dev = 0;
     EARS_CUDA(cudaGetDevice(&dev));
-    void* ws = nullptr;
+    void* word = nullptr;
     {
         std::lock_guard<std::mutex> lock(g_mutex);
         auto it = g_workspaces.find(std::make_pair(dev, stream_));
-        if (it != g_workspaces.end()) ws = it->second.ptr;
+        if (it != g_workspaces.end()) word = it->second.status_word;
     }
-    if (!ws) {
+    if (!word) {
         EARS_CUDA(cudaStreamSynchronize((cudaStream_t)stream_));
         return 0;
     }
-    return ears_workspace_device_status(ws, stream_);
+    return read_status((int*)word - 2, (cudaStream_t)stream_);
 }
 
 int ears_workspace_device_status(void* workspace, void* stream_) {

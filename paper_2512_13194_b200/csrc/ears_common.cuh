@@ -82,8 +82,16 @@ struct Params {
     // segment sums (double [nseg]); a sequence never needs both at once.
     unsigned char* seg_base;
     size_t seg_stride;
+    int stop_first;       // 1: what lies after a sequence's first rejection is neither validated nor reported
+    int* zero_ptr;        // counter block of the next call, cleared by this kernel (zero_words ints; may be 0)
+    int zero_words;
     Plan plan;
 };
+
+// All threads of the grid clear the other copy of the counter block (see the host side).
+template <class P> __device__ __forceinline__ void clear_next_counters(const P& p) {
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < p.zero_words; i += gridDim.x * blockDim.x) p.zero_ptr[i] = 0;
+}
 
 // Temperature and base tolerance of (local) sequence b: the per-sequence arrays where given,
 // else the call's scalars.  c = log2(e) / T is formed the way the host forms it for the scalar.

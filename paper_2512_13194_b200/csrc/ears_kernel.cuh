@@ -34,7 +34,7 @@ namespace ears {
 enum ChunkKind : int { kStats = 0, kFinal = 1, kEnd = 4 };
 enum MsgKind : int { kMsgPiece = 0, kMsgJobPiece = 1, kMsgExit = 3, kMsgNone = 6 };
 
-struct StageMeta {
+struct alignas(16) StageMeta {   // 32 bytes: two 16-byte shared-memory accesses
     int kind;    // ChunkKind
     int id;      // unit index (statistics) or sequence index (final-token rows)
     int nelem;   // valid elements per row in the slot
@@ -42,6 +42,7 @@ struct StageMeta {
     int elem0;   // index of the slot's first element within its row
     int aux;     // statistics: 1 for the extra target row; final-token rows: position n
     float c;     // log2(e) / temperature of the slot's sequence
+    int pad;
 };
 
 struct Msg { int kind, a, b, c; };
@@ -345,6 +346,10 @@ __device__ int finalize_sequence(const Params& p, int b, int lane) {
     const E* d = reinterpret_cast<const E*>(p.d);
     const float cb = seq_c(p, b);
     const double Tb = seq_temperature(p, b), betab = seq_beta(p, b);
+    // `bad`: something that invalidates the sequence wherever it is; with stop_first only what lies
+    // at or before the first rejection counts [Sec. 3.1: later draft tokens are discarded anyway],
+    // tracked per position in `stop` (the first position that is rejected or unusable ends the scan).
+    const bool stop_first = p.stop_first != 0;
     bool bad = !seq_params_ok(Tb, betab);
     for (int r = lane; r < R; r += 32) {
         float m = -INFINITY, s = 0.0f;
@@ -353,21 +358,23 @@ __device__ int finalize_sequence(const Params& p, int b, int lane) {
             float2 v = __ldcg(pp + i);
             merge_ms(m, s, v.x, v.y, cb);
         }
-        if (!rowstat_ok(m, s)) bad = true;
+        if (!rowstat_ok(m, s) && !stop_first) bad = true;
         p.rowstat[(size_t)b * R + r] = make_float2(m, s);
     }
     __syncwarp();
     int first_reject = K;
+    bool stopped_on_bad = false;
     for (int k0 = 0; k0 < K; k0 += 32) {
         const int k = k0 + lane;
-        bool reject = false;
+        bool reject = false, posbad = false;
         if (k < K) {
             const int tok = p.x[(size_t)b * K + k];
+            const float2 st = __ldcg(&p.rowstat[(size_t)b * R + 2 * k]);
+            const float2 sd = __ldcg(&p.rowstat[(size_t)b * R + 2 * k + 1]);
+            posbad = tok < 0 || tok >= V || !rowstat_ok(st.x, st.y) || !rowstat_ok(sd.x, sd.y);
             if (tok < 0 || tok >= V) {
-                bad = true;
+                if (!stop_first) bad = true;
             } else {
-                const float2 st = __ldcg(&p.rowstat[(size_t)b * R + 2 * k]);
-                const float2 sd = __ldcg(&p.rowstat[(size_t)b * R + 2 * k + 1]);
                 const double lt = (double)load_logit(t + (size_t)target_row(b, k, K) * V + tok);
                 const double ld = (double)load_logit(d + (size_t)draft_row(b, k, K) * V + tok);
                 const double U = uniform_accept(p.seed, p.offset, (uint32_t)(p.b_first + b), (uint32_t)k);
@@ -380,8 +387,19 @@ __device__ int finalize_sequence(const Params& p, int b, int lane) {
                 p.cls[i] = dc.cls;
             }
         }
-        const unsigned rej = __ballot_sync(0xffffffffu, reject);
-        if (rej != 0 && first_reject == K) first_reject = k0 + __ffs(rej) - 1;
+        const unsigned rej = __ballot_sync(0xffffffffu, stop_first ? (reject || posbad) : reject);
+        const unsigned pb = __ballot_sync(0xffffffffu, posbad);
+        if (rej != 0 && first_reject == K) {
+            first_reject = k0 + __ffs(rej) - 1;
+            stopped_on_bad = ((pb >> (__ffs(rej) - 1)) & 1u) != 0;
+        }
+    }
+    if (stop_first) {
+        if (stopped_on_bad) bad = true;
+        if (first_reject == K) {   // everything accepted: now the extra target row matters too
+            const float2 sb = __ldcg(&p.rowstat[(size_t)b * R + 2 * K]);
+            if (!rowstat_ok(sb.x, sb.y)) bad = true;
+        }
     }
     bad = __any_sync(0xffffffffu, bad);
     int32_t* ot = p.out_tok + (size_t)b * (K + 1);
@@ -592,7 +610,9 @@ __device__ void select_token(const Params& p, int b, int n, int lane) {
 }
 
 // ---- the kernel -------------------------------------------------------------------
-template <typename E, int STAGES>
+// PER_SEQ: the call carries per-sequence temperatures, so log2(e)/T comes with every slot;
+// otherwise it is the kernel parameter (kept apart: the consumers' code is sensitive to it).
+template <typename E, int STAGES, bool PER_SEQ>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const Params p) {
     extern __shared__ unsigned char smem_raw[];
     using Smem = PipeSmem<STAGES>;
@@ -606,6 +626,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
     const E* tbase = reinterpret_cast<const E*>(p.t);
     const E* dbase = reinterpret_cast<const E*>(p.d);
 
+    clear_next_counters(p);
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(&sm.full[s], use_tma ? 1u : 32u);
@@ -684,7 +705,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
                     ok = loader_acquire(sm, q, lane);
                     if (!ok) break;
                     const int ne = min(step, e_end - e0);
-                    const StageMeta mt{kFinal, b, ne, (e0 == e_begin ? 1 : 0) | (e0 + step >= e_end ? 2 : 0), e0, n, cj};
+                    const StageMeta mt{kFinal, b, ne, (e0 == e_begin ? 1 : 0) | (e0 + step >= e_end ? 2 : 0), e0, n, cj, 0};
                     loader_fill<E>(sm, q % STAGES, mt, use_tma, trow + e0, drow + e0, lane, pol_last_use);
                 }
                 if (!ok) break;
@@ -709,7 +730,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
                         ok = loader_acquire(sm, q, lane);
                         if (!ok) break;
                         const int e0 = ch * CHUNK_ELEMS;
-                        const StageMeta mt{kStats, (int)u, min(CHUNK_ELEMS, V - e0), (ch == ch0 ? 1 : 0) | (ch == ch1 - 1 ? 2 : 0), e0, ridx == 2 * K ? 1 : 0, cu};
+                        const StageMeta mt{kStats, (int)u, min(CHUNK_ELEMS, V - e0), (ch == ch0 ? 1 : 0) | (ch == ch1 - 1 ? 2 : 0), e0, ridx == 2 * K ? 1 : 0, cu, 0};
                         // the extra target row is never streamed again (its sums are kept); the other
                         // rows may be, if their position turns out to be the first rejection
                         loader_fill<E>(sm, q % STAGES, mt, use_tma, row + e0, nullptr, lane, ridx == 2 * K ? pol_last_use : pol_keep);
@@ -742,7 +763,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
             }
         }
         if (ok && loader_acquire(sm, q, lane)) {
-            loader_fill<E>(sm, q % STAGES, StageMeta{kEnd, 0, 0, 0, 0, 0, 0.f}, use_tma, (const E*)nullptr, (const E*)nullptr, lane, pol_keep);
+            loader_fill<E>(sm, q % STAGES, StageMeta{kEnd, 0, 0, 0, 0, 0, 0.f, 0}, use_tma, (const E*)nullptr, (const E*)nullptr, lane, pol_keep);
         } else if (use_tma && lane == 0) {
             loader_drain(sm, q);
         }
@@ -906,9 +927,9 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
                 if (mt.flags & 1) { m_run = -INFINITY; s[0] = s[1] = s[2] = s[3] = 0.f; }
                 if (mt.aux) {  // a piece of the extra target row
                     BonusSeg* out = bonus_segs(p, mt.id / (R * P)) + (size_t)(mt.elem0 / CHUNK_ELEMS) * kConsumerWarps + warp;
-                    chunk_stats<E, true>(sm.buf[stage], mt.nelem, warp, lane, mt.c, m_run, s, out);
+                    chunk_stats<E, true>(sm.buf[stage], mt.nelem, warp, lane, PER_SEQ ? mt.c : p.c, m_run, s, out);
                 } else {
-                    chunk_stats<E, false>(sm.buf[stage], mt.nelem, warp, lane, mt.c, m_run, s, nullptr);
+                    chunk_stats<E, false>(sm.buf[stage], mt.nelem, warp, lane, PER_SEQ ? mt.c : p.c, m_run, s, nullptr);
                 }
                 if (!(mt.flags & 2)) {
                     __syncwarp();
@@ -921,7 +942,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
                 for (int off = 16; off > 0; off >>= 1) {
                     float m2 = __shfl_xor_sync(0xffffffffu, m, off);
                     float s2 = __shfl_xor_sync(0xffffffffu, sum, off);
-                    merge_ms(m, sum, m2, s2, mt.c);
+                    merge_ms(m, sum, m2, s2, PER_SEQ ? mt.c : p.c);
                 }
                 if (lane == 0) {
                     const int us = unit_ends % kUnitSlots;
@@ -941,7 +962,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
                 rn = make_rownorm(st, sd);
             }
             double* seg_out = seg_sums(p, b) + mt.elem0 / kSegElems;
-            chunk_segments<E, true>(sm.buf[stage], sm.buf[stage] + kChunkBytes / 2, mt.nelem, warp, lane, rn, mt.c, seg_out);
+            chunk_segments<E, true>(sm.buf[stage], sm.buf[stage] + kChunkBytes / 2, mt.nelem, warp, lane, rn, PER_SEQ ? mt.c : p.c, seg_out);
             if (mt.flags & 2) {
                 // last chunk of the piece: publish the sums; the epilogue warp counts the piece once
                 // all warps are through and, when it is the sequence's last, picks the token

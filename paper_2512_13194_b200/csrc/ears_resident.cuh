@@ -64,6 +64,10 @@ struct RParams {
     int use_tma;
     int n_clusters;
     int want_stats;       // the caller asked for P_t(x), P_d(x), max P_t or the class of every position
+    int* zero_ptr;        // counter block of the next call, cleared by this kernel (zero_words ints; may be 0)
+    int zero_words;
+    int ordered;          // 1: a cluster takes a whole sequence, position by position, and stops at its first
+                          //    rejection [Sec. 3.1]: later rows are never read
 };
 
 struct RSmem {
@@ -304,11 +308,14 @@ __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RPara
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int rank = (int)cluster_ctarank();
     const int cluster_id = blockIdx.x / C;
-    const long long n_items = (long long)p.B * (K + 1);
+    const bool ordered = p.ordered != 0;
+    // queue entries: positions (b, j) in sequence-major order, or whole sequences when ordered
+    const long long n_items = ordered ? (long long)p.B : (long long)p.B * (K + 1);
     const bool use_tma = p.use_tma != 0;
     const E* tbase = reinterpret_cast<const E*>(p.t);
     const E* dbase = reinterpret_cast<const E*>(p.d);
 
+    clear_next_counters(p);
     if (tid == 0) {
         for (int q = 0; q < kRMaxSub; ++q) mbar_init(&sm.full[q], 1);
         for (int i = 0; i < 2; ++i) { mbar_init(&sm.xbar[i], (unsigned)(C * kRWarps)); mbar_init(&sm.mbar2[i], (unsigned)C); }
@@ -333,10 +340,10 @@ __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RPara
     double U = 0.0;
     bool tok_ok = true;
 
-    // Brings in the slices of item `it` and (thread 0) fetches what its decision needs.
-    auto issue_item = [&](long long it) {
-        b = (int)(it / (K + 1));
-        j = (int)(it % (K + 1));
+    // Brings in the slices of position j of sequence b and (thread 0) fetches what its decision needs.
+    auto issue_item = [&](int nb, int nj) {
+        b = nb;
+        j = nj;
         pair = j < K;
         const E* trow = tbase + (size_t)target_row(b, j, K) * V + e0;
         const E* drow = dbase + (size_t)draft_row(b, pair ? j : 0, K) * V + e0;
@@ -360,7 +367,8 @@ __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RPara
             __syncthreads();
         }
         if (tid == 0) {
-            if (rank == 0) next_item = atomicAdd(&p.heads[0], 1) + p.n_clusters;
+            // the cluster's next queue entry: one per position, or one per sequence when ordered
+            if (rank == 0 && (!ordered || j == 0)) next_item = atomicAdd(&p.heads[0], 1) + p.n_clusters;
             tok_ok = true;
             if (pair) {
                 const int tok = p.x[(size_t)b * K + j];
@@ -375,7 +383,10 @@ __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RPara
     };
 
     bool have = item < n_items;
-    if (have) issue_item(item);
+    if (have) {
+        if (ordered) issue_item((int)item, 0);
+        else issue_item((int)(item / (K + 1)), (int)(item % (K + 1)));
+    }
     // barriers of every CTA are initialised before any peer arrives on them; the first copies
     // (into this CTA's own memory only) are already under way
     cluster_sync_all();
@@ -579,9 +590,34 @@ __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RPara
         //         CTA report this item and count it; the sequence's last item finishes the sequence
         __syncthreads();
         const int rb = b, rj = j;
-        have = nxt < n_items;
-        if (have) issue_item(nxt);
-        if (rank == writer && warp == 0) {
+        if (ordered && dec > 0 && pair) {
+            issue_item(b, j + 1);          // accepted: on to the next position (or the extra row) of this sequence
+        } else {
+            have = nxt < n_items;           // (ordered: the sequence ended here, by rejection, bonus token or bad data)
+            if (have) {
+                if (ordered) issue_item((int)nxt, 0);
+                else issue_item((int)(nxt / (K + 1)), (int)(nxt % (K + 1)));
+            }
+        }
+        if (ordered) {
+            // the cluster owns the whole sequence: one CTA writes its outputs when it ends
+            if (rank == writer && warp == 0 && (dec < 0 || rj == K || dec == 0)) {
+                int32_t* ot = p.out_tok + (size_t)rb * (K + 1);
+                if (dec < 0) {
+                    for (int q = lane; q <= K; q += 32) ot[q] = -1;
+                    if (lane == 0) {
+                        p.out_len[rb] = -1;
+                        atomicOr(&p.heads[2], kDevInvalidInput);
+                    }
+                } else {
+                    for (int q = lane; q <= K; q += 32) ot[q] = q < rj ? p.x[(size_t)rb * K + q] : (q == rj ? token : -1);
+                    if (lane == 0) {
+                        p.out_len[rb] = rj;
+                        p.resid[rb] = mass;
+                    }
+                }
+            }
+        } else if (rank == writer && warp == 0) {
             int last = 0;
             if (lane == 0) {
                 const size_t s = (size_t)rb * (K + 1) + rj;

@@ -30,11 +30,14 @@ def main():
     threads = min(oracle.max_threads(), len(os.sched_getaffinity(0)))
     while tally.rows < want_rows:
         acc, tok, st = ears.verify(t, d, x, w.temperature, beta, w.verify_seed, offset, stats=True)
+        # without the optional outputs the resident kernel decides in fp32 away from the threshold
+        acc2, tok2 = ears.verify(t, d, x, w.temperature, beta, w.verify_seed, offset)
         torch.cuda.synchronize()
+        assert torch.equal(acc, acc2) and torch.equal(tok, tok2), f"step {offset}: outputs depend on stats"
         ora = oracle.verify(th, dh, xh, w.temperature, beta, seed=w.verify_seed, offset=offset, nthreads=threads)
         tally.merge(compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, w.K, {k: v.cpu().numpy() for k, v in st.items()}))
         offset += 1
-    print(f"{w.name} beta={beta}: steps={offset} rows={tally.rows} sequences={tally.sequences} "
+    print(f"{w.name} beta={beta} [{ears.describe_plan(w.dtype, w.B, w.K, w.V).split(':')[0]} kernel]: steps={offset} rows={tally.rows} sequences={tally.sequences} "
           f"explained decisions={tally.explained_decisions} tokens={tally.explained_tokens} "
           f"({tally.explained / tally.rows:.2e} of rows) unexplained={len(tally.unexplained)} "
           f"flagged decisions={tally.flagged_decisions} tokens={tally.flagged_tokens} "

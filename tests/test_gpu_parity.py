@@ -362,3 +362,74 @@ def test_parity_per_sequence_temperature_and_beta(ears, forced_path, B, K, V, dt
     ora = oracle.verify(t, d, x, 1.0, 0.0, seed=7, offset=0, b_first=3, nthreads=8, seq_temperature=badT, seq_beta=badb)
     assert ora.accept_len[[1, 2, 4]].tolist() == [-1, -1, -1]
     assert_parity(compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, K), max_explained=1)
+
+
+@pytest.mark.parametrize("path", [1, 2])
+def test_status_and_counters_start_clean_on_every_call_of_one_shape(ears, forced_path, path):
+    """Calls of one shape on the library's workspace alternate between two counter blocks without
+    a memset in between: a call that saw invalid input must not leak its status or counters."""
+    forced_path(path)
+    dev = "cuda:0"
+    w, t, d, x = synth.tiny_inputs(7, 3, 6000, "fp32", seed=91)
+    bad = x.clone()
+    bad[2, 1] = 6000
+    tg, dg, xg, bg = t.to(dev), d.to(dev), x.to(dev), bad.to(dev)
+    ref = ears.verify(tg, dg, xg, 1.0, 0.2, 3, 0)
+    assert ears.last_device_status() == 0
+    for rep in range(4):
+        a, k = ears.verify(tg, dg, bg, 1.0, 0.2, 3, 0)
+        assert ears.last_device_status() == ears.DEV_INVALID_INPUT and a[2].item() == -1
+        for _ in range(1 + rep % 2):       # odd and even numbers of clean calls in between
+            a, k = ears.verify(tg, dg, xg, 1.0, 0.2, 3, 0)
+            assert ears.last_device_status() == 0
+            assert torch.equal(a, ref[0]) and torch.equal(k, ref[1])
+
+
+@pytest.mark.parametrize("path,cluster", [(1, 0), (2, 0), (2, 2), (2, 8)])
+@pytest.mark.parametrize("B,K,V,dtype", [(24, 4, 9000, "fp32"), (200, 3, 1500, "bf16"), (5, 6, 20001, "bf16")])
+def test_parity_stop_at_first_reject(ears, forced_path, B, K, V, dtype, path, cluster):
+    """EARS_FLAG_STOP_AT_FIRST_REJECT against the oracle in the same mode: same lengths and tokens
+    as the full evaluation on clean data, and data planted after the first rejection (NaN, token out
+    of range, a broken extra row) is ignored, while planted at the rejected position it invalidates."""
+    forced_path(path, cluster)
+    dev = "cuda:0"
+    w, t, d, x = synth.tiny_inputs(B, K, V, dtype, seed=640 + K, noise=1.8)
+    T, beta = 1.0, 0.05
+    full = oracle.verify(t, d, x, T, beta, seed=4, offset=2, nthreads=8)
+    n = full.accept_len
+    assert (n < K).sum() >= 3
+    t2, d2, x2 = t.clone(), d.clone(), x.clone()
+    rej = [b for b in range(B) if n[b] < K]
+    for i, b in enumerate(rej):
+        if n[b] + 1 < K:
+            k = int(n[b]) + 1
+            if i % 3 == 0:
+                t2[b, k, 3] = float("nan")
+            elif i % 3 == 1:
+                x2[b, k] = V + 7
+            else:
+                d2[b, k, :] = float("-inf")
+        if i % 2 == 0:
+            t2[b, K, 0] = float("inf")
+    if len(rej) > 4:
+        b = rej[-1]
+        t2[b, int(n[b]), 1] = float("nan")      # at the rejected position: invalid in either mode
+    tally = Tally()
+    for tt, dd, xx in ((t, d, x), (t2, d2, x2)):
+        acc, tok, st = ears.verify(tt.to(dev), dd.to(dev), xx.to(dev), T, beta, 4, 2, stats=True, stop_at_first_reject=True)
+        acc2, tok2 = ears.verify(tt.to(dev), dd.to(dev), xx.to(dev), T, beta, 4, 2, stop_at_first_reject=True)
+        torch.cuda.synchronize()
+        assert ears.last_device_status() & ears.DEV_TIMEOUT == 0
+        assert torch.equal(acc, acc2) and torch.equal(tok, tok2)
+        ora = oracle.verify(tt, dd, xx, T, beta, seed=4, offset=2, nthreads=8, stop_at_first_reject=True)
+        tally.merge(compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, K))
+        # per-position outputs exist up to the first rejection
+        pt = st["pt_tok"].cpu().numpy()
+        for b in range(B):
+            if ora.accept_len[b] >= 0:
+                upto = min(int(ora.accept_len[b]) + 1, K)
+                np.testing.assert_allclose(pt[b, :upto], ora.pt_tok[b, :upto], rtol=1e-5, atol=1e-30)
+    assert_parity(tally, max_explained=1)
+    clean = ears.verify(t.to(dev), d.to(dev), x.to(dev), T, beta, 4, 2)
+    stop = ears.verify(t.to(dev), d.to(dev), x.to(dev), T, beta, 4, 2, stop_at_first_reject=True)
+    assert torch.equal(clean[0], stop[0]) and torch.equal(clean[1], stop[1])

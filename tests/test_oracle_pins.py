@@ -398,3 +398,51 @@ def test_per_sequence_parameters_match_closed_forms_and_scalar_calls():
     assert bad.accept_len[[1, 2, 4]].tolist() == [-1, -1, -1] and (bad.tokens[[1, 2, 4]] == -1).all()
     for b in (0, 3, 5):
         assert bad.accept_len[b] == res.accept_len[b] and np.array_equal(bad.tokens[b], res.tokens[b])
+
+
+# --------------------------------------------------------------------------- stopping at the first rejection
+def test_stop_at_first_reject_reads_nothing_beyond_it():
+    """Sec. 3.1: rejecting x_i rejects every later draft token, so their rows cannot influence the
+    result.  Pins: identical lengths, tokens and masses as the full evaluation on clean data; data
+    planted after the first rejection (NaN rows, tokens out of range, a broken extra row) changes
+    nothing in this mode but invalidates the sequence in the full one; data planted at or before
+    the first rejection invalidates it in both."""
+    rng = np.random.default_rng(5)
+    B, K, V = 40, 4, 30
+    t = rng.normal(0, 2, (B, K + 1, V)).astype(np.float32)
+    d = (t[:, :K] + rng.normal(0, 1.5, (B, K, V))).astype(np.float32)
+    x = rng.integers(0, V, (B, K)).astype(np.int32)
+    full = oracle.verify(t, d, x, 1.0, 0.05, seed=2, offset=1)
+    stop = oracle.verify(t, d, x, 1.0, 0.05, seed=2, offset=1, stop_at_first_reject=True)
+    assert np.array_equal(full.accept_len, stop.accept_len) and np.array_equal(full.tokens, stop.tokens)
+    assert np.array_equal(full.resid_mass, stop.resid_mass)
+    n = full.accept_len
+    assert (n < K).sum() > 10 and (n == K).sum() > 2 and (n < K - 1).sum() > 5
+    for b in range(B):       # diagnostics exist up to the first rejection only
+        upto = min(n[b] + 1, K)
+        assert np.array_equal(stop.pt_tok[b, :upto], full.pt_tok[b, :upto])
+        assert (stop.pt_tok[b, upto:] == 0).all()
+    t2, d2, x2 = t.copy(), d.copy(), x.copy()
+    early = [b for b in range(B) if n[b] < K - 1]
+    for i, b in enumerate(early):
+        k = n[b] + 1                      # a position after the first rejection
+        if i % 3 == 0:
+            t2[b, k, 3] = np.nan
+        elif i % 3 == 1:
+            x2[b, k] = V + 7
+        else:
+            d2[b, k, :] = -np.inf
+    rej = [b for b in range(B) if n[b] < K]
+    for b in rej[::2]:
+        t2[b, K, 0] = np.inf              # the extra row is not needed after a rejection
+    stop2 = oracle.verify(t2, d2, x2, 1.0, 0.05, seed=2, offset=1, stop_at_first_reject=True)
+    full2 = oracle.verify(t2, d2, x2, 1.0, 0.05, seed=2, offset=1)
+    assert np.array_equal(stop2.accept_len, full.accept_len) and np.array_equal(stop2.tokens, full.tokens)
+    assert (full2.accept_len[early] == -1).all() and (full2.accept_len[rej[::2]] == -1).all()
+    t3 = t.copy()
+    for b in rej:
+        t3[b, n[b], 1] = np.nan           # at the rejected position itself
+    stop3 = oracle.verify(t3, d, x, 1.0, 0.05, seed=2, offset=1, stop_at_first_reject=True)
+    assert (stop3.accept_len[rej] == -1).all()
+    ok = [b for b in range(B) if n[b] == K]
+    assert np.array_equal(stop3.tokens[ok], full.tokens[ok])
