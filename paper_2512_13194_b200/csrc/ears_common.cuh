@@ -101,8 +101,13 @@ template <class P> __device__ __forceinline__ double seq_temperature(const P& p,
 template <class P> __device__ __forceinline__ double seq_beta(const P& p, int b) {
     return p.seq_beta ? (double)__ldg(p.seq_beta + b) : p.beta;
 }
+// (kept out of line: the fp64 division would otherwise sit in every role's hot loop, and the
+// streaming kernel is sensitive to the size of those loops)
+__device__ __noinline__ float seq_c_from_array(const float* seq_T, int b) {
+    return (float)(1.4426950408889634 / (double)__ldg(seq_T + b));
+}
 template <class P> __device__ __forceinline__ float seq_c(const P& p, int b) {
-    return p.seq_T ? (float)(1.4426950408889634 / (double)__ldg(p.seq_T + b)) : p.c;
+    return p.seq_T ? seq_c_from_array(p.seq_T, b) : p.c;
 }
 // What the host refuses in the scalar form makes a sequence invalid in the per-sequence form.
 __device__ __forceinline__ bool seq_params_ok(double T, double beta) {

@@ -698,7 +698,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
                 const int step = CHUNK_ELEMS / 2;  // half a slot of each of the two rows
                 const E* trow = tbase + (size_t)target_row(b, n, K) * V;
                 const E* drow = dbase + (size_t)draft_row(b, n, K) * V;
-                const float cj = seq_c(p, b);
+                const float cj = PER_SEQ ? seq_c(p, b) : p.c;
                 const int e_begin = jpart * p.plan.job_elems;
                 const int e_end = min(V, e_begin + p.plan.job_elems);
                 for (int e0 = e_begin; e0 < e_end; e0 += step, ++q) {
@@ -723,7 +723,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
                     const E* row = (ridx == 2 * K) ? tbase + (size_t)target_row(b, K, K) * V
                                                    : ((ridx & 1) ? dbase + (size_t)draft_row(b, ridx >> 1, K) * V
                                                                  : tbase + (size_t)target_row(b, ridx >> 1, K) * V);
-                    const float cu = seq_c(p, b);
+                    const float cu = PER_SEQ ? seq_c(p, b) : p.c;
                     const int ch0 = part * cpp;
                     const int ch1 = min(chunks_per_row, ch0 + cpp);
                     for (int ch = ch0; ch < ch1; ++ch, ++q) {
@@ -793,7 +793,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
             }
             float pm = -INFINITY, ps = 0.f;
             if (m.kind == kMsgPiece && slot_ok) {
-                const float cu = seq_c(p, m.a / (R * P));
+                const float cu = PER_SEQ ? seq_c(p, m.a / (R * P)) : p.c;
                 for (int w = 0; w < kConsumerWarps; ++w) {
                     const float2 v = sm.scratch[m.c % kUnitSlots][w];
                     merge_ms(pm, ps, v.x, v.y, cu);
