@@ -55,6 +55,8 @@ struct Buffer {
     int clean_set = -1;            // copy that is known to be all zero, -1: none
     unsigned long long sig = 0;    // kernel kind and sizes the copies were laid out for
     void* status_word = nullptr;   // status word of the most recent call
+    bool captured = false;         // a call on this workspace was recorded into a CUDA graph: its replays use
+                                   // copy 0 behind the host's back, so from then on every call clears copy 0 itself
 };
 std::map<std::pair<int, void*>, Buffer> g_workspaces;  // (device, stream) -> scratch
 std::map<std::pair<int, void*>, Buffer> g_staging;     // (device, stream) -> host-entry staging
@@ -355,13 +357,16 @@ int pick_counters(void* caller_ws, int dev, void* stream_, int kind, size_t coun
     Buffer& b = g_workspaces[std::make_pair(dev, stream_)];
     char* set[2] = {(char*)ws, (char*)ws + main_bytes};
     const unsigned long long sig = ((unsigned long long)kind << 60) ^ ((unsigned long long)counters_bytes << 32) ^ (unsigned long long)total;
-    int use = b.clean_set;
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    EARS_CUDA(cudaStreamIsCapturing(stream, &capturing));
+    if (capturing != cudaStreamCaptureStatusNone) b.captured = true;
+    int use = b.captured ? -1 : b.clean_set;
     if (use < 0 || b.sig != sig) {
         use = 0;
         EARS_CUDA(cudaMemsetAsync(set[0], 0, counters_bytes, stream));
     }
     b.sig = sig;
-    b.clean_set = 1 - use;          // the kernel of this call clears it
+    b.clean_set = b.captured ? -1 : 1 - use;   // the kernel of this call clears the other copy
     b.status_word = set[use] + 2 * sizeof(int);
     *base = (char*)ws;
     *counters = set[use];

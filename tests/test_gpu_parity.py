@@ -433,3 +433,37 @@ def test_parity_stop_at_first_reject(ears, forced_path, B, K, V, dtype, path, cl
     clean = ears.verify(t.to(dev), d.to(dev), x.to(dev), T, beta, 4, 2)
     stop = ears.verify(t.to(dev), d.to(dev), x.to(dev), T, beta, 4, 2, stop_at_first_reject=True)
     assert torch.equal(clean[0], stop[0]) and torch.equal(clean[1], stop[1])
+
+
+def test_graph_replays_and_eager_calls_share_the_library_workspace(ears):
+    """A call recorded into a CUDA graph (after a warm-up call, so nothing allocates during the
+    capture) replays correctly any number of times, also interleaved with eager calls on the same
+    stream: the counters of every execution start at zero."""
+    dev = "cuda:0"
+    w, t, d, x = synth.tiny_inputs(6, 3, 7000, "fp32", seed=17)
+    tg, dg, xg = t.to(dev), d.to(dev), x.to(dev)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        ref = ears.verify(tg, dg, xg, 1.0, 0.2, 5, 3, stream=side)
+        ref = ears.verify(tg, dg, xg, 1.0, 0.2, 5, 3, stream=side)
+        side.synchronize()
+        acc = torch.empty_like(ref[0])
+        tok = torch.empty_like(ref[1])
+        lib = ears.load_library()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            rc = lib.ears_verify_f32(tg.data_ptr(), dg.data_ptr(), xg.data_ptr(), 6, 3, 7000, 1.0, 0.2, 5, 3,
+                                     acc.data_ptr(), tok.data_ptr(), torch.cuda.current_stream().cuda_stream)
+        assert rc == 0
+        cap_stream = side
+    for rep in range(5):
+        acc.fill_(-7)
+        tok.fill_(-7)
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(acc, ref[0]) and torch.equal(tok, ref[1]), rep
+        if rep % 2:
+            with torch.cuda.stream(cap_stream):
+                a, k = ears.verify(tg, dg, xg, 1.0, 0.2, 5, 3, stream=cap_stream)
+            cap_stream.synchronize()
+            assert torch.equal(a, ref[0]) and torch.equal(k, ref[1])
