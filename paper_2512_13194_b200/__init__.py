@@ -9,6 +9,7 @@ from .binding import (  # noqa: F401
     DEV_INVALID_INPUT,
     DEV_TIMEOUT,
     EarsError,
+    class_counts,
     describe_plan,
     last_device_status,
     load_library,

@@ -243,6 +243,19 @@ def verify_noalloc(target_logits, draft_logits, draft_tokens, temperature, beta,
     _check(rc)
 
 
+def class_counts(stats: dict, accept_len: torch.Tensor) -> dict:
+    """Counts of the three-way decision of Sec. 3.2 step 5 over the positions that were decided,
+    i.e. up to and including each sequence's first rejection: {"direct": .., "pardon": .., "reject": ..}
+    from the ``cls`` output of ``verify(..., stats=True)``."""
+    cls = stats["cls"]
+    B, K = cls.shape
+    n = accept_len.clamp(min=-1).to(torch.int64)
+    upto = torch.where(n < 0, torch.zeros_like(n), torch.clamp(n + 1, max=K))
+    live = torch.arange(K, device=cls.device)[None, :] < upto[:, None]
+    return {"direct": int(((cls == 1) & live).sum()), "pardon": int(((cls == 2) & live).sum()),
+            "reject": int(((cls == 0) & live).sum())}
+
+
 def workspace_bytes(B: int, K: int, V: int) -> int:
     return int(load_library().ears_workspace_bytes(B, K, V))
 

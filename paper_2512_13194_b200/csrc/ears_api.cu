@@ -4,6 +4,7 @@
 
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <mutex>
@@ -35,7 +36,22 @@ int cuda_fail(cudaError_t e, const char* what) {
     } while (0)
 
 struct PlanOverride { int loader = 0, parts1 = 0, path = 0, cluster = 0; };
-PlanOverride g_override;
+
+// Initial choice of kernel from the environment (EARS_PATH=streaming|resident, EARS_CLUSTER=1..16),
+// for trying a launch plan on an unmodified caller; ears_set_path overrides it.
+PlanOverride override_from_env() {
+    PlanOverride ov;
+    if (const char* e = getenv("EARS_PATH")) {
+        if (!strcmp(e, "streaming") || !strcmp(e, "1")) ov.path = 1;
+        else if (!strcmp(e, "resident") || !strcmp(e, "2")) ov.path = 2;
+    }
+    if (const char* e = getenv("EARS_CLUSTER")) {
+        const int c = atoi(e);
+        if (c == 1 || c == 2 || c == 4 || c == 8 || c == 16) ov.cluster = c;
+    }
+    return ov;
+}
+PlanOverride g_override = override_from_env();
 std::mutex g_mutex;
 
 struct DeviceInfo {

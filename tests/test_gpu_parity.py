@@ -467,3 +467,17 @@ def test_graph_replays_and_eager_calls_share_the_library_workspace(ears):
                 a, k = ears.verify(tg, dg, xg, 1.0, 0.2, 5, 3, stream=cap_stream)
             cap_stream.synchronize()
             assert torch.equal(a, ref[0]) and torch.equal(k, ref[1])
+
+
+def test_decision_class_counts_match_the_oracle(ears):
+    """direct / pardon / reject (Sec. 3.2 step 5) counted over the decided positions."""
+    w, t, d, x = synth.tiny_inputs(64, 4, 3000, "fp32", seed=77, noise=1.2)
+    acc, tok, st = ears.verify(t.cuda(), d.cuda(), x.cuda(), 1.0, 0.3, 2, 0, stats=True)
+    got = ears.class_counts(st, acc)
+    ora = oracle.verify(t, d, x, 1.0, 0.3, seed=2, offset=0)
+    want = {"direct": 0, "pardon": 0, "reject": 0}
+    for b in range(64):
+        for k in range(min(int(ora.accept_len[b]) + 1, 4)):
+            want[("reject", "direct", "pardon")[int(ora.cls[b, k])]] += 1
+    assert got == want and got["pardon"] > 0 and got["reject"] > 0
+    assert got["reject"] == int((ora.accept_len < 4).sum())
