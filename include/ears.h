@@ -163,6 +163,21 @@ int ears_verify_var(int dtype, const void* target_logits, const void* draft_logi
                     void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The temperature -> 0 limit of the step (Sec. 1 names temperature = 0 as the deterministic
+ * regime; the entry points above refuse temperature <= 0 because their arithmetic divides by it).
+ * In the limit every softmax is one-hot at its row's largest logit (the smallest index among
+ * equal ones), max P_t = 1, the tolerance beta (1 - max P_t) of Sec. 3.2 is zero, and for a
+ * greedily drafted token R_k is 1 or 0: x_k is accepted iff it is the top token of target row k.
+ * The first mismatch n ends the accepted prefix (Sec. 3.1); out_tokens[b, n] is the top token of
+ * target row n (row K if all K matched).  Draft logits, beta, seed and offset play no role.
+ * Outputs, invalid-sequence marking (NaN, +inf, no finite logit in ANY of the K+1 target rows; a
+ * draft token outside [0, V)), workspace rules and status words are those of ears_verify_ex.
+ */
+int ears_verify_greedy(int dtype, const void* target_logits, const int32_t* draft_tokens,
+                       int B, int K, int V, int32_t* out_accept_len, int32_t* out_tokens,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Same step with HOST buffers: copies the inputs to library-owned device staging
  * buffers, runs the step, copies out_accept_len / out_tokens back and waits for
  * completion.  All pointers are host memory (pinned memory makes the copies
@@ -255,8 +270,9 @@ int ears_set_plan(int loader, int parts);
 
 /*
  * Choice between the two kernels, for tests and measurements (0 = automatic for both fields):
- *   path 1 = streaming kernel (rows pass through a ring of shared-memory slots; the rows of a
- *            rejected position are read a second time), 2 = resident kernel (the two rows of a
+ *   path 1 = streaming kernel with a ring of shared-memory slots filled by bulk copies (the rows of
+ *            a rejected position are read a second time), 3 = streaming kernel whose warps read
+ *            straight from global memory (same second pass), 2 = resident kernel (the two rows of a
  *            position stay in the shared memory of a thread-block cluster; every logit is read
  *            once).  Forcing path 2 on a shape whose rows do not fit a cluster makes the
  *            verification calls return EARS_ERR_SHAPE.  A non-zero `parts` of ears_set_plan

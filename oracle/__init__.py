@@ -15,4 +15,5 @@ from .ears_oracle import (  # noqa: F401
     uniform_accept,
     uniform_final,
     verify,
+    verify_greedy,
 )

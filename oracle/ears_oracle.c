@@ -361,6 +361,63 @@ int ears_oracle_verify(const void* target_logits, const void* draft_logits, int 
                                   band_lo, band_hi, nthreads);
 }
 
+/*
+ * The temperature -> 0 limit of the step (the deterministic regime of Sec. 1): every softmax
+ * becomes one-hot at its row's largest logit (the smallest index among equal ones), so
+ * max_v P_t = 1, the tolerance beta (1 - max P_t) vanishes [Sec. 3.2], and for a draft token
+ * drawn greedily (P_d(x_k) = 1) the ratio R_k is 1 if x_k is the target's top token and 0
+ * otherwise: x_k is accepted iff it equals argmax of target row k.  The token at the first
+ * rejected position n is argmax of target row n (the residual of two different one-hot
+ * distributions is the target's), the bonus token argmax of row K.  No random numbers, no draft
+ * logits.  Rows are validated like everywhere else (NaN, +inf, no finite entry: the sequence is
+ * marked invalid); a draft token outside [0, V) is invalid too.
+ */
+int ears_oracle_verify_greedy(const void* target_logits, int dtype, const int32_t* draft_tokens,
+                              int B, int K, int V, int32_t* out_accept_len, int32_t* out_tokens,
+                              int32_t* argmax_out /* [B,K+1] or NULL */)
+{
+    if (!target_logits || !draft_tokens || !out_accept_len || !out_tokens) return -1;
+    if (B < 1 || K < 1 || V < 1 || (dtype != 0 && dtype != 1)) return -1;
+    for (int b = 0; b < B; ++b) {
+        int valid = 1, n = K;
+        for (int k = 0; k <= K; ++k) {
+            int best = -1;
+            double top = -INFINITY;
+            for (int v = 0; v < V; ++v) {
+                double l = logit_at(target_logits, dtype, ((int64_t)b * (K + 1) + k) * V + v);
+                if (isnan(l) || l == INFINITY) valid = 0;
+                if (l > top) { top = l; best = v; }   /* strict: the first of equal entries stays */
+            }
+            if (best < 0) valid = 0;                  /* nothing finite */
+            if (argmax_out) argmax_out[(int64_t)b * (K + 1) + k] = best;
+            if (k < K) {
+                int tok = draft_tokens[(int64_t)b * K + k];
+                if (tok < 0 || tok >= V) valid = 0;
+                if (tok != best && n == K) n = k;     /* first rejection [Sec. 3.1] */
+            }
+        }
+        if (!valid) { mark_invalid(b, K, out_accept_len, out_tokens); continue; }
+        out_accept_len[b] = n;
+        for (int j = 0; j <= K; ++j) {
+            int64_t o = (int64_t)b * (K + 1) + j;
+            out_tokens[o] = j < n ? draft_tokens[(int64_t)b * K + j] : -1;
+        }
+    }
+    /* second sweep for the emitted token keeps the first one simple to read */
+    for (int b = 0; b < B; ++b) {
+        int n = out_accept_len[b];
+        if (n < 0) continue;
+        int best = -1;
+        double top = -INFINITY;
+        for (int v = 0; v < V; ++v) {
+            double l = logit_at(target_logits, dtype, ((int64_t)b * (K + 1) + n) * V + v);
+            if (l > top) { top = l; best = v; }
+        }
+        out_tokens[(int64_t)b * (K + 1) + n] = best;
+    }
+    return 0;
+}
+
 /* Softmax of one stored row, for tests that need the full distribution. */
 int ears_oracle_row_softmax(const void* logits, int dtype, int64_t row_index, int V,
                             float temperature, double* p_out)

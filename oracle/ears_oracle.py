@@ -57,6 +57,9 @@ def _load():
          c.c_float, c.c_float, c.c_void_p, c.c_void_p, c.c_int, c.c_uint64, c.c_uint64, c.c_int64, c.c_double]
         + [c.c_void_p] * 11 + [c.c_int])
     lib.ears_oracle_verify_var.restype = c.c_int
+    lib.ears_oracle_verify_greedy.argtypes = [c.c_void_p, c.c_int, c.c_void_p, c.c_int, c.c_int, c.c_int,
+                                              c.c_void_p, c.c_void_p, c.c_void_p]
+    lib.ears_oracle_verify_greedy.restype = c.c_int
     lib.ears_oracle_row_softmax.argtypes = [c.c_void_p, c.c_int, c.c_int64, c.c_int, c.c_float, c.c_void_p]
     lib.ears_oracle_row_softmax.restype = c.c_int
     lib.ears_oracle_max_threads.argtypes = []
@@ -199,3 +202,22 @@ def verify(target_logits, draft_logits, draft_tokens, temperature: float, beta: 
     if rc:
         raise ValueError(f"ears_oracle_verify rejected its arguments (rc={rc})")
     return res
+
+
+def verify_greedy(target_logits, draft_tokens):
+    """The temperature -> 0 limit of the step: -> (accept_len [B], tokens [B,K+1], argmax [B,K+1])."""
+    lib = _load()
+    t, ct = _as_logits(target_logits)
+    x = _as_tokens(draft_tokens)
+    B, K1, V = t.shape
+    K = K1 - 1
+    if x.shape != (B, K):
+        raise ValueError("shape mismatch")
+    acc = np.empty(B, np.int32)
+    tok = np.empty((B, K + 1), np.int32)
+    am = np.empty((B, K + 1), np.int32)
+    rc = lib.ears_oracle_verify_greedy(t.ctypes.data, ct, x.ctypes.data, B, K, V, acc.ctypes.data, tok.ctypes.data,
+                                       am.ctypes.data)
+    if rc:
+        raise ValueError(f"ears_oracle_verify_greedy rejected its arguments (rc={rc})")
+    return acc, tok, am

@@ -22,6 +22,7 @@ from .binding import (  # noqa: F401
     shutdown,
     verify,
     verify_abi,
+    verify_greedy,
     verify_host,
     verify_noalloc,
     version,

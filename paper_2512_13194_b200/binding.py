@@ -46,6 +46,9 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ears_verify_var.argtypes = ([c.c_int] + common[:8] + [c.c_void_p, c.c_void_p, c.c_uint] + common[8:] + [c.c_int64]
                                     + [c.c_void_p] * 7 + [c.c_void_p, c.c_size_t, c.c_void_p])
     lib.ears_verify_var.restype = c.c_int
+    lib.ears_verify_greedy.argtypes = [c.c_int, c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p,
+                                       c.c_void_p, c.c_size_t, c.c_void_p]
+    lib.ears_verify_greedy.restype = c.c_int
     lib.ears_verify_host.argtypes = [c.c_int] + common + [c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p]
     lib.ears_verify_host.restype = c.c_int
     lib.ears_verify_noalloc.argtypes = [c.c_int] + common + [c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
@@ -172,6 +175,32 @@ def verify(target_logits: torch.Tensor, draft_logits: torch.Tensor, draft_tokens
                                      acc.data_ptr(), tok.data_ptr(), *ptrs, ws_ptr, ws_bytes, _stream_ptr(stream))
     _check(rc)
     return (acc, tok, st) if stats else (acc, tok)
+
+
+def verify_greedy(target_logits: torch.Tensor, draft_tokens: torch.Tensor, *, workspace: Optional[torch.Tensor] = None,
+                  stream=None):
+    """The temperature -> 0 limit of the step (ears_verify_greedy): a draft token is accepted iff it is
+    the top token of its target row.  Returns (accept_len [B] int32, tokens [B,K+1] int32)."""
+    lib = load_library()
+    if target_logits.dim() != 3 or draft_tokens.dim() != 2:
+        raise ValueError("expected target_logits [B,K+1,V] and draft_tokens [B,K]")
+    B, K1, V = target_logits.shape
+    K = K1 - 1
+    if draft_tokens.shape != (B, K) or K < 1:
+        raise ValueError("shape mismatch")
+    dev = target_logits.device
+    if dev.type != "cuda" or draft_tokens.device != dev:
+        raise ValueError("all inputs must live on the same CUDA device")
+    t = target_logits.contiguous()
+    x = draft_tokens.to(torch.int32).contiguous()
+    with torch.cuda.device(dev):
+        acc = torch.empty(B, dtype=torch.int32, device=dev)
+        tok = torch.empty((B, K + 1), dtype=torch.int32, device=dev)
+        ws_ptr, ws_bytes = (None, 0) if workspace is None else (workspace.data_ptr(), workspace.numel() * workspace.element_size())
+        rc = lib.ears_verify_greedy(_dtype_code(t), t.data_ptr(), x.data_ptr(), B, K, V, acc.data_ptr(), tok.data_ptr(),
+                                    ws_ptr, ws_bytes, _stream_ptr(stream))
+    _check(rc)
+    return acc, tok
 
 
 def verify_abi(name: str, target_logits, draft_logits, draft_tokens, temperature, beta, seed, offset,

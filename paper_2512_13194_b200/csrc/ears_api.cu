@@ -14,6 +14,8 @@
 #include "ears_common.cuh"
 #include "ears_kernel.cuh"
 #include "ears_resident.cuh"
+#include "ears_greedy.cuh"
+#include "ears_direct.cuh"
 
 namespace {
 
@@ -206,6 +208,34 @@ RLayout make_rlayout(int B, int K) {
     return L;
 }
 
+// ---- the greedy (temperature -> 0) form ----
+struct GLayout { size_t heads, ticket, counters_bytes, partial, total; int P, piece_elems; };
+
+GLayout make_glayout(int B, int K, int V, int esize, int sms) {
+    GLayout L;
+    const long long rows = (long long)B * (K + 1);
+    // pieces of at least 16 KB, enough of them to give every CTA several
+    const long long row_bytes = (long long)V * esize;
+    long long maxp = row_bytes / 16384;
+    if (maxp < 1) maxp = 1;
+    long long want = (8LL * sms + rows - 1) / rows;
+    if (want < 1) want = 1;
+    long long P = want < maxp ? want : maxp;
+    if (P > 4096) P = 4096;
+    long long pe = (V + P - 1) / P;
+    pe = (long long)align_up((size_t)pe, kSegElems);
+    L.piece_elems = (int)pe;
+    L.P = (int)((V + pe - 1) / pe);
+    size_t o = 0;
+    L.heads = o; o += 32;
+    L.ticket = o; o += (size_t)B * 4;
+    L.counters_bytes = o;
+    o = align_up(o, 256);
+    L.partial = o; o = align_up(o + (size_t)rows * L.P * sizeof(int4), 256);
+    L.total = o;
+    return L;
+}
+
 int check_shape(int B, int K, int V) {
     if (B < 1 || K < 1 || V < 1) return EARS_ERR_SHAPE;
     if (K > EARS_MAX_K || V > (1 << 30)) return EARS_ERR_SHAPE;
@@ -309,15 +339,23 @@ int launch_resident(RParams& p, const RPlan& rp, int max_clusters, cudaStream_t 
 }
 
 template <typename E>
-int launch(const Params& p, int sms, cudaStream_t stream) {
+int launch(const Params& p, int sms, bool direct, cudaStream_t stream) {
     const long long units = (long long)p.B * (2 * p.K + 1) * p.plan.parts1;
     const long long cap = (long long)sms * kCtasPerSm;
     const int grid = (int)(units < cap ? units : cap);
     const bool timed = g_profile.active && (int)g_profile.events.size() + 2 <= 2 * g_profile.max_calls;
     int rc = profile_mark(stream, timed);
     if (rc) return rc;
-    if (p.seq_T) ears_verify_kernel<E, kStages, true><<<grid, kThreads, smem_bytes(), stream>>>(p);
-    else ears_verify_kernel<E, kStages, false><<<grid, kThreads, smem_bytes(), stream>>>(p);
+    if (direct) {
+        const long long dcap = (long long)sms * kDCtasPerSm;
+        const int dgrid = (int)(units < dcap ? units : dcap);
+        if (p.seq_T) ears_direct_kernel<E, true><<<dgrid, kDThreads + 32, 0, stream>>>(p);
+        else ears_direct_kernel<E, false><<<dgrid, kDThreads + 32, 0, stream>>>(p);
+    } else if (p.seq_T) {
+        ears_verify_kernel<E, kStages, true><<<grid, kThreads, smem_bytes(), stream>>>(p);
+    } else {
+        ears_verify_kernel<E, kStages, false><<<grid, kThreads, smem_bytes(), stream>>>(p);
+    }
     EARS_CUDA(cudaGetLastError());
     return profile_mark(stream, timed);
 }
@@ -395,7 +433,7 @@ int pick_counters(void* caller_ws, int dev, void* stream_, int kind, size_t coun
 int choose_resident(int dtype, int B, int K, int V, DeviceInfo* di, const PlanOverride& ov, RPlan* rp, int* max_clusters) {
     *rp = RPlan();
     *max_clusters = 0;
-    if (ov.path == 1 || ov.parts1 != 0) return EARS_OK;
+    if (ov.path == 1 || ov.path == 3 || ov.parts1 != 0) return EARS_OK;
     const int esize = dtype == EARS_DTYPE_F32 ? 4 : 2;
     *rp = make_rplan(B, K, V, esize, di->sms, di->cluster16 ? kRMaxCluster : 8, ov.cluster);
     if (rp->ok && ov.path == 0) {
@@ -546,7 +584,12 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
     p.seg_stride = L.seg_stride;
     p.stop_first = stop_first;
     p.plan = plan;
-    rc = dtype == EARS_DTYPE_F32 ? launch<float>(p, di->sms, stream) : launch<uint16_t>(p, di->sms, stream);
+    // Long rows: 2-byte logits go to the kernel that reads straight from global memory (its warps
+    // do not march in step, which the special-function pipe rewards), 4-byte logits to the kernel
+    // with the shared-memory ring (HBM-bound either way; measured 570 against 592 us on B=512,
+    // K=3, V=256000).  Path 1 / 3 force one or the other.
+    const bool direct = ov.path == 3 || (ov.path != 1 && esize == 2);
+    rc = dtype == EARS_DTYPE_F32 ? launch<float>(p, di->sms, direct, stream) : launch<uint16_t>(p, di->sms, direct, stream);
     if (rc && !workspace) forget_clean_counters(dev, stream_);
     return rc;
 }
@@ -568,7 +611,13 @@ size_t workspace_bound(int B, int K, int V) {
             if (tot > best) best = tot;
         }
     const size_t res = make_rlayout(B, K).total;
-    return res > best ? res : best;
+    if (res > best) best = res;
+    for (int esize = 2; esize <= 4; esize += 2)
+        for (int s = 0; s < 2; ++s) {
+            const size_t tot = make_glayout(B, K, V, esize, sm_counts[s]).total;
+            if (tot > best) best = tot;
+        }
+    return best;
 }
 
 // Scratch of the allocation-free entry point.  Part of the library image: each GPU that
@@ -650,6 +699,53 @@ int ears_verify_var(int dtype, const void* target_logits, const void* draft_logi
     return verify_impl(dtype, target_logits, draft_logits, draft_tokens, B, K, V, temperature, beta,
                        seq_temperature, seq_beta, flags, seed, offset, b_first, out_accept_len, out_tokens, out_pt_tok,
                        out_pd_tok, out_max_pt, out_class, out_resid_mass, workspace, workspace_bytes, stream);
+}
+
+int ears_verify_greedy(int dtype, const void* target_logits, const int32_t* draft_tokens, int B, int K, int V,
+                       int32_t* out_accept_len, int32_t* out_tokens, void* workspace, size_t workspace_bytes,
+                       void* stream_) {
+    if (!target_logits || !draft_tokens || !out_accept_len || !out_tokens) return EARS_ERR_NULL;
+    if (dtype != EARS_DTYPE_F32 && dtype != EARS_DTYPE_BF16) return EARS_ERR_PARAM;
+    int rc = check_shape(B, K, V);
+    if (rc) return rc;
+    const int esize = dtype == EARS_DTYPE_F32 ? 4 : 2;
+    if (((uintptr_t)target_logits % esize) || ((uintptr_t)draft_tokens % 4)) return EARS_ERR_ALIGN;
+    if (workspace && ((uintptr_t)workspace % 256)) return EARS_ERR_ALIGN;
+    if (!workspace && workspace_bytes != 0) return EARS_ERR_WORKSPACE;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    int dev = 0;
+    EARS_CUDA(cudaGetDevice(&dev));
+    DeviceInfo* di = nullptr;
+    rc = device_info(dev, &di);
+    if (rc) return rc;
+    const GLayout L = make_glayout(B, K, V, esize, di->sms);
+    if (workspace && workspace_bytes < L.total) return EARS_ERR_WORKSPACE;
+    GParams p;
+    char *w = nullptr, *cw = nullptr;
+    rc = pick_counters(workspace, dev, stream_, 3, L.counters_bytes, L.total, &w, &cw, &p.zero_ptr, &p.zero_words);
+    if (rc) return rc;
+    p.t = target_logits; p.x = draft_tokens;
+    p.B = B; p.K = K; p.V = V;
+    p.P = L.P; p.piece_elems = L.piece_elems;
+    p.vec = ((uintptr_t)target_logits % 16 == 0) && (((size_t)V * esize) % 16 == 0);
+    p.units = (long long)B * (K + 1) * L.P;
+    p.partial = (int4*)(w + L.partial);
+    p.ticket = (int*)(cw + L.ticket);
+    p.heads = (int*)(cw + L.heads);
+    p.out_len = out_accept_len; p.out_tok = out_tokens;
+    const long long cap = (long long)kGCtasPerSm * di->sms;
+    const int grid = (int)(p.units < cap ? p.units : cap);
+    const bool timed = g_profile.active && (int)g_profile.events.size() + 2 <= 2 * g_profile.max_calls;
+    rc = profile_mark(stream, timed);
+    if (rc) return rc;
+    if (dtype == EARS_DTYPE_F32) ears_greedy_kernel<float><<<grid, kGThreads, 0, stream>>>(p);
+    else ears_greedy_kernel<uint16_t><<<grid, kGThreads, 0, stream>>>(p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        if (!workspace) forget_clean_counters(dev, stream_);
+        return cuda_fail(e, "ears_greedy_kernel launch");
+    }
+    return profile_mark(stream, timed);
 }
 
 int ears_verify_f32(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
@@ -819,14 +915,20 @@ int ears_describe_plan(int dtype, int B, int K, int V, char* out, size_t out_byt
     } else {
         const Plan pl = make_plan(B, K, V, esize, true, di->sms, ov);
         const long long units = (long long)B * (2 * K + 1) * pl.parts1, cap = (long long)di->sms * kCtasPerSm;
-        snprintf(out, out_bytes, "streaming: pieces_per_row=%d chunks_per_piece=%d ctas=%lld second_pass_pieces=%d",
-                 pl.parts1, pl.cpp1, units < cap ? units : cap, pl.parts2);
+        if (!(ov.path == 3 || (ov.path != 1 && esize == 2))) {
+            snprintf(out, out_bytes, "streaming: pieces_per_row=%d chunks_per_piece=%d ctas=%lld second_pass_pieces=%d",
+                     pl.parts1, pl.cpp1, units < cap ? units : cap, pl.parts2);
+        } else {
+            const long long dcap = (long long)di->sms * kDCtasPerSm;
+            snprintf(out, out_bytes, "direct: pieces_per_row=%d chunks_per_piece=%d ctas=%lld second_pass_pieces=%d",
+                     pl.parts1, pl.cpp1, units < dcap ? units : dcap, pl.parts2);
+        }
     }
     return EARS_OK;
 }
 
 int ears_set_path(int path, int cluster) {
-    if (path < 0 || path > 2) return EARS_ERR_PARAM;
+    if (path < 0 || path > 3) return EARS_ERR_PARAM;
     if (cluster != 0 && cluster != 1 && cluster != 2 && cluster != 4 && cluster != 8 && cluster != 16) return EARS_ERR_PARAM;
     std::lock_guard<std::mutex> lock(g_mutex);
     g_override.path = path;

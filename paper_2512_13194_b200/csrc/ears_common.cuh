@@ -25,6 +25,7 @@ constexpr int kSequenceWarp = kConsumerWarps + 2;    // per-sequence decisions a
 constexpr int kThreads = kConsumers + 96;
 constexpr int kChunkBytes = 16384;                   // bytes staged per pipeline slot
 constexpr int kSegElems = 256;                       // elements per final-token segment sum
+constexpr int kMaxK = 64;                            // largest K (EARS_MAX_K of the C ABI)
 constexpr double kEps = 1e-10;                       // division guard, Sec. 3.3 item 2
 constexpr double kTinyMass = 1e-300;                 // below this a residual is treated as empty
 

@@ -59,8 +59,9 @@ SHAPES = [
 ]
 
 
-# (path, cluster): 1 = streaming kernel; 2 = resident kernel with 1..16 CTAs per cluster (0 = automatic)
-PATHS = [(1, 0), (2, 0), (2, 1), (2, 2), (2, 4), (2, 8), (2, 16)]
+# (path, cluster): 1 = streaming kernel with the shared-memory ring; 3 = streaming kernel reading straight from
+# global memory; 2 = resident kernel with 1..16 CTAs per cluster (0 = automatic)
+PATHS = [(1, 0), (3, 0), (2, 0), (2, 1), (2, 2), (2, 4), (2, 8), (2, 16)]
 
 
 @pytest.fixture
@@ -92,7 +93,7 @@ def test_parity_shapes(ears, forced_path, B, K, V, dtype, path, cluster):
     assert tally.max_rel_prob_err < 1e-5
 
 
-@pytest.mark.parametrize("path", [0, 1])
+@pytest.mark.parametrize("path", [0, 1, 3])
 @pytest.mark.parametrize("idx", [1, 2, 3, 4])
 def test_parity_workloads(ears, forced_path, idx, path):
     """Workloads 1-4 at full size, in the automatic launch configuration (the resident kernel for
@@ -160,7 +161,7 @@ def test_kernels_agree(ears, forced_path):
     tg, dg, xg = t.to(dev), d.to(dev), x.to(dev)
     results = []
     try:
-        for path, cluster, loader in [(1, 0, 0), (2, 0, 0), (2, 1, 0), (2, 2, 2), (2, 4, 0), (2, 8, 2), (2, 16, 0)]:
+        for path, cluster, loader in [(1, 0, 0), (3, 0, 0), (3, 0, 2), (2, 0, 0), (2, 1, 0), (2, 2, 2), (2, 4, 0), (2, 8, 2), (2, 16, 0)]:
             forced_path(path, cluster)
             ears.set_plan(loader, 0)
             acc, tok = ears.verify(tg, dg, xg, 1.0, 0.1, 4, 9)
@@ -184,7 +185,7 @@ def test_forced_resident_path_refuses_rows_that_do_not_fit(ears, forced_path):
     assert e.value.status == -2
 
 
-@pytest.mark.parametrize("path", [1, 2])
+@pytest.mark.parametrize("path", [1, 2, 3])
 def test_invalid_sequences_are_marked(ears, forced_path, path):
     forced_path(path)
     w, t, d, x = synth.tiny_inputs(8, 3, 5000, "fp32", seed=9)
@@ -316,7 +317,7 @@ def test_bounded_wait_gives_up_and_context_survives(ears):
     assert ears.load_library().ears_selftest_bounded_wait(0, None) == -3
 
 
-@pytest.mark.parametrize("path,cluster", [(1, 0), (2, 0), (2, 4)])
+@pytest.mark.parametrize("path,cluster", [(1, 0), (3, 0), (2, 0), (2, 4)])
 @pytest.mark.parametrize("B,K,V,dtype", [(12, 3, 9000, "fp32"), (9, 4, 20001, "bf16"), (300, 2, 700, "bf16")])
 def test_parity_per_sequence_temperature_and_beta(ears, forced_path, B, K, V, dtype, path, cluster):
     """ears_verify_var: every sequence with its own temperature and beta, against the oracle run
@@ -364,7 +365,7 @@ def test_parity_per_sequence_temperature_and_beta(ears, forced_path, B, K, V, dt
     assert_parity(compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, K), max_explained=1)
 
 
-@pytest.mark.parametrize("path", [1, 2])
+@pytest.mark.parametrize("path", [1, 2, 3])
 def test_status_and_counters_start_clean_on_every_call_of_one_shape(ears, forced_path, path):
     """Calls of one shape on the library's workspace alternate between two counter blocks without
     a memset in between: a call that saw invalid input must not leak its status or counters."""
@@ -385,7 +386,7 @@ def test_status_and_counters_start_clean_on_every_call_of_one_shape(ears, forced
             assert torch.equal(a, ref[0]) and torch.equal(k, ref[1])
 
 
-@pytest.mark.parametrize("path,cluster", [(1, 0), (2, 0), (2, 2), (2, 8)])
+@pytest.mark.parametrize("path,cluster", [(1, 0), (3, 0), (2, 0), (2, 2), (2, 8)])
 @pytest.mark.parametrize("B,K,V,dtype", [(24, 4, 9000, "fp32"), (200, 3, 1500, "bf16"), (5, 6, 20001, "bf16")])
 def test_parity_stop_at_first_reject(ears, forced_path, B, K, V, dtype, path, cluster):
     """EARS_FLAG_STOP_AT_FIRST_REJECT against the oracle in the same mode: same lengths and tokens

@@ -446,3 +446,46 @@ def test_stop_at_first_reject_reads_nothing_beyond_it():
     assert (stop3.accept_len[rej] == -1).all()
     ok = [b for b in range(B) if n[b] == K]
     assert np.array_equal(stop3.tokens[ok], full.tokens[ok])
+
+
+# --------------------------------------------------------------------------- the deterministic limit
+def test_greedy_limit_matches_argmax_and_the_low_temperature_step():
+    """Sec. 1 names temperature = 0 as the regime where plain verification works.  Pins of the
+    greedy form: (i) its per-row choice is numpy's argmax (first index on ties); (ii) lengths and
+    tokens follow from it by the first-mismatch rule; (iii) it is the limit of the stochastic step:
+    with one-hot drafts (the draft token's logit far above the rest) and a temperature far below
+    the gap between the two best target logits, the ordinary oracle gives the same lengths and
+    tokens for any beta and any seed."""
+    rng = np.random.default_rng(11)
+    B, K, V = 30, 4, 40
+    t = rng.normal(0, 3, (B, K + 1, V)).astype(np.float32)
+    top2 = np.sort(t, axis=-1)[..., -2:]
+    t[np.arange(B)[:, None], np.arange(K + 1)[None, :], t.argmax(-1)] += (top2[..., 1] - top2[..., 0] < 1.0) * 1.5   # clear winners
+    am = t.argmax(-1)
+    x = am[:, :K].astype(np.int32).copy()
+    flip = rng.random((B, K)) < 0.3
+    x[flip] = (x[flip] + 1 + rng.integers(0, V - 1, flip.sum())) % V            # some drafts miss
+    acc, tok, am_o = oracle.verify_greedy(t, x)
+    assert np.array_equal(am_o, am)
+    for b in range(B):
+        miss = np.nonzero(x[b] != am[b, :K])[0]
+        n = int(miss[0]) if miss.size else K
+        assert acc[b] == n
+        assert tok[b, :n].tolist() == x[b, :n].tolist() and tok[b, n] == am[b, n] and (tok[b, n + 1:] == -1).all()
+    assert (acc < K).sum() > 5 and (acc == K).sum() > 2
+    d = np.full((B, K, V), -50.0, np.float32)
+    d[np.arange(B)[:, None], np.arange(K)[None, :], x] = 50.0                     # greedy drafts: P_d(x) = 1
+    for beta, seed in ((0.0, 1), (0.3, 2), (1.0, 3)):
+        res = oracle.verify(t, d, x, 0.02, beta, seed=seed, offset=5)
+        assert np.array_equal(res.accept_len, acc) and np.array_equal(res.tokens, tok)
+    # ties go to the smallest index; invalid rows and tokens mark the sequence
+    t2 = t.copy()
+    t2[0, 0, :] = 0.0
+    t2[0, 0, [7, 3, 9]] = 5.0
+    assert oracle.verify_greedy(t2, x)[2][0, 0] == 3
+    t2[1, 2, 5] = np.nan
+    t2[2, K, :] = -np.inf
+    x2 = x.copy()
+    x2[3, 1] = V
+    acc2, tok2, _ = oracle.verify_greedy(t2, x2)
+    assert acc2[1:4].tolist() == [-1, -1, -1] and (tok2[1:4] == -1).all() and np.array_equal(acc2[4:], acc[4:])
