@@ -109,16 +109,39 @@ void split_rows(long long items, int chunks, int sms, int forced_parts, int* par
     *parts = (chunks + c - 1) / c;
 }
 
-Plan make_plan(int B, int K, int V, int esize, bool aligned, int sms, const PlanOverride& ov) {
+// Which of the two streaming kernels takes a shape the resident kernel does not.  The kernel that
+// reads straight from global memory wins on 2-byte logits (its warps do not march in step, which
+// the special-function pipe rewards) and on short rows (no per-slot costs), from a few hundred
+// positions on; the ring kernel keeps long 4-byte rows (HBM-bound either way) and small batches
+// (shorter tail).  Measured on B200, us direct / ring: 1024,4,152064,bf16: 562 / 734;
+// 128,4,152064,bf16: 120 / 144; 64,4,152064,bf16: 100 / 94; 2048,4,32000,fp32: 485 / 1200;
+// 512,3,256000,fp32: 592 / 571.
+bool use_direct(const PlanOverride& ov, int esize, int V, long long items) {
+    if (ov.path == 1) return false;
+    if (ov.path == 3) return true;
+    if (ov.parts1 != 0) return false;               // the piece count is a knob of the ring kernel's tests
+    if (items < 400) return false;
+    return esize == 2 || (long long)V * esize <= 512 * 1024;
+}
+
+Plan make_plan(int B, int K, int V, int esize, bool aligned, int sms, const PlanOverride& ov, bool direct = false) {
     Plan pl;
     const int chunk_elems = kChunkBytes / esize;
     const int chunks = (V + chunk_elems - 1) / chunk_elems;
     pl.use_tma = aligned && ov.loader != 2;
     split_rows((long long)B * (2 * K + 1), chunks, sms, ov.parts1, &pl.parts1, &pl.cpp1);
+    if (direct && ov.parts1 == 0 && pl.cpp1 < 4) {
+        // the kernel that reads straight from global memory keeps eight 16-byte loads per thread
+        // in flight: pieces below 64 KB would leave most of that unused
+        const int n = (chunks + 3) / 4;
+        pl.cpp1 = (chunks + n - 1) / n;
+        pl.parts1 = (chunks + pl.cpp1 - 1) / pl.cpp1;
+    }
     pl.nseg = (V + kSegElems - 1) / kSegElems;
     const long long ctas = (long long)sms * kCtasPerSm;
     // second pass (rejected positions): 64 KB of each row per piece, single chunks when there are few sequences
-    const int job_chunks = (long long)B * ((chunks + 3) / 4) >= ctas ? 4 : 1;
+    int job_chunks = (long long)B * ((chunks + 3) / 4) >= ctas ? 4 : 1;
+    if (direct && job_chunks < 2 && esize == 4) job_chunks = 2;   // a round of its second pass covers 8192 entries
     pl.job_elems = job_chunks * chunk_elems;
     pl.parts2 = (V + pl.job_elems - 1) / pl.job_elems;
     return pl;
@@ -441,10 +464,11 @@ int choose_resident(int dtype, int B, int K, int V, DeviceInfo* di, const PlanOv
         // nothing else in that CTA can hide.  It wins when rows are short (a cluster of at most
         // four CTAs holds a pair) and when there are few positions, where the streaming kernel's
         // second pass and its queues dominate; long rows in large batches stream faster.
-        // Measured on B200 (B, K, V, dtype: us resident / streaming): 8,5,32000,bf16: 20 / 47;
-        // 4096,5,32000,bf16: 976 / 2624; 32,7,128256,bf16: 72 / 75; 128,4,152064,bf16: 195 / 148.
+        // Measured on B200 (B, K, V, dtype: us resident / best streaming kernel): 8,5,32000,bf16: 19 / 43;
+        // 512,5,32000,bf16: 148 / 150; 4096,5,32000,bf16: 1009 / 910; 32,7,128256,bf16: 72 / 75;
+        // 64,7,128256,bf16: 123 / 102; 128,4,152064,bf16: 195 / 120.
         const long long items = (long long)B * (K + 1);
-        const long long limit = !rp->roomy ? 64 : (rp->C >= 8 ? 256 : (1LL << 62));
+        const long long limit = !rp->roomy ? 64 : (rp->C >= 8 ? 256 : 3072);
         if (items > limit) rp->ok = false;
     }
     if (rp->ok) {
@@ -550,7 +574,12 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
         return rc;
     }
 
-    const Plan plan = make_plan(B, K, V, esize, aligned, di->sms, ov);
+    // Long rows: 2-byte logits go to the kernel that reads straight from global memory (its warps
+    // do not march in step, which the special-function pipe rewards), 4-byte logits to the kernel
+    // with the shared-memory ring (HBM-bound either way; measured 570 against 592 us on B=512,
+    // K=3, V=256000).  Path 1 / 3 force one or the other.
+    const bool direct = use_direct(ov, esize, V, (long long)B * (K + 1));
+    const Plan plan = make_plan(B, K, V, esize, aligned, di->sms, ov, direct);
     const Layout L = make_layout(B, K, V, plan.parts1);
     if (workspace && workspace_bytes < L.total) return EARS_ERR_WORKSPACE;
     char *w = nullptr, *cw = nullptr;
@@ -584,11 +613,6 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
     p.seg_stride = L.seg_stride;
     p.stop_first = stop_first;
     p.plan = plan;
-    // Long rows: 2-byte logits go to the kernel that reads straight from global memory (its warps
-    // do not march in step, which the special-function pipe rewards), 4-byte logits to the kernel
-    // with the shared-memory ring (HBM-bound either way; measured 570 against 592 us on B=512,
-    // K=3, V=256000).  Path 1 / 3 force one or the other.
-    const bool direct = ov.path == 3 || (ov.path != 1 && esize == 2);
     rc = dtype == EARS_DTYPE_F32 ? launch<float>(p, di->sms, direct, stream) : launch<uint16_t>(p, di->sms, direct, stream);
     if (rc && !workspace) forget_clean_counters(dev, stream_);
     return rc;
@@ -913,9 +937,10 @@ int ears_describe_plan(int dtype, int B, int K, int V, char* out, size_t out_byt
         snprintf(out, out_bytes, "resident: cluster=%d slice_elems=%d smem_bytes=%zu ctas_per_sm=%d clusters_resident=%d clusters_launched=%lld",
                  rp.C, rp.slice, rp.smem, per_sm, max_clusters, items < max_clusters ? items : (long long)max_clusters);
     } else {
-        const Plan pl = make_plan(B, K, V, esize, true, di->sms, ov);
+        const bool direct = use_direct(ov, esize, V, (long long)B * (K + 1));
+        const Plan pl = make_plan(B, K, V, esize, true, di->sms, ov, direct);
         const long long units = (long long)B * (2 * K + 1) * pl.parts1, cap = (long long)di->sms * kCtasPerSm;
-        if (!(ov.path == 3 || (ov.path != 1 && esize == 2))) {
+        if (!direct) {
             snprintf(out, out_bytes, "streaming: pieces_per_row=%d chunks_per_piece=%d ctas=%lld second_pass_pieces=%d",
                      pl.parts1, pl.cpp1, units < cap ? units : cap, pl.parts2);
         } else {

@@ -70,6 +70,16 @@ template <> struct Words<float> {
     __device__ static __forceinline__ void unpack(uint4 w, float (&x)[4]) {
         x[0] = __uint_as_float(w.x); x[1] = __uint_as_float(w.y); x[2] = __uint_as_float(w.z); x[3] = __uint_as_float(w.w);
     }
+    __device__ static __forceinline__ uint4 minus_inf() { return make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u); }
+    // up to N entries from p (fewer, or none, when `left` says so), the rest -inf
+    __device__ static __forceinline__ uint4 gather(const float* p, int left) {
+        uint4 w = minus_inf();
+        if (left > 0) w.x = __float_as_uint(__ldg(p));
+        if (left > 1) w.y = __float_as_uint(__ldg(p + 1));
+        if (left > 2) w.z = __float_as_uint(__ldg(p + 2));
+        if (left > 3) w.w = __float_as_uint(__ldg(p + 3));
+        return w;
+    }
 };
 template <> struct Words<uint16_t> {
     static constexpr int N = 8;
@@ -82,6 +92,13 @@ template <> struct Words<uint16_t> {
         x[2] = __uint_as_float(w.y << 16); x[3] = __uint_as_float(w.y & 0xffff0000u);
         x[4] = __uint_as_float(w.z << 16); x[5] = __uint_as_float(w.z & 0xffff0000u);
         x[6] = __uint_as_float(w.w << 16); x[7] = __uint_as_float(w.w & 0xffff0000u);
+    }
+    __device__ static __forceinline__ uint4 minus_inf() { return make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u); }
+    __device__ static __forceinline__ uint4 gather(const uint16_t* p, int left) {
+        uint32_t h[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) h[i] = i < left ? (uint32_t)__ldg(p + i) : 0xff80u;
+        return make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
     }
 };
 
@@ -120,6 +137,10 @@ __device__ __forceinline__ float2 stream_piece(const E* row, int e0, int e1, boo
             for (int j = 0; j < kDUnroll; ++j) w[j] = ld_stream16(vs + v + j * kDThreads);
             fold_vectors<E, kDUnroll>(w, c, a);
         }
+        for (; v + kDThreads < nvec; v += 2 * kDThreads) {   // what is left of a piece: two, then one at a time
+            uint4 w[2] = {ld_stream16(vs + v), ld_stream16(vs + v + kDThreads)};
+            fold_vectors<E, 2>(w, c, a);
+        }
         for (; v < nvec; v += kDThreads) {
             uint4 w[1] = {ld_stream16(vs + v)};
             fold_vectors<E, 1>(w, c, a);
@@ -135,8 +156,9 @@ __device__ __forceinline__ float2 stream_piece(const E* row, int e0, int e1, boo
 }
 
 // A piece [e0, e1) of the extra target row: warp w takes the segments w, w + kDWarps, ... of
-// kBonusSegBytes each, keeps a warp-uniform running maximum and stores (sum, reference
-// maximum) of every segment.  -> the lane's (m, s) relative to the warp's final maximum.
+// kBonusSegBytes each, two per round (eight loads in flight per lane), keeps a warp-uniform
+// running maximum and stores (sum, reference maximum) of every segment.
+// -> the lane's (m, s) relative to the warp's final maximum.
 template <typename E>
 __device__ __forceinline__ float2 stream_bonus_piece(const E* row, int e0, int e1, bool vec, float c, int warp, int lane,
                                                      BonusSeg* segs /* of the whole row */) {
@@ -145,55 +167,69 @@ __device__ __forceinline__ float2 stream_bonus_piece(const E* row, int e0, int e
     constexpr int VPL = SEG / N / 32;                        // vectors per lane per segment
     float m_run = -INFINITY;
     float s = 0.f;
-    for (int g0 = e0 + warp * SEG; g0 < e1; g0 += kDWarps * SEG) {
-        const int cnt = min(SEG, e1 - g0);
-        float x[VPL][N];
-        if (vec) {
-            const uint4* vs = reinterpret_cast<const uint4*>(row + g0);
+    for (int ga = e0 + warp * SEG; ga < e1; ga += 2 * kDWarps * SEG) {
+        // the loads stay packed (16 bytes per vector) until they are used; rows that are not
+        // 16-byte aligned are gathered element by element into the same form
+        uint4 w[2][VPL];
+        float cm[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int g0 = ga + h * kDWarps * SEG;
+            const int cnt = max(0, min(SEG, e1 - g0));
 #pragma unroll
             for (int j = 0; j < VPL; ++j) {
-                const int v = j * 32 + lane;
-                if (v * N < cnt) {
-                    Words<E>::unpack(ld_stream16(vs + v), x[j]);
+                const int k0 = (j * 32 + lane) * N;
+                if (vec) {
+                    w[h][j] = k0 < cnt ? ld_stream16(row + g0 + k0) : Words<E>::minus_inf();
                 } else {
-#pragma unroll
-                    for (int i = 0; i < N; ++i) x[j][i] = -INFINITY;
+                    w[h][j] = Words<E>::gather(row + g0 + k0, cnt - k0);
                 }
             }
-        } else {
-#pragma unroll
-            for (int j = 0; j < VPL; ++j)
-#pragma unroll
-                for (int i = 0; i < N; ++i) {
-                    const int k = (j * 32 + lane) * N + i;
-                    x[j][i] = k < cnt ? load_logit(row + g0 + k) : -INFINITY;
-                }
         }
-        float cm = -INFINITY;
 #pragma unroll
-        for (int j = 0; j < VPL; ++j)
+        for (int h = 0; h < 2; ++h) {
+            cm[h] = Words<E>::vmax(w[h][0]);
 #pragma unroll
-            for (int i = 0; i < N; ++i) cm = fmaxf(cm, x[j][i]);
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, off));
-        if (cm > m_run) {
-            s *= ex2_approx((m_run - cm) * c);   // m_run = -inf gives 0
-            m_run = cm;
+            for (int j = 1; j < VPL; ++j) cm[h] = fmaxf(cm[h], Words<E>::vmax(w[h][j]));
         }
-        const float mu = (m_run == -INFINITY) ? 0.0f : m_run;
-        float cs[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int j = 0; j < VPL; ++j)
+        for (int off = 16; off > 0; off >>= 1) {
+            cm[0] = fmaxf(cm[0], __shfl_xor_sync(0xffffffffu, cm[0], off));
+            cm[1] = fmaxf(cm[1], __shfl_xor_sync(0xffffffffu, cm[1], off));
+        }
+        double tot[2];
+        float ref[2];
 #pragma unroll
-            for (int i = 0; i < N; ++i) cs[i & 3] += ex2_approx(__fmul_rn(__fsub_rn(x[j][i], mu), c));
-        const float part = (cs[0] + cs[1]) + (cs[2] + cs[3]);
-        s += part;
+        for (int h = 0; h < 2; ++h) {
+            if (cm[h] > m_run) {
+                s *= ex2_approx((m_run - cm[h]) * c);   // m_run = -inf gives 0
+                m_run = cm[h];
+            }
+            ref[h] = m_run;
+            const float mu = (m_run == -INFINITY) ? 0.0f : m_run;
+            float cs[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int j = 0; j < VPL; ++j) {
+                float x[N];
+                Words<E>::unpack(w[h][j], x);
+#pragma unroll
+                for (int i = 0; i < N; ++i) cs[i & 3] += ex2_approx(__fmul_rn(__fsub_rn(x[i], mu), c));
+            }
+            const float part = (cs[0] + cs[1]) + (cs[2] + cs[3]);
+            s += part;
+            tot[h] = (double)part;
+        }
         // a lane's few terms add up in fp32; across lanes in fp64 (the running sums of the final
         // draw stay exact to ~1e-9 of the row's mass)
-        double tot = (double)part;
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, off);
-        if (lane == 0) segs[g0 / SEG] = BonusSeg{tot, m_run, 0.f};
+        for (int off = 16; off > 0; off >>= 1) {
+            tot[0] += __shfl_xor_sync(0xffffffffu, tot[0], off);
+            tot[1] += __shfl_xor_sync(0xffffffffu, tot[1], off);
+        }
+        if (lane == 0) {
+            segs[ga / SEG] = BonusSeg{tot[0], ref[0], 0.f};
+            if (ga + kDWarps * SEG < e1) segs[(ga + kDWarps * SEG) / SEG] = BonusSeg{tot[1], ref[1], 0.f};
+        }
     }
     // the draw looks at whole 16 KB chunks: segments of the row's last chunk that lie beyond its
     // end hold no mass
@@ -205,44 +241,59 @@ __device__ __forceinline__ float2 stream_bonus_piece(const E* row, int e0, int e
 }
 
 // A second-pass piece [e0, e1) of the two rows of a rejected position: sums of
-// max(0, e_t - e_d Z_t / Z_d) per kSegElems entries; warp w takes groups of two segments.
+// max(0, e_t - e_d Z_t / Z_d) per kSegElems entries; warp w takes groups of four segments and
+// keeps the loads of a group (packed, as they come) in flight together.
 template <typename E>
 __device__ __forceinline__ void stream_job_piece(const E* trow, const E* drow, int e0, int e1, bool vec, const RowNorm& rn,
                                                  float c, int warp, int lane, double* seg_out /* of the whole row */) {
     constexpr int N = Words<E>::N;
     constexpr int VPL = kSegElems / N / 32;   // vectors per lane per segment and row
-    constexpr int GROUP = 2;                  // segments per round: 2 VPL loads of each row in flight
+    constexpr int GROUP = 4;                  // segments per round
     for (int g0 = e0 + warp * GROUP * kSegElems; g0 < e1; g0 += kDWarps * GROUP * kSegElems) {
-        float xt[GROUP][VPL][N], xd[GROUP][VPL][N];
+        double acc[GROUP];
+        if (vec) {
+            uint4 wt[GROUP][VPL], wd[GROUP][VPL];
 #pragma unroll
-        for (int h = 0; h < GROUP; ++h)
+            for (int h = 0; h < GROUP; ++h)
 #pragma unroll
-            for (int j = 0; j < VPL; ++j) {
-                const int k0 = g0 + h * kSegElems + (j * 32 + lane) * N;
-                if (vec && k0 < e1) {
-                    Words<E>::unpack(ld_stream16(trow + k0), xt[h][j]);
-                    Words<E>::unpack(ld_stream16(drow + k0), xd[h][j]);
-                } else {
-#pragma unroll
-                    for (int i = 0; i < N; ++i) {
-                        const bool in = k0 + i < e1;
-                        xt[h][j][i] = in ? load_logit(trow + k0 + i) : -INFINITY;
-                        xd[h][j][i] = in ? load_logit(drow + k0 + i) : -INFINITY;
+                for (int j = 0; j < VPL; ++j) {
+                    const int k0 = g0 + h * kSegElems + (j * 32 + lane) * N;
+                    if (k0 < e1) {
+                        wt[h][j] = ld_stream16(trow + k0);
+                        wd[h][j] = ld_stream16(drow + k0);
+                    } else {
+                        wt[h][j] = make_uint4(0, 0, 0, 0);
+                        wd[h][j] = make_uint4(0, 0, 0, 0);
                     }
                 }
-            }
-        double acc[GROUP];
 #pragma unroll
-        for (int h = 0; h < GROUP; ++h) {
-            float a = 0.f;
+            for (int h = 0; h < GROUP; ++h) {
+                float a = 0.f;
 #pragma unroll
-            for (int j = 0; j < VPL; ++j)
+                for (int j = 0; j < VPL; ++j) {
+                    float xt[N], xd[N];
+                    Words<E>::unpack(wt[h][j], xt);
+                    Words<E>::unpack(wd[h][j], xd);
+                    const bool in = g0 + h * kSegElems + (j * 32 + lane) * N < e1;   // whole vectors here
 #pragma unroll
-                for (int i = 0; i < N; ++i) {
-                    const float r = entry_mass<true>(xt[h][j][i], xd[h][j][i], rn, c);
-                    if (g0 + h * kSegElems + (j * 32 + lane) * N + i < e1) a += r;
+                    for (int i = 0; i < N; ++i) {
+                        const float r = entry_mass<true>(xt[i], xd[i], rn, c);
+                        if (in) a += r;
+                    }
                 }
-            acc[h] = (double)a;
+                acc[h] = (double)a;
+            }
+        } else {
+#pragma unroll
+            for (int h = 0; h < GROUP; ++h) {
+                float a = 0.f;
+                for (int j = 0; j < VPL; ++j)
+                    for (int i = 0; i < N; ++i) {
+                        const int k = g0 + h * kSegElems + (j * 32 + lane) * N + i;
+                        if (k < e1) a += entry_mass<true>(load_logit(trow + k), load_logit(drow + k), rn, c);
+                    }
+                acc[h] = (double)a;
+            }
         }
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1)
