@@ -32,7 +32,7 @@
  *
  * Conventions for every entry point unless stated otherwise:
  *   - logits are row-major and contiguous: target [B, K+1, V], draft [B, K, V],
- *     fp32 or bf16 (bit pattern of the upper half of an fp32); draft tokens [B, K]
+ *     fp32, bf16 (bit pattern of the upper half of an fp32) or fp16 (IEEE binary16); draft tokens [B, K]
  *     int32.  -inf logits (masked vocabulary) are legal.
  *   - pointers are DEVICE pointers owned by the caller; the library neither
  *     retains nor frees them.  Logits must be aligned to their element size.
@@ -73,7 +73,7 @@ enum {
     EARS_ERR_TIMEOUT = -7    /* a bounded device-side wait gave up (reported by ears_last_device_status) */
 };
 
-enum { EARS_DTYPE_F32 = 0, EARS_DTYPE_BF16 = 1 };
+enum { EARS_DTYPE_F32 = 0, EARS_DTYPE_BF16 = 1, EARS_DTYPE_F16 = 2 };
 
 /* bits of the device status word of a call */
 enum { EARS_DEV_INVALID_INPUT = 1, EARS_DEV_TIMEOUT = 2 };
@@ -104,7 +104,7 @@ int ears_verify(const void* target_logits, const void* draft_logits,
 
 /*
  * General form.  Beyond the arguments above:
- *   dtype       EARS_DTYPE_F32 or EARS_DTYPE_BF16.
+ *   dtype       EARS_DTYPE_F32, EARS_DTYPE_BF16 or EARS_DTYPE_F16 (IEEE binary16).
  *   b_first     global index of local sequence 0; it enters the random counter so
  *               that a batch sharded across GPUs (Sec. 3.3 item 3 treats all active
  *               sequences independently) reproduces the unsharded result.

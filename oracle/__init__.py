@@ -8,6 +8,7 @@ from .ears_oracle import (  # noqa: F401
     OracleResult,
     build,
     inverse_cdf,
+    half_to_double,
     max_threads,
     philox4x32_10,
     row_softmax,

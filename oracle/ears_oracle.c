@@ -91,12 +91,25 @@ double ears_oracle_uniform_final(uint64_t seed, uint64_t offset, int64_t b, int 
 }
 
 /* ------------------------------------------------------------------------- */
-/* Row access: logits are fp32 (dtype 0) or bf16 bit patterns (dtype 1).      */
-/* Both widen to double without rounding.                                     */
+/* Row access: logits are fp32 (dtype 0), bf16 bit patterns (dtype 1) or IEEE  */
+/* binary16 bit patterns (dtype 2).  All widen to double without rounding.    */
 /* ------------------------------------------------------------------------- */
+
+/* IEEE 754 binary16: 1 sign bit, 5 exponent bits (bias 15), 10 fraction bits. */
+double ears_oracle_half_to_double(uint16_t h)
+{
+    const int sign = h >> 15, e = (h >> 10) & 31, f = h & 1023;
+    double v;
+    if (e == 31) v = f ? NAN : INFINITY;
+    else if (e == 0) v = ldexp((double)f, -24);               /* subnormal: f * 2^-10 * 2^-14 */
+    else v = ldexp(1.0 + (double)f / 1024.0, e - 15);
+    return sign ? -v : v;
+}
+
 static double logit_at(const void* base, int dtype, int64_t index)
 {
     if (dtype == 0) return (double)((const float*)base)[index];
+    if (dtype == 2) return ears_oracle_half_to_double(((const uint16_t*)base)[index]);
     uint32_t bits = (uint32_t)((const uint16_t*)base)[index] << 16;
     float f;
     memcpy(&f, &bits, sizeof f);
@@ -278,7 +291,7 @@ static void verify_one(const void* tl, const void* dl, int dtype, const int32_t*
 /*
  * One verification step over B independent sequences [Sec. 3.3 item 3 batches
  * "all active sequences"].  All pointers are host memory.
- *   target_logits [B,K+1,V], draft_logits [B,K,V] (dtype 0 fp32, 1 bf16 bits),
+ *   target_logits [B,K+1,V], draft_logits [B,K,V] (dtype 0 fp32, 1 bf16 bits, 2 fp16 bits),
  *   draft_tokens [B,K]; b_first = global index of local sequence 0 (batch shards);
  *   band = half-width, in probability, used for the near-boundary token range.
  * Outputs: out_accept_len [B] (n in [0,K], or -1 for an invalid sequence),
@@ -303,7 +316,7 @@ int ears_oracle_verify_var(const void* target_logits, const void* draft_logits, 
                            int32_t* band_lo, int32_t* band_hi, int nthreads)
 {
     if (!target_logits || !draft_logits || !draft_tokens || !out_accept_len || !out_tokens) return -1;
-    if (B < 1 || K < 1 || V < 1 || (dtype != 0 && dtype != 1)) return -1;
+    if (B < 1 || K < 1 || V < 1 || (dtype < 0 || dtype > 2)) return -1;
     if (!seq_temperature && (!(temperature > 0.0f) || !isfinite(temperature))) return -1;
     if (!seq_beta && (!(beta >= 0.0f) || !isfinite(beta))) return -1;
     ears_oracle_diag dg = { pt_tok, pd_tok, max_pt, margin, cls, resid_mass, cdf_margin, band_lo, band_hi };
@@ -377,7 +390,7 @@ int ears_oracle_verify_greedy(const void* target_logits, int dtype, const int32_
                               int32_t* argmax_out /* [B,K+1] or NULL */)
 {
     if (!target_logits || !draft_tokens || !out_accept_len || !out_tokens) return -1;
-    if (B < 1 || K < 1 || V < 1 || (dtype != 0 && dtype != 1)) return -1;
+    if (B < 1 || K < 1 || V < 1 || (dtype < 0 || dtype > 2)) return -1;
     for (int b = 0; b < B; ++b) {
         int valid = 1, n = K;
         for (int k = 0; k <= K; ++k) {

@@ -1,7 +1,7 @@
 """ctypes binding of the fp64 C oracle (TEST INFRASTRUCTURE, see ears_oracle.c).
 
 Argument marshalling only; every number is computed in ``ears_oracle.c``.
-Logits may be numpy float32 arrays, numpy uint16 arrays holding bf16 bit
+Logits may be numpy float32 or float16 arrays, numpy uint16 arrays holding bf16 bit
 patterns, or CPU torch tensors of dtype float32 / bfloat16.
 """
 from __future__ import annotations
@@ -62,6 +62,8 @@ def _load():
     lib.ears_oracle_verify_greedy.restype = c.c_int
     lib.ears_oracle_row_softmax.argtypes = [c.c_void_p, c.c_int, c.c_int64, c.c_int, c.c_float, c.c_void_p]
     lib.ears_oracle_row_softmax.restype = c.c_int
+    lib.ears_oracle_half_to_double.argtypes = [c.c_uint16]
+    lib.ears_oracle_half_to_double.restype = c.c_double
     lib.ears_oracle_max_threads.argtypes = []
     lib.ears_oracle_max_threads.restype = c.c_int
     _lib = lib
@@ -69,7 +71,7 @@ def _load():
 
 
 def _as_logits(a):
-    """-> (contiguous numpy array, dtype code 0=fp32 / 1=bf16 bits)."""
+    """-> (contiguous numpy array, dtype code 0=fp32 / 1=bf16 bits / 2=fp16 bits)."""
     if not isinstance(a, np.ndarray):  # torch tensor on the CPU
         import torch
         a = a.detach().contiguous()
@@ -77,12 +79,16 @@ def _as_logits(a):
             return a.view(torch.int16).numpy().view(np.uint16), 1
         if a.dtype == torch.float32:
             return a.numpy(), 0
+        if a.dtype == torch.float16:
+            return a.view(torch.int16).numpy().view(np.uint16), 2
         raise TypeError(f"unsupported logits dtype {a.dtype}")
     a = np.ascontiguousarray(a)
     if a.dtype == np.float32:
         return a, 0
     if a.dtype == np.uint16:
         return a, 1
+    if a.dtype == np.float16:
+        return a.view(np.uint16), 2
     raise TypeError(f"unsupported logits dtype {a.dtype}")
 
 
@@ -144,6 +150,10 @@ def row_softmax(logits, row_index: int, V: int, temperature: float):
     if rc:
         raise ValueError("row has no softmax")
     return p
+
+
+def half_to_double(bits: int) -> float:
+    return float(_load().ears_oracle_half_to_double(int(bits) & 0xFFFF))
 
 
 def max_threads() -> int:

@@ -11,7 +11,7 @@ import torch
 
 from . import build as _build
 
-EARS_DTYPE_F32, EARS_DTYPE_BF16 = 0, 1
+EARS_DTYPE_F32, EARS_DTYPE_BF16, EARS_DTYPE_F16 = 0, 1, 2
 DEV_INVALID_INPUT, DEV_TIMEOUT = 1, 2
 
 _lib = None
@@ -98,7 +98,9 @@ def _dtype_code(t: torch.Tensor) -> int:
         return EARS_DTYPE_F32
     if t.dtype == torch.bfloat16:
         return EARS_DTYPE_BF16
-    raise TypeError(f"logits must be float32 or bfloat16, got {t.dtype}")
+    if t.dtype == torch.float16:
+        return EARS_DTYPE_F16
+    raise TypeError(f"logits must be float32, bfloat16 or float16, got {t.dtype}")
 
 
 def _shapes(target_logits, draft_logits, draft_tokens):
@@ -323,14 +325,15 @@ def set_plan(loader: int = 0, parts: int = 0) -> None:
 
 
 def set_path(path: int = 0, cluster: int = 0) -> None:
-    """0 = automatic; path 1 streaming kernel, 2 resident (cluster) kernel; cluster = CTAs per cluster."""
+    """0 = automatic; path 1 streaming kernel with the shared-memory ring, 2 resident (cluster) kernel,
+    3 streaming kernel reading straight from global memory; cluster = CTAs per cluster."""
     _check(load_library().ears_set_path(path, cluster))
 
 
 def describe_plan(dtype: str, B: int, K: int, V: int) -> str:
-    """The launch plan a call with these sizes would use on the current device ("fp32" or "bf16")."""
+    """The launch plan a call with these sizes would use on the current device ("fp32", "bf16" or "fp16")."""
     buf = ctypes.create_string_buffer(256)
-    _check(load_library().ears_describe_plan(0 if dtype == "fp32" else 1, B, K, V, buf, len(buf)))
+    _check(load_library().ears_describe_plan({"fp32": 0, "bf16": 1, "fp16": 2}[dtype], B, K, V, buf, len(buf)))
     return buf.value.decode()
 
 

@@ -8,6 +8,7 @@
 #include <cstring>
 #include <map>
 #include <mutex>
+#include <type_traits>
 #include <utility>
 #include <vector>
 
@@ -20,6 +21,17 @@
 namespace {
 
 using namespace ears;
+
+bool dtype_ok(int dtype) { return dtype == EARS_DTYPE_F32 || dtype == EARS_DTYPE_BF16 || dtype == EARS_DTYPE_F16; }
+int dtype_size(int dtype) { return dtype == EARS_DTYPE_F32 ? 4 : 2; }
+
+// Calls f with a null pointer to the element type of `dtype` (float, uint16_t = bfloat16 bits, f16_t).
+template <typename F>
+int by_dtype(int dtype, F&& f) {
+    if (dtype == EARS_DTYPE_F32) return f((float*)nullptr);
+    if (dtype == EARS_DTYPE_F16) return f((f16_t*)nullptr);
+    return f((uint16_t*)nullptr);
+}
 
 // 256 KB of one row per unit when there is plenty of work (smaller units cost more per-unit
 // bookkeeping than they gain in balance; measured on B=512, V=256000).
@@ -313,8 +325,8 @@ int set_attrs(bool* cluster16) {
 
 // How many clusters of this shape the device can hold at once (cached per device).
 template <typename E>
-int resident_clusters(DeviceInfo* di, const RPlan& rp, int* out) {
-    const std::pair<int, int> key(rp.C * 8 + (int)sizeof(E), (int)rp.smem);
+int resident_clusters(DeviceInfo* di, const RPlan& rp, int dtype, int* out) {
+    const std::pair<int, int> key(rp.C * 8 + dtype, (int)rp.smem);
     {
         std::lock_guard<std::mutex> lock(g_mutex);
         auto it = di->clusters.find(key);
@@ -457,7 +469,7 @@ int choose_resident(int dtype, int B, int K, int V, DeviceInfo* di, const PlanOv
     *rp = RPlan();
     *max_clusters = 0;
     if (ov.path == 1 || ov.path == 3 || ov.parts1 != 0) return EARS_OK;
-    const int esize = dtype == EARS_DTYPE_F32 ? 4 : 2;
+    const int esize = dtype_size(dtype);
     *rp = make_rplan(B, K, V, esize, di->sms, di->cluster16 ? kRMaxCluster : 8, ov.cluster);
     if (rp->ok && ov.path == 0) {
         // Holding rows in shared memory costs a few microseconds of latency per position that
@@ -472,8 +484,9 @@ int choose_resident(int dtype, int B, int K, int V, DeviceInfo* di, const PlanOv
         if (items > limit) rp->ok = false;
     }
     if (rp->ok) {
-        const int rc = dtype == EARS_DTYPE_F32 ? resident_clusters<float>(di, *rp, max_clusters)
-                                               : resident_clusters<uint16_t>(di, *rp, max_clusters);
+        const int rc = by_dtype(dtype, [&](auto* e) {
+            return resident_clusters<std::remove_pointer_t<decltype(e)>>(di, *rp, dtype, max_clusters);
+        });
         if (rc) return rc;
         if (*max_clusters < 1) rp->ok = false;
     }
@@ -488,6 +501,8 @@ int ensure_attrs(DeviceInfo* di) {
     if (rc) return rc;
     rc = set_attrs<uint16_t>(&c16);
     if (rc) return rc;
+    rc = set_attrs<f16_t>(&c16);
+    if (rc) return rc;
     di->cluster16 = c16;
     di->attrs_set = true;
     return EARS_OK;
@@ -499,7 +514,7 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
                 int32_t* out_len, int32_t* out_tok, double* o_pt, double* o_pd, double* o_max,
                 uint8_t* o_cls, double* o_resid, void* workspace, size_t workspace_bytes, void* stream_) {
     if (!t || !d || !x || !out_len || !out_tok) return EARS_ERR_NULL;
-    if (dtype != EARS_DTYPE_F32 && dtype != EARS_DTYPE_BF16) return EARS_ERR_PARAM;
+    if (!dtype_ok(dtype)) return EARS_ERR_PARAM;
     if (flags & ~(unsigned)EARS_FLAG_STOP_AT_FIRST_REJECT) return EARS_ERR_PARAM;
     const int stop_first = (flags & EARS_FLAG_STOP_AT_FIRST_REJECT) ? 1 : 0;
     int rc = check_shape(B, K, V);
@@ -511,7 +526,7 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
     if (!(beta >= 0.0f) || !std::isfinite(beta)) return EARS_ERR_PARAM;
     if (((uintptr_t)seq_T % 4) || ((uintptr_t)seq_beta % 4)) return EARS_ERR_ALIGN;
     if (b_first < 0 || (unsigned long long)b_first + (unsigned long long)B > 0xffffffffull) return EARS_ERR_PARAM;
-    const int esize = dtype == EARS_DTYPE_F32 ? 4 : 2;
+    const int esize = dtype_size(dtype);
     if (((uintptr_t)t % esize) || ((uintptr_t)d % esize) || ((uintptr_t)x % 4)) return EARS_ERR_ALIGN;
     if (workspace && ((uintptr_t)workspace % 256)) return EARS_ERR_ALIGN;
     if (!workspace && workspace_bytes != 0) return EARS_ERR_WORKSPACE;
@@ -568,8 +583,9 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
         p.n_clusters = 0;
         p.want_stats = (o_pt || o_pd || o_max || o_cls) ? 1 : 0;
         p.ordered = stop_first;
-        rc = dtype == EARS_DTYPE_F32 ? launch_resident<float>(p, rp, max_clusters, stream)
-                                     : launch_resident<uint16_t>(p, rp, max_clusters, stream);
+        rc = by_dtype(dtype, [&](auto* e) {
+            return launch_resident<std::remove_pointer_t<decltype(e)>>(p, rp, max_clusters, stream);
+        });
         if (rc && !workspace) forget_clean_counters(dev, stream_);
         return rc;
     }
@@ -613,7 +629,7 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
     p.seg_stride = L.seg_stride;
     p.stop_first = stop_first;
     p.plan = plan;
-    rc = dtype == EARS_DTYPE_F32 ? launch<float>(p, di->sms, direct, stream) : launch<uint16_t>(p, di->sms, direct, stream);
+    rc = by_dtype(dtype, [&](auto* e) { return launch<std::remove_pointer_t<decltype(e)>>(p, di->sms, direct, stream); });
     if (rc && !workspace) forget_clean_counters(dev, stream_);
     return rc;
 }
@@ -729,10 +745,10 @@ int ears_verify_greedy(int dtype, const void* target_logits, const int32_t* draf
                        int32_t* out_accept_len, int32_t* out_tokens, void* workspace, size_t workspace_bytes,
                        void* stream_) {
     if (!target_logits || !draft_tokens || !out_accept_len || !out_tokens) return EARS_ERR_NULL;
-    if (dtype != EARS_DTYPE_F32 && dtype != EARS_DTYPE_BF16) return EARS_ERR_PARAM;
+    if (!dtype_ok(dtype)) return EARS_ERR_PARAM;
     int rc = check_shape(B, K, V);
     if (rc) return rc;
-    const int esize = dtype == EARS_DTYPE_F32 ? 4 : 2;
+    const int esize = dtype_size(dtype);
     if (((uintptr_t)target_logits % esize) || ((uintptr_t)draft_tokens % 4)) return EARS_ERR_ALIGN;
     if (workspace && ((uintptr_t)workspace % 256)) return EARS_ERR_ALIGN;
     if (!workspace && workspace_bytes != 0) return EARS_ERR_WORKSPACE;
@@ -762,8 +778,10 @@ int ears_verify_greedy(int dtype, const void* target_logits, const int32_t* draf
     const bool timed = g_profile.active && (int)g_profile.events.size() + 2 <= 2 * g_profile.max_calls;
     rc = profile_mark(stream, timed);
     if (rc) return rc;
-    if (dtype == EARS_DTYPE_F32) ears_greedy_kernel<float><<<grid, kGThreads, 0, stream>>>(p);
-    else ears_greedy_kernel<uint16_t><<<grid, kGThreads, 0, stream>>>(p);
+    by_dtype(dtype, [&](auto* e) {
+        ears_greedy_kernel<std::remove_pointer_t<decltype(e)>><<<grid, kGThreads, 0, stream>>>(p);
+        return 0;
+    });
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) {
         if (!workspace) forget_clean_counters(dev, stream_);
@@ -800,10 +818,10 @@ int ears_verify_host(int dtype, const void* target_logits, const void* draft_log
                      uint64_t seed, uint64_t offset, int64_t b_first, int32_t* out_accept_len,
                      int32_t* out_tokens, void* stream_) {
     if (!target_logits || !draft_logits || !draft_tokens || !out_accept_len || !out_tokens) return EARS_ERR_NULL;
-    if (dtype != EARS_DTYPE_F32 && dtype != EARS_DTYPE_BF16) return EARS_ERR_PARAM;
+    if (!dtype_ok(dtype)) return EARS_ERR_PARAM;
     int rc = check_shape(B, K, V);
     if (rc) return rc;
-    const size_t esize = dtype == EARS_DTYPE_F32 ? 4 : 2;
+    const size_t esize = (size_t)dtype_size(dtype);
     const size_t tb = (size_t)B * (K + 1) * V * esize, db = (size_t)B * K * V * esize;
     const size_t xb = (size_t)B * K * 4, lb = (size_t)B * 4, ob = (size_t)B * (K + 1) * 4;
     size_t o_t = 0, o_d = align_up(o_t + tb, 256), o_x = align_up(o_d + db, 256);
@@ -909,7 +927,7 @@ int ears_set_plan(int loader, int parts) {
 
 int ears_describe_plan(int dtype, int B, int K, int V, char* out, size_t out_bytes) {
     if (!out || out_bytes == 0) return EARS_ERR_NULL;
-    if (dtype != EARS_DTYPE_F32 && dtype != EARS_DTYPE_BF16) return EARS_ERR_PARAM;
+    if (!dtype_ok(dtype)) return EARS_ERR_PARAM;
     int rc = check_shape(B, K, V);
     if (rc) return rc;
     int dev = 0;
@@ -928,12 +946,14 @@ int ears_describe_plan(int dtype, int B, int K, int V, char* out, size_t out_byt
     int max_clusters = 0;
     rc = choose_resident(dtype, B, K, V, di, ov, &rp, &max_clusters);
     if (rc) return rc;
-    const int esize = dtype == EARS_DTYPE_F32 ? 4 : 2;
+    const int esize = dtype_size(dtype);
     if (rp.ok) {
         const long long items = (long long)B * (K + 1);
         int per_sm = 0;
-        if (dtype == EARS_DTYPE_F32) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ears_resident_kernel<float>, kRThreads, rp.smem);
-        else cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ears_resident_kernel<uint16_t>, kRThreads, rp.smem);
+        by_dtype(dtype, [&](auto* e) {
+            return (int)cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ears_resident_kernel<std::remove_pointer_t<decltype(e)>>,
+                                                                      kRThreads, rp.smem);
+        });
         snprintf(out, out_bytes, "resident: cluster=%d slice_elems=%d smem_bytes=%zu ctas_per_sm=%d clusters_resident=%d clusters_launched=%lld",
                  rp.C, rp.slice, rp.smem, per_sm, max_clusters, items < max_clusters ? items : (long long)max_clusters);
     } else {

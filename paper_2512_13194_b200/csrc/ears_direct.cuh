@@ -101,6 +101,21 @@ template <> struct Words<uint16_t> {
         return make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
     }
 };
+template <> struct Words<f16_t> {
+    static constexpr int N = 8;
+    __device__ static __forceinline__ float vmax(uint4 w) {   // exact on packed pairs
+        const float2 m = f16x2_to_float2(max_f16x2(max_f16x2(w.x, w.y), max_f16x2(w.z, w.w)));
+        return fmaxf(m.x, m.y);
+    }
+    __device__ static __forceinline__ void unpack(uint4 w, float (&x)[8]) { Vec<f16_t>::unpack(w, x); }
+    __device__ static __forceinline__ uint4 minus_inf() { return make_uint4(0xfc00fc00u, 0xfc00fc00u, 0xfc00fc00u, 0xfc00fc00u); }
+    __device__ static __forceinline__ uint4 gather(const f16_t* p, int left) {
+        uint32_t h[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) h[i] = i < left ? (uint32_t)__ldg(&p[i].bits) : 0xfc00u;
+        return make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
+    }
+};
 
 // G vectors of one thread: maximum first, one rescale of the running sums if it grew, then one
 // fused multiply-add and one exp2 per entry (RowAcc convention, see ears_math.cuh).

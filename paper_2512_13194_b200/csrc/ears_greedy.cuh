@@ -86,6 +86,15 @@ template <> struct GVec<uint16_t> {
         top_take(a, __uint_as_float(w.w << 16), i0 + 6); top_take(a, __uint_as_float(w.w & 0xffff0000u), i0 + 7);
     }
 };
+template <> struct GVec<f16_t> {
+    static constexpr int N = 8;
+    __device__ static __forceinline__ void take(Top& a, uint4 w, int i0) {
+        float x[8];
+        Vec<f16_t>::unpack(w, x);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) top_take(a, x[i], i0 + i);
+    }
+};
 
 // One warp: combines the pieces of every target row of sequence b, compares the draft tokens
 // with the rows' top tokens and writes accept length and tokens.

@@ -171,7 +171,7 @@ __device__ __forceinline__ bool loader_acquire(PipeSmem<STAGES>& sm, uint32_t q,
 template <typename E>
 __device__ __forceinline__ void lane_copy(void* dst, const E* src, int n, int lane) {
     E* o = reinterpret_cast<E*>(dst);
-    for (int i = lane; i < n; i += 32) o[i] = __ldg(src + i);
+    for (int i = lane; i < n; i += 32) o[i] = ld_elem(src + i);
 }
 
 // After an abort: give copies that may still be in flight a bounded time to land

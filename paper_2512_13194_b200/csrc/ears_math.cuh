@@ -24,9 +24,20 @@ template <> struct Vec<uint16_t> {
         x[6] = __uint_as_float(v.w << 16); x[7] = __uint_as_float(v.w & 0xffff0000u);
     }
 };
+template <> struct Vec<f16_t> {
+    static constexpr int N = 8;
+    __device__ static __forceinline__ void unpack(uint4 v, float (&x)[8]) {
+        const float2 a = f16x2_to_float2(v.x), b = f16x2_to_float2(v.y), c = f16x2_to_float2(v.z), d = f16x2_to_float2(v.w);
+        x[0] = a.x; x[1] = a.y; x[2] = b.x; x[3] = b.y; x[4] = c.x; x[5] = c.y; x[6] = d.x; x[7] = d.y;
+    }
+    __device__ static __forceinline__ void load(const unsigned char* buf, int vec_index, float (&x)[8]) {
+        unpack(reinterpret_cast<const uint4*>(buf)[vec_index], x);
+    }
+};
 
 __device__ __forceinline__ float load_logit(const float* p) { return __ldg(p); }
 __device__ __forceinline__ float load_logit(const uint16_t* p) { return bf16_bits_to_float(__ldg(p)); }
+__device__ __forceinline__ float load_logit(const f16_t* p) { return f16_bits_to_float(__ldg(&p->bits)); }
 
 struct RowNorm {
     float mt, md;          // row maxima
@@ -93,6 +104,12 @@ __device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
     return r;
 }
 
+__device__ __forceinline__ uint32_t max_f16x2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("max.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+
 // ---- statistics of a slice ------------------------------------------------------
 // Running (m, s) of one thread: s = sum exp2(fl(l c - mu)), mu = fl(m c) (0 while m = -inf).
 // One fused multiply-add per entry; the rounding of m c is taken out again in acc_close.
@@ -151,6 +168,18 @@ template <> struct SubLoad<uint16_t> {
         x[1][4] = __uint_as_float(b.z << 16); x[1][5] = __uint_as_float(b.z & 0xffff0000u);
         x[1][6] = __uint_as_float(b.w << 16); x[1][7] = __uint_as_float(b.w & 0xffff0000u);
         return fmaxf(__uint_as_float(pm << 16), __uint_as_float(pm & 0xffff0000u));
+    }
+};
+template <> struct SubLoad<f16_t> {
+    __device__ static __forceinline__ float load(const unsigned char* buf, int v0, int v1, float (&x)[2][8]) {
+        const uint4 a = reinterpret_cast<const uint4*>(buf)[v0];
+        const uint4 b = reinterpret_cast<const uint4*>(buf)[v1];
+        const uint32_t pm = max_f16x2(max_f16x2(max_f16x2(a.x, a.y), max_f16x2(a.z, a.w)),
+                                      max_f16x2(max_f16x2(b.x, b.y), max_f16x2(b.z, b.w)));
+        Vec<f16_t>::unpack(a, x[0]);
+        Vec<f16_t>::unpack(b, x[1]);
+        const float2 m = f16x2_to_float2(pm);
+        return fmaxf(m.x, m.y);
     }
 };
 

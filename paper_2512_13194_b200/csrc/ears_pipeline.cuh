@@ -117,6 +117,27 @@ __device__ __forceinline__ float ex2_approx(float x) {
 
 __device__ __forceinline__ float bf16_bits_to_float(uint32_t bits16) { return __uint_as_float(bits16 << 16); }
 
+// IEEE binary16 logits: a 2-byte element type of its own (uint16_t stands for bfloat16 bits).
+struct f16_t { uint16_t bits; };
+
+// both halves of a packed pair -> fp32 (exact)
+__device__ __forceinline__ float2 f16x2_to_float2(uint32_t w) {
+    float lo, hi;
+    asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\tcvt.f32.f16 %0, l;\n\tcvt.f32.f16 %1, h;\n\t}"
+        : "=f"(lo), "=f"(hi) : "r"(w));
+    return make_float2(lo, hi);
+}
+// one element through the read-only path, unconverted
+__device__ __forceinline__ float ld_elem(const float* p) { return __ldg(p); }
+__device__ __forceinline__ uint16_t ld_elem(const uint16_t* p) { return __ldg(p); }
+__device__ __forceinline__ f16_t ld_elem(const f16_t* p) { f16_t r; r.bits = __ldg(&p->bits); return r; }
+
+__device__ __forceinline__ float f16_bits_to_float(uint16_t bits) {
+    float r;
+    asm("cvt.f32.f16 %0, %1;" : "=f"(r) : "h"(bits));
+    return r;
+}
+
 // (m, s) pairs describe sum_v exp2((l_v - m) * c) = s.  Merging keeps the larger m.
 // -inf maxima (nothing finite seen yet) contribute nothing; NaN sums propagate.
 __device__ __forceinline__ void merge_ms(float& m, float& s, float m2, float s2, float c) {

@@ -361,8 +361,8 @@ __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RPara
             E* st = reinterpret_cast<E*>(buf_t);
             E* sd = reinterpret_cast<E*>(buf_d);
             for (int i = tid; i < n; i += kRThreads) {
-                st[i] = __ldg(trow + i);
-                if (pair) sd[i] = __ldg(drow + i);
+                st[i] = ld_elem(trow + i);
+                if (pair) sd[i] = ld_elem(drow + i);
             }
             __syncthreads();
         }

@@ -6,8 +6,8 @@ logits and draft tokens with the shapes and value distributions of the five
 workload configurations (they stand in for logits a target/draft model pair
 would produce during serving; no model or dataset is involved).
 
-Conventions: ``N(0, s)`` means standard deviation ``s``.  bf16 tensors are made
-in fp32 and rounded to bf16 *before* the draft tokens are drawn, so every
+Conventions: ``N(0, s)`` means standard deviation ``s``.  bf16 and fp16 tensors are made
+in fp32 and rounded *before* the draft tokens are drawn, so every
 consumer sees identical bits.  Draft tokens are drawn from the softmax of the
 (rounded) draft logits at the call's temperature, as a draft model would.
 Generation runs in fixed blocks of sequences so peak memory stays bounded and the
@@ -22,6 +22,7 @@ from typing import Tuple
 import torch
 
 _BLOCK = 16  # sequences generated at a time
+TORCH_DTYPES = {"fp32": torch.float32, "bf16": torch.bfloat16, "fp16": torch.float16}
 
 
 @dataclass(frozen=True)
@@ -30,7 +31,7 @@ class Workload:
     B: int
     K: int
     V: int
-    dtype: str            # "fp32" | "bf16"
+    dtype: str            # "fp32" | "bf16" | "fp16"
     temperature: float
     beta: float
     recipe: str           # which generator below
@@ -127,7 +128,7 @@ def make_inputs(w: Workload, device="cpu", temperature: float | None = None):
     """
     device = torch.device(device)
     T = w.temperature if temperature is None else float(temperature)
-    tdt = torch.float32 if w.dtype == "fp32" else torch.bfloat16
+    tdt = TORCH_DTYPES[w.dtype]
     gen = torch.Generator(device=device)
     gen.manual_seed(w.data_seed)
     t_out = torch.empty((w.B, w.K + 1, w.V), dtype=tdt, device=device)
@@ -152,7 +153,7 @@ def tiny_inputs(B: int, K: int, V: int, dtype: str = "fp32", seed: int = 0, scal
     device = torch.device(device)
     gen = torch.Generator(device=device)
     gen.manual_seed(seed)
-    tdt = torch.float32 if dtype == "fp32" else torch.bfloat16
+    tdt = TORCH_DTYPES[dtype]
     t = (torch.randn(B, K + 1, V, generator=gen, device=device) * scale)
     d = (t[:, :K] + torch.randn(B, K, V, generator=gen, device=device) * noise).to(tdt)
     t = t.to(tdt)

@@ -31,6 +31,7 @@ def make(B, K, V, dtype, seed, miss=0.25):
 @pytest.mark.parametrize("B,K,V,dtype", [
     (1, 1, 1, "fp32"), (2, 3, 7, "bf16"), (3, 2, 1023, "fp32"), (2, 2, 4097, "bf16"), (4, 5, 32000, "fp32"),
     (3, 4, 32001, "bf16"), (6, 7, 128256, "bf16"), (1, 64, 515, "fp32"), (700, 2, 130, "fp32"), (2, 1, 1000003, "fp32"),
+    (2, 3, 7, "fp16"), (2, 2, 4097, "fp16"), (6, 7, 128256, "fp16"), (300, 2, 1400, "fp16"),
 ])
 def test_greedy_parity_shapes(ears, B, K, V, dtype):
     t, x = make(B, K, V, dtype, seed=B + K + V)

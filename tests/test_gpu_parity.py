@@ -56,6 +56,8 @@ SHAPES = [
     (2, 3, 1023, "fp32"), (3, 1, 1025, "bf16"), (2, 2, 4096, "fp32"), (2, 2, 4097, "fp32"),
     (2, 2, 8192, "bf16"), (1, 4, 8200, "bf16"), (4, 5, 32000, "fp32"), (3, 4, 32001, "bf16"),
     (2, 3, 70001, "fp32"), (5, 7, 50000, "bf16"), (1, 64, 515, "fp32"), (700, 2, 130, "fp32"),
+    (3, 2, 8, "fp16"), (3, 1, 1025, "fp16"), (1, 4, 8200, "fp16"), (3, 4, 32001, "fp16"), (5, 7, 50000, "fp16"),
+    (300, 2, 700, "fp16"),
 ]
 
 
@@ -115,6 +117,24 @@ def test_parity_workloads(ears, forced_path, idx, path):
     assert tally.max_rel_prob_err < 1e-5
     print(f"\n{w.name}: rows={tally.rows} explained={tally.explained} flagged_dec={tally.flagged_decisions} "
           f"flagged_tok={tally.flagged_tokens} max_rel={tally.max_rel_prob_err:.2e} mean_len={np.mean(lens):.2f}")
+
+
+@pytest.mark.parametrize("path", [0, 1, 3])
+@pytest.mark.parametrize("idx,B", [(2, 8), (3, 32), (4, 128), (4, 24)])
+def test_parity_fp16_workload_shapes(ears, forced_path, idx, B, path):
+    """The 2-byte workloads with IEEE binary16 logits instead of bfloat16 (same values before
+    rounding), in the automatic launch configuration and with each streaming kernel forced."""
+    from dataclasses import replace
+    forced_path(path)
+    w = replace(synth.workload(idx), dtype="fp16", B=B)
+    t, d, x = synth.make_inputs(w, "cpu")
+    assert t.dtype == torch.float16
+    tally = Tally()
+    for offset, beta in enumerate([w.beta, 0.0]):
+        tl, *_ = run_both(ears, w, t, d, x, w.temperature, beta, seed=w.verify_seed, offset=offset)
+        tally.merge(tl)
+    assert_parity(tally)
+    assert tally.max_rel_prob_err < 1e-5
 
 
 @pytest.mark.parametrize("beta", [1.0, 0.0])
@@ -185,10 +205,11 @@ def test_forced_resident_path_refuses_rows_that_do_not_fit(ears, forced_path):
     assert e.value.status == -2
 
 
+@pytest.mark.parametrize("dtype", ["fp32", "fp16"])
 @pytest.mark.parametrize("path", [1, 2, 3])
-def test_invalid_sequences_are_marked(ears, forced_path, path):
+def test_invalid_sequences_are_marked(ears, forced_path, path, dtype):
     forced_path(path)
-    w, t, d, x = synth.tiny_inputs(8, 3, 5000, "fp32", seed=9)
+    w, t, d, x = synth.tiny_inputs(8, 3, 5000, dtype, seed=9)
     t = t.clone(); d = d.clone(); x = x.clone()
     x[1, 0] = 5000
     x[2, 2] = -3

@@ -337,6 +337,30 @@ def test_bf16_rows_widen_exactly():
     assert np.array_equal(a.tokens, b.tokens) and np.array_equal(a.pt_tok, b.pt_tok)
 
 
+def test_fp16_bits_widen_like_the_library_conversion():
+    """All 65536 binary16 patterns against numpy's float16 -> float64 conversion; fp16 rows give the
+    same step as the same values held in fp32."""
+    import torch
+    bits = np.arange(65536, dtype=np.uint16)
+    want = bits.view(np.float16).astype(np.float64)
+    got = np.array([oracle.half_to_double(int(b)) for b in bits])
+    assert np.array_equal(np.isnan(want), np.isnan(got))
+    ok = ~np.isnan(want)
+    assert np.array_equal(want[ok], got[ok]) and np.array_equal(np.signbit(want[ok]), np.signbit(got[ok]))
+    g = torch.Generator().manual_seed(3)
+    B, K, V = 4, 2, 200
+    t = (3 * torch.randn(B, K + 1, V, generator=g)).to(torch.float16)
+    d = (3 * torch.randn(B, K, V, generator=g)).to(torch.float16)
+    t[0, 1, 5] = float("-inf")
+    t[1, 0, 7] = 6e-8   # subnormal in binary16
+    x = torch.randint(0, V, (B, K), generator=g).to(torch.int32)
+    a = oracle.verify(t, d, x, 0.9, 0.2, seed=1)
+    b = oracle.verify(t.float(), d.float(), x, 0.9, 0.2, seed=1)
+    c = oracle.verify(t.numpy(), d.numpy(), x, 0.9, 0.2, seed=1)
+    assert np.array_equal(a.tokens, b.tokens) and np.array_equal(a.pt_tok, b.pt_tok) and np.array_equal(a.margin, b.margin)
+    assert np.array_equal(a.tokens, c.tokens) and np.array_equal(a.pt_tok, c.pt_tok)
+
+
 def test_invalid_sequences_are_marked_not_fatal():
     rng = np.random.default_rng(15)
     B, K, V = 6, 2, 32
