@@ -373,6 +373,53 @@ def run_table(args):
             del t, d, x
 
 
+def run_shard_table(args):
+    """One rank's share of the vocabulary-sharded step, phase by phase, on one GPU: this rank's
+    columns of every row with the synthetic distributions of the workload, the other ranks'
+    statistics and masses stood in for by copies of this rank's own (same sizes; the exchanges
+    themselves are not timed here).  L2 flushed before every step.  Not the benchmark line."""
+    import torch
+
+    import paper_2512_13194_b200 as ears
+    from dataclasses import replace
+    from paper_2512_13194_b200 import synth
+    from paper_2512_13194_b200.shard import vocab_range
+
+    torch.cuda.set_device(0)
+    ears.load_library()
+    peak, peak_kind = measured_peak()
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    print(f"| workload | B | ranks | columns per rank | dtype | statistics us (GB/s, of {peak:.0f} {peak_kind}) | decisions + mass us "
+          f"| pick us | exchanged bytes per rank |")
+    print("|---|---|---|---|---|---|---|---|---|")
+    for idx, B, n in ((5, 512, 8), (5, 512, 2), (4, 1024, 8), (4, 128, 4), (3, 32, 2), (2, 4096, 2)):
+        w = replace(synth.workload(idx), B=B)
+        _, Vs = vocab_range(w.V, 0, n)
+        t, d, x = synth.make_inputs(replace(w, V=Vs), "cuda:0")
+        step = ears.ShardStep(t, d, x, 0, w.V, w.temperature, w.beta, 0, 1)
+        res = []
+        for it in range(args.warmup + 9):
+            flush.zero_()
+            e = [ev() for _ in range(6)]
+            e[0].record(); st = step.stats(); e[1].record()
+            all_stats = st[None].repeat(n, 1, 1)
+            all_stats[1:, :, 3] = 0          # every token claimed once
+            e[2].record(); m = step.decide(all_stats); e[3].record()
+            all_mass = m[None].repeat(n, 1)
+            e[4].record(); step.pick(0, all_stats, all_mass); e[5].record()
+            torch.cuda.synchronize()
+            if it >= args.warmup:
+                res.append(tuple(e[2 * i].elapsed_time(e[2 * i + 1]) * 1e3 for i in range(3)))
+        res = sorted(res, key=sum)[len(res) // 2]
+        nbytes = (t.numel() + d.numel()) * t.element_size()
+        gbs = nbytes / res[0] / 1e3
+        xbytes = B * (2 * w.K + 1) * 16 + B * 8 + B * (w.K + 1) * 4
+        print(f"| {idx} | {B} | {n} | {Vs} | {w.dtype} | {res[0]:.1f} ({gbs:.0f}, {gbs / peak:.2f}) | {res[1]:.1f} | {res[2]:.1f} | {xbytes} |",
+              flush=True)
+        del t, d, x, step
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -386,8 +433,12 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--table", action="store_true", help="print the five-workload results table instead")
     ap.add_argument("--table-full", action="store_true", help="also time the 1-thread oracle on workload 5")
+    ap.add_argument("--shard-table", action="store_true",
+                    help="print per-phase times of one rank of the vocabulary-sharded step instead")
     args = ap.parse_args()
-    if args.table:
+    if args.shard_table:
+        run_shard_table(args)
+    elif args.table:
         run_table(args)
     elif args.impl == "reference":
         run_reference(args)

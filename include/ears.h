@@ -178,6 +178,61 @@ int ears_verify_greedy(int dtype, const void* target_logits, const int32_t* draf
                        void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Verification with the VOCABULARY split across devices (tensor-parallel logits).  Device r of
+ * n_shards holds the columns [v_first, v_first + Vs) of every row: target_shard [B, K+1, Vs],
+ * draft_shard [B, K, Vs], row-major and contiguous; the devices' column ranges are disjoint,
+ * cover [0, V) and ascend with r.  draft_tokens [B, K] (ids in [0, V)) are the same everywhere.
+ * The step is the one of ears_verify_ex [Sec. 3.1-3.3] on the concatenated rows, computed in
+ * three local phases with two small exchanges the CALLER performs (all-gathers of device
+ * buffers, e.g. NCCL; logits never move):
+ *
+ *   ears_shard_stats   -> out_stats [B (2K+1)] x 4 floats per row of this device's columns:
+ *                         (max m, sum of exp((l - m)/T), logit of the row's draft token if its
+ *                         column lies here else 0, 1 or 0 saying which).  Rows of a sequence:
+ *                         target 0..K, then draft 0..K-1.
+ *   -- all-gather out_stats over devices into all_stats [n_shards][B (2K+1)][4] --
+ *   ears_shard_decide  -> every device combines the statistics in device order (so decisions
+ *                         are bitwise identical everywhere), applies the acceptance rule of
+ *                         Sec. 3.2 per position with U_k from the counter stream of ears_verify,
+ *                         writes out_accept_len [B] and the accepted prefix of out_tokens
+ *                         [B, K+1] (-1 elsewhere), and out_mass [B]: the mass this device's
+ *                         columns hold of the row to draw from, in units of 1/Z_t
+ *                         (max(0, P_t - P_d) of the rejected position, P_t of row K after K
+ *                         acceptances).  Invalid sequences (as in ears_verify, or a token whose
+ *                         column no device or more than one device claimed): length -1, tokens -1.
+ *   -- all-gather out_mass over devices into all_mass [n_shards][B] --
+ *   ears_shard_pick    -> the device whose columns contain the point u S of the cumulative mass
+ *                         (devices in order; u the final uniform of ears_verify, S the total)
+ *                         writes the drawn token's id into out_tokens[b, n]; the others leave
+ *                         -1 there.  An element-wise MAX of out_tokens over devices completes
+ *                         the step on every device.
+ *
+ * All pointers are device memory.  `workspace` (256-byte aligned, at least
+ * ears_shard_workspace_bytes(dtype, B, K, Vs) bytes, caller-owned) carries state from phase to
+ * phase: pass the same buffer, untouched, to the three calls of one step.  Calls are enqueued
+ * on `stream`; nothing synchronises.  temperature, seed, offset, b_first as in ears_verify_ex.
+ * Errors: as ears_verify_ex; EARS_ERR_SHAPE also for v_first / Vs outside [0, V];
+ * EARS_ERR_PARAM for n_shards outside [1, EARS_MAX_SHARDS] or shard outside [0, n_shards).
+ */
+#define EARS_MAX_SHARDS 64
+size_t ears_shard_workspace_bytes(int dtype, int B, int K, int Vs);
+int ears_shard_stats(int dtype, const void* target_shard, const void* draft_shard,
+                     const int32_t* draft_tokens, int B, int K, int Vs, int V, int v_first,
+                     float temperature, float* out_stats,
+                     void* workspace, size_t workspace_bytes, void* stream);
+int ears_shard_decide(int dtype, const void* target_shard, const void* draft_shard,
+                      const int32_t* draft_tokens, int B, int K, int Vs, int V, int v_first,
+                      int n_shards, const float* all_stats, float temperature, float beta,
+                      uint64_t seed, uint64_t offset, int64_t b_first,
+                      int32_t* out_accept_len, int32_t* out_tokens, double* out_mass,
+                      void* workspace, size_t workspace_bytes, void* stream);
+int ears_shard_pick(int dtype, const void* target_shard, const void* draft_shard,
+                    const int32_t* draft_tokens, int B, int K, int Vs, int V, int v_first,
+                    int n_shards, int shard, const float* all_stats, const double* all_mass,
+                    float temperature, uint64_t seed, uint64_t offset, int64_t b_first,
+                    int32_t* out_tokens, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Same step with HOST buffers: copies the inputs to library-owned device staging
  * buffers, runs the step, copies out_accept_len / out_tokens back and waits for
  * completion.  All pointers are host memory (pinned memory makes the copies

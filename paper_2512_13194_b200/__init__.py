@@ -2,13 +2,15 @@
 
 ``verify`` and friends call the C-ABI library built from ``csrc/`` (declared in
 ``include/ears.h``); there is no CPU fallback.  ``synth`` holds the seeded
-synthetic workloads, ``shard`` the batch partition used across GPUs.
+synthetic workloads, ``shard`` the batch partition used across GPUs and
+the driver of the vocabulary-sharded step.
 """
 from . import shard, synth  # noqa: F401
 from .binding import (  # noqa: F401
     DEV_INVALID_INPUT,
     DEV_TIMEOUT,
     EarsError,
+    ShardStep,
     class_counts,
     describe_plan,
     last_device_status,

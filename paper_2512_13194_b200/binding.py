@@ -53,6 +53,18 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ears_verify_host.restype = c.c_int
     lib.ears_verify_noalloc.argtypes = [c.c_int] + common + [c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
     lib.ears_verify_noalloc.restype = c.c_int
+    shard_head = [c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_int, c.c_int, c.c_int]
+    lib.ears_shard_workspace_bytes.argtypes = [c.c_int, c.c_int, c.c_int, c.c_int]
+    lib.ears_shard_workspace_bytes.restype = c.c_size_t
+    lib.ears_shard_stats.argtypes = shard_head + [c.c_float, c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p]
+    lib.ears_shard_stats.restype = c.c_int
+    lib.ears_shard_decide.argtypes = shard_head + [c.c_int, c.c_void_p, c.c_float, c.c_float, c.c_uint64, c.c_uint64,
+                                                   c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p,
+                                                   c.c_void_p, c.c_size_t, c.c_void_p]
+    lib.ears_shard_decide.restype = c.c_int
+    lib.ears_shard_pick.argtypes = shard_head + [c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_float, c.c_uint64,
+                                                 c.c_uint64, c.c_int64, c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p]
+    lib.ears_shard_pick.restype = c.c_int
     lib.ears_workspace_bytes.argtypes = [c.c_int, c.c_int, c.c_int]
     lib.ears_workspace_bytes.restype = c.c_size_t
     lib.ears_last_device_status.argtypes = [c.c_void_p]
@@ -322,6 +334,79 @@ def philox_device(ctr_key: torch.Tensor) -> torch.Tensor:
 
 def set_plan(loader: int = 0, parts: int = 0) -> None:
     _check(load_library().ears_set_plan(loader, parts))
+
+
+class ShardStep:
+    """One device's part of a verification step whose vocabulary is split across devices: the
+    three local phases of ``ears_shard_stats`` / ``_decide`` / ``_pick``.  The caller exchanges the
+    small results between the phases (``shard.verify_vocab_sharded`` does it with a communicator).
+
+    target_shard [B,K+1,Vs] and draft_shard [B,K,Vs] hold columns [v_first, v_first+Vs) of a
+    vocabulary of V entries; draft_tokens [B,K] int32 are ids in [0, V)."""
+
+    def __init__(self, target_shard: torch.Tensor, draft_shard: torch.Tensor, draft_tokens: torch.Tensor,
+                 v_first: int, V: int, temperature: float, beta: float, seed: int = 0, offset: int = 0,
+                 b_first: int = 0):
+        if not target_shard.is_cuda:
+            raise RuntimeError("ears: the step runs on CUDA devices only")
+        self.t, self.d, self.x = target_shard.contiguous(), draft_shard.contiguous(), draft_tokens.contiguous()
+        self.B, K1, self.Vs = self.t.shape
+        self.K = K1 - 1
+        if self.d.shape != (self.B, self.K, self.Vs) or self.x.shape != (self.B, self.K) or self.x.dtype != torch.int32:
+            raise ValueError("shape or dtype mismatch")
+        if self.d.dtype != self.t.dtype:
+            raise TypeError("target and draft logits must share a dtype")
+        self.dtype = _dtype_code(self.t)
+        self.v_first, self.V = int(v_first), int(V)
+        self.T, self.beta, self.seed, self.offset, self.b_first = float(temperature), float(beta), int(seed), int(offset), int(b_first)
+        self.lib = load_library()
+        dev = self.t.device
+        nbytes = self.lib.ears_shard_workspace_bytes(self.dtype, self.B, self.K, self.Vs)
+        if nbytes == 0:
+            raise EarsError(-2, "bad shape")
+        self.ws = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        self.acc = torch.empty(self.B, dtype=torch.int32, device=dev)
+        self.tok = torch.empty((self.B, self.K + 1), dtype=torch.int32, device=dev)
+
+    def _head(self):
+        return (self.dtype, self.t.data_ptr(), self.d.data_ptr(), self.x.data_ptr(), self.B, self.K, self.Vs, self.V,
+                self.v_first)
+
+    def _stream(self):
+        return torch.cuda.current_stream(self.t.device).cuda_stream
+
+    def stats(self) -> torch.Tensor:
+        """-> [B (2K+1), 4] float32: (m, s, token logit, token column here) per row of the local columns."""
+        out = torch.empty((self.B * (2 * self.K + 1), 4), dtype=torch.float32, device=self.t.device)
+        with torch.cuda.device(self.t.device):
+            _check(self.lib.ears_shard_stats(*self._head(), self.T, out.data_ptr(), self.ws.data_ptr(), self.ws.numel(),
+                                             self._stream()))
+        return out
+
+    def decide(self, all_stats: torch.Tensor) -> torch.Tensor:
+        """all_stats [n_shards, B (2K+1), 4] -> [B] float64: local mass of the row each sequence draws from."""
+        all_stats = all_stats.contiguous()
+        self.n_shards = int(all_stats.shape[0])
+        if all_stats.shape[1:] != (self.B * (2 * self.K + 1), 4) or all_stats.dtype != torch.float32:
+            raise ValueError("all_stats must be [n_shards, B (2K+1), 4] float32")
+        mass = torch.empty(self.B, dtype=torch.float64, device=self.t.device)
+        with torch.cuda.device(self.t.device):
+            _check(self.lib.ears_shard_decide(*self._head(), self.n_shards, all_stats.data_ptr(), self.T, self.beta,
+                                              self.seed, self.offset, self.b_first, self.acc.data_ptr(), self.tok.data_ptr(),
+                                              mass.data_ptr(), self.ws.data_ptr(), self.ws.numel(), self._stream()))
+        return mass
+
+    def pick(self, shard: int, all_stats: torch.Tensor, all_mass: torch.Tensor):
+        """-> (accept_len [B], tokens [B,K+1]); tokens[b, n] holds the drawn token only on the device
+        that owns it (-1 elsewhere): an element-wise MAX over devices completes it."""
+        all_stats, all_mass = all_stats.contiguous(), all_mass.contiguous()
+        if all_mass.shape != (self.n_shards, self.B) or all_mass.dtype != torch.float64:
+            raise ValueError("all_mass must be [n_shards, B] float64")
+        with torch.cuda.device(self.t.device):
+            _check(self.lib.ears_shard_pick(*self._head(), self.n_shards, int(shard), all_stats.data_ptr(),
+                                            all_mass.data_ptr(), self.T, self.seed, self.offset, self.b_first,
+                                            self.tok.data_ptr(), self.ws.data_ptr(), self.ws.numel(), self._stream()))
+        return self.acc, self.tok
 
 
 def set_path(path: int = 0, cluster: int = 0) -> None:

@@ -2,6 +2,7 @@
 // launch plan, workspace management and the kernel launch.
 #include "../../include/ears.h"
 
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -17,6 +18,7 @@
 #include "ears_resident.cuh"
 #include "ears_greedy.cuh"
 #include "ears_direct.cuh"
+#include "ears_shard.cuh"
 
 namespace {
 
@@ -714,6 +716,74 @@ int read_status(int* heads, cudaStream_t stream) {
     return status;
 }
 
+
+// ---- vocabulary-sharded verification (three local phases, see ears_shard.cuh) ----
+constexpr long long kShardWarpRowBytes = 256 * 1024;   // rows up to this size may go one per warp
+
+struct SLayout {
+    int P, piece_elems, nseg;
+    size_t counters_bytes, ticket_row, ticket_seq, partial, rowstat, sel, seg, total;
+};
+
+SLayout make_slayout(int B, int K, int Vs, int esize) {
+    SLayout L;
+    const long long rows = (long long)B * (2 * K + 1);
+    // about a thousand units (a few per CTA of a full grid), pieces of at least 16 KB
+    long long P = (1024 + rows - 1) / rows;
+    const long long most = std::max<long long>(1, (long long)Vs * esize / 16384);
+    P = std::max<long long>(1, std::min<long long>(std::min<long long>(P, most), 64));
+    L.piece_elems = (int)((((long long)Vs + P - 1) / P + 255) / 256 * 256);
+    L.P = (Vs + L.piece_elems - 1) / L.piece_elems;
+    L.nseg = (Vs + kSegElems - 1) / kSegElems;
+    auto up = [](size_t v) { return (v + 255) / 256 * 256; };
+    size_t o = 0;
+    L.ticket_row = o; o = up(o + (size_t)rows * 4);
+    L.ticket_seq = o; o = up(o + (size_t)B * 4);
+    L.counters_bytes = o;
+    L.partial = o; o = up(o + (size_t)rows * L.P * 8);
+    L.rowstat = o; o = up(o + (size_t)rows * 16);
+    L.sel = o; o = up(o + (size_t)B * 4);
+    L.seg = o; o = up(o + (size_t)B * L.nseg * 8);
+    L.total = o;
+    return L;
+}
+
+int shard_common(int dtype, const void* t, const void* d, const int32_t* x, int B, int K, int Vs, int V, int v_first,
+                 int n_shards, int shard, float temperature, void* workspace, size_t workspace_bytes, SParams* p, SLayout* L,
+                 DeviceInfo** di) {
+    if (!t || !d || !x || !workspace) return EARS_ERR_NULL;
+    if (!dtype_ok(dtype)) return EARS_ERR_PARAM;
+    int rc = check_shape(B, K, Vs);
+    if (rc) return rc;
+    if (V < Vs || V > (1 << 30) || v_first < 0 || v_first > V - Vs) return EARS_ERR_SHAPE;
+    if (n_shards < 1 || n_shards > EARS_MAX_SHARDS || shard < 0 || shard >= n_shards) return EARS_ERR_PARAM;
+    if (!(temperature > 0.0f) || !std::isfinite(temperature)) return EARS_ERR_PARAM;
+    const int esize = dtype_size(dtype);
+    if (((uintptr_t)t % esize) || ((uintptr_t)d % esize) || ((uintptr_t)x % 4) || ((uintptr_t)workspace % 256)) return EARS_ERR_ALIGN;
+    *L = make_slayout(B, K, Vs, esize);
+    if (workspace_bytes < L->total) return EARS_ERR_WORKSPACE;
+    int dev = 0;
+    EARS_CUDA(cudaGetDevice(&dev));
+    rc = device_info(dev, di);
+    if (rc) return rc;
+    char* w = (char*)workspace;
+    *p = SParams();
+    p->t = t; p->d = d; p->x = x;
+    p->B = B; p->K = K; p->Vs = Vs; p->V = V; p->v_first = v_first; p->n_shards = n_shards;
+    p->P = L->P; p->piece_elems = L->piece_elems;
+    p->vec = ((uintptr_t)t % 16 == 0) && ((uintptr_t)d % 16 == 0) && (((size_t)Vs * esize) % 16 == 0);
+    p->c = (float)(1.4426950408889634 / (double)temperature);
+    p->T = (double)temperature;
+    p->ticket_row = (int*)(w + L->ticket_row);
+    p->ticket_seq = (int*)(w + L->ticket_seq);
+    p->partial = (float2*)(w + L->partial);
+    p->rowstat = (float4*)(w + L->rowstat);
+    p->sel = (int*)(w + L->sel);
+    p->seg = (double*)(w + L->seg);
+    p->nseg = L->nseg;
+    return EARS_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -1023,6 +1093,104 @@ const char* ears_status_string(int status) {
         case EARS_ERR_TIMEOUT: return "a device-side wait timed out";
         default: return "unknown status";
     }
+}
+
+size_t ears_shard_workspace_bytes(int dtype, int B, int K, int Vs) {
+    if (!dtype_ok(dtype) || check_shape(B, K, Vs)) return 0;
+    return make_slayout(B, K, Vs, dtype_size(dtype)).total;
+}
+
+int ears_shard_stats(int dtype, const void* target_shard, const void* draft_shard, const int32_t* draft_tokens,
+                     int B, int K, int Vs, int V, int v_first, float temperature, float* out_stats,
+                     void* workspace, size_t workspace_bytes, void* stream_) {
+    if (!out_stats) return EARS_ERR_NULL;
+    if ((uintptr_t)out_stats % 16) return EARS_ERR_ALIGN;
+    SParams p; SLayout L; DeviceInfo* di = nullptr;
+    int rc = shard_common(dtype, target_shard, draft_shard, draft_tokens, B, K, Vs, V, v_first, 1, 0, temperature,
+                          workspace, workspace_bytes, &p, &L, &di);
+    if (rc) return rc;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    p.stats = (float4*)out_stats;
+    const long long rows = (long long)B * (2 * K + 1), cap = (long long)kSCtasPerSm * di->sms;
+    if (L.P == 1 && (long long)Vs * dtype_size(dtype) <= kShardWarpRowBytes && rows >= 2 * cap * (kSThreads / 32)) {
+        // many short rows (several rounds of one row per warp): a warp per row
+        const long long want = (rows + kSThreads / 32 - 1) / (kSThreads / 32);
+        const int grid = (int)(want < cap ? want : cap);
+        by_dtype(dtype, [&](auto* e) {
+            ears_shard_stats_rows_kernel<std::remove_pointer_t<decltype(e)>><<<grid, kSThreads, 0, stream>>>(p);
+            return 0;
+        });
+    } else {
+        EARS_CUDA(cudaMemsetAsync(p.ticket_row, 0, (size_t)rows * 4, stream));
+        const long long units = rows * L.P;
+        const int grid = (int)(units < cap ? units : cap);
+        by_dtype(dtype, [&](auto* e) {
+            ears_shard_stats_kernel<std::remove_pointer_t<decltype(e)>><<<grid, kSThreads, 0, stream>>>(p);
+            return 0;
+        });
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "ears_shard_stats_kernel launch");
+    return EARS_OK;
+}
+
+int ears_shard_decide(int dtype, const void* target_shard, const void* draft_shard, const int32_t* draft_tokens,
+                      int B, int K, int Vs, int V, int v_first, int n_shards, const float* all_stats,
+                      float temperature, float beta, uint64_t seed, uint64_t offset, int64_t b_first,
+                      int32_t* out_accept_len, int32_t* out_tokens, double* out_mass,
+                      void* workspace, size_t workspace_bytes, void* stream_) {
+    if (!all_stats || !out_accept_len || !out_tokens || !out_mass) return EARS_ERR_NULL;
+    if (((uintptr_t)all_stats % 16) || ((uintptr_t)out_mass % 8)) return EARS_ERR_ALIGN;
+    if (!(beta >= 0.0f) || !std::isfinite(beta)) return EARS_ERR_PARAM;
+    if (b_first < 0 || (unsigned long long)b_first + (unsigned long long)B > 0xffffffffull) return EARS_ERR_PARAM;
+    SParams p; SLayout L; DeviceInfo* di = nullptr;
+    int rc = shard_common(dtype, target_shard, draft_shard, draft_tokens, B, K, Vs, V, v_first, n_shards, 0, temperature,
+                          workspace, workspace_bytes, &p, &L, &di);
+    if (rc) return rc;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    p.all_stats = (const float4*)all_stats;
+    p.beta = (double)beta;
+    p.seed = seed; p.offset = offset; p.b_first = b_first;
+    p.out_len = out_accept_len; p.out_tok = out_tokens; p.mass = out_mass;
+    EARS_CUDA(cudaMemsetAsync(p.ticket_seq, 0, (size_t)B * 4, stream));
+    ears_shard_decide_kernel<<<(B + kSSeqPerCta - 1) / kSSeqPerCta, kSSeqPerCta * 32, 0, stream>>>(p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "ears_shard_decide_kernel launch");
+    const int cps = (L.nseg + kSSegsPerCta - 1) / kSSegsPerCta;
+    if ((long long)B * cps > 0x7fffffffll) return EARS_ERR_SHAPE;
+    by_dtype(dtype, [&](auto* el) {
+        ears_shard_mass_kernel<std::remove_pointer_t<decltype(el)>><<<B * cps, kSThreads, 0, stream>>>(p, cps);
+        return 0;
+    });
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "ears_shard_mass_kernel launch");
+    return EARS_OK;
+}
+
+int ears_shard_pick(int dtype, const void* target_shard, const void* draft_shard, const int32_t* draft_tokens,
+                    int B, int K, int Vs, int V, int v_first, int n_shards, int shard, const float* all_stats,
+                    const double* all_mass, float temperature, uint64_t seed, uint64_t offset, int64_t b_first,
+                    int32_t* out_tokens, void* workspace, size_t workspace_bytes, void* stream_) {
+    if (!all_stats || !all_mass || !out_tokens) return EARS_ERR_NULL;
+    if (((uintptr_t)all_stats % 16) || ((uintptr_t)all_mass % 8)) return EARS_ERR_ALIGN;
+    if (b_first < 0 || (unsigned long long)b_first + (unsigned long long)B > 0xffffffffull) return EARS_ERR_PARAM;
+    SParams p; SLayout L; DeviceInfo* di = nullptr;
+    int rc = shard_common(dtype, target_shard, draft_shard, draft_tokens, B, K, Vs, V, v_first, n_shards, shard, temperature,
+                          workspace, workspace_bytes, &p, &L, &di);
+    if (rc) return rc;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    p.all_stats = (const float4*)all_stats;
+    p.all_mass = all_mass;
+    p.seed = seed; p.offset = offset; p.b_first = b_first;
+    p.out_tok = out_tokens;
+    by_dtype(dtype, [&](auto* el) {
+        ears_shard_pick_kernel<std::remove_pointer_t<decltype(el)>>
+            <<<(B + kSSeqPerCta - 1) / kSSeqPerCta, kSSeqPerCta * 32, 0, stream>>>(p, shard);
+        return 0;
+    });
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "ears_shard_pick_kernel launch");
+    return EARS_OK;
 }
 
 const char* ears_last_cuda_error(void) { return g_cuda_error; }

@@ -136,8 +136,9 @@ __device__ __forceinline__ void fold_vectors(const uint4 (&w)[G], float c, RowAc
     }
 }
 
-// An ordinary row piece [e0, e1): every thread strides over it.  -> the thread's (m, s).
-template <typename E>
+// An ordinary row piece [e0, e1): THREADS threads (tid = 0 .. THREADS-1) stride over it.
+// -> the thread's (m, s).
+template <typename E, int THREADS = kDThreads>
 __device__ __forceinline__ float2 stream_piece(const E* row, int e0, int e1, bool vec, float c, int tid) {
     constexpr int N = Words<E>::N;
     RowAcc a;
@@ -146,22 +147,22 @@ __device__ __forceinline__ float2 stream_piece(const E* row, int e0, int e1, boo
         const uint4* vs = reinterpret_cast<const uint4*>(row + e0);
         const int nvec = (e1 - e0) / N;   // rows and pieces are whole vectors here
         int v = tid;
-        for (; v + (kDUnroll - 1) * kDThreads < nvec; v += kDUnroll * kDThreads) {
+        for (; v + (kDUnroll - 1) * THREADS < nvec; v += kDUnroll * THREADS) {
             uint4 w[kDUnroll];
 #pragma unroll
-            for (int j = 0; j < kDUnroll; ++j) w[j] = ld_stream16(vs + v + j * kDThreads);
+            for (int j = 0; j < kDUnroll; ++j) w[j] = ld_stream16(vs + v + j * THREADS);
             fold_vectors<E, kDUnroll>(w, c, a);
         }
-        for (; v + kDThreads < nvec; v += 2 * kDThreads) {   // what is left of a piece: two, then one at a time
-            uint4 w[2] = {ld_stream16(vs + v), ld_stream16(vs + v + kDThreads)};
+        for (; v + THREADS < nvec; v += 2 * THREADS) {   // what is left of a piece: two, then one at a time
+            uint4 w[2] = {ld_stream16(vs + v), ld_stream16(vs + v + THREADS)};
             fold_vectors<E, 2>(w, c, a);
         }
-        for (; v < nvec; v += kDThreads) {
+        for (; v < nvec; v += THREADS) {
             uint4 w[1] = {ld_stream16(vs + v)};
             fold_vectors<E, 1>(w, c, a);
         }
     } else {  // rows that are not 16-byte aligned: element by element
-        for (int i = e0 + tid; i < e1; i += kDThreads) {
+        for (int i = e0 + tid; i < e1; i += THREADS) {
             const float x = load_logit(row + i);
             acc_raise(a, x, c);
             a.s[0] += ex2_approx(__fmaf_rn(x, c, -a.mu));
