@@ -8,6 +8,8 @@ as the ordinary entry point, on two calls in a row (the array keeps the first ca
 contents, so the second call proves that what must start at zero is cleared), and that
 shapes too large for the array are refused.  It is collected last on purpose.
 """
+import gc
+
 import pytest
 import torch
 
@@ -28,6 +30,7 @@ def test_noalloc_matches_ordinary_entry_twice_in_a_row(ears):
             ref_len, ref_tok = ears.verify(tg, dg, xg, 0.9, beta, 5, offset, b_first=2)
             acc.fill_(-9)
             tok.fill_(-9)
+            gc.collect()                       # tensors that earlier tests left in reference cycles go now, not mid-call
             torch.cuda.synchronize()
             before = torch.cuda.memory_allocated()
             free_before = torch.cuda.mem_get_info()[0]
