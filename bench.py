@@ -393,7 +393,10 @@ def run_shard_table(args):
     print(f"| workload | B | ranks | columns per rank | dtype | statistics us (GB/s, of {peak:.0f} {peak_kind}) | decisions + mass us "
           f"| pick us | exchanged bytes per rank |")
     print("|---|---|---|---|---|---|---|---|---|")
-    for idx, B, n in ((5, 512, 8), (5, 512, 2), (4, 1024, 8), (4, 128, 4), (3, 32, 2), (2, 4096, 2)):
+    cases = ((5, 512, 8), (5, 512, 2), (4, 1024, 8), (4, 128, 4), (3, 32, 2), (2, 4096, 2))
+    if args.batch:   # one case (small ones for profiler captures)
+        cases = ((args.workload, args.batch, args.ranks),)
+    for idx, B, n in cases:
         w = replace(synth.workload(idx), B=B)
         _, Vs = vocab_range(w.V, 0, n)
         t, d, x = synth.make_inputs(replace(w, V=Vs), "cuda:0")
@@ -433,6 +436,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--table", action="store_true", help="print the five-workload results table instead")
     ap.add_argument("--table-full", action="store_true", help="also time the 1-thread oracle on workload 5")
+    ap.add_argument("--ranks", type=int, default=2, help="with --shard-table --batch: ranks the vocabulary is split over")
     ap.add_argument("--shard-table", action="store_true",
                     help="print per-phase times of one rank of the vocabulary-sharded step instead")
     args = ap.parse_args()

@@ -37,8 +37,9 @@
  *   - pointers are DEVICE pointers owned by the caller; the library neither
  *     retains nor frees them.  Logits must be aligned to their element size.
  *     When both logits bases are 16-byte aligned and V * elem_size is a multiple
- *     of 16 the rows are fetched with bulk asynchronous copies (TMA); otherwise a
- *     slower element-wise loader is used with identical results.
+ *     of 16 the rows are fetched with bulk asynchronous copies (TMA) or 16-byte
+ *     vector loads, depending on the kernel the call's shape selects; otherwise
+ *     slower element-wise loads are used with identical results.
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls
  *     enqueue work and return; they do not synchronise.
  *   - outputs: out_accept_len[b] = n in [0, K]; out_tokens[b, 0:n] = the accepted

@@ -128,17 +128,19 @@ __device__ __forceinline__ void acc_raise(RowAcc& a, float cm, float c) {
 }
 
 // -> (m, s) with s relative to the exact product m c: fl(m c) differs from m c by
-// delta = fma(m, c, -fl(m c)) exactly, and 2^delta = 1 + delta ln 2 to first order (|delta| < 1e-5).
+// delta = fma(m, c, -fl(m c)) exactly; the terms were taken relative to fl(m c) = m c - delta, so
+// every one carries the factor 2^delta, which is divided out: 2^-delta = 1 - delta ln 2 to first
+// order (|delta| < 1e-5).
 __device__ __forceinline__ float2 acc_close(const RowAcc& a, float c) {
     float s = (a.s[0] + a.s[1]) + (a.s[2] + a.s[3]);
-    if (a.m > -INFINITY && a.m < INFINITY) s = __fmaf_rn(s, 0.6931471805599453f * __fmaf_rn(a.m, c, -a.mu), s);
+    if (a.m > -INFINITY && a.m < INFINITY) s = __fmaf_rn(s, -0.6931471805599453f * __fmaf_rn(a.m, c, -a.mu), s);
     return make_float2(a.m, s);
 }
 
 // s, a sum of exp2((l - m) c), expressed relative to the maximum M >= m instead.  An empty part
 // (m = -inf) contributes nothing; NaN sums stay NaN.
 __device__ __forceinline__ float rebase_sum(float m, float s, float M, float c) {
-    const float sc = (m == -INFINITY) ? 0.f : ex2_approx((m - M) * c);
+    const float sc = (m == -INFINITY) ? 0.f : exp2f((m - M) * c);   // full precision: the factor scales a whole part
     return s * sc;
 }
 

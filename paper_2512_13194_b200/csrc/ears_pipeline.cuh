@@ -143,8 +143,10 @@ __device__ __forceinline__ float f16_bits_to_float(uint16_t bits) {
 __device__ __forceinline__ void merge_ms(float& m, float& s, float m2, float s2, float c) {
     float mn = fmaxf(m, m2);
     if (mn == -INFINITY) { s = s + s2; return; }  // both empty (sums are 0 unless NaN)
-    float a = ex2_approx((m - mn) * c);           // (-inf - finite) -> 0
-    float b = ex2_approx((m2 - mn) * c);
+    // full-precision exp2 (one of the two factors is exactly 1): merges happen once per piece, and
+    // the error of an approximate factor would be common to everything merged so far
+    float a = exp2f((m - mn) * c);                // (-inf - finite) -> 0
+    float b = exp2f((m2 - mn) * c);
     s = s * a + s2 * b;
     m = mn;
 }
