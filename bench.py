@@ -34,7 +34,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of ears_verify_kernel<float,6> from one ncu capture on
 # a 96-sequence batch of the default workload (691.07 MB + 4.24 MB), per sequence.  The traffic grows
 # in proportion to the number of sequences; set to None whenever the kernel changes after a capture.
-NCU_DRAM_BYTES_PER_SEQUENCE = (691068928 + 4242176) / 96
+NCU_DRAM_BYTES_PER_SEQUENCE = (690650624 + 4477440) / 96
 
 
 def measured_peak():
