@@ -336,7 +336,7 @@ int ears_set_plan(int loader, int parts);
  *   cluster = CTAs per cluster of the resident kernel: 1, 2, 4, 8 or 16.
  * Both kernels implement the same step (Sec. 3.1-3.3); results differ only through
  * floating-point summation order.  The initial values can also come from the environment,
- * read once when the library is loaded: EARS_PATH=streaming|resident, EARS_CLUSTER=1|2|4|8|16.
+ * read once when the library is loaded: EARS_PATH=streaming|resident|direct, EARS_CLUSTER=1|2|4|8|16.
  */
 int ears_set_path(int path, int cluster);
 

@@ -53,13 +53,14 @@ int cuda_fail(cudaError_t e, const char* what) {
 
 struct PlanOverride { int loader = 0, parts1 = 0, path = 0, cluster = 0; };
 
-// Initial choice of kernel from the environment (EARS_PATH=streaming|resident, EARS_CLUSTER=1..16),
+// Initial choice of kernel from the environment (EARS_PATH=streaming|resident|direct, EARS_CLUSTER=1..16),
 // for trying a launch plan on an unmodified caller; ears_set_path overrides it.
 PlanOverride override_from_env() {
     PlanOverride ov;
     if (const char* e = getenv("EARS_PATH")) {
         if (!strcmp(e, "streaming") || !strcmp(e, "1")) ov.path = 1;
         else if (!strcmp(e, "resident") || !strcmp(e, "2")) ov.path = 2;
+        else if (!strcmp(e, "direct") || !strcmp(e, "3")) ov.path = 3;
     }
     if (const char* e = getenv("EARS_CLUSTER")) {
         const int c = atoi(e);
