@@ -425,6 +425,41 @@ def run_shard_table(args):
         del t, d, x, step
 
 
+def run_greedy_table(args):
+    """The temperature -> 0 form (ears_verify_greedy: target rows only) on the five workloads' target
+    rows and two larger batches, L2 flushed before every step.  Not the benchmark line."""
+    import torch
+
+    import paper_2512_13194_b200 as ears
+    from dataclasses import replace
+    from paper_2512_13194_b200 import synth
+
+    torch.cuda.set_device(0)
+    ears.load_library()
+    peak, peak_kind = measured_peak()
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    print(f"| workload | B | dtype | target-row bytes | us per step | GB/s | of {peak:.0f} ({peak_kind}) |")
+    print("|---|---|---|---|---|---|---|")
+    for idx, B in ((1, 0), (2, 0), (3, 0), (4, 0), (5, 0), (4, 1024), (2, 4096)):
+        w = synth.workload(idx)
+        if B:
+            w = replace(w, B=B)
+        t, d, x = synth.make_inputs(w, "cuda:0")
+        del d
+        ts = []
+        for it in range(args.warmup + 21):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); ears.verify_greedy(t, x); b.record()
+            torch.cuda.synchronize()
+            if it >= args.warmup:
+                ts.append(a.elapsed_time(b) * 1e3)
+        us = statistics.median(ts)
+        nbytes = t.numel() * t.element_size()
+        print(f"| {idx} | {w.B} | {w.dtype} | {nbytes} | {us:.1f} | {nbytes / us / 1e3:.0f} | {nbytes / us / 1e3 / peak:.2f} |", flush=True)
+        del t, x
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -441,8 +476,11 @@ def main():
     ap.add_argument("--ranks", type=int, default=2, help="with --shard-table --batch: ranks the vocabulary is split over")
     ap.add_argument("--shard-table", action="store_true",
                     help="print per-phase times of one rank of the vocabulary-sharded step instead")
+    ap.add_argument("--greedy-table", action="store_true", help="print times of the temperature -> 0 form instead")
     args = ap.parse_args()
-    if args.shard_table:
+    if args.greedy_table:
+        run_greedy_table(args)
+    elif args.shard_table:
         run_shard_table(args)
     elif args.table:
         run_table(args)

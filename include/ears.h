@@ -97,6 +97,12 @@ int ears_verify_bf16(const void* target_logits, const void* draft_logits,
                      float temperature, float beta, uint64_t seed, uint64_t offset,
                      int32_t* out_accept_len, int32_t* out_tokens, void* stream);
 
+/* Same, fp16 (IEEE binary16) logits. */
+int ears_verify_f16(const void* target_logits, const void* draft_logits,
+                    const int32_t* draft_tokens, int B, int K, int V,
+                    float temperature, float beta, uint64_t seed, uint64_t offset,
+                    int32_t* out_accept_len, int32_t* out_tokens, void* stream);
+
 /* Alias of ears_verify_f32 (the element type cannot be inferred from the arguments). */
 int ears_verify(const void* target_logits, const void* draft_logits,
                 const int32_t* draft_tokens, int B, int K, int V,

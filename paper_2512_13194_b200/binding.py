@@ -36,7 +36,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     c = ctypes
     common = [c.c_void_p, c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_int, c.c_float, c.c_float,
               c.c_uint64, c.c_uint64]
-    for name in ("ears_verify_f32", "ears_verify_bf16", "ears_verify"):
+    for name in ("ears_verify_f32", "ears_verify_bf16", "ears_verify_f16", "ears_verify"):
         fn = getattr(lib, name)
         fn.argtypes = common + [c.c_void_p, c.c_void_p, c.c_void_p]
         fn.restype = c.c_int
@@ -219,7 +219,7 @@ def verify_greedy(target_logits: torch.Tensor, draft_tokens: torch.Tensor, *, wo
 
 def verify_abi(name: str, target_logits, draft_logits, draft_tokens, temperature, beta, seed, offset,
                stream=None):
-    """Calls one of the 13-argument entry points (ears_verify, ears_verify_f32, ears_verify_bf16) as is."""
+    """Calls one of the 13-argument entry points (ears_verify, ears_verify_f32, ears_verify_bf16, ears_verify_f16) as is."""
     lib = load_library()
     B, K, V = _shapes(target_logits, draft_logits, draft_tokens)
     dev = target_logits.device

@@ -877,6 +877,14 @@ int ears_verify_bf16(const void* target_logits, const void* draft_logits, const 
                        nullptr, 0, stream);
 }
 
+int ears_verify_f16(const void* target_logits, const void* draft_logits, const int32_t* draft_tokens,
+                    int B, int K, int V, float temperature, float beta, uint64_t seed, uint64_t offset,
+                    int32_t* out_accept_len, int32_t* out_tokens, void* stream) {
+    return verify_impl(EARS_DTYPE_F16, target_logits, draft_logits, draft_tokens, B, K, V, temperature, beta,
+                       nullptr, nullptr, 0u, seed, offset, 0, out_accept_len, out_tokens, nullptr, nullptr, nullptr, nullptr, nullptr,
+                       nullptr, 0, stream);
+}
+
 int ears_verify(const void* target_logits, const void* draft_logits, const int32_t* draft_tokens,
                 int B, int K, int V, float temperature, float beta, uint64_t seed, uint64_t offset,
                 int32_t* out_accept_len, int32_t* out_tokens, void* stream) {

@@ -143,15 +143,19 @@ __device__ void greedy_finish(const GParams& p, int b, int lane, int* row_top /*
 template <typename E>
 __global__ void __launch_bounds__(kGThreads, kGCtasPerSm) ears_greedy_kernel(const GParams p) {
     constexpr int N = GVec<E>::N;
-    __shared__ float s_v[kGThreads / 32];
-    __shared__ int s_i[kGThreads / 32];
-    __shared__ int s_bad[kGThreads / 32];
+    // two copies, used alternately: one barrier per unit suffices, because a copy is rewritten only
+    // after warp 0, which reads it, has arrived at the next unit's barrier
+    __shared__ float s_v[2][kGThreads / 32];
+    __shared__ int s_i[2][kGThreads / 32];
+    __shared__ int s_bad[2][kGThreads / 32];
     __shared__ int s_top[kMaxK + 1];
     clear_next_counters(p);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int K = p.K, V = p.V, P = p.P;
     const E* base = reinterpret_cast<const E*>(p.t);
-    for (long long u = blockIdx.x; u < p.units; u += gridDim.x) {
+    int it = 0;
+    for (long long u = blockIdx.x; u < p.units; u += gridDim.x, ++it) {
+        const int h = it & 1;
         const long long row = u / P;
         const int piece = (int)(u % P);
         const int b = (int)(row / (K + 1));
@@ -180,11 +184,11 @@ __global__ void __launch_bounds__(kGThreads, kGCtasPerSm) ears_greedy_kernel(con
             const int ob = __shfl_xor_sync(0xffffffffu, a.bad, off);
             top_merge(a, ov, oi, ob);
         }
-        if (lane == 0) { s_v[warp] = a.v; s_i[warp] = a.i; s_bad[warp] = a.bad; }
+        if (lane == 0) { s_v[h][warp] = a.v; s_i[h][warp] = a.i; s_bad[h][warp] = a.bad; }
         __syncthreads();
         if (warp == 0) {
             Top c{-INFINITY, INT_MAX, 0};
-            if (lane < kGThreads / 32) c = Top{s_v[lane], s_i[lane], s_bad[lane]};
+            if (lane < kGThreads / 32) c = Top{s_v[h][lane], s_i[h][lane], s_bad[h][lane]};
 #pragma unroll
             for (int off = kGThreads / 64; off > 0; off >>= 1) {
                 const float ov = __shfl_xor_sync(0xffffffffu, c.v, off);
@@ -203,7 +207,6 @@ __global__ void __launch_bounds__(kGThreads, kGCtasPerSm) ears_greedy_kernel(con
                 greedy_finish(p, b, lane, s_top);
             }
         }
-        __syncthreads();
     }
 }
 

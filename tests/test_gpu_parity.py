@@ -264,7 +264,8 @@ def test_batch_shards_match_full_batch(ears):
 def test_entry_points_agree(ears):
     """13-argument symbols, caller-owned workspace, a side stream and the host-buffer entry."""
     dev = "cuda:0"
-    for dtype, name in (("fp32", "ears_verify_f32"), ("bf16", "ears_verify_bf16"), ("fp32", "ears_verify")):
+    for dtype, name in (("fp32", "ears_verify_f32"), ("bf16", "ears_verify_bf16"), ("fp16", "ears_verify_f16"),
+                        ("fp32", "ears_verify")):
         w, t, d, x = synth.tiny_inputs(5, 3, 12000, dtype, seed=33)
         tg, dg, xg = t.to(dev), d.to(dev), x.to(dev)
         ref_len, ref_tok = ears.verify(tg, dg, xg, 1.1, 0.2, 9, 4)
