@@ -83,7 +83,7 @@ class ClockSampler(threading.Thread):
         self._halt.set()
         self.join(timeout=2)
         out = {"sm_mhz": statistics.median(self.samples) if self.samples else None,
-               "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+               "sm_min_mhz": min(self.samples) if self.samples else None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
         if self.error:
             out["error"] = self.error
         return out
@@ -440,7 +440,10 @@ def run_greedy_table(args):
     flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
     print(f"| workload | B | dtype | target-row bytes | us per step | GB/s | of {peak:.0f} ({peak_kind}) |")
     print("|---|---|---|---|---|---|---|")
-    for idx, B in ((1, 0), (2, 0), (3, 0), (4, 0), (5, 0), (4, 1024), (2, 4096)):
+    cases = ((1, 0), (2, 0), (3, 0), (4, 0), (5, 0), (4, 1024), (2, 4096))
+    if args.batch:   # one case (small ones for profiler captures)
+        cases = ((args.workload, args.batch),)
+    for idx, B in cases:
         w = synth.workload(idx)
         if B:
             w = replace(w, B=B)
