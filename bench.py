@@ -31,10 +31,14 @@ METRIC = "verify rows/s"
 UNIT = "rows/s"
 DATASHEET_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of ears_verify_kernel<float,6> from one ncu capture on
-# a 96-sequence batch of the default workload (691.07 MB + 4.24 MB), per sequence.  The traffic grows
-# in proportion to the number of sequences; set to None whenever the kernel changes after a capture.
-NCU_DRAM_BYTES_PER_SEQUENCE = (690650624 + 4477440) / 96
+# dram__bytes_read.sum + dram__bytes_write.sum per sequence from one ncu capture of the named kernel on a
+# small batch of the default workload (see profiles/); the traffic grows in proportion to the number
+# of sequences.  Reported only while the kernel the plan names is the captured one; an entry is taken
+# out (None) whenever its kernel changes after the capture.
+NCU_DRAM_BYTES_PER_SEQUENCE = {
+    # kernel name: (bytes per sequence, what was captured)
+    "ears_verify_kernel": None,
+}
 
 
 def measured_peak():
@@ -59,6 +63,7 @@ class ClockSampler(threading.Thread):
         super().__init__(daemon=True)
         self.index, self.period = index, period_s
         self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.trace = []          # (host time, SM MHz, reason names, watts) per sample
         self._halt = threading.Event()
         self.error = None
 
@@ -69,12 +74,18 @@ class ClockSampler(threading.Thread):
             h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
             self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM)
             while not self._halt.is_set():
-                self.samples.append(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM))
+                now = time.perf_counter()
+                mhz = pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)
+                self.samples.append(mhz)
                 mask = pynvml.nvmlDeviceGetCurrentClocksEventReasons(h) if hasattr(
                     pynvml, "nvmlDeviceGetCurrentClocksEventReasons") else pynvml.nvmlDeviceGetCurrentClocksThrottleReasons(h)
-                for bit, name in self.REASONS.items():
-                    if mask & bit:
-                        self.reasons.add(name)
+                names = tuple(name for bit, name in self.REASONS.items() if mask & bit)
+                self.reasons.update(names)
+                try:
+                    watts = pynvml.nvmlDeviceGetPowerUsage(h) / 1000.0
+                except Exception:
+                    watts = None
+                self.trace.append((now, mhz, names, watts))
                 time.sleep(self.period)
         except Exception as e:  # NVML missing: report it rather than guess
             self.error = repr(e)
@@ -97,6 +108,95 @@ def physical_gpu_index(local_index: int) -> int:
         except Exception:
             return local_index
     return local_index
+
+
+def back_to_back(step, ears, gpu_index: int, n: int):
+    """n steps back to back with the library's per-launch events and NVML samples beside them.
+    -> (kernel_ms per launch, estimated host time of each launch, clock trace, clocks summary)."""
+    import torch
+    sampler = ClockSampler(gpu_index, period_s=0.004)
+    sampler.start()
+    time.sleep(0.03)
+    ears.profile_begin(n)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for i in range(n):
+        step(5000 + i)
+    torch.cuda.synchronize()
+    t1 = time.perf_counter()
+    kernel_ms = ears.profile_end(n)
+    clocks = sampler.stop()
+    # launches fill [t0, t1] in order; place each by its share of the summed kernel time
+    total = sum(kernel_ms) or 1.0
+    at, run = [], 0.0
+    for k in kernel_ms:
+        at.append(t0 + (t1 - t0) * (run + 0.5 * k) / total)
+        run += k
+    return kernel_ms, at, sampler.trace, clocks
+
+
+def clock_at(trace, when):
+    """The NVML sample nearest in time to `when` -> (MHz, reasons, watts) or None."""
+    if not trace:
+        return None
+    import bisect
+    times = [s[0] for s in trace]
+    i = bisect.bisect_left(times, when)
+    cand = [j for j in (i - 1, i) if 0 <= j < len(trace)]
+    j = min(cand, key=lambda j: abs(times[j] - when))
+    return trace[j][1:]
+
+
+def bins_by_clock(kernel_ms, at, trace, logits_bytes, peak, width_mhz=50):
+    """Kernel time binned by the SM clock sampled beside each launch."""
+    groups = {}
+    for k, when in zip(kernel_ms, at):
+        c = clock_at(trace, when)
+        if c is None:
+            continue
+        lo = int(c[0] // width_mhz) * width_mhz
+        g = groups.setdefault(lo, {"ms": [], "mhz": [], "reasons": set(), "watts": []})
+        g["ms"].append(k)
+        g["mhz"].append(c[0])
+        g["reasons"].update(c[1])
+        if c[2] is not None:
+            g["watts"].append(c[2])
+    out = []
+    for lo in sorted(groups, reverse=True):
+        g = groups[lo]
+        med = statistics.median(g["ms"])
+        q = sorted(g["ms"])
+        out.append({"sm_mhz_bin": [lo, lo + width_mhz], "launches": len(q), "kernel_us_median": med * 1e3,
+                    "kernel_us_p10_p90": [q[len(q) // 10] * 1e3, q[(9 * len(q)) // 10 - (1 if len(q) >= 10 else 0)] * 1e3],
+                    "gbs": logits_bytes / (med * 1e-3) / 1e9, "frac": logits_bytes / (med * 1e-3) / 1e9 / peak,
+                    "us_x_mhz": med * 1e3 * statistics.median(g["mhz"]), "reasons": sorted(g["reasons"]),
+                    "watts_median": statistics.median(g["watts"]) if g["watts"] else None})
+    return out
+
+
+def sustained(step, ears, gpu_index: int, ms_step: float, logits_bytes: int, peak: float, seconds: float = 0.6):
+    """The kernel under continuous load: >= `seconds` of back-to-back steps appended after the timed
+    region; the figure is the mean over the last half, with the clocks sampled during that half."""
+    n = int(min(60000, max(100, seconds * 1e3 / max(ms_step, 1e-3))))
+    kernel_ms, at, trace, _ = back_to_back(step, ears, gpu_index, n)
+    half = kernel_ms[len(kernel_ms) // 2:]
+    t_half = at[len(at) // 2]
+    late = [s for s in trace if s[0] >= t_half]
+    k = statistics.fmean(half)
+    gbs = logits_bytes / (k * 1e-3) / 1e9
+    return {"kernel_ms": k, "achieved": gbs, "frac": gbs / peak, "launches": n,
+            "seconds": sum(kernel_ms) * 1e-3, "over": "last half of the launches",
+            "clocks": {"sm_mhz": statistics.median(s[1] for s in late) if late else None,
+                       "sm_min_mhz": min((s[1] for s in late), default=None),
+                       "reasons": sorted({r for s in late for r in s[2]}), "samples": len(late)}}
+
+
+def config_of(w, world: int) -> dict:
+    """The workload as both arms of the benchmark report it."""
+    return {"workload": w.name, "B_per_gpu": w.B, "K": w.K, "V": w.V, "logits_dtype": w.dtype,
+            "temperature": w.temperature, "beta": w.beta, "parallelism": f"batch-shard x{world}",
+            "l2": "inputs exceed L2 several times over; no flush needed" if w.logit_bytes > 512e6
+                  else "inputs fit L2: warm-cache number"}
 
 
 def final_token_bytes(accept_len, K: int, V: int, esize: int):
@@ -191,6 +291,12 @@ def run_ours(args):
     # algorithmic HBM bytes of the kernel: every logit once.  The rows of the final token are a second
     # pass over bytes already counted (normally served by L2), so they are left out of the roofline.
     achieved = logits_bytes / (k_avg * 1e-3) / 1e9
+    # the same kernel under continuous load (the timed region above may be too short for the power
+    # management of the device to settle)
+    sus = None
+    if rank == 0 and world == 1 and not args.no_sustained:
+        sus = sustained(step, ears, physical_gpu_index(local), ms_step, logits_bytes, peak)
+    captured = NCU_DRAM_BYTES_PER_SEQUENCE.get(kernel_name) if args.workload == 5 else None
 
     # end to end through the host-buffer entry point: H2D of the inputs and D2H of the results every step
     th, dh, xh = (a.cpu().pin_memory() for a in (t, d, x))
@@ -225,11 +331,8 @@ def run_ours(args):
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
-            "config": {"workload": w.name, "B_per_gpu": w.B, "K": K, "V": V, "logits_dtype": w.dtype,
-                       "temperature": w.temperature, "beta": w.beta, "parallelism": f"batch-shard x{world}",
-                       "l2": "inputs (3.67 GB at the default workload) exceed L2; no flush needed"
-                             if logits_bytes > 512e6 else "inputs fit L2: warm-cache number",
-                       "mean_accept_len": float(acc.float().mean().item()), "launch_plan": plan},
+            "config": config_of(w, world),
+            "mean_accept_len": float(acc.float().mean().item()), "launch_plan": plan,
             "gbs_step_formula": step_bytes / (ms_step * 1e-3) / 1e9,
             "bytes_per_step": {"logits": logits_bytes, "final_token_rows_formula": rs_formula,
                                "final_token_rows_streamed_again": rs_again},
@@ -237,9 +340,10 @@ def run_ours(args):
             "roofline": {"bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                          "frac_of_datasheet_8000": achieved / DATASHEET_HBM_GBS,
-                         "traffic": (NCU_DRAM_BYTES_PER_SEQUENCE * w.B
-                                     if NCU_DRAM_BYTES_PER_SEQUENCE and args.workload == 5 else None),
-                         "traffic_note": "ncu DRAM read+write bytes of a 96-sequence capture scaled by sequences"},
+                         "traffic": captured[0] * w.B if captured else None,
+                         "traffic_note": (captured[1] if captured else
+                                          "no ncu capture of this kernel since it last changed"),
+                         "sustained": sus},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps},
             "gpu_launches": args.steps,
@@ -301,8 +405,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": warm, "ms_per_step": dt * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "B_per_step": n, "K": w.K, "V": w.V, "logits_dtype": w.dtype,
-                   "temperature": w.temperature, "beta": w.beta},
+        "config": config_of(w, args.gpus),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -319,8 +422,7 @@ def run_table(args):
     import oracle
     import paper_2512_13194_b200 as ears
     from paper_2512_13194_b200 import synth
-    sys.path.insert(0, os.path.join(ROOT, "tests"))
-    from parity import Tally, compare
+    from oracle.parity import compare
 
     torch.cuda.set_device(0)
     ears.load_library()
@@ -366,13 +468,71 @@ def run_table(args):
                     o_1 = f"{time.perf_counter() - t0:.3f}"
                 else:
                     o_1 = f"~{o_n * cores:.1f} (threads x wall)"
-                tl = compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, w.K, {k: v.cpu().numpy() for k, v in st.items()})
+                tl = compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, w.K, {k: v.cpu().numpy() for k, v in st.items()},
+                             inputs=(th, dh, T))
                 gbs = w.logit_bytes / (cold * 1e-6) / 1e9
                 print(f"| {idx} | {w.B} | {w.K} | {w.V} | {w.dtype} | {T} | {beta} | {float(ora.accept_len.mean()):.2f} | "
                       f"{cold:.1f} / {warm:.1f} | {w.rows / (cold * 1e-6):.3g} | {gbs:.0f} | {100 * gbs / peak:.1f} | "
                       f"{100 * gbs / DATASHEET_HBM_GBS:.1f} | {o_1} | {o_n:.3f} | {tl.explained + len(tl.unexplained)} / {tl.rows} "
                       f"({tl.explained} / {len(tl.unexplained)}) | {tl.max_rel_prob_err:.1e} |", flush=True)
             del t, d, x
+
+
+def run_series(args):
+    """The kernel under continuous load: --series N steps back to back on one GPU (N >= 1000 for the
+    default workload keeps the device busy for more than half a second), the library's events around
+    every launch, NVML sampled beside them.  Prints kernel time by position in the series and by
+    sampled SM clock, and one JSON line with the bins.  Not the benchmark line."""
+    import torch
+
+    import paper_2512_13194_b200 as ears
+    from paper_2512_13194_b200 import synth
+
+    torch.cuda.set_device(0)
+    ears.load_library()
+    w = synth.workload(args.workload)
+    if args.batch:
+        w = w.with_batch(args.batch)
+    t, d, x = synth.make_inputs(w, "cuda:0")
+    peak, peak_kind = measured_peak()
+    step = lambda i: ears.verify(t, d, x, w.temperature, w.beta, w.verify_seed, i)
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    torch.cuda.synchronize()
+    time.sleep(0.5)      # let the device idle first: the series then shows the change of state from its start
+    n = min(args.series, 60000)
+    kernel_ms, at, trace, clocks = back_to_back(step, ears, physical_gpu_index(0), n)
+    plan = ears.describe_plan(w.dtype, w.B, w.K, w.V)
+    print(f"# {w.name}: {n} launches back to back, {sum(kernel_ms) * 1e-3:.2f} s of kernel time; plan: {plan}")
+    print(f"# peak for the fractions: {peak:.1f} GB/s ({peak_kind})")
+    print("| launches | kernel us (median) | GB/s | of peak | SM MHz beside (median) | reasons | W |")
+    print("|---|---|---|---|---|---|---|")
+    edges = sorted({0, 20, 50, 100, 200, 400, 800, 1600, 3200, 6400, 12800, 25600, n} & set(range(n + 1)) | {n})
+    for a, b in zip(edges[:-1], edges[1:]):
+        seg = kernel_ms[a:b]
+        if not seg:
+            continue
+        med = statistics.median(seg)
+        cs = [c for c in (clock_at(trace, when) for when in at[a:b]) if c]
+        mhz = statistics.median(c[0] for c in cs) if cs else float("nan")
+        reasons = sorted({r for c in cs for r in c[1]})
+        watts = [c[2] for c in cs if c[2] is not None]
+        gbs = w.logit_bytes / (med * 1e-3) / 1e9
+        print(f"| {a + 1}-{b} | {med * 1e3:.1f} | {gbs:.0f} | {gbs / peak:.3f} | {mhz:.0f} | {','.join(reasons) or '-'} | "
+              f"{statistics.median(watts) if watts else float('nan'):.0f} |")
+    bins = bins_by_clock(kernel_ms, at, trace, w.logit_bytes, peak)
+    print()
+    print("| SM MHz bin | launches | kernel us median (p10-p90) | GB/s | of peak | us x MHz | reasons | W |")
+    print("|---|---|---|---|---|---|---|---|")
+    for b in bins:
+        print(f"| {b['sm_mhz_bin'][0]}-{b['sm_mhz_bin'][1]} | {b['launches']} | {b['kernel_us_median']:.1f} "
+              f"({b['kernel_us_p10_p90'][0]:.1f}-{b['kernel_us_p10_p90'][1]:.1f}) | {b['gbs']:.0f} | {b['frac']:.3f} | "
+              f"{b['us_x_mhz']:.3g} | {','.join(b['reasons']) or '-'} | {b['watts_median'] or float('nan'):.0f} |")
+    half = kernel_ms[n // 2:]
+    k = statistics.fmean(half)
+    print(json.dumps({"series": n, "workload": w.name, "plan": plan, "kernel_ms_first_20": statistics.fmean(kernel_ms[:20]),
+                      "kernel_ms_last_half": k, "frac_last_half": w.logit_bytes / (k * 1e-3) / 1e9 / peak,
+                      "peak": peak, "peak_kind": peak_kind, "clocks": clocks, "bins": bins}), flush=True)
 
 
 def run_shard_table(args):
@@ -474,6 +634,10 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-sample", type=int, default=512, help="sequences given to the CPU baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the appended run under continuous load")
+    ap.add_argument("--series", type=int, default=0,
+                    help="instead of the benchmark line: this many steps back to back, kernel time per launch "
+                         "binned by the SM clock sampled beside it")
     ap.add_argument("--table", action="store_true", help="print the five-workload results table instead")
     ap.add_argument("--table-full", action="store_true", help="also time the 1-thread oracle on workload 5")
     ap.add_argument("--ranks", type=int, default=2, help="with --shard-table --batch: ranks the vocabulary is split over")
@@ -481,7 +645,9 @@ def main():
                     help="print per-phase times of one rank of the vocabulary-sharded step instead")
     ap.add_argument("--greedy-table", action="store_true", help="print times of the temperature -> 0 form instead")
     args = ap.parse_args()
-    if args.greedy_table:
+    if args.series:
+        run_series(args)
+    elif args.greedy_table:
         run_greedy_table(args)
     elif args.shard_table:
         run_shard_table(args)

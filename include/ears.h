@@ -159,6 +159,7 @@ int ears_verify_ex(int dtype, const void* target_logits, const void* draft_logit
  * Everything else is as in ears_verify_ex.
  */
 #define EARS_FLAG_STOP_AT_FIRST_REJECT 1u
+#define EARS_FLAGS_ALL (EARS_FLAG_STOP_AT_FIRST_REJECT)
 int ears_verify_var(int dtype, const void* target_logits, const void* draft_logits,
                     const int32_t* draft_tokens, int B, int K, int V,
                     float temperature, float beta,
@@ -277,6 +278,11 @@ int ears_verify_host(int dtype, const void* target_logits, const void* draft_log
  *   - The first call on each device looks up the array's device address (and sets the
  *     kernels' shared-memory attribute); make that first call outside any stream
  *     capture.  The device must be current, as for every other entry point.
+ *   - "Allocates nothing" holds once the code a call needs is resident: the CUDA driver loads
+ *     a kernel when it is first launched (one kernel per element type and per launch plan:
+ *     rows that stay in shared memory, long rows, 2- or 4-byte logits), and loading
+ *     allocates.  Make one warm-up call per element type and kind of shape you will use,
+ *     outside any capture, before the phase in which allocation is forbidden.
  *   - All calls on a device share the one array.  It keeps the previous call's
  *     contents; the counters that must start at zero are cleared at the start of every
  *     call, on the call's stream.  Calls that can overlap on the GPU (different streams

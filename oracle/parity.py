@@ -1,9 +1,11 @@
-"""Comparison of the CUDA path's outputs with the oracle's, with the near-tie rules.
+"""Comparison of the CUDA path's outputs with the oracle's, with the near-tie rules
+(TEST INFRASTRUCTURE: the checker's side, like everything under oracle/).
 
 accept lengths and tokens must be bit-exact except
   - a decision whose oracle margin |R - max(U - Tol, 0)| is below 1e-5, or
   - a final token that lies in the oracle's band of tokens whose CDF interval comes
-    within 1e-6 (in probability) of the uniform;
+    within 1e-6 (in probability) of the uniform AND carries mass in the oracle's own row
+    (a token of zero mass is never a legitimate draw, wherever it sits in the band);
 such explained disagreements are counted (one per sequence at most), anything else is
 unexplained and fails.  Probabilities must agree to 1e-5 relative (or 1e-30 absolute:
 fp32 cannot hold what fp64 underflows to).
@@ -13,6 +15,8 @@ from __future__ import annotations
 from dataclasses import dataclass, field
 
 import numpy as np
+
+from . import ears_oracle as _oracle
 
 DECISION_BAND = 1e-5
 CDF_BAND = 1e-6
@@ -47,8 +51,31 @@ class Tally:
         return self
 
 
-def compare(gpu_len, gpu_tok, ora, K: int, stats=None) -> Tally:
-    """gpu_len [B], gpu_tok [B,K+1] numpy int32; ora an oracle.OracleResult; stats the GPU's dict."""
+def final_token_mass(inputs, b: int, n: int, K: int, token: int) -> float:
+    """Mass the oracle's row gives `token` as the final token of sequence b after n acceptances:
+    max(0, P_t - P_d) of position n after a rejection (P_t if that residual is empty, as in the
+    oracle), P_t of the extra row when n = K.  inputs = (target_logits, draft_logits, temperature),
+    temperature a scalar or a [B] array."""
+    t, d, temperature = inputs
+    V = t.shape[-1]
+    if not 0 <= token < V:
+        return 0.0
+    T = float(np.asarray(temperature).reshape(-1)[b]) if np.ndim(temperature) else float(temperature)
+    pt = _oracle.row_softmax(t, b * (K + 1) + n, V, T)
+    if n >= K:
+        return float(pt[token])
+    pd = _oracle.row_softmax(d, b * K + n, V, T)
+    r = np.maximum(pt - pd, 0.0)
+    if r.sum() < 1e-300:
+        return float(pt[token])
+    return float(r[token])
+
+
+def compare(gpu_len, gpu_tok, ora, K: int, stats=None, inputs=None) -> Tally:
+    """gpu_len [B], gpu_tok [B,K+1] numpy int32; ora an oracle.OracleResult; stats the GPU's dict;
+    inputs = (target_logits, draft_logits, temperature) as given to the oracle (CPU).  A token
+    disagreement counts as explained only if the other token lies in the oracle's band and has
+    positive mass in the oracle's row, which needs `inputs`; without them it stays unexplained."""
     gpu_len = np.asarray(gpu_len)
     gpu_tok = np.asarray(gpu_tok)
     B = gpu_len.shape[0]
@@ -75,10 +102,12 @@ def compare(gpu_len, gpu_tok, ora, K: int, stats=None) -> Tally:
             continue
         g, o = int(gpu_tok[b, n]), int(ora.tokens[b, n])
         if g != o:
-            if ora.band_lo[b] <= g <= ora.band_hi[b]:
+            in_band = ora.band_lo[b] <= g <= ora.band_hi[b]
+            if in_band and inputs is not None and final_token_mass(inputs, b, n, K, g) > 0.0:
                 t.explained_tokens += 1
             else:
-                t.unexplained.append((b, "token", g, o, int(ora.band_lo[b]), int(ora.band_hi[b]),
+                why = "token" if not in_band else ("token-unchecked" if inputs is None else "token-zero-mass")
+                t.unexplained.append((b, why, g, o, int(ora.band_lo[b]), int(ora.band_hi[b]),
                                       float(ora.cdf_margin[b])))
     if stats is not None:
         for key in ("pt_tok", "pd_tok", "max_pt"):

@@ -93,11 +93,14 @@ struct Buffer {
 };
 std::map<std::pair<int, void*>, Buffer> g_workspaces;  // (device, stream) -> scratch
 std::map<std::pair<int, void*>, Buffer> g_staging;     // (device, stream) -> host-entry staging
+// Workspaces that a CUDA graph may still point at: kept until ears_shutdown (device, pointer).
+std::vector<std::pair<int, void*>> g_parked;
 
 struct Profile {
     bool active = false;
     int max_calls = 0;
-    std::vector<cudaEvent_t> events;  // 2 per timed call
+    size_t used = 0;                  // events recorded so far
+    std::vector<cudaEvent_t> events;  // 2 per timed call, created by ears_profile_begin
 } g_profile;
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -298,12 +301,12 @@ int device_info(int dev, DeviceInfo** out) {
 
 size_t smem_bytes() { return sizeof(PipeSmem<kStages>) + 128; }
 
+// The events exist already (ears_profile_begin): a timed call only records them.
+bool profile_wanted() { return g_profile.active && g_profile.used + 2 <= g_profile.events.size(); }
+
 int profile_mark(cudaStream_t stream, bool timed) {
     if (!timed) return EARS_OK;
-    cudaEvent_t ev;
-    EARS_CUDA(cudaEventCreate(&ev));
-    g_profile.events.push_back(ev);
-    EARS_CUDA(cudaEventRecord(ev, stream));
+    EARS_CUDA(cudaEventRecord(g_profile.events[g_profile.used++], stream));
     return EARS_OK;
 }
 
@@ -369,7 +372,7 @@ int launch_resident(RParams& p, const RPlan& rp, int max_clusters, cudaStream_t 
     attr[0].val.clusterDim.x = (unsigned)rp.C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const bool timed = g_profile.active && (int)g_profile.events.size() + 2 <= 2 * g_profile.max_calls;
+    const bool timed = profile_wanted();
     int rc = profile_mark(stream, timed);
     if (rc) return rc;
     EARS_CUDA(cudaLaunchKernelEx(&cfg, ears_resident_kernel<E>, p));
@@ -381,7 +384,7 @@ int launch(const Params& p, int sms, bool direct, cudaStream_t stream) {
     const long long units = (long long)p.B * (2 * p.K + 1) * p.plan.parts1;
     const long long cap = (long long)sms * kCtasPerSm;
     const int grid = (int)(units < cap ? units : cap);
-    const bool timed = g_profile.active && (int)g_profile.events.size() + 2 <= 2 * g_profile.max_calls;
+    const bool timed = profile_wanted();
     int rc = profile_mark(stream, timed);
     if (rc) return rc;
     if (direct) {
@@ -402,7 +405,15 @@ int get_buffer(std::map<std::pair<int, void*>, Buffer>& pool, int dev, void* str
     std::lock_guard<std::mutex> lock(g_mutex);
     Buffer& b = pool[std::make_pair(dev, stream)];
     if (b.bytes < bytes) {
-        if (b.ptr) {
+        if (b.ptr && b.captured) {
+            // A call on this buffer was recorded into a CUDA graph whose replays will use these very
+            // addresses: the buffer is never freed before ears_shutdown.  Later eager calls move to
+            // a new one (replays and eager calls stay ordered by the stream they share).
+            g_parked.emplace_back(dev, b.ptr);
+            b.ptr = nullptr;
+            b.bytes = 0;
+            b.captured = false;
+        } else if (b.ptr) {
             // work enqueued earlier on this stream may still use the old buffer
             EARS_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
             EARS_CUDA(cudaFree(b.ptr));
@@ -498,6 +509,8 @@ int choose_resident(int dtype, int B, int K, int V, DeviceInfo* di, const PlanOv
 }
 
 int ensure_attrs(DeviceInfo* di) {
+    static std::mutex attrs_mutex;   // two threads making their first call on a device set the attributes once
+    std::lock_guard<std::mutex> lock(attrs_mutex);
     if (di->attrs_set) return EARS_OK;
     bool c16 = true;
     int rc = set_attrs<float>(&c16);
@@ -511,26 +524,36 @@ int ensure_attrs(DeviceInfo* di) {
     return EARS_OK;
 }
 
+// Everything about a call's arguments that the host can judge without a device.
+int check_arguments(int dtype, const void* t, const void* d, const int32_t* x, int B, int K, int V,
+                    float temperature, float beta, const float* seq_T, const float* seq_beta, unsigned flags,
+                    int64_t b_first, const int32_t* out_len, const int32_t* out_tok) {
+    if (!t || !d || !x || !out_len || !out_tok) return EARS_ERR_NULL;
+    if (!dtype_ok(dtype)) return EARS_ERR_PARAM;
+    if (flags & ~(unsigned)EARS_FLAGS_ALL) return EARS_ERR_PARAM;
+    const int rc = check_shape(B, K, V);
+    if (rc) return rc;
+    // a per-sequence array replaces its scalar, which is then not looked at
+    if (!seq_T && (!(temperature > 0.0f) || !std::isfinite(temperature))) return EARS_ERR_PARAM;
+    if (!seq_beta && (!(beta >= 0.0f) || !std::isfinite(beta))) return EARS_ERR_PARAM;
+    if (((uintptr_t)seq_T % 4) || ((uintptr_t)seq_beta % 4)) return EARS_ERR_ALIGN;
+    if (b_first < 0 || (unsigned long long)b_first + (unsigned long long)B > 0xffffffffull) return EARS_ERR_PARAM;
+    const int esize = dtype_size(dtype);
+    if (((uintptr_t)t % esize) || ((uintptr_t)d % esize) || ((uintptr_t)x % 4)) return EARS_ERR_ALIGN;
+    return EARS_OK;
+}
+
 int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B, int K, int V,
                 float temperature, float beta, const float* seq_T, const float* seq_beta, unsigned flags,
                 uint64_t seed, uint64_t offset, int64_t b_first,
                 int32_t* out_len, int32_t* out_tok, double* o_pt, double* o_pd, double* o_max,
                 uint8_t* o_cls, double* o_resid, void* workspace, size_t workspace_bytes, void* stream_) {
-    if (!t || !d || !x || !out_len || !out_tok) return EARS_ERR_NULL;
-    if (!dtype_ok(dtype)) return EARS_ERR_PARAM;
-    if (flags & ~(unsigned)EARS_FLAG_STOP_AT_FIRST_REJECT) return EARS_ERR_PARAM;
-    const int stop_first = (flags & EARS_FLAG_STOP_AT_FIRST_REJECT) ? 1 : 0;
-    int rc = check_shape(B, K, V);
+    int rc = check_arguments(dtype, t, d, x, B, K, V, temperature, beta, seq_T, seq_beta, flags, b_first, out_len, out_tok);
     if (rc) return rc;
-    // a per-sequence array replaces its scalar, which is then not looked at
+    const int stop_first = (flags & EARS_FLAG_STOP_AT_FIRST_REJECT) ? 1 : 0;
     if (seq_T) temperature = 1.0f;
     if (seq_beta) beta = 0.0f;
-    if (!(temperature > 0.0f) || !std::isfinite(temperature)) return EARS_ERR_PARAM;
-    if (!(beta >= 0.0f) || !std::isfinite(beta)) return EARS_ERR_PARAM;
-    if (((uintptr_t)seq_T % 4) || ((uintptr_t)seq_beta % 4)) return EARS_ERR_ALIGN;
-    if (b_first < 0 || (unsigned long long)b_first + (unsigned long long)B > 0xffffffffull) return EARS_ERR_PARAM;
     const int esize = dtype_size(dtype);
-    if (((uintptr_t)t % esize) || ((uintptr_t)d % esize) || ((uintptr_t)x % 4)) return EARS_ERR_ALIGN;
     if (workspace && ((uintptr_t)workspace % 256)) return EARS_ERR_ALIGN;
     if (!workspace && workspace_bytes != 0) return EARS_ERR_WORKSPACE;
 
@@ -846,7 +869,7 @@ int ears_verify_greedy(int dtype, const void* target_logits, const int32_t* draf
     p.out_len = out_accept_len; p.out_tok = out_tokens;
     const long long cap = (long long)kGCtasPerSm * di->sms;
     const int grid = (int)(p.units < cap ? p.units : cap);
-    const bool timed = g_profile.active && (int)g_profile.events.size() + 2 <= 2 * g_profile.max_calls;
+    const bool timed = profile_wanted();
     rc = profile_mark(stream, timed);
     if (rc) return rc;
     by_dtype(dtype, [&](auto* e) {
@@ -930,8 +953,9 @@ int ears_verify_noalloc(int dtype, const void* target_logits, const void* draft_
                         const int32_t* draft_tokens, int B, int K, int V, float temperature, float beta,
                         uint64_t seed, uint64_t offset, int64_t b_first, int32_t* out_accept_len,
                         int32_t* out_tokens, int32_t* out_device_status, void* stream) {
-    if (!target_logits || !draft_logits || !draft_tokens || !out_accept_len || !out_tokens) return EARS_ERR_NULL;
-    int rc = check_shape(B, K, V);
+    // what the host can judge comes first: a bad argument is reported as such, device or no device
+    int rc = check_arguments(dtype, target_logits, draft_logits, draft_tokens, B, K, V, temperature, beta, nullptr, nullptr,
+                             0u, b_first, out_accept_len, out_tokens);
     if (rc) return rc;
     if (workspace_bound(B, K, V) > (size_t)EARS_NOALLOC_SCRATCH_BYTES) return EARS_ERR_WORKSPACE;
     int dev = 0;
@@ -1061,10 +1085,18 @@ int ears_set_path(int path, int cluster) {
 }
 
 int ears_profile_begin(int max_calls) {
-    if (max_calls < 1 || max_calls > (1 << 20)) return EARS_ERR_PARAM;
+    if (max_calls < 1 || max_calls > (1 << 16)) return EARS_ERR_PARAM;
     for (cudaEvent_t ev : g_profile.events) cudaEventDestroy(ev);
     g_profile.events.clear();
+    g_profile.used = 0;
+    g_profile.active = false;
+    // all events are created here, so that a timed call adds two cudaEventRecord and nothing else
     g_profile.events.reserve((size_t)2 * max_calls);
+    for (int i = 0; i < 2 * max_calls; ++i) {
+        cudaEvent_t ev;
+        EARS_CUDA(cudaEventCreate(&ev));
+        g_profile.events.push_back(ev);
+    }
     g_profile.max_calls = max_calls;
     g_profile.active = true;
     return EARS_OK;
@@ -1073,7 +1105,7 @@ int ears_profile_begin(int max_calls) {
 int ears_profile_end(float* kernel_ms, int capacity, int* n_calls) {
     if (!kernel_ms || !n_calls) return EARS_ERR_NULL;
     g_profile.active = false;
-    const int calls = (int)(g_profile.events.size() / 2);
+    const int calls = (int)(g_profile.used / 2);
     int rc = EARS_OK;
     if (calls > 0) {
         cudaError_t e = cudaEventSynchronize(g_profile.events[(size_t)2 * calls - 1]);
@@ -1086,6 +1118,7 @@ int ears_profile_end(float* kernel_ms, int capacity, int* n_calls) {
     }
     for (cudaEvent_t ev : g_profile.events) cudaEventDestroy(ev);
     g_profile.events.clear();
+    g_profile.used = 0;
     *n_calls = n;
     return rc;
 }
@@ -1219,6 +1252,12 @@ void ears_shutdown(void) {
         }
         pool->clear();
     }
+    for (auto& dp : g_parked) {
+        cudaSetDevice(dp.first);
+        cudaDeviceSynchronize();
+        cudaFree(dp.second);
+    }
+    g_parked.clear();
     cudaSetDevice(cur);
 }
 

@@ -128,7 +128,11 @@ constexpr int kSeqCap = 4;
 // warp 0 holds back while kUnitGuard ends are unread, hence the slots cannot be overrun.
 constexpr int kUnitSlots = 16;
 constexpr int kUnitGuard = 8;
-constexpr unsigned long long kIdleLimitNs = 30000000000ull;  // an idle warp may wait for the whole kernel
+// A warp that is idle by design (the epilogue and sequence warps between messages, a CTA that ran
+// out of units and stays to help) may wait for as long as the rest of the kernel runs.  The largest
+// input that fits this GPU's 180 GB of HBM streams in under 30 ms, so half a second is a limit no
+// healthy launch comes near, and a slip in the hand-over logic costs the GPU half a second, not half a minute.
+constexpr unsigned long long kIdleLimitNs = 500000000ull;
 
 template <int STAGES>
 struct PipeSmem {

@@ -18,12 +18,11 @@ import numpy as np
 import torch
 
 sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
-sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
 import oracle  # noqa: E402
 import paper_2512_13194_b200 as ears  # noqa: E402
 from paper_2512_13194_b200 import synth  # noqa: E402
 from paper_2512_13194_b200.shard import vocab_range  # noqa: E402
-from parity import Tally, compare  # noqa: E402
+from oracle.parity import Tally, compare  # noqa: E402
 
 
 def main():
@@ -49,7 +48,7 @@ def main():
         tok = torch.stack([o[1] for o in outs]).max(0).values
         assert all(torch.equal(o[0], acc) for o in outs), f"step {offset}: ranks disagree on accept lengths"
         ora = oracle.verify(th, dh, xh, w.temperature, beta, seed=w.verify_seed, offset=offset, nthreads=threads)
-        tally.merge(compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, w.K))
+        tally.merge(compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, w.K, inputs=(th, dh, w.temperature)))
         offset += 1
     while tally.rows < want_rows:
         acc, tok, st = ears.verify(t, d, x, w.temperature, beta, w.verify_seed, offset, stats=True)
@@ -58,7 +57,8 @@ def main():
         torch.cuda.synchronize()
         assert torch.equal(acc, acc2) and torch.equal(tok, tok2), f"step {offset}: outputs depend on stats"
         ora = oracle.verify(th, dh, xh, w.temperature, beta, seed=w.verify_seed, offset=offset, nthreads=threads)
-        tally.merge(compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, w.K, {k: v.cpu().numpy() for k, v in st.items()}))
+        tally.merge(compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, w.K, {k: v.cpu().numpy() for k, v in st.items()},
+                            inputs=(th, dh, w.temperature)))
         offset += 1
     how = f"{shards} vocabulary shards" if shards else ears.describe_plan(w.dtype, w.B, w.K, w.V).split(':')[0] + " kernel"
     print(f"{w.name} {w.dtype} beta={beta} [{how}]: steps={offset} rows={tally.rows} sequences={tally.sequences} "

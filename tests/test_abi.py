@@ -62,6 +62,19 @@ def test_bad_arguments_are_rejected_on_the_host():
     assert lib.ears_verify_ex(0, p, p, p, 1, 1, 4, 1.0, 0.1, 0, 0, 0, p, p, None, None, None, None, None,
                               p + 4, 1 << 20, None) == -4
     assert lib.ears_verify_host(0, None, p, p, 1, 1, 4, 1.0, 0.1, 0, 0, 0, p, p, None) == -1
+    # the allocation-free entry point judges its arguments before it looks for a device
+    lib.ears_verify_noalloc.argtypes = ([ctypes.c_int] + [ctypes.c_void_p] * 3 + [ctypes.c_int] * 3 + [ctypes.c_float] * 2
+                                        + [ctypes.c_uint64] * 2 + [ctypes.c_int64] + [ctypes.c_void_p] * 4)
+
+    def noalloc(dtype=0, t=p, B=1, K=1, V=4, T=1.0, beta=0.1, b_first=0):
+        return lib.ears_verify_noalloc(dtype, t, p, p, B, K, V, T, beta, 0, 0, b_first, p, p, None, None)
+
+    assert noalloc(t=None) == -1
+    assert noalloc(dtype=9) == -3 and noalloc(T=0.0) == -3 and noalloc(T=float("nan")) == -3 and noalloc(beta=-1.0) == -3
+    assert noalloc(b_first=-1) == -3
+    assert noalloc(B=0) == -2 and noalloc(K=65) == -2
+    assert noalloc(t=p + 2) == -4
+    assert noalloc(B=40000, K=8, V=16) == -5          # beyond the fixed scratch array
     assert lib.ears_set_plan(3, 0) == -3 and lib.ears_set_plan(0, 0) == 0
     assert lib.ears_philox_device(None, None, -1, None) == -2
     assert lib.ears_philox_device(None, None, 0, None) == 0

@@ -58,21 +58,31 @@ def test_greedy_parity_workloads(ears, idx):
     assert np.array_equal(acc.cpu().numpy(), o_acc) and np.array_equal(tok.cpu().numpy(), o_tok)
 
 
-def test_greedy_invalid_sequences_workspace_and_repeats(ears):
-    t, x = make(8, 3, 5000, "fp32", seed=5)
-    t[1, 2, 77] = float("nan")
+@pytest.mark.parametrize("dtype", ["fp32", "bf16", "fp16"])
+def test_greedy_invalid_sequences_are_marked(ears, dtype):
+    """NaN in an odd and an even lane of a packed pair (2-byte types), +inf, a fully masked row,
+    tokens out of range: each marks its own sequence only."""
+    t, x = make(10, 3, 5000, dtype, seed=5)
+    t[1, 2, 77] = float("nan")                        # odd lane
     t[2, 0, 4999] = float("inf")
     t[3, 3, :] = float("-inf")
     x[4, 1] = 5000
     x[5, 0] = -1
+    t[6, 1, 78] = float("nan")                        # even lane
+    top = int(t[7, 0].float().argmax())
+    t[7, 0, top ^ 1] = float("nan")                   # beside the row's top entry
     t[0, 0, 10:500] = float("-inf")                   # masked entries are legal
     dev = "cuda:0"
     acc, tok = ears.verify_greedy(t.to(dev), x.to(dev))
     torch.cuda.synchronize()
     assert ears.last_device_status() & ears.DEV_INVALID_INPUT
     o_acc, o_tok, _ = oracle.verify_greedy(t, x)
-    assert o_acc[1:6].tolist() == [-1] * 5
+    assert o_acc[1:8].tolist() == [-1] * 7 and (o_acc[[0, 8, 9]] >= 0).all()
     assert np.array_equal(acc.cpu().numpy(), o_acc) and np.array_equal(tok.cpu().numpy(), o_tok)
+
+
+def test_greedy_workspace_and_repeats(ears):
+    dev = "cuda:0"
     # caller workspace, repeated calls, clean status afterwards
     t2, x2 = make(8, 3, 5000, "bf16", seed=6)
     ws = torch.empty(ears.workspace_bytes(8, 3, 5000) + 256, dtype=torch.uint8, device=dev)

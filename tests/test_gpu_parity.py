@@ -8,7 +8,7 @@ import torch
 
 import oracle
 from paper_2512_13194_b200 import synth
-from parity import Tally, assert_parity, compare
+from oracle.parity import Tally, assert_parity, compare
 
 pytestmark = pytest.mark.gpu
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "philox4x32_10_kat.txt")
@@ -26,7 +26,7 @@ def run_both(ears, w, t, d, x, T, beta, seed=0, offset=0, b_first=0, nthreads=8)
     ora = oracle.verify(t.cpu(), d.cpu(), x.cpu(), T, beta, seed=seed, offset=offset, b_first=b_first,
                         nthreads=nthreads)
     stats = {k: v.cpu().numpy() for k, v in st.items()}
-    tally = compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, w.K, stats)
+    tally = compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, w.K, stats, inputs=(t.cpu(), d.cpu(), T))
     # the mass the final token was drawn from
     ok = ora.accept_len >= 0
     np.testing.assert_allclose(stats["resid_mass"][ok], ora.resid_mass[ok], rtol=2e-5)
@@ -152,18 +152,28 @@ def test_probabilities_are_tight_on_rows_far_below_their_maximum(ears, forced_pa
     assert tl.max_rel_prob_err < 7e-7
 
 
+@pytest.mark.parametrize("path,V", [(0, 256000), (3, 256000), (0, 131072), (3, 131072), (1, 131072)])
 @pytest.mark.parametrize("beta", [1.0, 0.0])
-def test_parity_largest_workload(ears, beta):
-    """Full size of the largest configuration, in the launch configuration the benchmark times;
-    beta = 0 is added because at beta = 1 nearly everything is accepted and the residual path idles."""
-    w = synth.workload(5)
+def test_parity_largest_workload(ears, forced_path, beta, path, V):
+    """Full size of the largest configuration, in the launch configuration the benchmark times
+    (path 0, V = 256000: the ring kernel) and with the kernel that reads straight from global memory
+    forced; and the same batch with rows of 512 KB (V = 131072), which the automatic rule gives to
+    that kernel.  beta = 0 is added because at beta = 1 nearly everything is accepted and the
+    residual path idles."""
+    from dataclasses import replace
+    forced_path(path)
+    w = replace(synth.workload(5), V=V)
+    plan = ears.describe_plan(w.dtype, w.B, w.K, w.V).split(":")[0]
+    assert plan == {(0, 256000): "streaming", (0, 131072): "direct", 1: "streaming", 3: "direct"}.get((path, V), None) \
+        or plan == {1: "streaming", 3: "direct"}[path]
     t, d, x = synth.make_inputs(w, "cuda:0")
     acc, tok, st = ears.verify(t, d, x, w.temperature, beta, 0, 3, stats=True)
     torch.cuda.synchronize()
     assert ears.last_device_status() == 0
     ora = oracle.verify(t.cpu(), d.cpu(), x.cpu(), w.temperature, beta, seed=0, offset=3,
                         nthreads=oracle.max_threads())
-    tally = compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, w.K, {k: v.cpu().numpy() for k, v in st.items()})
+    tally = compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, w.K, {k: v.cpu().numpy() for k, v in st.items()},
+                    inputs=(t.cpu(), d.cpu(), w.temperature))
     assert_parity(tally)
     assert tally.max_rel_prob_err < 1e-5
     if beta == 0.0:
@@ -220,32 +230,43 @@ def test_forced_resident_path_refuses_rows_that_do_not_fit(ears, forced_path):
     assert e.value.status == -2
 
 
-@pytest.mark.parametrize("dtype", ["fp32", "fp16"])
+@pytest.mark.parametrize("dtype", ["fp32", "fp16", "bf16"])
 @pytest.mark.parametrize("path", [1, 2, 3])
 def test_invalid_sequences_are_marked(ears, forced_path, path, dtype):
+    """Unusable data marks its own sequence and nothing else.  For the 2-byte types the NaNs sit in
+    an odd and in an even lane of a packed pair (the packed maximum drops NaNs, so they must reach
+    the sum), alone in a row that is otherwise ordinary, and next to the row's maximum."""
     forced_path(path)
-    w, t, d, x = synth.tiny_inputs(8, 3, 5000, dtype, seed=9)
+    B, V = 13, 5000
+    w, t, d, x = synth.tiny_inputs(B, 3, V, dtype, seed=9)
     t = t.clone(); d = d.clone(); x = x.clone()
-    x[1, 0] = 5000
+    x[1, 0] = V
     x[2, 2] = -3
-    t[3, 1, 77] = float("nan")
+    t[3, 1, 77] = float("nan")        # odd lane
     d[4, 0, 4999] = float("inf")
-    t[5, 3, :] = float("-inf")
+    t[5, 3, :] = float("-inf")        # a row with nothing finite
+    t[6, 2, 78] = float("nan")        # even lane
+    d[7, 1, 4096] = float("nan")      # first entry of a 16-byte vector, draft row
+    top = int(t[8, 0].float().argmax())
+    t[8, 0, top ^ 1] = float("nan")   # the partner of the row's maximum in its packed pair
+    t[9, 3, 4999] = float("inf")      # +inf in the extra row, last entry
     t[0, 0, 10:500] = float("-inf")   # masked vocabulary entries are legal
     d[0, 0, 10:500] = float("-inf")
     x[0, 0] = 5
+    bad = list(range(1, 10))
     dev = "cuda:0"
     acc, tok = ears.verify(t.to(dev), d.to(dev), x.to(dev), 1.0, 0.1, 1, 2)
     torch.cuda.synchronize()
     assert ears.last_device_status() & ears.DEV_INVALID_INPUT
     ora = oracle.verify(t, d, x, 1.0, 0.1, seed=1, offset=2)
-    assert ora.accept_len[1:6].tolist() == [-1] * 5
-    tl = compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, 3)
+    assert ora.accept_len[bad].tolist() == [-1] * len(bad)
+    assert (ora.accept_len[[0, 10, 11, 12]] >= 0).all()
+    tl = compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, 3, inputs=(t, d, 1.0))
     assert_parity(tl, max_explained=0)
     # the next call starts from a clean status
-    acc, tok = ears.verify(t[6:].to(dev), d[6:].to(dev), x[6:].to(dev), 1.0, 0.1, 1, 2, b_first=6)
+    acc, tok = ears.verify(t[10:].to(dev), d[10:].to(dev), x[10:].to(dev), 1.0, 0.1, 1, 2, b_first=10)
     assert ears.last_device_status() == 0
-    assert torch.equal(acc.cpu(), torch.from_numpy(ora.accept_len[6:]))
+    assert torch.equal(acc.cpu(), torch.from_numpy(ora.accept_len[10:]))
 
 
 def test_batch_shards_match_full_batch(ears):
@@ -378,7 +399,8 @@ def test_parity_per_sequence_temperature_and_beta(ears, forced_path, B, K, V, dt
         assert torch.equal(acc, acc2) and torch.equal(tok, tok2)
         ora = oracle.verify(t, d, x, 1.0, 0.0, seed=7, offset=offset, b_first=3, nthreads=8, seq_temperature=Ts,
                             seq_beta=betas)
-        tally.merge(compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, K, {k: v.cpu().numpy() for k, v in st.items()}))
+        tally.merge(compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, K, {k: v.cpu().numpy() for k, v in st.items()},
+                            inputs=(t, d, Ts)))
     assert_parity(tally, max_explained=1)
     assert tally.max_rel_prob_err < 1e-5
     # equal entries == the scalar call
@@ -399,7 +421,8 @@ def test_parity_per_sequence_temperature_and_beta(ears, forced_path, B, K, V, dt
     assert ears.last_device_status() & ears.DEV_INVALID_INPUT
     ora = oracle.verify(t, d, x, 1.0, 0.0, seed=7, offset=0, b_first=3, nthreads=8, seq_temperature=badT, seq_beta=badb)
     assert ora.accept_len[[1, 2, 4]].tolist() == [-1, -1, -1]
-    assert_parity(compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, K), max_explained=1)
+    assert_parity(compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, K, inputs=(t, d, np.where(np.isfinite(badT) & (badT > 0), badT, 1.0))),
+                  max_explained=1)
 
 
 @pytest.mark.parametrize("path", [1, 2, 3])
@@ -460,7 +483,7 @@ def test_parity_stop_at_first_reject(ears, forced_path, B, K, V, dtype, path, cl
         assert ears.last_device_status() & ears.DEV_TIMEOUT == 0
         assert torch.equal(acc, acc2) and torch.equal(tok, tok2)
         ora = oracle.verify(tt, dd, xx, T, beta, seed=4, offset=2, nthreads=8, stop_at_first_reject=True)
-        tally.merge(compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, K))
+        tally.merge(compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, K, inputs=(tt, dd, T)))
         # per-position outputs exist up to the first rejection
         pt = st["pt_tok"].cpu().numpy()
         for b in range(B):
@@ -505,6 +528,43 @@ def test_graph_replays_and_eager_calls_share_the_library_workspace(ears):
                 a, k = ears.verify(tg, dg, xg, 1.0, 0.2, 5, 3, stream=cap_stream)
             cap_stream.synchronize()
             assert torch.equal(a, ref[0]) and torch.equal(k, ref[1])
+
+
+def test_workspace_recorded_in_a_graph_outlives_a_larger_call(ears):
+    """A call recorded into a CUDA graph keeps pointing at the library's workspace of that moment.
+    A later, larger call on the same stream needs a bigger workspace: the recorded one must stay
+    allocated (the library parks it until shutdown), so that further replays still work."""
+    dev = "cuda:0"
+    w, t, d, x = synth.tiny_inputs(4, 2, 6000, "fp32", seed=23)
+    wl, tl_, dl, xl = synth.tiny_inputs(40, 6, 90000, "fp32", seed=24)     # needs a much larger workspace
+    assert ears.workspace_bytes(40, 6, 90000) > 4 * ears.workspace_bytes(4, 2, 6000)
+    tg, dg, xg = t.to(dev), d.to(dev), x.to(dev)
+    side = torch.cuda.Stream()
+    lib = ears.load_library()
+    with torch.cuda.stream(side):
+        ref = ears.verify(tg, dg, xg, 1.0, 0.2, 5, 3, stream=side)
+        side.synchronize()
+        acc, tok = torch.empty_like(ref[0]), torch.empty_like(ref[1])
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            rc = lib.ears_verify_f32(tg.data_ptr(), dg.data_ptr(), xg.data_ptr(), 4, 2, 6000, 1.0, 0.2, 5, 3,
+                                     acc.data_ptr(), tok.data_ptr(), torch.cuda.current_stream().cuda_stream)
+        assert rc == 0
+        big_ref = oracle.verify(tl_, dl, xl, 1.0, 0.2, seed=5, offset=3, nthreads=8)
+        a, k = ears.verify(tl_.to(dev), dl.to(dev), xl.to(dev), 1.0, 0.2, 5, 3, stream=side)   # grows the workspace
+        side.synchronize()
+        assert_parity(compare(a.cpu().numpy(), k.cpu().numpy(), big_ref, 6, inputs=(tl_, dl, 1.0)), max_explained=1)
+    for rep in range(3):
+        acc.fill_(-7)
+        tok.fill_(-7)
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(acc, ref[0]) and torch.equal(tok, ref[1]), rep
+    with torch.cuda.stream(side):
+        again = ears.verify(tg, dg, xg, 1.0, 0.2, 5, 3, stream=side)
+    side.synchronize()
+    assert torch.equal(again[0], ref[0]) and torch.equal(again[1], ref[1])
+    assert ears.last_device_status(side) == 0
 
 
 def test_decision_class_counts_match_the_oracle(ears):

@@ -84,6 +84,109 @@ def test_inverse_cdf_hand_cases():
     assert (near["token"], near["band_lo"], near["band_hi"]) == (3, 1, 3)
 
 
+def test_inverse_cdf_band_width_is_the_stated_one():
+    """The band lists the tokens whose CDF interval comes within `band` of u: a neighbour whose
+    interval ends 5e-6 from u is outside at band 1e-6 and inside at band 1e-5, on either side of u;
+    a band ten times too wide (or too narrow) fails one of these."""
+    r = [0.25, 0.25, 0.5]                                   # boundaries at 0.25 and 0.5
+    below = oracle.inverse_cdf(r, 0.25 + 5e-6, band=1e-6)   # token 0 ends 5e-6 below u
+    assert (below["token"], below["band_lo"], below["band_hi"]) == (1, 1, 1)
+    below = oracle.inverse_cdf(r, 0.25 + 5e-6, band=1e-5)
+    assert (below["token"], below["band_lo"], below["band_hi"]) == (1, 0, 1)
+    above = oracle.inverse_cdf(r, 0.5 - 5e-6, band=1e-6)    # token 2 starts 5e-6 above u
+    assert (above["token"], above["band_lo"], above["band_hi"]) == (1, 1, 1)
+    above = oracle.inverse_cdf(r, 0.5 - 5e-6, band=1e-5)
+    assert (above["token"], above["band_lo"], above["band_hi"]) == (1, 1, 2)
+    # just inside and just outside the stated width, both sides
+    assert oracle.inverse_cdf(r, 0.25 + 0.9e-6, band=1e-6)["band_lo"] == 0
+    assert oracle.inverse_cdf(r, 0.25 + 1.1e-6, band=1e-6)["band_lo"] == 1
+    assert oracle.inverse_cdf(r, 0.5 - 0.9e-6, band=1e-6)["band_hi"] == 2
+    assert oracle.inverse_cdf(r, 0.5 - 1.1e-6, band=1e-6)["band_hi"] == 1
+    # the band is in probability units, not in units of mass: scaling the masses changes nothing
+    scaled = oracle.inverse_cdf([250.0, 250.0, 500.0], 0.25 + 5e-6, band=1e-5)
+    assert (scaled["token"], scaled["band_lo"], scaled["band_hi"]) == (1, 0, 1)
+    # zero-mass tokens may sit between the ends of a band but are never its ends
+    gap = oracle.inverse_cdf([0.25, 0.0, 0.0, 0.25, 0.5], 0.25 + 1e-9, band=1e-6)
+    assert (gap["token"], gap["band_lo"], gap["band_hi"]) == (3, 0, 3)
+
+
+def test_cdf_margin_is_the_distance_to_the_nearer_interval_end():
+    """verify() reports min(u - lo, hi - u) of the drawn token's interval.  Bonus draw from
+    P_t = (1/4, 1/4, 1/2) (identical rows: everything accepted); u comes from the pinned Philox
+    stream, the interval ends are known by hand."""
+    K, V = 2, 3
+    row = np.log(np.array([1.0, 1.0, 2.0])).astype(np.float32)
+    t = np.broadcast_to(row, (64, K + 1, V)).copy()
+    d = np.broadcast_to(row, (64, K, V)).copy()
+    x = np.zeros((64, K), np.int32)
+    res = oracle.verify(t, d, x, 1.0, 0.0, seed=12, offset=34)
+    assert (res.accept_len == K).all()
+    edges = np.array([0.0, 0.25, 0.5, 1.0])
+    seen = set()
+    for b in range(64):
+        u = oracle.uniform_final(12, 34, b, K)
+        j = int(np.searchsorted(edges, u, side="right")) - 1
+        assert res.tokens[b, K] == j
+        want = min(u - edges[j], edges[j + 1] - u)
+        assert abs(res.cdf_margin[b] - want) < 1e-7, (b, u, res.cdf_margin[b], want)
+        assert res.band_lo[b] == res.band_hi[b] == j or want < 1e-6
+        seen.add(j)
+    assert seen == {0, 1, 2}
+
+
+def test_compare_refuses_a_zero_mass_token_inside_the_band():
+    """The parity helper accepts a token disagreement only when the other token lies in the oracle's
+    band AND has mass in the oracle's row.  Planted here: a 'GPU' answer that differs from the
+    oracle's by a zero-mass token inside the band (refused), by the positive-mass neighbour (accepted)
+    and by a token outside the band (refused)."""
+    from oracle.parity import compare
+    K, V = 1, 6
+    # P_t = (1/4, 0, 0, 1/4, 1/2, 0) on the extra row; tokens 1, 2, 5 are masked out
+    row = np.array([0.0, -np.inf, -np.inf, 0.0, np.log(2.0), -np.inf], np.float32)
+    t = np.broadcast_to(row, (1, K + 1, V)).copy()
+    d = np.broadcast_to(row, (1, K, V)).copy()
+    x = np.zeros((1, K), np.int32)
+    # find a (seed, offset) whose final uniform falls just above the boundary at 0.25
+    hit = None
+    for off in range(200000):
+        u = oracle.uniform_final(3, off, 0, K)
+        if 0.25 < u < 0.25 + 1e-6:
+            hit = off
+            break
+    if hit is None:      # no such draw among these offsets: plant the band through a wide one instead
+        hit, band = 0, 1.0
+    else:
+        band = 1e-6
+    ora = oracle.verify(t, d, x, 1.0, 0.0, seed=3, offset=hit, band=band)
+    n = int(ora.accept_len[0])
+    assert n == K
+    o = int(ora.tokens[0, n])
+    lo, hi = int(ora.band_lo[0]), int(ora.band_hi[0])
+    assert lo <= 0 and hi >= 3                  # the band spans tokens 0..3, of which 1 and 2 have no mass
+    inputs = (t, d, 1.0)
+
+    def gpu_answer(g):
+        tok = ora.tokens.copy()
+        tok[0, n] = g
+        return compare(ora.accept_len.copy(), tok, ora, K, inputs=inputs)
+
+    other = 0 if o == 3 else 3
+    ok = gpu_answer(other)
+    assert ok.explained_tokens == 1 and not ok.unexplained
+    for zero in (1, 2):
+        bad = gpu_answer(zero)
+        assert bad.explained_tokens == 0 and bad.unexplained and bad.unexplained[0][1] == "token-zero-mass"
+    out = gpu_answer(5)
+    assert out.unexplained and out.unexplained[0][1] in ("token", "token-zero-mass")
+    # without the inputs nothing can be explained
+    tok = ora.tokens.copy()
+    tok[0, n] = other
+    assert compare(ora.accept_len.copy(), tok, ora, K).unexplained[0][1] == "token-unchecked"
+    # and an exact match is clean
+    clean = compare(ora.accept_len.copy(), ora.tokens.copy(), ora, K, inputs=inputs)
+    assert not clean.unexplained and clean.explained == 0
+
+
 # -------------------------------------------------- closed-form acceptance probability
 @pytest.mark.parametrize("beta,T", [(0.0, 1.0), (0.1, 0.9), (0.5, 1.3), (1.0, 1.0)])
 def test_acceptance_probability_closed_form(beta, T):

@@ -10,9 +10,12 @@ shapes too large for the array are refused.  It is collected last on purpose.
 """
 import gc
 
+import numpy as np
 import pytest
 import torch
 
+import oracle
+from oracle.parity import assert_parity, compare
 from paper_2512_13194_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -43,6 +46,35 @@ def test_noalloc_matches_ordinary_entry_twice_in_a_row(ears):
             # same kernels, same launch plan, same inputs: bit-exact, the bar of the parity tests
             assert torch.equal(acc, ref_len), (call, acc, ref_len)
             assert torch.equal(tok, ref_tok), (call, tok, ref_tok)
+            # and against the oracle, with the near-tie rules of the parity tests
+            ora = oracle.verify(t, d, x, 0.9, beta, seed=5, offset=offset, b_first=2)
+            assert_parity(compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, w.K, inputs=(t, d, 0.9)), max_explained=1)
+
+
+def test_noalloc_allocates_nothing_once_its_kernels_are_loaded(ears):
+    """The first use of an element type and kernel on a device loads code (the driver allocates for
+    that once); the call after it must not allocate at all.  Here the allocation-free entry point
+    itself makes the first use: fp16 logits under each kernel, a warm-up call, then a measured one."""
+    dev = "cuda:0"
+    for path, (B, K, V) in ((2, (3, 2, 9000)), (3, (3, 2, 70000)), (1, (3, 2, 70000))):
+        w, t, d, x = synth.tiny_inputs(B, K, V, "fp16", seed=64 + path)
+        tg, dg, xg = t.to(dev), d.to(dev), x.to(dev)
+        acc = torch.empty(B, dtype=torch.int32, device=dev)
+        tok = torch.empty((B, K + 1), dtype=torch.int32, device=dev)
+        ears.set_path(path, 0)
+        try:
+            ears.verify_noalloc(tg, dg, xg, 1.1, 0.2, 8, 1, out_accept_len=acc, out_tokens=tok)    # warm-up: loads the kernel
+            gc.collect()
+            torch.cuda.synchronize()
+            before, free_before = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
+            ears.verify_noalloc(tg, dg, xg, 1.1, 0.2, 8, 2, out_accept_len=acc, out_tokens=tok)
+            torch.cuda.synchronize()
+            assert torch.cuda.memory_allocated() == before
+            assert torch.cuda.mem_get_info()[0] >= free_before
+        finally:
+            ears.set_path(0, 0)
+        ora = oracle.verify(t, d, x, 1.1, 0.2, seed=8, offset=2)
+        assert_parity(compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, K, inputs=(t, d, 1.1)), max_explained=1)
 
 
 def test_noalloc_marks_invalid_sequences_and_reports_status(ears):
