@@ -33,8 +33,9 @@ constexpr double kTinyMass = 1e-300;                 // below this a residual is
 constexpr int kDevInvalidInput = 1;
 constexpr int kDevTimeout = 2;
 
-// Sum of exp2((l - ref) c) over one consumer warp's share of a chunk of the extra target row.
-struct BonusSeg { double sum; float ref; float pad; };
+// Sum of exp2(l c - mu) over one consumer warp's share of a chunk of the extra target row; mu is
+// the fp32 product (running maximum) x c that the terms were taken relative to.
+struct BonusSeg { double sum; float mu; float pad; };
 
 struct Plan {
     int use_tma;   // 1: bulk asynchronous copies, 0: element-wise loader

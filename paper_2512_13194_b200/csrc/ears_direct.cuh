@@ -61,81 +61,6 @@ __device__ __forceinline__ uint4 ld_stream16(const void* p) {
     return r;
 }
 
-template <typename E> struct Words;
-template <> struct Words<float> {
-    static constexpr int N = 4;
-    __device__ static __forceinline__ float vmax(uint4 w) {
-        return fmaxf(fmaxf(__uint_as_float(w.x), __uint_as_float(w.y)), fmaxf(__uint_as_float(w.z), __uint_as_float(w.w)));
-    }
-    __device__ static __forceinline__ void unpack(uint4 w, float (&x)[4]) {
-        x[0] = __uint_as_float(w.x); x[1] = __uint_as_float(w.y); x[2] = __uint_as_float(w.z); x[3] = __uint_as_float(w.w);
-    }
-    __device__ static __forceinline__ uint4 minus_inf() { return make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u); }
-    // up to N entries from p (fewer, or none, when `left` says so), the rest -inf
-    __device__ static __forceinline__ uint4 gather(const float* p, int left) {
-        uint4 w = minus_inf();
-        if (left > 0) w.x = __float_as_uint(__ldg(p));
-        if (left > 1) w.y = __float_as_uint(__ldg(p + 1));
-        if (left > 2) w.z = __float_as_uint(__ldg(p + 2));
-        if (left > 3) w.w = __float_as_uint(__ldg(p + 3));
-        return w;
-    }
-};
-template <> struct Words<uint16_t> {
-    static constexpr int N = 8;
-    __device__ static __forceinline__ float vmax(uint4 w) {   // exact on packed pairs
-        const uint32_t pm = max_bf16x2(max_bf16x2(w.x, w.y), max_bf16x2(w.z, w.w));
-        return fmaxf(__uint_as_float(pm << 16), __uint_as_float(pm & 0xffff0000u));
-    }
-    __device__ static __forceinline__ void unpack(uint4 w, float (&x)[8]) {
-        x[0] = __uint_as_float(w.x << 16); x[1] = __uint_as_float(w.x & 0xffff0000u);
-        x[2] = __uint_as_float(w.y << 16); x[3] = __uint_as_float(w.y & 0xffff0000u);
-        x[4] = __uint_as_float(w.z << 16); x[5] = __uint_as_float(w.z & 0xffff0000u);
-        x[6] = __uint_as_float(w.w << 16); x[7] = __uint_as_float(w.w & 0xffff0000u);
-    }
-    __device__ static __forceinline__ uint4 minus_inf() { return make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u); }
-    __device__ static __forceinline__ uint4 gather(const uint16_t* p, int left) {
-        uint32_t h[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) h[i] = i < left ? (uint32_t)__ldg(p + i) : 0xff80u;
-        return make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
-    }
-};
-template <> struct Words<f16_t> {
-    static constexpr int N = 8;
-    __device__ static __forceinline__ float vmax(uint4 w) {   // exact on packed pairs
-        const float2 m = f16x2_to_float2(max_f16x2(max_f16x2(w.x, w.y), max_f16x2(w.z, w.w)));
-        return fmaxf(m.x, m.y);
-    }
-    __device__ static __forceinline__ void unpack(uint4 w, float (&x)[8]) { Vec<f16_t>::unpack(w, x); }
-    __device__ static __forceinline__ uint4 minus_inf() { return make_uint4(0xfc00fc00u, 0xfc00fc00u, 0xfc00fc00u, 0xfc00fc00u); }
-    __device__ static __forceinline__ uint4 gather(const f16_t* p, int left) {
-        uint32_t h[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) h[i] = i < left ? (uint32_t)__ldg(&p[i].bits) : 0xfc00u;
-        return make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
-    }
-};
-
-// G vectors of one thread: maximum first, one rescale of the running sums if it grew, then one
-// fused multiply-add and one exp2 per entry (RowAcc convention, see ears_math.cuh).
-template <typename E, int G>
-__device__ __forceinline__ void fold_vectors(const uint4 (&w)[G], float c, RowAcc& a) {
-    constexpr int N = Words<E>::N;
-    float cm = Words<E>::vmax(w[0]);
-#pragma unroll
-    for (int j = 1; j < G; ++j) cm = fmaxf(cm, Words<E>::vmax(w[j]));
-    acc_raise(a, cm, c);
-    const float nmu = -a.mu;
-#pragma unroll
-    for (int j = 0; j < G; ++j) {
-        float x[N];
-        Words<E>::unpack(w[j], x);
-#pragma unroll
-        for (int i = 0; i < N; ++i) a.s[i & 3] += ex2_approx(__fmaf_rn(x[i], c, nmu));
-    }
-}
-
 // An ordinary row piece [e0, e1): THREADS threads (tid = 0 .. THREADS-1) stride over it.
 // -> the thread's (m, s).
 template <typename E, int THREADS = kDThreads>
@@ -165,7 +90,7 @@ __device__ __forceinline__ float2 stream_piece(const E* row, int e0, int e1, boo
         for (int i = e0 + tid; i < e1; i += THREADS) {
             const float x = load_logit(row + i);
             acc_raise(a, x, c);
-            a.s[0] += ex2_approx(__fmaf_rn(x, c, -a.mu));
+            acc_add_one(a, x, c);
         }
     }
     return acc_close(a, c);
@@ -181,8 +106,9 @@ __device__ __forceinline__ float2 stream_bonus_piece(const E* row, int e0, int e
     constexpr int N = Words<E>::N;
     constexpr int SEG = kBonusSegBytes / (int)sizeof(E);   // entries per segment
     constexpr int VPL = SEG / N / 32;                        // vectors per lane per segment
-    float m_run = -INFINITY;
-    float s = 0.f;
+    constexpr int PN = N / 2;
+    RowAcc a;            // the maximum is kept warp-uniform
+    acc_open(a);
     for (int ga = e0 + warp * SEG; ga < e1; ga += 2 * kDWarps * SEG) {
         // the loads stay packed (16 bytes per vector) until they are used; rows that are not
         // 16-byte aligned are gathered element by element into the same form
@@ -203,37 +129,36 @@ __device__ __forceinline__ float2 stream_bonus_piece(const E* row, int e0, int e
             }
         }
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            cm[h] = Words<E>::vmax(w[h][0]);
-#pragma unroll
-            for (int j = 1; j < VPL; ++j) cm[h] = fmaxf(cm[h], Words<E>::vmax(w[h][j]));
-        }
+        for (int h = 0; h < 2; ++h) cm[h] = Words<E>::template vmax_all<VPL>(w[h]);
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) {
             cm[0] = fmaxf(cm[0], __shfl_xor_sync(0xffffffffu, cm[0], off));
             cm[1] = fmaxf(cm[1], __shfl_xor_sync(0xffffffffu, cm[1], off));
         }
         double tot[2];
-        float ref[2];
+        float ref[2];   // the fp32 product (running maximum) x c the segment's terms are relative to
+        const f32x2 c2 = pack2(c, c);
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            if (cm[h] > m_run) {
-                s *= ex2_approx((m_run - cm[h]) * c);   // m_run = -inf gives 0
-                m_run = cm[h];
-            }
-            ref[h] = m_run;
-            const float mu = (m_run == -INFINITY) ? 0.0f : m_run;
-            float cs[4] = {0.f, 0.f, 0.f, 0.f};
+            acc_raise(a, cm[h], c);
+            ref[h] = a.mu;
+            const f32x2 nmu2 = pack2(-a.mu, -a.mu);
+            f32x2 cs[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
 #pragma unroll
             for (int j = 0; j < VPL; ++j) {
-                float x[N];
-                Words<E>::unpack(w[h][j], x);
+                f32x2 p[PN];
+                Words<E>::pairs(w[h][j], p);
 #pragma unroll
-                for (int i = 0; i < N; ++i) cs[i & 3] += ex2_approx(__fmul_rn(__fsub_rn(x[i], mu), c));
+                for (int i = 0; i < PN; i += 2) {
+                    cs[0] = add2(cs[0], ex2_pair(fma2(p[i], c2, nmu2)));
+                    cs[1] = add2(cs[1], ex2_pair(fma2(p[i + 1], c2, nmu2)));
+                }
             }
-            const float part = (cs[0] + cs[1]) + (cs[2] + cs[3]);
-            s += part;
-            tot[h] = (double)part;
+            a.s[0] = add2(a.s[0], cs[0]);
+            a.s[1] = add2(a.s[1], cs[1]);
+            float q0, q1;
+            unpack2(add2(cs[0], cs[1]), q0, q1);
+            tot[h] = (double)(q0 + q1);
         }
         // a lane's few terms add up in fp32; across lanes in fp64 (the running sums of the final
         // draw stay exact to ~1e-9 of the row's mass)
@@ -253,7 +178,7 @@ __device__ __forceinline__ float2 stream_bonus_piece(const E* row, int e0, int e
     const int e_pad = (e1 + CHUNK - 1) / CHUNK * CHUNK;
     for (int g0 = (e1 + SEG - 1) / SEG * SEG + warp * SEG; g0 < e_pad; g0 += kDWarps * SEG)
         if (lane == 0) segs[g0 / SEG] = BonusSeg{0.0, 0.f, 0.f};
-    return make_float2(m_run, s);
+    return acc_close(a, c);
 }
 
 // A second-pass piece [e0, e1) of the two rows of a rejected position: sums of

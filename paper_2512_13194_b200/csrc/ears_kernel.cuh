@@ -221,63 +221,57 @@ __device__ __forceinline__ void loader_fill(PipeSmem<STAGES>& sm, int stage, con
 }
 
 // ---- consumer arithmetic --------------------------------------------------------
-// Running (m, s) of one thread over its share of a staged chunk:
-// s = sum exp2((l - m) * c), m = running maximum; s is rescaled when m grows.
+// Running (m, s) of one thread over its share of a staged chunk, in the RowAcc form: one
+// multiply-add, one exp2 and one addition per entry, the first and the last on pairs of entries.
 // Warp w owns the w-th eighth of the slot (contiguous), lane-interleaved in 16-byte vectors.
 //
-// BONUS (the extra target row K): the maximum is kept warp-uniform and the warp also emits
-// (sum, reference maximum) of its eighth of the chunk.  If every draft token turns out to be
-// accepted, the final token is drawn from exactly these sums and the row is not read again.
+// BONUS (the extra target row K): the maximum is kept warp-uniform and the warp also emits the sum
+// of its eighth of the chunk together with the reference the terms were taken against.  If every
+// draft token turns out to be accepted, the final token is drawn from exactly these sums and the
+// row is not read again.
 template <typename E, bool BONUS>
 __device__ __forceinline__ void chunk_stats(const unsigned char* buf, int nelem, int warp, int lane, float c,
-                                            float& m_run, float (&s)[4], BonusSeg* warp_chunk_out) {
-    constexpr int N = Vec<E>::N;
+                                            RowAcc& a, BonusSeg* warp_chunk_out) {
+    constexpr int N = Words<E>::N, PN = N / 2;
     constexpr int VECS = kChunkBytes / 16 / kConsumers;  // 16-byte vectors per thread per chunk
     constexpr int CHUNK_ELEMS = kChunkBytes / (int)sizeof(E);
-    float x[VECS][N];
+    uint4 w[VECS];
 #pragma unroll
-    for (int j = 0; j < VECS; ++j) Vec<E>::load(buf, (warp * VECS + j) * 32 + lane, x[j]);
+    for (int j = 0; j < VECS; ++j) w[j] = reinterpret_cast<const uint4*>(buf)[(warp * VECS + j) * 32 + lane];
     if (nelem < CHUNK_ELEMS) {  // ragged last chunk of a row: mask what lies beyond it
 #pragma unroll
-        for (int j = 0; j < VECS; ++j)
-#pragma unroll
-            for (int i = 0; i < N; ++i)
-                if (((warp * VECS + j) * 32 + lane) * N + i >= nelem) x[j][i] = -INFINITY;
+        for (int j = 0; j < VECS; ++j) w[j] = Words<E>::mask_tail(w[j], nelem - ((warp * VECS + j) * 32 + lane) * N);
     }
-    float cm = -INFINITY;
-#pragma unroll
-    for (int j = 0; j < VECS; ++j)
-#pragma unroll
-        for (int i = 0; i < N; ++i) cm = fmaxf(cm, x[j][i]);
-    if (BONUS) {
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, off));
-    }
-    if (cm > m_run) {
-        float sc = ex2_approx((m_run - cm) * c);  // m_run = -inf gives 0
-        s[0] *= sc; s[1] *= sc; s[2] *= sc; s[3] *= sc;
-        m_run = cm;
-    }
-    const float mu = (m_run == -INFINITY) ? 0.0f : m_run;
     if (!BONUS) {
-#pragma unroll
-        for (int j = 0; j < VECS; ++j)
-#pragma unroll
-            for (int i = 0; i < N; ++i) s[(j * N + i) & 3] += ex2_approx(__fmul_rn(__fsub_rn(x[j][i], mu), c));
-    } else {
-        float cs[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int j = 0; j < VECS; ++j)
-#pragma unroll
-            for (int i = 0; i < N; ++i) cs[(j * N + i) & 3] += ex2_approx(__fmul_rn(__fsub_rn(x[j][i], mu), c));
-        s[0] += cs[0]; s[1] += cs[1]; s[2] += cs[2]; s[3] += cs[3];
-        // a lane's few terms add up in fp32; across lanes in fp64, so that the running sums of the
-        // final draw stay exact to ~1e-9 of the row's mass
-        double tot = (double)((cs[0] + cs[1]) + (cs[2] + cs[3]));
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, off);
-        if (lane == 0) *warp_chunk_out = BonusSeg{tot, m_run, 0.f};   // m_run is warp-uniform here
+        fold_vectors<E, VECS>(w, c, a);
+        return;
     }
+    float cm = Words<E>::template vmax_all<VECS>(w);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, off));
+    acc_raise(a, cm, c);   // warp-uniform
+    const f32x2 c2 = pack2(c, c), nmu2 = pack2(-a.mu, -a.mu);
+    f32x2 cs[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
+#pragma unroll
+    for (int j = 0; j < VECS; ++j) {
+        f32x2 p[PN];
+        Words<E>::pairs(w[j], p);
+#pragma unroll
+        for (int i = 0; i < PN; i += 2) {
+            cs[0] = add2(cs[0], ex2_pair(fma2(p[i], c2, nmu2)));
+            cs[1] = add2(cs[1], ex2_pair(fma2(p[i + 1], c2, nmu2)));
+        }
+    }
+    a.s[0] = add2(a.s[0], cs[0]);
+    a.s[1] = add2(a.s[1], cs[1]);
+    // a lane's few terms add up in fp32; across lanes in fp64, so that the running sums of the
+    // final draw stay exact to ~1e-9 of the row's mass
+    float q0, q1;
+    unpack2(add2(cs[0], cs[1]), q0, q1);
+    double tot = (double)(q0 + q1);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, off);
+    if (lane == 0) *warp_chunk_out = BonusSeg{tot, a.mu, 0.f};
 }
 
 // Sums of kSegElems-element segments of a staged chunk; warp w takes segments w, w+8, ...
@@ -587,15 +581,15 @@ __device__ void select_token(const Params& p, int b, int n, int lane) {
         seg = pick_block([ss](int g) { return __ldcg(ss + g); }, nseg, u, lane, &S, &before);
         seg_elems = kSegElems;
     } else {
-        // one entry per (chunk, consumer warp) of the extra row: (sum, reference maximum)
+        // one entry per (chunk, consumer warp) of the extra row: (sum, reference of its terms)
         const int chunks = (V + CHUNK_ELEMS - 1) / CHUNK_ELEMS;
         const BonusSeg* bs = bonus_segs(p, b);
-        const double m = (double)rn.mt, c = (double)cb;
-        seg = pick_block([bs, m, c](int g) {
+        const double mc = (double)rn.mt * (double)cb;   // exact: two fp32 factors
+        seg = pick_block([bs, mc](int g) {
                   const double sum = __ldcg(&bs[g].sum);
-                  const float ref = __ldcg(&bs[g].ref);
-                  // bring the sum from its own reference maximum to the row's (fp64: no new error)
-                  return sum > 0.0 ? sum * exp2(((double)ref - m) * c) : 0.0;
+                  const float mu = __ldcg(&bs[g].mu);
+                  // the terms were exp2(l c - mu): bring the sum to the row's own maximum (fp64: no new error)
+                  return sum > 0.0 ? sum * exp2((double)mu - mc) : 0.0;
               }, chunks * kConsumerWarps, u, lane, &S, &before);
         seg_elems = CHUNK_ELEMS / kConsumerWarps;
     }
@@ -915,8 +909,8 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
         }
     } else {
         // =============================== consumer warps
-        float m_run = -INFINITY;
-        float s[4] = {0.f, 0.f, 0.f, 0.f};
+        RowAcc acc;
+        acc_open(acc);
         int unit_ends = 0;   // ends of units and pieces seen so far (same in every consumer warp)
         RowNorm rn{0.f, 0.f, 0.f, 0.f, 0.0};
         for (uint32_t q = 0;; ++q) {
@@ -928,26 +922,28 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
                 break;
             }
             if (mt.kind == kStats) {
-                if (mt.flags & 1) { m_run = -INFINITY; s[0] = s[1] = s[2] = s[3] = 0.f; }
+                if (mt.flags & 1) acc_open(acc);
                 if (mt.aux) {  // a piece of the extra target row
                     BonusSeg* out = bonus_segs(p, mt.id / (R * P)) + (size_t)(mt.elem0 / CHUNK_ELEMS) * kConsumerWarps + warp;
-                    chunk_stats<E, true>(sm.buf[stage], mt.nelem, warp, lane, PER_SEQ ? mt.c : p.c, m_run, s, out);
+                    chunk_stats<E, true>(sm.buf[stage], mt.nelem, warp, lane, PER_SEQ ? mt.c : p.c, acc, out);
                 } else {
-                    chunk_stats<E, false>(sm.buf[stage], mt.nelem, warp, lane, PER_SEQ ? mt.c : p.c, m_run, s, nullptr);
+                    chunk_stats<E, false>(sm.buf[stage], mt.nelem, warp, lane, PER_SEQ ? mt.c : p.c, acc, nullptr);
                 }
                 if (!(mt.flags & 2)) {
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&sm.empty[stage]);
                     continue;
                 }
-                // last chunk of the unit: reduce the CTA's (m, s)
-                float m = m_run, sum = (s[0] + s[1]) + (s[2] + s[3]);
+                // last chunk of the unit: (max, sum) of the warp -- the maximum first (shuffles only),
+                // then one rescale per thread and a sum
+                const float cu = PER_SEQ ? mt.c : p.c;
+                const float2 ms = acc_close(acc, cu);
+                float m = ms.x;
 #pragma unroll
-                for (int off = 16; off > 0; off >>= 1) {
-                    float m2 = __shfl_xor_sync(0xffffffffu, m, off);
-                    float s2 = __shfl_xor_sync(0xffffffffu, sum, off);
-                    merge_ms(m, sum, m2, s2, PER_SEQ ? mt.c : p.c);
-                }
+                for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+                float sum = rebase_sum(ms.x, ms.y, m, cu);
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
                 if (lane == 0) {
                     const int us = unit_ends % kUnitSlots;
                     sm.scratch[us][warp] = make_float2(m, sum);

@@ -110,21 +110,79 @@ __device__ __forceinline__ uint32_t max_f16x2(uint32_t a, uint32_t b) {
     return r;
 }
 
+// ---- two fp32 lanes per instruction ---------------------------------------------
+// sm_100 issues fused multiply-adds, additions and multiplications on pairs of fp32 values held in
+// a 64-bit register (fma.rn.f32x2 and friends): the same roundings as the scalar forms, half the
+// issue slots.  The streaming loops spend one multiply-add and one addition per logit, so this is
+// where their instruction count comes from.
+typedef unsigned long long f32x2;
+
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+    f32x2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+// exp2 of both lanes (the special-function unit has no paired form)
+__device__ __forceinline__ f32x2 ex2_pair(f32x2 v) {
+    float lo, hi;
+    unpack2(v, lo, hi);
+    return pack2(ex2_approx(lo), ex2_approx(hi));
+}
+// the largest of three (sm_100 takes three operands in one instruction); a NaN operand is
+// ignored, like fmaxf does
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+
 // ---- statistics of a slice ------------------------------------------------------
 // Running (m, s) of one thread: s = sum exp2(fl(l c - mu)), mu = fl(m c) (0 while m = -inf).
 // One fused multiply-add per entry; the rounding of m c is taken out again in acc_close.
-struct RowAcc { float m, mu, s[4]; };
+// The sum is kept in four lanes (two register pairs) so that consecutive additions overlap.
+struct RowAcc { float m, mu; f32x2 s[2]; };
 
-__device__ __forceinline__ void acc_open(RowAcc& a) { a.m = -INFINITY; a.mu = 0.f; a.s[0] = a.s[1] = a.s[2] = a.s[3] = 0.f; }
+__device__ __forceinline__ void acc_open(RowAcc& a) { a.m = -INFINITY; a.mu = 0.f; a.s[0] = a.s[1] = pack2(0.f, 0.f); }
 
 __device__ __forceinline__ void acc_raise(RowAcc& a, float cm, float c) {
     if (cm > a.m) {  // false for NaN: a NaN entry reaches the sum instead
         const float mu_new = cm * c;
         const float sc = (a.m == -INFINITY) ? 0.f : ex2_approx(a.mu - mu_new);
-        a.s[0] *= sc; a.s[1] *= sc; a.s[2] *= sc; a.s[3] *= sc;
+        const f32x2 sc2 = pack2(sc, sc);
+        a.s[0] = mul2(a.s[0], sc2);
+        a.s[1] = mul2(a.s[1], sc2);
         a.m = cm;
         a.mu = mu_new;
     }
+}
+
+// One more entry (loops that go element by element: rows that are not 16-byte aligned).
+__device__ __forceinline__ void acc_add_one(RowAcc& a, float x, float c) {
+    a.s[0] = add2(a.s[0], pack2(ex2_approx(__fmaf_rn(x, c, -a.mu)), 0.f));
+}
+
+// Two more pairs of entries: sum += exp2(x c - mu) in each of the four lanes.
+__device__ __forceinline__ void acc_add_pairs(RowAcc& a, f32x2 x01, f32x2 x23, f32x2 c2, f32x2 nmu2) {
+    a.s[0] = add2(a.s[0], ex2_pair(fma2(x01, c2, nmu2)));
+    a.s[1] = add2(a.s[1], ex2_pair(fma2(x23, c2, nmu2)));
 }
 
 // -> (m, s) with s relative to the exact product m c: fl(m c) differs from m c by
@@ -132,7 +190,9 @@ __device__ __forceinline__ void acc_raise(RowAcc& a, float cm, float c) {
 // every one carries the factor 2^delta, which is divided out: 2^-delta = 1 - delta ln 2 to first
 // order (|delta| < 1e-5).
 __device__ __forceinline__ float2 acc_close(const RowAcc& a, float c) {
-    float s = (a.s[0] + a.s[1]) + (a.s[2] + a.s[3]);
+    float s0, s1;
+    unpack2(add2(a.s[0], a.s[1]), s0, s1);
+    float s = s0 + s1;
     if (a.m > -INFINITY && a.m < INFINITY) s = __fmaf_rn(s, -0.6931471805599453f * __fmaf_rn(a.m, c, -a.mu), s);
     return make_float2(a.m, s);
 }
@@ -144,73 +204,145 @@ __device__ __forceinline__ float rebase_sum(float m, float s, float M, float c) 
     return s * sc;
 }
 
-template <typename E> struct SubLoad;
-template <> struct SubLoad<float> {
-    // two 16-byte vectors of a full sub-chunk and their maximum
-    __device__ static __forceinline__ float load(const unsigned char* buf, int v0, int v1, float (&x)[2][4]) {
-        Vec<float>::load(buf, v0, x[0]);
-        Vec<float>::load(buf, v1, x[1]);
-        return fmaxf(fmaxf(fmaxf(x[0][0], x[0][1]), fmaxf(x[0][2], x[0][3])),
-                     fmaxf(fmaxf(x[1][0], x[1][1]), fmaxf(x[1][2], x[1][3])));
+// ---- packed 16-byte vectors of logits ---------------------------------------------
+// A vector stays packed (four 32-bit words, as loaded) until it is used.  Per element type:
+//   N            entries per vector
+//   vmax_all     the largest entry of G vectors (on packed pairs for the 2-byte types, which is exact;
+//                three operands per instruction for fp32); NaN entries are ignored here and reach the
+//                sum instead
+//   pairs        the entries widened to fp32, two per 64-bit register
+//   unpack       the entries widened to fp32, one per register
+//   minus_inf    a vector of -inf entries;  mask_tail: entries from index `keep` on become -inf
+//   gather       up to N entries fetched one by one (rows that are not 16-byte aligned)
+template <typename E> struct Words;
+template <> struct Words<float> {
+    static constexpr int N = 4;
+    template <int G>
+    __device__ static __forceinline__ float vmax_all(const uint4 (&w)[G]) {
+        float cm = max3(__uint_as_float(w[0].x), __uint_as_float(w[0].y), __uint_as_float(w[0].z));
+        cm = fmaxf(cm, __uint_as_float(w[0].w));
+#pragma unroll
+        for (int j = 1; j < G; ++j) {
+            cm = max3(cm, __uint_as_float(w[j].x), __uint_as_float(w[j].y));
+            cm = max3(cm, __uint_as_float(w[j].z), __uint_as_float(w[j].w));
+        }
+        return cm;
+    }
+    __device__ static __forceinline__ void pairs(uint4 w, f32x2 (&p)[2]) {
+        p[0] = pack2(__uint_as_float(w.x), __uint_as_float(w.y));
+        p[1] = pack2(__uint_as_float(w.z), __uint_as_float(w.w));
+    }
+    __device__ static __forceinline__ void unpack(uint4 w, float (&x)[4]) {
+        x[0] = __uint_as_float(w.x); x[1] = __uint_as_float(w.y); x[2] = __uint_as_float(w.z); x[3] = __uint_as_float(w.w);
+    }
+    __device__ static __forceinline__ uint4 minus_inf() { return make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u); }
+    __device__ static __forceinline__ uint4 mask_tail(uint4 w, int keep) {
+        if (keep < 1) w.x = 0xff800000u;
+        if (keep < 2) w.y = 0xff800000u;
+        if (keep < 3) w.z = 0xff800000u;
+        if (keep < 4) w.w = 0xff800000u;
+        return w;
+    }
+    // up to N entries from p (fewer, or none, when `left` says so), the rest -inf
+    __device__ static __forceinline__ uint4 gather(const float* p, int left) {
+        uint4 w = minus_inf();
+        if (left > 0) w.x = __float_as_uint(__ldg(p));
+        if (left > 1) w.y = __float_as_uint(__ldg(p + 1));
+        if (left > 2) w.z = __float_as_uint(__ldg(p + 2));
+        if (left > 3) w.w = __float_as_uint(__ldg(p + 3));
+        return w;
     }
 };
-template <> struct SubLoad<uint16_t> {
-    __device__ static __forceinline__ float load(const unsigned char* buf, int v0, int v1, float (&x)[2][8]) {
-        const uint4 a = reinterpret_cast<const uint4*>(buf)[v0];
-        const uint4 b = reinterpret_cast<const uint4*>(buf)[v1];
-        // the maximum of bf16 pairs is exact in packed form: half an instruction per entry
-        const uint32_t pm = max_bf16x2(max_bf16x2(max_bf16x2(a.x, a.y), max_bf16x2(a.z, a.w)),
-                                       max_bf16x2(max_bf16x2(b.x, b.y), max_bf16x2(b.z, b.w)));
-        x[0][0] = __uint_as_float(a.x << 16); x[0][1] = __uint_as_float(a.x & 0xffff0000u);
-        x[0][2] = __uint_as_float(a.y << 16); x[0][3] = __uint_as_float(a.y & 0xffff0000u);
-        x[0][4] = __uint_as_float(a.z << 16); x[0][5] = __uint_as_float(a.z & 0xffff0000u);
-        x[0][6] = __uint_as_float(a.w << 16); x[0][7] = __uint_as_float(a.w & 0xffff0000u);
-        x[1][0] = __uint_as_float(b.x << 16); x[1][1] = __uint_as_float(b.x & 0xffff0000u);
-        x[1][2] = __uint_as_float(b.y << 16); x[1][3] = __uint_as_float(b.y & 0xffff0000u);
-        x[1][4] = __uint_as_float(b.z << 16); x[1][5] = __uint_as_float(b.z & 0xffff0000u);
-        x[1][6] = __uint_as_float(b.w << 16); x[1][7] = __uint_as_float(b.w & 0xffff0000u);
+// entries from `keep` on of a vector of eight 2-byte entries become `ninf` (the type's -inf pattern)
+__device__ __forceinline__ uint4 mask_tail16(uint4 w, int keep, uint32_t ninf) {
+    uint32_t h[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if (keep <= 2 * i) h[i] = ninf | (ninf << 16);
+        else if (keep == 2 * i + 1) h[i] = (h[i] & 0xffffu) | (ninf << 16);
+    }
+    return make_uint4(h[0], h[1], h[2], h[3]);
+}
+template <> struct Words<uint16_t> {
+    static constexpr int N = 8;
+    template <int G>
+    __device__ static __forceinline__ float vmax_all(const uint4 (&w)[G]) {   // exact on packed pairs
+        uint32_t pm = max_bf16x2(max_bf16x2(w[0].x, w[0].y), max_bf16x2(w[0].z, w[0].w));
+#pragma unroll
+        for (int j = 1; j < G; ++j) pm = max_bf16x2(max_bf16x2(pm, w[j].x), max_bf16x2(max_bf16x2(w[j].y, w[j].z), w[j].w));
         return fmaxf(__uint_as_float(pm << 16), __uint_as_float(pm & 0xffff0000u));
     }
+    __device__ static __forceinline__ f32x2 widen(uint32_t h) { return pack2(__uint_as_float(h << 16), __uint_as_float(h & 0xffff0000u)); }
+    __device__ static __forceinline__ void pairs(uint4 w, f32x2 (&p)[4]) {
+        p[0] = widen(w.x); p[1] = widen(w.y); p[2] = widen(w.z); p[3] = widen(w.w);
+    }
+    __device__ static __forceinline__ void unpack(uint4 w, float (&x)[8]) {
+        x[0] = __uint_as_float(w.x << 16); x[1] = __uint_as_float(w.x & 0xffff0000u);
+        x[2] = __uint_as_float(w.y << 16); x[3] = __uint_as_float(w.y & 0xffff0000u);
+        x[4] = __uint_as_float(w.z << 16); x[5] = __uint_as_float(w.z & 0xffff0000u);
+        x[6] = __uint_as_float(w.w << 16); x[7] = __uint_as_float(w.w & 0xffff0000u);
+    }
+    __device__ static __forceinline__ uint4 minus_inf() { return make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u); }
+    __device__ static __forceinline__ uint4 mask_tail(uint4 w, int keep) { return mask_tail16(w, keep, 0xff80u); }
+    __device__ static __forceinline__ uint4 gather(const uint16_t* p, int left) {
+        uint32_t h[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) h[i] = i < left ? (uint32_t)__ldg(p + i) : 0xff80u;
+        return make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
+    }
 };
-template <> struct SubLoad<f16_t> {
-    __device__ static __forceinline__ float load(const unsigned char* buf, int v0, int v1, float (&x)[2][8]) {
-        const uint4 a = reinterpret_cast<const uint4*>(buf)[v0];
-        const uint4 b = reinterpret_cast<const uint4*>(buf)[v1];
-        const uint32_t pm = max_f16x2(max_f16x2(max_f16x2(a.x, a.y), max_f16x2(a.z, a.w)),
-                                      max_f16x2(max_f16x2(b.x, b.y), max_f16x2(b.z, b.w)));
-        Vec<f16_t>::unpack(a, x[0]);
-        Vec<f16_t>::unpack(b, x[1]);
+template <> struct Words<f16_t> {
+    static constexpr int N = 8;
+    template <int G>
+    __device__ static __forceinline__ float vmax_all(const uint4 (&w)[G]) {   // exact on packed pairs
+        uint32_t pm = max_f16x2(max_f16x2(w[0].x, w[0].y), max_f16x2(w[0].z, w[0].w));
+#pragma unroll
+        for (int j = 1; j < G; ++j) pm = max_f16x2(max_f16x2(pm, w[j].x), max_f16x2(max_f16x2(w[j].y, w[j].z), w[j].w));
         const float2 m = f16x2_to_float2(pm);
         return fmaxf(m.x, m.y);
     }
+    __device__ static __forceinline__ f32x2 widen(uint32_t h) { const float2 v = f16x2_to_float2(h); return pack2(v.x, v.y); }
+    __device__ static __forceinline__ void pairs(uint4 w, f32x2 (&p)[4]) {
+        p[0] = widen(w.x); p[1] = widen(w.y); p[2] = widen(w.z); p[3] = widen(w.w);
+    }
+    __device__ static __forceinline__ void unpack(uint4 w, float (&x)[8]) { Vec<f16_t>::unpack(w, x); }
+    __device__ static __forceinline__ uint4 minus_inf() { return make_uint4(0xfc00fc00u, 0xfc00fc00u, 0xfc00fc00u, 0xfc00fc00u); }
+    __device__ static __forceinline__ uint4 mask_tail(uint4 w, int keep) { return mask_tail16(w, keep, 0xfc00u); }
+    __device__ static __forceinline__ uint4 gather(const f16_t* p, int left) {
+        uint32_t h[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) h[i] = i < left ? (uint32_t)__ldg(&p[i].bits) : 0xfc00u;
+        return make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
+    }
 };
+
+// G vectors of one thread: maximum first, one rescale of the running sums if it grew, then one
+// multiply-add, one exp2 and one addition per entry, the first and the last on pairs.
+template <typename E, int G>
+__device__ __forceinline__ void fold_vectors(const uint4 (&w)[G], float c, RowAcc& a) {
+    constexpr int PN = Words<E>::N / 2;
+    acc_raise(a, Words<E>::template vmax_all<G>(w), c);
+    const f32x2 c2 = pack2(c, c), nmu2 = pack2(-a.mu, -a.mu);
+#pragma unroll
+    for (int j = 0; j < G; ++j) {
+        f32x2 p[PN];
+        Words<E>::pairs(w[j], p);
+#pragma unroll
+        for (int i = 0; i < PN; i += 2) acc_add_pairs(a, p[i], p[i + 1], c2, nmu2);
+    }
+}
 
 // Two 16-byte vectors (indices v0, v1) of a staged row piece holding n valid entries from its
 // start; `full` says that both vectors lie wholly inside the piece.
 template <typename E>
 __device__ __forceinline__ void stats_two_vectors(const unsigned char* buf, int v0, int v1, bool full, int n, float c, RowAcc& a) {
-    constexpr int N = Vec<E>::N;
-    float x[2][N];
-    float cm;
-    if (full) {
-        cm = SubLoad<E>::load(buf, v0, v1, x);
-    } else {  // ragged end: what lies beyond the piece counts as -inf
-        Vec<E>::load(buf, v0, x[0]);
-        Vec<E>::load(buf, v1, x[1]);
-        cm = -INFINITY;
-#pragma unroll
-        for (int i = 0; i < N; ++i) {
-            if (v0 * N + i >= n) x[0][i] = -INFINITY;
-            if (v1 * N + i >= n) x[1][i] = -INFINITY;
-            cm = fmaxf(cm, fmaxf(x[0][i], x[1][i]));
-        }
+    constexpr int N = Words<E>::N;
+    uint4 w[2] = {reinterpret_cast<const uint4*>(buf)[v0], reinterpret_cast<const uint4*>(buf)[v1]};
+    if (!full) {  // ragged end: what lies beyond the piece counts as -inf
+        w[0] = Words<E>::mask_tail(w[0], n - v0 * N);
+        w[1] = Words<E>::mask_tail(w[1], n - v1 * N);
     }
-    acc_raise(a, cm, c);
-    const float nmu = -a.mu;
-#pragma unroll
-    for (int j = 0; j < 2; ++j)
-#pragma unroll
-        for (int i = 0; i < N; ++i) a.s[i & 3] += ex2_approx(__fmaf_rn(x[j][i], c, nmu));
+    fold_vectors<E, 2>(w, c, a);
 }
 
 }  // namespace ears
