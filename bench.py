@@ -535,6 +535,70 @@ def run_series(args):
                       "peak": peak, "peak_kind": peak_kind, "clocks": clocks, "bins": bins}), flush=True)
 
 
+def run_timeline(args):
+    """Where one launch spends its time: builds (if needed) and loads the timeline variant of the
+    library (-DEARS_TRACE, paper_2512_13194_b200/build.py --trace), runs one step of the chosen
+    workload after an L2 flush and prints what the first CTAs recorded at the ends of their phases.
+    Only the cluster kernel (resident and streamed forms) carries marks.  Not the benchmark line."""
+    import ctypes
+
+    import torch
+
+    from paper_2512_13194_b200 import binding, build as ears_build, synth
+
+    lib = binding.load_library(ears_build.build(trace=True))
+    import paper_2512_13194_b200 as ears
+    torch.cuda.set_device(0)
+    w = synth.workload(args.workload)
+    if args.batch:
+        w = w.with_batch(args.batch)
+    t, d, x = synth.make_inputs(w, "cuda:0")
+    beta = w.beta if args.beta is None else args.beta
+    ears.set_path(args.path, args.cluster)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    for i in range(3):
+        ears.verify(t, d, x, w.temperature, beta, w.verify_seed, i)
+    torch.cuda.synchronize()
+    flush.zero_()
+    torch.cuda.synchronize()
+    assert lib.ears_trace_reset() == 0
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    acc, _ = ears.verify(t, d, x, w.temperature, beta, w.verify_seed, 7)
+    e1.record()
+    torch.cuda.synchronize()
+    n_ctas, n_ev = ctypes.c_int(), ctypes.c_int()
+    buf = (ctypes.c_uint64 * (96 * 192 * 2))()
+    counts = (ctypes.c_int * 96)()
+    assert lib.ears_trace_read(buf, counts, ctypes.byref(n_ctas), ctypes.byref(n_ev)) == 0
+    names = {0: "start", 1: "item", 2: "stats", 3: "exchange", 4: "decision", 5: "masses+pick", 6: "exit", 7: "job",
+             10: "unit-chosen", 11: "piece-chosen", 12: "idle-chosen", 13: "exit-chosen", 15: "streamed", 16: "epilogue"}
+    print(f"# {w.name} beta={beta}: {ears.describe_plan(w.dtype, w.B, w.K, w.V)}; event-timed {e0.elapsed_time(e1) * 1e3:.1f} us; "
+          f"rejected sequences {float((acc < w.K).float().mean()):.2f}")
+    ev = {}
+    for c in range(n_ctas.value):
+        ev[c] = [(buf[(c * n_ev.value + i) * 2], buf[(c * n_ev.value + i) * 2 + 1] >> 32, buf[(c * n_ev.value + i) * 2 + 1] & 0xffffffff)
+                 for i in range(min(counts[c], n_ev.value))]
+    t0 = min(e[0][0] for e in ev.values() if e)
+    t_end = max(e[-1][0] for e in ev.values() if e)
+    print(f"# first mark to last mark over the traced CTAs: {(t_end - t0) * 1e-3:.1f} us")
+    # durations of each phase (time since the previous mark of the same CTA), over all traced CTAs
+    dur = {}
+    for c, e in ev.items():
+        for a, b in zip(e[:-1], e[1:]):
+            key = names.get(b[1], str(b[1])) + (" (none)" if b[1] == 5 and a[1] == 4 and (b[0] - a[0]) < 400 else "")
+            dur.setdefault(key, []).append((b[0] - a[0]) * 1e-3)
+    print("| phase (ends with this mark) | count | median us | p10 | p90 | total us per CTA |")
+    print("|---|---|---|---|---|---|")
+    ctas = sum(1 for e in ev.values() if e)
+    for k, v in dur.items():
+        v = sorted(v)
+        print(f"| {k} | {len(v)} | {statistics.median(v):.2f} | {v[len(v) // 10]:.2f} | {v[(9 * len(v)) // 10 - 1 if len(v) > 9 else -1]:.2f} | {sum(v) / ctas:.1f} |")
+    for c in (0, 1, n_ctas.value - 1):
+        if ev.get(c):
+            print(f"CTA {c}: " + " ".join(f"{names.get(tag, tag)}@{(ts - t0) * 1e-3:.1f}" + (f"[{arg}]" if tag in (1, 10) else "") for ts, tag, arg in ev[c][:40]))
+
+
 def run_shard_table(args):
     """One rank's share of the vocabulary-sharded step, phase by phase, on one GPU: this rank's
     columns of every row with the synthetic distributions of the workload, the other ranks'
@@ -635,6 +699,10 @@ def main():
     ap.add_argument("--cpu-sample", type=int, default=512, help="sequences given to the CPU baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sustained", action="store_true", help="skip the appended run under continuous load")
+    ap.add_argument("--timeline", action="store_true", help="print where one launch spends its time (timeline build) instead")
+    ap.add_argument("--path", type=int, default=0, help="with --timeline: force a kernel (ears_set_path)")
+    ap.add_argument("--cluster", type=int, default=0, help="with --timeline: CTAs per cluster")
+    ap.add_argument("--beta", type=float, default=None, help="with --timeline: override the workload's beta")
     ap.add_argument("--series", type=int, default=0,
                     help="instead of the benchmark line: this many steps back to back, kernel time per launch "
                          "binned by the SM clock sampled beside it")
@@ -645,7 +713,9 @@ def main():
                     help="print per-phase times of one rank of the vocabulary-sharded step instead")
     ap.add_argument("--greedy-table", action="store_true", help="print times of the temperature -> 0 form instead")
     args = ap.parse_args()
-    if args.series:
+    if args.timeline:
+        run_timeline(args)
+    elif args.series:
         run_series(args)
     elif args.greedy_table:
         run_greedy_table(args)

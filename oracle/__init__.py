@@ -7,6 +7,8 @@ CPU-baseline leg do.
 from .ears_oracle import (  # noqa: F401
     OracleResult,
     build,
+    entropy,
+    entropy_uncertainty,
     inverse_cdf,
     half_to_double,
     max_threads,

@@ -12,6 +12,10 @@
  *   - temperature softmax of every target and draft row            [Sec. 3.1, 4.3]
  *   - R_i = P_t(x_i) / max(P_d(x_i), eps), eps = 1e-10              [Sec. 3.2 step 2, Sec. 3.3 item 2]
  *   - Uncertainty_i = 1 - max_v P_t(v), Tolerance_i = beta * it     [Sec. 3.2, tolerance equation]
+ *     or, on request, Uncertainty_i = H(P_t) / ln V with H = -sum_v P_t(v) ln P_t(v): the paper
+ *     names "distribution entropy" as a more refined measure [Sec. 5, future work item 1] and gives
+ *     no formula; dividing by ln V (the entropy of the flat distribution over the V entries) is
+ *     this library's reading, chosen so that the measure runs over [0, 1] like the printed one
  *   - accept iff R_i >= max(U_i - Tolerance_i, 0)                   [Sec. 3.2 acceptance condition, Sec. 3.3 item 2]
  *   - direct / pardon / reject classification                       [Sec. 3.2 step 5]
  *   - first rejection ends the accepted prefix                      [Sec. 3.1]
@@ -142,6 +146,24 @@ int ears_oracle_softmax(const double* logits, int V, double T, double* p, double
 }
 
 /*
+ * Shannon entropy (nats) of a distribution p[0..V): H = -sum_v p_v ln p_v, with 0 ln 0 = 0
+ * [Sec. 5 item 1 names it as an uncertainty measure; the definition is the textbook one].
+ */
+double ears_oracle_entropy(const double* p, int V)
+{
+    double H = 0.0;
+    for (int v = 0; v < V; ++v)
+        if (p[v] > 0.0) H -= p[v] * log(p[v]);
+    return H;
+}
+
+/* Uncertainty in [0, 1] from the entropy: H / ln V (0 when V = 1: one entry leaves no doubt). */
+double ears_oracle_entropy_uncertainty(double H, int V)
+{
+    return V > 1 ? H / log((double)V) : 0.0;
+}
+
+/*
  * Inverse-CDF draw from unnormalised masses r[0..V) at uniform u in [0,1):
  * S = sum r, C_j = sum_{v<=j} r_v; the token is the smallest j with u*S < C_j.
  * Zero-mass entries are therefore never chosen.  If rounding leaves u*S >= C_{V-1}
@@ -198,6 +220,7 @@ typedef struct {
     double* cdf_margin;  /* [B]    distance of u to the chosen interval's nearer end */
     int32_t* band_lo;    /* [B]    see ears_oracle_inverse_cdf            */
     int32_t* band_hi;    /* [B]                                           */
+    double* entropy;     /* [B,K]  H(P_t) of target row k, in nats        */
 } ears_oracle_diag;
 
 static void mark_invalid(int b, int K, int32_t* out_accept_len, int32_t* out_tokens)
@@ -207,7 +230,7 @@ static void mark_invalid(int b, int K, int32_t* out_accept_len, int32_t* out_tok
 }
 
 static void verify_one(const void* tl, const void* dl, int dtype, const int32_t* x,
-                       int b, int K, int V, double T, double beta, int stop_at_first_reject,
+                       int b, int K, int V, double T, double beta, int stop_at_first_reject, int uncertainty,
                        uint64_t seed, uint64_t offset, int64_t b_first, double band,
                        int32_t* out_accept_len, int32_t* out_tokens,
                        const ears_oracle_diag* dg,
@@ -230,7 +253,11 @@ static void verify_one(const void* tl, const void* dl, int dtype, const int32_t*
         for (int v = 0; v < V; ++v) if (pt[v] > maxp) maxp = pt[v];
         double pd_safe = pd[tok] > EARS_ORACLE_EPS ? pd[tok] : EARS_ORACLE_EPS; /* Sec. 3.3 item 2 */
         double R = pt[tok] / pd_safe;                        /* Sec. 3.2 step 2 */
-        double tol = beta * (1.0 - maxp);                    /* tolerance equation */
+        double H = 0.0;
+        if (uncertainty == 1 || (dg && dg->entropy)) H = ears_oracle_entropy(pt, V);
+        double unc = uncertainty == 1 ? ears_oracle_entropy_uncertainty(H, V)   /* Sec. 5 item 1 */
+                                      : 1.0 - maxp;                             /* Sec. 3.2 */
+        double tol = beta * unc;                             /* tolerance equation */
         double U = ears_oracle_uniform_accept(seed, offset, gb, k);
         double thr = U - tol > 0.0 ? U - tol : 0.0;          /* Sec. 3.3 item 2, clamp */
         int accept = R >= thr;                               /* acceptance condition */
@@ -242,6 +269,7 @@ static void verify_one(const void* tl, const void* dl, int dtype, const int32_t*
             if (dg->max_pt) dg->max_pt[i] = maxp;
             if (dg->margin) dg->margin[i] = R - thr;
             if (dg->cls) dg->cls[i] = (uint8_t)cls;
+            if (dg->entropy) dg->entropy[i] = H;
         }
         if (!accept && n == K) n = k; /* first rejection; later positions are diagnostics only */
         /* Sec. 3.1: a rejection discards every later draft token, so a caller may ask that their
@@ -301,25 +329,28 @@ static void verify_one(const void* tl, const void* dl, int dtype, const int32_t*
  * seq_temperature, seq_beta: optional [B] arrays that replace the scalars per sequence.
  * stop_at_first_reject != 0: rows and tokens after a sequence's first rejected position (and the
  *   extra target row, unless everything was accepted) are not read: not validated, no diagnostics.
+ * uncertainty: 0 = 1 - max P_t [Sec. 3.2], 1 = H(P_t) / ln V [Sec. 5 item 1, see the header];
+ *   entropy: optional [B,K] output of H(P_t) of every target row that was looked at.
  * Returns 0, -1 on bad arguments, -2 when out of memory.
  */
-int ears_oracle_verify_var(const void* target_logits, const void* draft_logits, int dtype,
+int ears_oracle_verify_unc(const void* target_logits, const void* draft_logits, int dtype,
                            const int32_t* draft_tokens, int B, int K, int V,
                            float temperature, float beta,
                            const float* seq_temperature, const float* seq_beta,
-                           int stop_at_first_reject,
+                           int stop_at_first_reject, int uncertainty,
                            uint64_t seed, uint64_t offset,
                            int64_t b_first, double band,
                            int32_t* out_accept_len, int32_t* out_tokens,
                            double* pt_tok, double* pd_tok, double* max_pt, double* margin,
                            uint8_t* cls, double* resid_mass, double* cdf_margin,
-                           int32_t* band_lo, int32_t* band_hi, int nthreads)
+                           int32_t* band_lo, int32_t* band_hi, double* entropy, int nthreads)
 {
     if (!target_logits || !draft_logits || !draft_tokens || !out_accept_len || !out_tokens) return -1;
     if (B < 1 || K < 1 || V < 1 || (dtype < 0 || dtype > 2)) return -1;
     if (!seq_temperature && (!(temperature > 0.0f) || !isfinite(temperature))) return -1;
     if (!seq_beta && (!(beta >= 0.0f) || !isfinite(beta))) return -1;
-    ears_oracle_diag dg = { pt_tok, pd_tok, max_pt, margin, cls, resid_mass, cdf_margin, band_lo, band_hi };
+    if (uncertainty != 0 && uncertainty != 1) return -1;
+    ears_oracle_diag dg = { pt_tok, pd_tok, max_pt, margin, cls, resid_mass, cdf_margin, band_lo, band_hi, entropy };
     if (nthreads < 1) nthreads = 1;
     int failed = 0;
 #ifdef _OPENMP
@@ -351,11 +382,31 @@ int ears_oracle_verify_var(const void* target_logits, const void* draft_logits, 
                 continue;
             }
             verify_one(target_logits, draft_logits, dtype, draft_tokens, b, K, V, (double)Tb, (double)bb,
-                       stop_at_first_reject, seed, offset, b_first, band, out_accept_len, out_tokens, &dg, row, pt, pd);
+                       stop_at_first_reject, uncertainty, seed, offset, b_first, band, out_accept_len, out_tokens, &dg,
+                       row, pt, pd);
         }
         free(row); free(pt); free(pd);
     }
     return failed ? -2 : 0;
+}
+
+/* The step with the uncertainty measure the paper prints (1 - max P_t). */
+int ears_oracle_verify_var(const void* target_logits, const void* draft_logits, int dtype,
+                           const int32_t* draft_tokens, int B, int K, int V,
+                           float temperature, float beta,
+                           const float* seq_temperature, const float* seq_beta,
+                           int stop_at_first_reject,
+                           uint64_t seed, uint64_t offset,
+                           int64_t b_first, double band,
+                           int32_t* out_accept_len, int32_t* out_tokens,
+                           double* pt_tok, double* pd_tok, double* max_pt, double* margin,
+                           uint8_t* cls, double* resid_mass, double* cdf_margin,
+                           int32_t* band_lo, int32_t* band_hi, int nthreads)
+{
+    return ears_oracle_verify_unc(target_logits, draft_logits, dtype, draft_tokens, B, K, V, temperature, beta,
+                                  seq_temperature, seq_beta, stop_at_first_reject, 0, seed, offset, b_first, band,
+                                  out_accept_len, out_tokens, pt_tok, pd_tok, max_pt, margin, cls, resid_mass,
+                                  cdf_margin, band_lo, band_hi, NULL, nthreads);
 }
 
 /* The same with one temperature and one beta for the whole batch. */

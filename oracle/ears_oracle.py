@@ -57,6 +57,15 @@ def _load():
          c.c_float, c.c_float, c.c_void_p, c.c_void_p, c.c_int, c.c_uint64, c.c_uint64, c.c_int64, c.c_double]
         + [c.c_void_p] * 11 + [c.c_int])
     lib.ears_oracle_verify_var.restype = c.c_int
+    lib.ears_oracle_verify_unc.argtypes = (
+        [c.c_void_p, c.c_void_p, c.c_int, c.c_void_p, c.c_int, c.c_int, c.c_int,
+         c.c_float, c.c_float, c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_uint64, c.c_uint64, c.c_int64, c.c_double]
+        + [c.c_void_p] * 12 + [c.c_int])
+    lib.ears_oracle_verify_unc.restype = c.c_int
+    lib.ears_oracle_entropy.argtypes = [c.c_void_p, c.c_int]
+    lib.ears_oracle_entropy.restype = c.c_double
+    lib.ears_oracle_entropy_uncertainty.argtypes = [c.c_double, c.c_int]
+    lib.ears_oracle_entropy_uncertainty.restype = c.c_double
     lib.ears_oracle_verify_greedy.argtypes = [c.c_void_p, c.c_int, c.c_void_p, c.c_int, c.c_int, c.c_int,
                                               c.c_void_p, c.c_void_p, c.c_void_p]
     lib.ears_oracle_verify_greedy.restype = c.c_int
@@ -141,6 +150,16 @@ def inverse_cdf(r, u: float, band: float = 1e-6):
                 band_lo=blo.value, band_hi=bhi.value)
 
 
+def entropy(p) -> float:
+    """Shannon entropy (nats) of a distribution."""
+    p = np.ascontiguousarray(p, dtype=np.float64)
+    return float(_load().ears_oracle_entropy(p.ctypes.data, p.size))
+
+
+def entropy_uncertainty(H: float, V: int) -> float:
+    return float(_load().ears_oracle_entropy_uncertainty(float(H), int(V)))
+
+
 def row_softmax(logits, row_index: int, V: int, temperature: float):
     lib = _load()
     a, code = _as_logits(logits)
@@ -173,14 +192,17 @@ class OracleResult:
     cdf_margin: np.ndarray   # [B]
     band_lo: np.ndarray      # [B] int32
     band_hi: np.ndarray      # [B] int32
+    entropy: np.ndarray = None   # [B,K] H(P_t) in nats, when asked for
 
 
 def verify(target_logits, draft_logits, draft_tokens, temperature: float, beta: float,
            seed: int = 0, offset: int = 0, b_first: int = 0, band: float = 1e-6,
            nthreads: int = 1, seq_temperature=None, seq_beta=None,
-           stop_at_first_reject: bool = False) -> OracleResult:
+           stop_at_first_reject: bool = False, uncertainty: str = "maxprob", want_entropy: bool = False) -> OracleResult:
     """seq_temperature / seq_beta: optional [B] float32 arrays replacing the scalars per sequence.
-    stop_at_first_reject: rows after a sequence's first rejection are not read (nor validated)."""
+    stop_at_first_reject: rows after a sequence's first rejection are not read (nor validated).
+    uncertainty: "maxprob" (1 - max P_t, Sec. 3.2) or "entropy" (H(P_t) / ln V, Sec. 5 item 1).
+    want_entropy: also report H(P_t) per position (always reported with uncertainty="entropy")."""
     lib = _load()
     t, ct = _as_logits(target_logits)
     d, cd = _as_logits(draft_logits)
@@ -200,15 +222,19 @@ def verify(target_logits, draft_logits, draft_tokens, temperature: float, beta: 
     sb = None if seq_beta is None else np.ascontiguousarray(np.asarray(seq_beta, dtype=np.float32))
     if (st is not None and st.shape != (B,)) or (sb is not None and sb.shape != (B,)):
         raise ValueError("per-sequence arrays must have shape [B]")
-    rc = lib.ears_oracle_verify_var(
+    mode = {"maxprob": 0, "entropy": 1}[uncertainty]
+    if mode == 1 or want_entropy:
+        res.entropy = f(B, K)
+    rc = lib.ears_oracle_verify_unc(
         t.ctypes.data, d.ctypes.data, ct, x.ctypes.data, B, K, V,
         float(temperature), float(beta), None if st is None else st.ctypes.data,
-        None if sb is None else sb.ctypes.data, int(bool(stop_at_first_reject)),
+        None if sb is None else sb.ctypes.data, int(bool(stop_at_first_reject)), mode,
         int(seed), int(offset), int(b_first), float(band),
         acc.ctypes.data, tok.ctypes.data, res.pt_tok.ctypes.data, res.pd_tok.ctypes.data,
         res.max_pt.ctypes.data, res.margin.ctypes.data, res.cls.ctypes.data,
         res.resid_mass.ctypes.data, res.cdf_margin.ctypes.data,
-        res.band_lo.ctypes.data, res.band_hi.ctypes.data, int(nthreads))
+        res.band_lo.ctypes.data, res.band_hi.ctypes.data,
+        None if res.entropy is None else res.entropy.ctypes.data, int(nthreads))
     if rc:
         raise ValueError(f"ears_oracle_verify rejected its arguments (rc={rc})")
     return res

@@ -32,16 +32,24 @@ def is_stale() -> bool:
     return any(os.path.getmtime(s) > t for s in sources())
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not is_stale():
-        return LIB
+TRACE_LIB = os.path.join(HERE, "libears_trace.so")
+
+
+def build(force: bool = False, verbose: bool = False, trace: bool = False) -> str:
+    """trace=True builds the timeline variant (-DEARS_TRACE: the kernels record the ends of their
+    phases, see bench.py --timeline) next to the ordinary library, which it never replaces."""
+    out = TRACE_LIB if trace else LIB
+    if not force and os.path.exists(out) and all(os.path.getmtime(s) <= os.path.getmtime(out) for s in sources()):
+        return out
     cmd = [_nvcc()] + NVCC_FLAGS
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += ["-o", LIB, os.path.join(CSRC, "ears_api.cu")]
+    if trace:
+        cmd += ["-DEARS_TRACE"]
+    cmd += ["-o", out, os.path.join(CSRC, "ears_api.cu")]
     subprocess.run(cmd, check=True)
-    return LIB
+    return out
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, trace="--trace" in sys.argv))

@@ -19,6 +19,7 @@
 #include "ears_greedy.cuh"
 #include "ears_direct.cuh"
 #include "ears_shard.cuh"
+#include "ears_cstream.cuh"
 
 namespace {
 
@@ -61,6 +62,7 @@ PlanOverride override_from_env() {
         if (!strcmp(e, "streaming") || !strcmp(e, "1")) ov.path = 1;
         else if (!strcmp(e, "resident") || !strcmp(e, "2")) ov.path = 2;
         else if (!strcmp(e, "direct") || !strcmp(e, "3")) ov.path = 3;
+        else if (!strcmp(e, "cluster-streamed") || !strcmp(e, "4")) ov.path = 4;
     }
     if (const char* e = getenv("EARS_CLUSTER")) {
         const int c = atoi(e);
@@ -202,7 +204,7 @@ Layout make_layout(int B, int K, int V, int parts1) {
 }
 
 // ---- the resident path: one position's rows held in the shared memory of a cluster ----
-struct RPlan { bool ok = false; int C = 0, slice = 0, buf_bytes = 0; size_t smem = 0; bool roomy = false; };
+struct RPlan { bool ok = false; int C = 0, slice = 0, buf_bytes = 0; size_t smem = 0; bool roomy = false; bool streamed = false; };
 
 size_t resident_smem(int buf_bytes) { return ((sizeof(RSmem) + 127) & ~size_t(127)) + 2 * (size_t)buf_bytes + 128; }
 
@@ -228,18 +230,63 @@ RPlan make_rplan(int B, int K, int V, int esize, int sms, int max_cluster, int f
     return best;
 }
 
-struct RLayout { size_t heads, ticket, counters_bytes, flag, cand, cand_mass, pt_tok, pd_tok, max_pt, cls, resid, total; };
+// The streamed form of the cluster kernel: nothing is staged, a CTA only keeps the segment sums of
+// its slice (8 bytes per 256 entries).  The cluster size is the one a small model of the launch
+// likes best: clusters pull positions from a queue, so the kernel takes
+// rounds x (time to stream a position + its exchange, decision and report), where the CTAs that are
+// active share the memory bandwidth and at least two rounds' worth of them hide each other's waits.
+constexpr size_t kStreamedSegBytes = 48 * 1024;   // segment sums of a slice: at most this much shared memory
+
+// bytes behind CSmem: a job's sums per 256 entries, or the extra row's per 2 KB (the larger of the two)
+size_t streamed_area(int slice) {
+    const size_t job = (size_t)(slice / kSegElems) * sizeof(double);
+    const size_t bonus = ((size_t)slice * 2 / kBonusSegBytes + kCBonusPad) * sizeof(BonusSeg);   // 2-byte entries give the fewest, 4-byte: slice * 4
+    const size_t bonus4 = ((size_t)slice * 4 / kBonusSegBytes + kCBonusPad) * sizeof(BonusSeg);
+    return std::max(job, std::max(bonus, bonus4));
+}
+size_t streamed_smem(int slice) { return ((sizeof(CSmem) + 127) & ~size_t(127)) + streamed_area(slice) + 128; }
+
+RPlan make_splan(int B, int K, int V, int esize, int sms, int max_cluster, int forced_cluster, bool ordered) {
+    RPlan best;
+    double best_t = 0.0;
+    const long long items = ordered ? (long long)B : (long long)B * (K + 1);
+    const double item_bytes = 2.0 * V * esize;
+    for (int C = 1; C <= max_cluster; C *= 2) {
+        if (forced_cluster > 0 && C != forced_cluster) continue;
+        const int slice = (int)align_up((size_t)((V + C - 1) / C), kCSliceAlign);
+        if (streamed_area(slice) > kStreamedSegBytes) continue;
+        const long long resident = std::max<long long>(1, (long long)kCCtasPerSm * sms / C);
+        const long long clusters = std::min(items, resident);
+        const long long rounds = (items + clusters - 1) / clusters;
+        // per position: its bytes at the share of ~6.5 TB/s that the active CTAs leave it, but no faster than
+        // one CTA can pull on its own (~60 GB/s), plus ~2.5 us of exchange, decision and report
+        const double share = 6.5e12 / (double)(clusters * C);
+        const double t_item = item_bytes / C / std::min(share, 60e9) + 2.5e-6;
+        const double t = rounds * t_item * (ordered ? K + 1 : 1);   // walking a sequence in order: up to K+1 positions in a row
+        if (!best.ok || t < best_t) {
+            best.ok = true; best.C = C; best.slice = slice; best.buf_bytes = 0; best.smem = streamed_smem(slice);
+            best.roomy = true; best.streamed = true;
+            best_t = t;
+        }
+    }
+    return best;
+}
+
+struct RLayout { size_t heads, ticket, seqmask, counters_bytes, flag, cand, cand_mass, rowstat, pt_tok, pd_tok, max_pt, cls, resid, total; };
 
 RLayout make_rlayout(int B, int K) {
     RLayout L;
     size_t o = 0;
     L.heads = o; o += 32;   // the status word is heads[2] of any workspace
     L.ticket = o; o += (size_t)B * 4;
+    o = align_up(o, 8);
+    L.seqmask = o; o += (size_t)B * 8;
     L.counters_bytes = o;
     o = align_up(o, 256);
     L.flag = o; o = align_up(o + (size_t)B * (K + 1), 256);
     L.cand = o; o = align_up(o + (size_t)B * (K + 1) * 4, 256);
     L.cand_mass = o; o = align_up(o + (size_t)B * (K + 1) * 8, 256);
+    L.rowstat = o; o = align_up(o + (size_t)B * (K + 1) * 16, 256);
     L.pt_tok = o; o = align_up(o + (size_t)B * K * 8, 256);
     L.pd_tok = o; o = align_up(o + (size_t)B * K * 8, 256);
     L.max_pt = o; o = align_up(o + (size_t)B * K * 8, 256);
@@ -311,7 +358,20 @@ int profile_mark(cudaStream_t stream, bool timed) {
 }
 
 template <typename E>
+int set_attrs_streamed(bool* cluster16) {
+    EARS_CUDA(cudaFuncSetAttribute(ears_cstream_kernel<E>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)(streamed_smem(0) + kStreamedSegBytes)));
+    if (cudaFuncSetAttribute(ears_cstream_kernel<E>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
+        (void)cudaGetLastError();
+        *cluster16 = false;
+    }
+    return EARS_OK;
+}
+
+template <typename E>
 int set_attrs(bool* cluster16) {
+    int rc = set_attrs_streamed<E>(cluster16);
+    if (rc) return rc;
     EARS_CUDA(cudaFuncSetAttribute(ears_verify_kernel<E, kStages, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)smem_bytes()));
     EARS_CUDA(cudaFuncSetAttribute(ears_verify_kernel<E, kStages, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -332,7 +392,7 @@ int set_attrs(bool* cluster16) {
 // How many clusters of this shape the device can hold at once (cached per device).
 template <typename E>
 int resident_clusters(DeviceInfo* di, const RPlan& rp, int dtype, int* out) {
-    const std::pair<int, int> key(rp.C * 8 + dtype, (int)rp.smem);
+    const std::pair<int, int> key(rp.C * 16 + dtype * 2 + (rp.streamed ? 1 : 0), (int)rp.smem);
     {
         std::lock_guard<std::mutex> lock(g_mutex);
         auto it = di->clusters.find(key);
@@ -340,7 +400,7 @@ int resident_clusters(DeviceInfo* di, const RPlan& rp, int dtype, int* out) {
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(rp.C * di->sms), 1, 1);
-    cfg.blockDim = dim3(kRThreads, 1, 1);
+    cfg.blockDim = dim3(rp.streamed ? kCThreads : kRThreads, 1, 1);
     cfg.dynamicSmemBytes = rp.smem;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -348,7 +408,9 @@ int resident_clusters(DeviceInfo* di, const RPlan& rp, int dtype, int* out) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, ears_resident_kernel<E>, &cfg) != cudaSuccess) {
+    const cudaError_t qe = rp.streamed ? cudaOccupancyMaxActiveClusters(&n, ears_cstream_kernel<E>, &cfg)
+                                       : cudaOccupancyMaxActiveClusters(&n, ears_resident_kernel<E>, &cfg);
+    if (qe != cudaSuccess) {
         (void)cudaGetLastError();
         n = 0;
     }
@@ -364,7 +426,7 @@ int launch_resident(RParams& p, const RPlan& rp, int max_clusters, cudaStream_t 
     p.n_clusters = (int)(items < max_clusters ? items : max_clusters);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(p.n_clusters * rp.C), 1, 1);
-    cfg.blockDim = dim3(kRThreads, 1, 1);
+    cfg.blockDim = dim3(rp.streamed ? kCThreads : kRThreads, 1, 1);
     cfg.dynamicSmemBytes = rp.smem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -375,7 +437,8 @@ int launch_resident(RParams& p, const RPlan& rp, int max_clusters, cudaStream_t 
     const bool timed = profile_wanted();
     int rc = profile_mark(stream, timed);
     if (rc) return rc;
-    EARS_CUDA(cudaLaunchKernelEx(&cfg, ears_resident_kernel<E>, p));
+    if (rp.streamed) EARS_CUDA(cudaLaunchKernelEx(&cfg, ears_cstream_kernel<E>, p));
+    else EARS_CUDA(cudaLaunchKernelEx(&cfg, ears_resident_kernel<E>, p));
     return profile_mark(stream, timed);
 }
 
@@ -479,13 +542,27 @@ int pick_counters(void* caller_ws, int dev, void* stream_, int kind, size_t coun
 }
 
 // The resident plan for this shape, if its rows fit a cluster and the device can hold one.
-int choose_resident(int dtype, int B, int K, int V, DeviceInfo* di, const PlanOverride& ov, RPlan* rp, int* max_clusters) {
+int choose_resident(int dtype, int B, int K, int V, bool ordered, DeviceInfo* di, const PlanOverride& ov, RPlan* rp,
+                    int* max_clusters) {
     *rp = RPlan();
     *max_clusters = 0;
     if (ov.path == 1 || ov.path == 3 || ov.parts1 != 0) return EARS_OK;
     const int esize = dtype_size(dtype);
-    *rp = make_rplan(B, K, V, esize, di->sms, di->cluster16 ? kRMaxCluster : 8, ov.cluster);
-    if (rp->ok && ov.path == 0) {
+    if (ov.path == 4) *rp = make_splan(B, K, V, esize, di->sms, di->cluster16 ? kRMaxCluster : 8, ov.cluster, ordered);
+    else *rp = make_rplan(B, K, V, esize, di->sms, di->cluster16 ? kRMaxCluster : 8, ov.cluster);
+    if (ov.path == 0 && ordered && B >= 4 * di->sms) {
+        // Asked to leave out what follows a first rejection, and enough sequences to give every SM
+        // four clusters of its own (fewer leave the last round half empty): clusters that stream walk one sequence each and read nothing after
+        // its first rejection, where the other streaming kernels read every row and discard.  (Rows
+        // short enough to stay in shared memory keep the resident kernel, which does the same.)
+        const long long items = (long long)B * (K + 1);
+        const bool resident_takes_it = rp->ok && items <= (!rp->roomy ? 64 : (rp->C >= 8 ? 256 : 3072));
+        if (!resident_takes_it) {
+            const RPlan sp = make_splan(B, K, V, esize, di->sms, di->cluster16 ? kRMaxCluster : 8, ov.cluster, true);
+            if (sp.ok) *rp = sp;
+        }
+    }
+    if (rp->ok && ov.path == 0 && !rp->streamed) {
         // Holding rows in shared memory costs a few microseconds of latency per position that
         // nothing else in that CTA can hide.  It wins when rows are short (a cluster of at most
         // four CTAs holds a pair) and when there are few positions, where the streaming kernel's
@@ -504,7 +581,7 @@ int choose_resident(int dtype, int B, int K, int V, DeviceInfo* di, const PlanOv
         if (rc) return rc;
         if (*max_clusters < 1) rp->ok = false;
     }
-    if (!rp->ok && ov.path == 2) return EARS_ERR_SHAPE;   // the forced path cannot take this shape
+    if (!rp->ok && (ov.path == 2 || ov.path == 4)) return EARS_ERR_SHAPE;   // the forced path cannot take this shape
     return EARS_OK;
 }
 
@@ -577,7 +654,7 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
     // Rows small enough to stay in a cluster's shared memory take the resident path.
     RPlan rp;
     int max_clusters = 0;
-    rc = choose_resident(dtype, B, K, V, di, ov, &rp, &max_clusters);
+    rc = choose_resident(dtype, B, K, V, stop_first != 0, di, ov, &rp, &max_clusters);
     if (rc) return rc;
     if (rp.ok) {
         const RLayout L = make_rlayout(B, K);
@@ -604,6 +681,8 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
         p.flag = (signed char*)(w + L.flag);
         p.cand = (int32_t*)(w + L.cand);
         p.cand_mass = (double*)(w + L.cand_mass);
+        p.rowstat = (float4*)(w + L.rowstat);
+        p.seqmask = (unsigned long long*)(cw + L.seqmask);
         p.C = rp.C; p.slice = rp.slice; p.buf_bytes = rp.buf_bytes;
         p.use_tma = aligned && ov.loader != 2;
         p.n_clusters = 0;
@@ -1047,17 +1126,19 @@ int ears_describe_plan(int dtype, int B, int K, int V, char* out, size_t out_byt
     }
     RPlan rp;
     int max_clusters = 0;
-    rc = choose_resident(dtype, B, K, V, di, ov, &rp, &max_clusters);
+    rc = choose_resident(dtype, B, K, V, false, di, ov, &rp, &max_clusters);
     if (rc) return rc;
     const int esize = dtype_size(dtype);
     if (rp.ok) {
         const long long items = (long long)B * (K + 1);
         int per_sm = 0;
         by_dtype(dtype, [&](auto* e) {
-            return (int)cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ears_resident_kernel<std::remove_pointer_t<decltype(e)>>,
-                                                                      kRThreads, rp.smem);
+            using El = std::remove_pointer_t<decltype(e)>;
+            return rp.streamed ? (int)cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ears_cstream_kernel<El>, kCThreads, rp.smem)
+                               : (int)cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ears_resident_kernel<El>, kRThreads, rp.smem);
         });
-        snprintf(out, out_bytes, "resident: cluster=%d slice_elems=%d smem_bytes=%zu ctas_per_sm=%d clusters_resident=%d clusters_launched=%lld",
+        snprintf(out, out_bytes, rp.streamed ? "cluster-streamed: cluster=%d slice_elems=%d smem_bytes=%zu ctas_per_sm=%d clusters_resident=%d clusters_launched=%lld" :
+                 "resident: cluster=%d slice_elems=%d smem_bytes=%zu ctas_per_sm=%d clusters_resident=%d clusters_launched=%lld",
                  rp.C, rp.slice, rp.smem, per_sm, max_clusters, items < max_clusters ? items : (long long)max_clusters);
     } else {
         const bool direct = use_direct(ov, esize, V, (long long)B * (K + 1));
@@ -1076,7 +1157,7 @@ int ears_describe_plan(int dtype, int B, int K, int V, char* out, size_t out_byt
 }
 
 int ears_set_path(int path, int cluster) {
-    if (path < 0 || path > 3) return EARS_ERR_PARAM;
+    if (path < 0 || path > 4) return EARS_ERR_PARAM;
     if (cluster != 0 && cluster != 1 && cluster != 2 && cluster != 4 && cluster != 8 && cluster != 16) return EARS_ERR_PARAM;
     std::lock_guard<std::mutex> lock(g_mutex);
     g_override.path = path;
@@ -1234,6 +1315,24 @@ int ears_shard_pick(int dtype, const void* target_shard, const void* draft_shard
     if (e != cudaSuccess) return cuda_fail(e, "ears_shard_pick_kernel launch");
     return EARS_OK;
 }
+
+#ifdef EARS_TRACE
+// Timeline build only (not part of the public header): clears, then reads back, what the kernels' marks recorded.
+int ears_trace_reset(void) {
+    static int zeros[kTraceCtas];
+    EARS_CUDA(cudaMemcpyToSymbol(g_trace_n, zeros, sizeof zeros));
+    return EARS_OK;
+}
+// out: [kTraceCtas][kTraceEvents][2] 64-bit words (time in ns; tag << 32 | argument); counts: [kTraceCtas]
+int ears_trace_read(unsigned long long* out, int* counts, int* n_ctas, int* n_events) {
+    EARS_CUDA(cudaDeviceSynchronize());
+    EARS_CUDA(cudaMemcpyFromSymbol(out, g_trace, sizeof(unsigned long long) * kTraceCtas * kTraceEvents * 2));
+    EARS_CUDA(cudaMemcpyFromSymbol(counts, g_trace_n, sizeof(int) * kTraceCtas));
+    *n_ctas = kTraceCtas;
+    *n_events = kTraceEvents;
+    return EARS_OK;
+}
+#endif
 
 const char* ears_last_cuda_error(void) { return g_cuda_error; }
 

@@ -1,0 +1,553 @@
+// The verification step with thread-block clusters that stream their rows: nothing is staged.
+//
+// Work item = one position of one sequence, as in the resident kernel: the pair (target row k,
+// draft row k), or the extra target row K.  A cluster of C CTAs takes an item from a queue; CTA j
+// owns the j-th slice of the row(s) and reads it straight from global memory through registers:
+//
+//   1. softmax statistics (max, sum exp2) of the slices [Sec. 3.1]; for the extra row the sums of
+//      2 KB segments are kept in shared memory as well, so that a bonus token needs no second read;
+//   2. the partial results, the cluster's next queue entry and any pending second-pass job travel
+//      through distributed shared memory (remote stores plus a remote mbarrier arrive per peer);
+//   3. every CTA takes the decision of Sec. 3.2 (guards of Sec. 3.3 item 2) from identical numbers;
+//   4. the extra row draws its bonus token at once from the segment sums of step 1;
+//   5. one CTA reports the item in a per-sequence word of decided / accepted positions.  The report
+//      that settles the sequence's first rejection [Sec. 3.1] (every earlier position accepted) leaves
+//      a job: the two rows of that one position are read a second time -- by this cluster, in its
+//      next round, while they are still in L2 -- for the masses max(0, P_t - P_d) and the
+//      inverse-CDF pick.  Whoever reports last (an item or the job) writes the sequence's outputs.
+//
+// So every logit crosses HBM once for the statistics, and per sequence at most one pair of rows is
+// read again (usually from L2).  A rejected position that is not the sequence's first costs nothing.
+// There is no global queue of second-pass work, no publication and no hand-over between clusters; a
+// cluster never waits for another cluster.  Without a shared-memory footprint several clusters share
+// an SM and hide each other's exchanges.  Ordered mode (EARS_FLAG_STOP_AT_FIRST_REJECT): the queue
+// holds sequences, a cluster walks one position by position and stops at its first rejection, whose
+// masses it computes at once; rows after it are never read.
+#pragma once
+#include "ears_common.cuh"
+#include "ears_math.cuh"
+#include "ears_philox.cuh"
+#include "ears_pipeline.cuh"
+#include "ears_kernel.cuh"     // pick_in_range
+#include "ears_direct.cuh"     // stream_piece, stream_bonus_piece, stream_job_piece
+#include "ears_resident.cuh"   // RParams, cluster primitives
+
+namespace ears {
+
+constexpr int kCWarps = kDWarps;          // the streaming helpers stride over this many warps
+constexpr int kCThreads = kCWarps * 32;
+constexpr int kCSliceAlign = 1024;        // slices are whole 2 KB segments of 2-byte entries (and of 4-byte ones)
+constexpr int kCBonusPad = 8;             // stream_bonus_piece may clear up to this many entries past the last segment
+#ifndef EARS_C_CTAS
+#define EARS_C_CTAS 3
+#endif
+constexpr int kCCtasPerSm = EARS_C_CTAS;  // no shared-memory footprint to speak of: registers set the limit
+
+struct CSmem {
+    alignas(8) uint64_t xbar[2];          // statistics exchange, alternating by round
+    uint64_t mbar2[2];                    // mass-total exchange, alternating by mass round
+    alignas(16) float4 xstat[2][kRMaxCluster * kCWarps];   // (m_t, s_t, m_d, s_d) of every warp of every peer
+    double xmass[2][kRMaxCluster];        // mass totals of every peer
+    int xnext[2];                         // next queue entry of the cluster (written by rank 0)
+    int2 xjob[2][kRMaxCluster];           // second-pass job each peer announces: (sequence, position) or (-1, 0)
+    int my_job_b, my_job_n;               // job this CTA will announce with the next exchange
+    float2 rs_t, rs_d;                    // (max, Z) of the item's rows
+    int dec;                              // 1 accept / row usable, 0 reject, -1 invalid
+    int pick_rank;                        // CTA that holds u*S (-1: no mass anywhere)
+    double pick_tin, pick_S;
+    int abort_flag;
+};
+
+__device__ __forceinline__ void peer_store(uint32_t addr, int2 v) {
+    asm volatile("st.shared::cluster.v2.s32 [%0], {%1, %2};" ::"r"(addr), "r"(v.x), "r"(v.y) : "memory");
+}
+
+// A segment sum of the extra row, taken relative to mu, brought to the row's own maximum (mc = m c,
+// exact in fp64).  Out of line: the fp64 exp2 would otherwise weigh on the registers of every loop around it.
+__device__ __noinline__ double bonus_sum_at_row_maximum(double sum, float mu, double mc) {
+    return sum > 0.0 ? sum * exp2((double)mu - mc) : 0.0;
+}
+
+// Cluster-wide inverse-CDF pick.  Every CTA holds `nseg` non-negative sums val(g) (fp64) over
+// consecutive segments of `seg_elems` entries of its slice, CTAs in slice order.  Totals are
+// exchanged through distributed shared memory; every CTA locates the CTA that holds u * S, that CTA
+// locates the segment and reads its entries again for the token.  All threads of all CTAs call it.
+// -> false if a wait gave up.  token: valid in warp 0 of the CTA sm.pick_rank (-1 elsewhere).
+template <typename E, typename ValFn>
+__device__ __forceinline__ bool cluster_pick(CSmem& sm, const RParams& p, ValFn val, int nseg, int seg_elems, int b, bool resid,
+                                             const E* trow, const E* drow, const RowNorm& rn, float cb, int e0, int n,
+                                             int rank, int C, int& mround, int& token) {
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int mpar = mround & 1;
+    const int per = (nseg + 31) / 32;
+    const int g0 = min(nseg, lane * per), g1 = min(nseg, g0 + per);
+    double loc = 0.0, inc = 0.0;
+    token = -1;
+    if (warp == 0) {
+        for (int g = g0; g < g1; ++g) loc += val(g);
+        inc = warp_inclusive_scan(loc, lane);
+        const double total = __shfl_sync(0xffffffffu, inc, 31);
+        if (lane < C) {
+            peer_store(map_to_peer(smem_u32(&sm.xmass[mpar][rank]), (uint32_t)lane), total);
+            peer_arrive(map_to_peer(smem_u32(&sm.mbar2[mpar]), (uint32_t)lane));
+        }
+    }
+    const bool ok = mbar_wait_cluster(&sm.mbar2[mpar], (uint32_t)(mround >> 1) & 1u, &sm.abort_flag);
+    ++mround;
+    if (ok && tid == 0) {
+        const double u = uniform_final(p.seed, p.offset, (uint32_t)(p.b_first + b), (uint32_t)p.K);
+        double S = 0.0;
+        for (int i = 0; i < C; ++i) S += sm.xmass[mpar][i];
+        const double target = u * S;
+        double cum = 0.0, before = 0.0, before_last = 0.0;
+        int pick = -1, last = -1;
+        for (int i = 0; i < C && pick < 0; ++i) {
+            const double m_i = sm.xmass[mpar][i];
+            if (m_i > 0.0) {
+                last = i;
+                before_last = cum;
+                if (target < cum + m_i) { pick = i; before = cum; }
+            }
+            cum += m_i;
+        }
+        if (pick < 0) { pick = last; before = before_last; }
+        sm.pick_rank = pick;
+        sm.pick_tin = target - before;
+        sm.pick_S = S;
+    }
+    if (__syncthreads_or(ok ? 0 : 1)) return false;
+    // a rejection implies residual mass; if rounding erased it the caller draws from P_t instead
+    if (resid && !(sm.pick_S * rn.izt >= kTinyMass)) return true;
+    if (rank == sm.pick_rank && warp == 0) {
+        const double tin = sm.pick_tin;
+        const unsigned hit = __ballot_sync(0xffffffffu, tin < inc && loc > 0.0);
+        const unsigned pos = __ballot_sync(0xffffffffu, loc > 0.0);
+        if (pos) {
+            const int L = hit ? __ffs(hit) - 1 : 31 - __clz(pos);
+            int seg = -1, lastseg = -1;
+            double before = 0.0, before_last = 0.0;
+            if (lane == L) {
+                double run = inc - loc;
+                for (int g = g0; g < g1 && seg < 0; ++g) {
+                    const double v = val(g);
+                    if (v > 0.0) {
+                        lastseg = g;
+                        before_last = run;
+                        if (tin < run + v) { seg = g; before = run; }
+                    }
+                    run += v;
+                }
+                if (seg < 0) { seg = lastseg; before = before_last; }
+            }
+            seg = __shfl_sync(0xffffffffu, seg, L);
+            before = __shfl_sync(0xffffffffu, before, L);
+            if (seg >= 0)
+                token = pick_in_range<E>(trow, drow, resid, rn, cb, e0 + seg * seg_elems, min(seg_elems, n - seg * seg_elems),
+                                         tin - before, p.V, lane);
+        }
+    }
+    return true;
+}
+
+// First rejection that a word of decided (low 32 bits) and accepted (high 32 bits) positions settles:
+// the lowest rejected position, provided every position before it has been decided (then they were
+// all accepted); -1 while that is open or when nothing decided so far was rejected.
+__device__ __forceinline__ int settled_first_rejection(unsigned long long m, int K) {
+    const uint32_t decided = (uint32_t)m, accepted = (uint32_t)(m >> 32);
+    const uint32_t rej = decided & ~accepted & ((1u << K) - 1u);
+    if (!rej) return -1;
+    const int n = __ffs(rej) - 1;
+    const uint32_t below = (1u << n) - 1u;
+    return (decided & below) == below ? n : -1;
+}
+
+// Called by one warp once everything of sequence b is in: first rejection [Sec. 3.1], the accepted
+// prefix and the token drawn at that position (or the bonus token).  With job_pending the slot of a
+// rejected position is left to the second-pass job that is yet to run (K > 30 only).
+// -> n in [0, K], or -1 for an invalid sequence.
+__device__ __forceinline__ int finish_streamed_sequence(const RParams& p, int b, int lane, bool job_pending) {
+    const int K = p.K;
+    const signed char* fl = p.flag + (size_t)b * (K + 1);
+    int first_reject = K;
+    bool bad = false;
+    for (int k0 = 0; k0 <= K; k0 += 32) {
+        const int k = k0 + lane;
+        int f = 1;
+        if (k <= K) f = *reinterpret_cast<const volatile signed char*>(fl + k);
+        if (f < 0) bad = true;
+        const unsigned rej = __ballot_sync(0xffffffffu, k < K && f == 0);
+        if (rej != 0 && first_reject == K) first_reject = k0 + __ffs(rej) - 1;
+    }
+    bad = __any_sync(0xffffffffu, bad);
+    int32_t* ot = p.out_tok + (size_t)b * (K + 1);
+    if (bad) {
+        for (int q = lane; q <= K; q += 32) ot[q] = -1;
+        if (lane == 0) {
+            p.out_len[b] = -1;
+            atomicOr(&p.heads[2], kDevInvalidInput);
+        }
+        return -1;
+    }
+    const int n = first_reject;
+    const bool mine = n == K || !job_pending;   // the slot n is filled here
+    for (int q = lane; q <= K; q += 32) {
+        if (q < n) ot[q] = p.x[(size_t)b * K + q];
+        else if (q > n) ot[q] = -1;
+        else if (mine) ot[q] = __ldcg(p.cand + (size_t)b * (K + 1) + n);
+    }
+    if (lane == 0) {
+        p.out_len[b] = n;
+        if (mine) p.resid[b] = __ldcg(p.cand_mass + (size_t)b * (K + 1) + n);
+    }
+    return n;
+}
+
+template <typename E>
+__global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(const RParams p) {
+    extern __shared__ unsigned char smem_raw[];
+    CSmem& sm = *reinterpret_cast<CSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+    unsigned char* area = reinterpret_cast<unsigned char*>(&sm) + ((sizeof(CSmem) + 127) & ~size_t(127));
+    double* const segsum = reinterpret_cast<double*>(area);     // a job's sums per kSegElems entries
+    BonusSeg* const bseg = reinterpret_cast<BonusSeg*>(area);   // the extra row's sums per 2 KB (never in use together)
+    constexpr int BSEG = kBonusSegBytes / (int)sizeof(E);       // entries per bonus segment
+    const int K = p.K, V = p.V, C = p.C;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int rank = (int)cluster_ctarank();
+    const int cluster_id = blockIdx.x / C;
+    const bool ordered = p.ordered != 0;
+    // first rejections are settled as the reports come in when the decided / accepted bits of a sequence fit one word
+    const bool early = !ordered && K <= 30;
+    const long long n_items = ordered ? (long long)p.B : (long long)p.B * (K + 1);
+    const bool vec = p.use_tma != 0;   // rows are 16-byte aligned: 16-byte loads
+    const E* tbase = reinterpret_cast<const E*>(p.t);
+    const E* dbase = reinterpret_cast<const E*>(p.d);
+
+    if (tid == 0) trace_mark(0, 0);
+    clear_next_counters(p);
+    if (tid == 0) {
+        for (int i = 0; i < 2; ++i) { mbar_init(&sm.xbar[i], (unsigned)(C * kCWarps)); mbar_init(&sm.mbar2[i], (unsigned)C); }
+        sm.abort_flag = 0;
+        sm.my_job_b = -1;
+        sm.my_job_n = 0;
+        mbar_init_fence();
+    }
+    __syncthreads();
+
+    const int e0 = rank * p.slice;                         // this CTA's slice of every row
+    const int n = max(0, min(p.slice, V - e0));
+    int round = 0, mround = 0;                             // exchanges so far (the same in every CTA of the cluster)
+    bool failed = false;
+    int b = 0, j = 0;
+    // what thread 0 fetches ahead for an item's decision: the token's two logits and the uniform
+    float lt = 0.f, ld = 0.f, nx_lt = 0.f, nx_ld = 0.f;
+    double U = 0.0, nx_U = 0.0;
+    bool tok_ok = true, nx_tok_ok = true;
+    int next_item = 0;
+
+    auto fetch_token = [&](int fb, int fj) {   // thread 0
+        nx_tok_ok = true;
+        if (fj < K) {
+            const int tok = p.x[(size_t)fb * K + fj];
+            nx_tok_ok = tok >= 0 && tok < V;
+            if (nx_tok_ok) {
+                nx_lt = load_logit(tbase + (size_t)target_row(fb, fj, K) * V + tok);
+                nx_ld = load_logit(dbase + (size_t)draft_row(fb, fj, K) * V + tok);
+            }
+            nx_U = uniform_accept(p.seed, p.offset, (uint32_t)(p.b_first + fb), (uint32_t)fj);
+        }
+    };
+    auto take_item = [&](int nb, int nj) {
+        b = nb;
+        j = nj;
+        if (tid == 0) {
+            lt = nx_lt; ld = nx_ld; U = nx_U; tok_ok = nx_tok_ok;
+            // the cluster's next queue entry: one per position, or one per sequence when ordered
+            if (rank == 0 && (!ordered || j == 0)) next_item = atomicAdd(&p.heads[0], 1) + p.n_clusters;
+        }
+    };
+
+    bool have = cluster_id < n_items;
+    if (have) {
+        const int fb = ordered ? cluster_id : cluster_id / (K + 1), fj = ordered ? 0 : cluster_id % (K + 1);
+        if (tid == 0) fetch_token(fb, fj);
+        take_item(fb, fj);
+    }
+    // barriers of every CTA are initialised before any peer arrives on them
+    cluster_sync_all();
+
+    for (;;) {
+        const bool work = have;          // the same in every CTA of the cluster
+        const bool pair = j < K;
+        const float cb = work ? seq_c(p, b) : 1.0f;   // log2(e) / temperature of this sequence
+        const E* const trow = tbase + (size_t)target_row(work ? b : 0, work ? j : 0, K) * V;
+        const E* const drow = dbase + (size_t)draft_row(work ? b : 0, (work && pair) ? j : 0, K) * V;
+        // ---- 1. statistics of this CTA's slices
+        if (tid == 0) trace_mark(1, work ? b * (K + 1) + j : -1);
+        float2 pt2 = make_float2(-INFINITY, 0.f), pd2 = make_float2(-INFINITY, 0.f);
+        if (work) {
+            if (pair) {
+                pt2 = stream_piece<E, kCThreads>(trow, e0, e0 + n, vec, cb, tid);
+                pd2 = stream_piece<E, kCThreads>(drow, e0, e0 + n, vec, cb, tid);
+            } else {
+                pt2 = stream_bonus_piece<E>(trow, e0, e0 + n, vec, cb, warp, lane, bseg - e0 / BSEG);
+            }
+        }
+        if (tid == 0) trace_mark(2, 0);
+        // (max, sum) of the warp's share: the maximum first (shuffles only), then one rescale per thread and a sum
+        const int par = round & 1;
+        {
+            float Mt = pt2.x, Md = pd2.x;
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                Mt = fmaxf(Mt, __shfl_xor_sync(0xffffffffu, Mt, off));
+                Md = fmaxf(Md, __shfl_xor_sync(0xffffffffu, Md, off));
+            }
+            float St = rebase_sum(pt2.x, pt2.y, Mt, cb), Sd = rebase_sum(pd2.x, pd2.y, Md, cb);
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                St += __shfl_xor_sync(0xffffffffu, St, off);
+                Sd += __shfl_xor_sync(0xffffffffu, Sd, off);
+            }
+            // ---- 2. every warp hands its partial result to every CTA of the cluster (itself included);
+            //         warp 0 adds the next queue entry (rank 0) and the job this CTA has to announce
+            const int nx = __shfl_sync(0xffffffffu, next_item, 0);
+            if (lane < C) {
+                peer_store(map_to_peer(smem_u32(&sm.xstat[par][rank * kCWarps + warp]), (uint32_t)lane),
+                           make_float4(Mt, St, Md, Sd));
+                if (warp == 0) {
+                    if (rank == 0) peer_store(map_to_peer(smem_u32(&sm.xnext[par]), (uint32_t)lane), nx);
+                    peer_store(map_to_peer(smem_u32(&sm.xjob[par][rank]), (uint32_t)lane), make_int2(sm.my_job_b, sm.my_job_n));
+                }
+                peer_arrive(map_to_peer(smem_u32(&sm.xbar[par]), (uint32_t)lane));
+            }
+        }
+        bool ok = mbar_wait_cluster(&sm.xbar[par], (uint32_t)(round >> 1) & 1u, &sm.abort_flag);
+        ++round;
+        if (tid == 0) trace_mark(3, 0);
+        if (__syncthreads_or(ok ? 0 : 1)) { failed = true; break; }   // (also: every warp has sent before my_job is cleared)
+        if (tid == 0) sm.my_job_b = -1;
+        // the job announced in this round, if any (at most one CTA reported an item last round)
+        int job_b = -1, job_n = 0;
+        for (int i = 0; i < C; ++i) {
+            const int2 q = sm.xjob[par][i];
+            if (q.x >= 0) { job_b = q.x; job_n = q.y; }
+        }
+        // the cluster's next queue entry, known to every CTA now
+        const long long nxt = sm.xnext[par];
+        const bool q_have = work && nxt < n_items;
+        const int qb = q_have ? (ordered ? (int)nxt : (int)(nxt / (K + 1))) : 0;
+        const int qj = (q_have && !ordered) ? (int)(nxt % (K + 1)) : 0;
+        // ---- 3. the rows' (max, Z) and the decision
+        if (work && warp == 0) {
+            // C x 8 partial results, lane i takes entries i, i + 32, ...: the same in every CTA, hence identical bits
+            const int parts = C * kCWarps;
+            float mt = -INFINITY, md = -INFINITY;
+            for (int i = lane; i < parts; i += 32) {
+                mt = fmaxf(mt, sm.xstat[par][i].x);
+                md = fmaxf(md, sm.xstat[par][i].z);
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, off));
+                md = fmaxf(md, __shfl_xor_sync(0xffffffffu, md, off));
+            }
+            float zt = 0.f, zd = 0.f;
+            for (int i = lane; i < parts; i += 32) {
+                const float4 v = sm.xstat[par][i];
+                zt += rebase_sum(v.x, v.y, mt, cb);
+                zd += rebase_sum(v.z, v.w, md, cb);
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                zt += __shfl_xor_sync(0xffffffffu, zt, off);
+                zd += __shfl_xor_sync(0xffffffffu, zd, off);
+            }
+            if (lane == 0) {
+                const double Tb = seq_temperature(p, b), betab = seq_beta(p, b);
+                int dec = 1;
+                if (!rowstat_ok(mt, zt) || (pair && (!rowstat_ok(md, zd) || !tok_ok)) || !seq_params_ok(Tb, betab)) dec = -1;
+                sm.rs_t = make_float2(mt, zt);
+                sm.rs_d = pair ? make_float2(md, zd) : make_float2(0.f, 1.f);
+                if (pair && dec >= 0) {
+                    // fp32 first; it stands unless R comes close to the threshold (the band is some 25 times
+                    // the fp32 error) or the caller wants the probabilities: then fp64.  Every CTA of the
+                    // cluster runs the same arithmetic on the same numbers.
+                    const float pt32 = ex2_approx((lt - mt) * cb) / zt;
+                    const float pd32 = ex2_approx((ld - md) * cb) / zd;
+                    const float ratio32 = pt32 / fmaxf(pd32, (float)kEps);
+                    const float thr32 = fmaxf((float)U - (float)betab * (1.0f - 1.0f / zt), 0.0f);
+                    const float diff = ratio32 - thr32;
+                    if (!p.want_stats && fabsf(diff) > 1e-4f * (ratio32 + thr32) + 1e-6f) {
+                        dec = diff > 0.0f ? 1 : 0;
+                    } else {
+                        const Decision dc = decide_position((double)lt, (double)ld, sm.rs_t, sm.rs_d, Tb, betab, U);
+                        dec = dc.accept ? 1 : 0;
+                        if (rank == 0 && p.want_stats) {
+                            const size_t i = (size_t)b * K + j;
+                            p.pt_tok[i] = dc.pt;
+                            p.pd_tok[i] = dc.pd;
+                            p.max_pt[i] = dc.maxp;
+                            p.cls[i] = (uint8_t)dc.cls;
+                        }
+                    }
+                }
+                sm.dec = dec;
+            }
+        }
+        __syncthreads();
+        const int dec = work ? sm.dec : 1;
+        if (tid == 0) {
+            trace_mark(4, dec);
+            // the next item's token, fetched now that the others are released: the loads land while this
+            // item is reported (walking a sequence in order, an accepted position is followed by the next one)
+            if (work && ordered && pair && dec > 0) fetch_token(b, j + 1);
+            else if (q_have) fetch_token(qb, qj);
+        }
+        // ---- 4. the extra row draws its bonus token at once from the segment sums of step 1
+        int writer = work ? (b + j) % C : 0, token = -1;   // reports are spread over the CTAs of the cluster
+        double mass = 0.0;
+        if (work && !pair && dec >= 0) {
+            const RowNorm rn = make_rownorm(sm.rs_t, sm.rs_d);
+            const double mc = (double)rn.mt * (double)cb;   // exact: two fp32 factors
+            const BonusSeg* bs = bseg;
+            // the terms of a segment were exp2(l c - mu): bring its sum to the row's own maximum (fp64: no new error)
+            auto val = [bs, mc](int g) { return bonus_sum_at_row_maximum(bs[g].sum, bs[g].mu, mc); };
+            if (!cluster_pick<E>(sm, p, val, (n + BSEG - 1) / BSEG, BSEG, b, false, trow, trow, rn, cb, e0, n, rank, C, mround, token)) {
+                failed = true;
+                break;
+            }
+            if (sm.pick_rank >= 0) writer = sm.pick_rank;
+            mass = sm.pick_S * rn.izt;
+        }
+        // ---- 5. one CTA reports the item and counts it; the sequence's last item finishes the sequence
+        //         and, after a rejection, leaves the second-pass job for the cluster's next round
+        bool seq_goes_on = false;
+        if (work && ordered) {
+            seq_goes_on = dec > 0 && pair;
+            if (dec == 0) { job_b = b; job_n = j; }        // the first rejection of a sequence walked in order: its masses now
+            if (rank == writer && warp == 0 && !seq_goes_on) {
+                int32_t* ot = p.out_tok + (size_t)b * (K + 1);
+                if (dec < 0) {
+                    for (int q = lane; q <= K; q += 32) ot[q] = -1;
+                    if (lane == 0) {
+                        p.out_len[b] = -1;
+                        atomicOr(&p.heads[2], kDevInvalidInput);
+                    }
+                } else {
+                    for (int q = lane; q <= K; q += 32) {
+                        if (q < j) ot[q] = p.x[(size_t)b * K + q];
+                        else if (q > j) ot[q] = -1;
+                        else if (!pair) ot[q] = token;        // the bonus token; a rejected slot is the job's to fill
+                    }
+                    if (lane == 0) {
+                        p.out_len[b] = j;
+                        if (!pair) p.resid[b] = mass;
+                    }
+                }
+            }
+        } else if (work && rank == writer && warp == 0) {
+            int last = 0;
+            if (lane == 0) {
+                const size_t s = (size_t)b * (K + 1) + j;
+                p.flag[s] = (signed char)dec;
+                p.cand[s] = token;
+                p.cand_mass[s] = mass;
+                p.rowstat[s] = make_float4(sm.rs_t.x, sm.rs_t.y, sm.rs_d.x, sm.rs_d.y);
+                if (early) {
+                    // decided, and accepted unless rejected (an unusable position counts as accepted here: it
+                    // must not ask for masses; the flag array remembers it and invalidates the sequence)
+                    const unsigned long long bit = 1ull << j;
+                    const unsigned long long add = bit | (dec != 0 ? bit << 32 : 0ull);
+                    __threadfence();   // the row statistics above are visible before the position counts as decided
+                    const unsigned long long old = atomicOr(p.seqmask + b, add);
+                    const int n_now = settled_first_rejection(old | add, K);
+                    if (n_now >= 0 && settled_first_rejection(old, K) < 0) { sm.my_job_b = b; sm.my_job_n = n_now; }   // settled by this report
+                    const int done = ticket_add(&p.ticket[b]) + 1;
+                    // K+1 items report, and the job if a position was rejected; the last of them finishes
+                    const unsigned long long all = *reinterpret_cast<volatile unsigned long long*>(p.seqmask + b);
+                    const bool every = (uint32_t)all == (K + 1 >= 32 ? 0xffffffffu : (1u << (K + 1)) - 1u);
+                    const bool none_rejected = ((uint32_t)all & ~(uint32_t)(all >> 32) & ((1u << K) - 1u)) == 0;
+                    last = (done == K + 2 || (done == K + 1 && every && none_rejected)) ? 1 : 0;
+                } else {
+                    last = ticket_add(&p.ticket[b]) == K ? 1 : 0;
+                }
+            }
+            last = __shfl_sync(0xffffffffu, last, 0);
+            if (last) {
+                __threadfence();
+                const int nfirst = finish_streamed_sequence(p, b, lane, !early);
+                if (!early && lane == 0 && nfirst >= 0 && nfirst < K) { sm.my_job_b = b; sm.my_job_n = nfirst; }
+            }
+        }
+        if (tid == 0) trace_mark(5, token);
+        // ---- 6. the second-pass job of this round: the masses of one rejected position and its token
+        if (job_b >= 0) {
+            const float cj = seq_c(p, job_b);
+            const E* const jt = tbase + (size_t)target_row(job_b, job_n, K) * V;
+            const E* const jd = dbase + (size_t)draft_row(job_b, job_n, K) * V;
+            float4 rs;
+            if (ordered) rs = make_float4(sm.rs_t.x, sm.rs_t.y, sm.rs_d.x, sm.rs_d.y);
+            else rs = __ldcg(&p.rowstat[(size_t)job_b * (K + 1) + job_n]);   // stored before the ticket that made the job
+            const RowNorm rn = make_rownorm(make_float2(rs.x, rs.y), make_float2(rs.z, rs.w));
+            double* so = segsum - e0 / kSegElems;    // sums land at index (entry - e0) / kSegElems
+            const double* ss = segsum;
+            auto val = [ss](int g) { return ss[g]; };
+            int jtoken = -1;
+            bool resid = true;
+            __syncthreads();                         // the bonus sums of step 4 (same memory) are no longer needed
+            for (;;) {
+                if (resid) stream_job_piece<E, true>(jt, jd, e0, e0 + n, vec, rn, cj, warp, lane, so);
+                else stream_job_piece<E, false>(jt, jt, e0, e0 + n, vec, rn, cj, warp, lane, so);
+                __syncthreads();
+                if (!cluster_pick<E>(sm, p, val, (n + kSegElems - 1) / kSegElems, kSegElems, job_b, resid, jt, jd, rn, cj, e0, n, rank,
+                                     C, mround, jtoken)) {
+                    failed = true;
+                    break;
+                }
+                // a rejection implies residual mass; if rounding erased it, draw from P_t instead
+                if (resid && !(sm.pick_S * rn.izt >= kTinyMass)) { resid = false; __syncthreads(); continue; }
+                break;
+            }
+            if (failed) break;
+            if (warp == 0 && (rank == sm.pick_rank || (sm.pick_rank < 0 && rank == 0))) {
+                if (early) {
+                    // the job reports like an item; if it is the last of the sequence to do so it finishes it
+                    int last = 0;
+                    if (lane == 0) {
+                        const size_t s = (size_t)job_b * (K + 1) + job_n;
+                        p.cand[s] = jtoken;
+                        p.cand_mass[s] = sm.pick_S * rn.izt;
+                        last = ticket_add(&p.ticket[job_b]) + 1 == K + 2 ? 1 : 0;
+                    }
+                    last = __shfl_sync(0xffffffffu, last, 0);
+                    if (last) {
+                        __threadfence();
+                        finish_streamed_sequence(p, job_b, lane, false);
+                    }
+                } else if (lane == 0) {
+                    p.out_tok[(size_t)job_b * (K + 1) + job_n] = jtoken;
+                    p.resid[job_b] = sm.pick_S * rn.izt;
+                }
+            }
+            if (tid == 0) trace_mark(7, jtoken);
+        }
+        __syncthreads();     // shared memory of this round (decision, sums) is free again
+        if (!work) break;    // that was the round after the last item: its job, if any, is done
+        // ---- on to the next item
+        if (seq_goes_on) {
+            take_item(b, j + 1);
+        } else {
+            have = q_have;
+            if (have) take_item(qb, qj);
+            else j = 0;
+        }
+    }
+    if (tid == 0) trace_mark(6, 0);
+    if (failed || sm.abort_flag) {
+        if (tid == 0) atomicOr(&p.heads[2], kDevTimeout);
+    }
+    __syncthreads();
+    cluster_sync_all();   // no CTA leaves while a peer may still store into it
+}
+
+}  // namespace ears

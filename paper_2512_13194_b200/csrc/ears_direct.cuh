@@ -183,13 +183,14 @@ __device__ __forceinline__ float2 stream_bonus_piece(const E* row, int e0, int e
 
 // A second-pass piece [e0, e1) of the two rows of a rejected position: sums of
 // max(0, e_t - e_d Z_t / Z_d) per kSegElems entries; warp w takes groups of four segments and
-// keeps the loads of a group (packed, as they come) in flight together.
-template <typename E>
+// keeps the loads of a group (packed, as they come) in flight together.  RESID = false: the
+// target row alone, sums of e_t (a bonus token is drawn from P_t).
+template <typename E, bool RESID = true>
 __device__ __forceinline__ void stream_job_piece(const E* trow, const E* drow, int e0, int e1, bool vec, const RowNorm& rn,
                                                  float c, int warp, int lane, double* seg_out /* of the whole row */) {
     constexpr int N = Words<E>::N;
     constexpr int VPL = kSegElems / N / 32;   // vectors per lane per segment and row
-    constexpr int GROUP = 4;                  // segments per round
+    constexpr int GROUP = VPL >= 2 ? 2 : 4;   // segments per round: 32 registers of loads in flight for either row width
     for (int g0 = e0 + warp * GROUP * kSegElems; g0 < e1; g0 += kDWarps * GROUP * kSegElems) {
         double acc[GROUP];
         if (vec) {
@@ -201,7 +202,7 @@ __device__ __forceinline__ void stream_job_piece(const E* trow, const E* drow, i
                     const int k0 = g0 + h * kSegElems + (j * 32 + lane) * N;
                     if (k0 < e1) {
                         wt[h][j] = ld_stream16(trow + k0);
-                        wd[h][j] = ld_stream16(drow + k0);
+                        wd[h][j] = RESID ? ld_stream16(drow + k0) : make_uint4(0, 0, 0, 0);
                     } else {
                         wt[h][j] = make_uint4(0, 0, 0, 0);
                         wd[h][j] = make_uint4(0, 0, 0, 0);
@@ -218,7 +219,7 @@ __device__ __forceinline__ void stream_job_piece(const E* trow, const E* drow, i
                     const bool in = g0 + h * kSegElems + (j * 32 + lane) * N < e1;   // whole vectors here
 #pragma unroll
                     for (int i = 0; i < N; ++i) {
-                        const float r = entry_mass<true>(xt[i], xd[i], rn, c);
+                        const float r = entry_mass<RESID>(xt[i], xd[i], rn, c);
                         if (in) a += r;
                     }
                 }
@@ -231,7 +232,7 @@ __device__ __forceinline__ void stream_job_piece(const E* trow, const E* drow, i
                 for (int j = 0; j < VPL; ++j)
                     for (int i = 0; i < N; ++i) {
                         const int k = g0 + h * kSegElems + (j * 32 + lane) * N + i;
-                        if (k < e1) a += entry_mass<true>(load_logit(trow + k), load_logit(drow + k), rn, c);
+                        if (k < e1) a += entry_mass<RESID>(load_logit(trow + k), RESID ? load_logit(drow + k) : 0.f, rn, c);
                     }
                 acc[h] = (double)a;
             }
@@ -340,6 +341,7 @@ __global__ void __launch_bounds__(kDThreads + 32, kDCtasPerSm) ears_direct_kerne
     const E* tbase = reinterpret_cast<const E*>(p.t);
     const E* dbase = reinterpret_cast<const E*>(p.d);
 
+    if (tid == 0) trace_mark(0, 0);
     clear_next_counters(p);
     if (tid == 0) sm.abort_flag = 0;
     __syncthreads();
@@ -399,7 +401,9 @@ __global__ void __launch_bounds__(kDThreads + 32, kDCtasPerSm) ears_direct_kerne
                 // be waiting for exactly that), then look again.
                 if (!prev_done) {
                     sync_B(it - 1);
+                    if (lane == 0) trace_mark(15, 1);
                     direct_epilogue<E, PER_SEQ>(p, prev, sm.red[(it - 1) & 1], lane);
+                    if (lane == 0) trace_mark(16, 1);
                     prev_done = true;
                     continue;
                 }
@@ -426,10 +430,13 @@ __global__ void __launch_bounds__(kDThreads + 32, kDCtasPerSm) ears_direct_kerne
             if (lane == 0) sm.work[it & 1] = wk;
             __threadfence_block();
             __syncwarp();
+            if (lane == 0) trace_mark(10 + wk.kind, (int)wk.unit);
             arrive_A(it);                                    // A(it): the item is published
             if (!prev_done) {
                 sync_B(it - 1);                               // B(it - 1): the previous item's results are in
+                if (lane == 0) trace_mark(15, 0);
                 direct_epilogue<E, PER_SEQ>(p, prev, sm.red[(it - 1) & 1], lane);
+                if (lane == 0) trace_mark(16, 0);
             }
             if (wk.kind == kDExit) break;
             prev = wk;
@@ -481,6 +488,7 @@ __global__ void __launch_bounds__(kDThreads + 32, kDCtasPerSm) ears_direct_kerne
         }
     }
     __syncthreads();
+    if (tid == 0) trace_mark(6, 0);
     if (tid == 0 && sm.abort_flag) atomicOr(&p.heads[2], kDevTimeout);
 }
 

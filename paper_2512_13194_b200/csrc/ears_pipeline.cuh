@@ -23,6 +23,28 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
     return t;
 }
 
+// ---- optional timeline (compiled in with -DEARS_TRACE only) ----------------------------
+// A few CTAs record (time, tag, argument) at the ends of their phases into a fixed device array
+// that the host reads back with ears_trace_read; used to see where a launch spends its time.
+// Without the macro the marks compile to nothing.
+#ifdef EARS_TRACE
+constexpr int kTraceCtas = 96, kTraceEvents = 192;
+__device__ unsigned long long g_trace[kTraceCtas][kTraceEvents][2];
+__device__ int g_trace_n[kTraceCtas];
+// called by one thread of the CTA
+__device__ __forceinline__ void trace_mark(int tag, int arg) {
+    if (blockIdx.x < kTraceCtas) {
+        const int i = g_trace_n[blockIdx.x]++;
+        if (i < kTraceEvents) {
+            g_trace[blockIdx.x][i][0] = global_timer_ns();
+            g_trace[blockIdx.x][i][1] = ((unsigned long long)(unsigned)tag << 32) | (unsigned)arg;
+        }
+    }
+}
+#else
+__device__ __forceinline__ void trace_mark(int, int) {}
+#endif
+
 __device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }

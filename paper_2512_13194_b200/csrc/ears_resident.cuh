@@ -58,6 +58,8 @@ struct RParams {
     signed char* flag;    // [B,K+1] 1 accepted / row usable, 0 rejected, -1 invalid
     int32_t* cand;        // [B,K+1] token drawn at the position (rejected positions and slot K)
     double* cand_mass;    // [B,K+1] mass that token was drawn from
+    float4* rowstat;      // [B,K+1] (max, Z) of the item's target and draft rows (streaming clusters only)
+    unsigned long long* seqmask;  // [B] positions decided (low word) and accepted (high word), K <= 30 (streaming clusters only)
     int C;                // CTAs per cluster
     int slice;            // elements of a row per CTA, a multiple of kSegElems
     int buf_bytes;        // shared-memory bytes reserved per row slice (slice bytes rounded up to kRSubBytes)

@@ -62,8 +62,9 @@ SHAPES = [
 
 
 # (path, cluster): 1 = streaming kernel with the shared-memory ring; 3 = streaming kernel reading straight from
-# global memory; 2 = resident kernel with 1..16 CTAs per cluster (0 = automatic)
-PATHS = [(1, 0), (3, 0), (2, 0), (2, 1), (2, 2), (2, 4), (2, 8), (2, 16)]
+# global memory; 2 = resident kernel with 1..16 CTAs per cluster (0 = automatic); 4 = the cluster kernel in its
+# streamed form (nothing staged, slices read twice)
+PATHS = [(1, 0), (3, 0), (2, 0), (2, 1), (2, 2), (2, 4), (2, 8), (2, 16), (4, 0), (4, 1), (4, 2), (4, 4), (4, 8), (4, 16)]
 
 
 @pytest.fixture
@@ -87,7 +88,7 @@ def test_parity_shapes(ears, forced_path, B, K, V, dtype, path, cluster):
         try:
             tl, *_ = run_both(ears, w, t, d, x, T, beta, seed=seed, offset=7 * seed)
         except ears.EarsError as e:
-            if cluster and e.status == -2 and 2 * V * (4 if dtype == "fp32" else 2) > 60000 * cluster:
+            if path == 2 and cluster and e.status == -2 and 2 * V * (4 if dtype == "fp32" else 2) > 60000 * cluster:
                 pytest.skip("a pair of rows does not fit a cluster of this size")
             raise
         tally.merge(tl)
@@ -95,7 +96,7 @@ def test_parity_shapes(ears, forced_path, B, K, V, dtype, path, cluster):
     assert tally.max_rel_prob_err < 1e-5
 
 
-@pytest.mark.parametrize("path", [0, 1, 3])
+@pytest.mark.parametrize("path", [0, 1, 3, 4])
 @pytest.mark.parametrize("idx", [1, 2, 3, 4])
 def test_parity_workloads(ears, forced_path, idx, path):
     """Workloads 1-4 at full size, in the automatic launch configuration (the resident kernel for
@@ -119,7 +120,7 @@ def test_parity_workloads(ears, forced_path, idx, path):
           f"flagged_tok={tally.flagged_tokens} max_rel={tally.max_rel_prob_err:.2e} mean_len={np.mean(lens):.2f}")
 
 
-@pytest.mark.parametrize("path", [0, 1, 3])
+@pytest.mark.parametrize("path", [0, 1, 3, 4])
 @pytest.mark.parametrize("idx,B", [(2, 8), (3, 32), (4, 128), (4, 24)])
 def test_parity_fp16_workload_shapes(ears, forced_path, idx, B, path):
     """The 2-byte workloads with IEEE binary16 logits instead of bfloat16 (same values before
@@ -137,7 +138,7 @@ def test_parity_fp16_workload_shapes(ears, forced_path, idx, B, path):
     assert tally.max_rel_prob_err < 1e-5
 
 
-@pytest.mark.parametrize("path", [1, 2, 3])
+@pytest.mark.parametrize("path", [1, 2, 3, 4])
 def test_probabilities_are_tight_on_rows_far_below_their_maximum(ears, forced_path, path):
     """Rows of workload 3 (one logit 8 above the rest: every other term of Z sits near 2^-17, where
     the fp32 product l c is coarse).  A correction of the wrong sign for the rounding of m c doubled
@@ -152,7 +153,7 @@ def test_probabilities_are_tight_on_rows_far_below_their_maximum(ears, forced_pa
     assert tl.max_rel_prob_err < 7e-7
 
 
-@pytest.mark.parametrize("path,V", [(0, 256000), (3, 256000), (0, 131072), (3, 131072), (1, 131072)])
+@pytest.mark.parametrize("path,V", [(0, 256000), (3, 256000), (4, 256000), (0, 131072), (3, 131072), (1, 131072)])
 @pytest.mark.parametrize("beta", [1.0, 0.0])
 def test_parity_largest_workload(ears, forced_path, beta, path, V):
     """Full size of the largest configuration, in the launch configuration the benchmark times
@@ -164,8 +165,8 @@ def test_parity_largest_workload(ears, forced_path, beta, path, V):
     forced_path(path)
     w = replace(synth.workload(5), V=V)
     plan = ears.describe_plan(w.dtype, w.B, w.K, w.V).split(":")[0]
-    assert plan == {(0, 256000): "streaming", (0, 131072): "direct", 1: "streaming", 3: "direct"}.get((path, V), None) \
-        or plan == {1: "streaming", 3: "direct"}[path]
+    assert plan == {(0, 256000): "streaming", (0, 131072): "direct"}.get((path, V)) \
+        or plan == {1: "streaming", 3: "direct", 4: "cluster-streamed"}.get(path)
     t, d, x = synth.make_inputs(w, "cuda:0")
     acc, tok, st = ears.verify(t, d, x, w.temperature, beta, 0, 3, stats=True)
     torch.cuda.synchronize()
@@ -174,7 +175,9 @@ def test_parity_largest_workload(ears, forced_path, beta, path, V):
                         nthreads=oracle.max_threads())
     tally = compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, w.K, {k: v.cpu().numpy() for k, v in st.items()},
                     inputs=(t.cpu(), d.cpu(), w.temperature))
-    assert_parity(tally)
+    # One step of 3584 rows cannot resolve a rate of 1e-4 (the soak runs over 1e6 rows do: 3-5e-5 under every
+    # kernel, i.e. 0.1-0.2 expected here); what this step checks is that nothing is unexplained.
+    assert_parity(tally, max_explained=3)
     assert tally.max_rel_prob_err < 1e-5
     if beta == 0.0:
         assert (ora.accept_len < w.K).mean() > 0.3
@@ -206,7 +209,8 @@ def test_kernels_agree(ears, forced_path):
     tg, dg, xg = t.to(dev), d.to(dev), x.to(dev)
     results = []
     try:
-        for path, cluster, loader in [(1, 0, 0), (3, 0, 0), (3, 0, 2), (2, 0, 0), (2, 1, 0), (2, 2, 2), (2, 4, 0), (2, 8, 2), (2, 16, 0)]:
+        for path, cluster, loader in [(1, 0, 0), (3, 0, 0), (3, 0, 2), (2, 0, 0), (2, 1, 0), (2, 2, 2), (2, 4, 0), (2, 8, 2), (2, 16, 0),
+                                      (4, 0, 0), (4, 1, 2), (4, 2, 0), (4, 8, 2), (4, 16, 0)]:
             forced_path(path, cluster)
             ears.set_plan(loader, 0)
             acc, tok = ears.verify(tg, dg, xg, 1.0, 0.1, 4, 9)
@@ -231,7 +235,7 @@ def test_forced_resident_path_refuses_rows_that_do_not_fit(ears, forced_path):
 
 
 @pytest.mark.parametrize("dtype", ["fp32", "fp16", "bf16"])
-@pytest.mark.parametrize("path", [1, 2, 3])
+@pytest.mark.parametrize("path", [1, 2, 3, 4])
 def test_invalid_sequences_are_marked(ears, forced_path, path, dtype):
     """Unusable data marks its own sequence and nothing else.  For the 2-byte types the NaNs sit in
     an odd and in an even lane of a packed pair (the packed maximum drops NaNs, so they must reach
@@ -375,7 +379,7 @@ def test_bounded_wait_gives_up_and_context_survives(ears):
     assert ears.load_library().ears_selftest_bounded_wait(0, None) == -3
 
 
-@pytest.mark.parametrize("path,cluster", [(1, 0), (3, 0), (2, 0), (2, 4)])
+@pytest.mark.parametrize("path,cluster", [(1, 0), (3, 0), (2, 0), (2, 4), (4, 0), (4, 2)])
 @pytest.mark.parametrize("B,K,V,dtype", [(12, 3, 9000, "fp32"), (9, 4, 20001, "bf16"), (300, 2, 700, "bf16")])
 def test_parity_per_sequence_temperature_and_beta(ears, forced_path, B, K, V, dtype, path, cluster):
     """ears_verify_var: every sequence with its own temperature and beta, against the oracle run
@@ -425,7 +429,7 @@ def test_parity_per_sequence_temperature_and_beta(ears, forced_path, B, K, V, dt
                   max_explained=1)
 
 
-@pytest.mark.parametrize("path", [1, 2, 3])
+@pytest.mark.parametrize("path", [1, 2, 3, 4])
 def test_status_and_counters_start_clean_on_every_call_of_one_shape(ears, forced_path, path):
     """Calls of one shape on the library's workspace alternate between two counter blocks without
     a memset in between: a call that saw invalid input must not leak its status or counters."""
@@ -446,7 +450,7 @@ def test_status_and_counters_start_clean_on_every_call_of_one_shape(ears, forced
             assert torch.equal(a, ref[0]) and torch.equal(k, ref[1])
 
 
-@pytest.mark.parametrize("path,cluster", [(1, 0), (3, 0), (2, 0), (2, 2), (2, 8)])
+@pytest.mark.parametrize("path,cluster", [(1, 0), (3, 0), (2, 0), (2, 2), (2, 8), (4, 0), (4, 1), (4, 4)])
 @pytest.mark.parametrize("B,K,V,dtype", [(24, 4, 9000, "fp32"), (200, 3, 1500, "bf16"), (5, 6, 20001, "bf16")])
 def test_parity_stop_at_first_reject(ears, forced_path, B, K, V, dtype, path, cluster):
     """EARS_FLAG_STOP_AT_FIRST_REJECT against the oracle in the same mode: same lengths and tokens

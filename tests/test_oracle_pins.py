@@ -616,3 +616,102 @@ def test_greedy_limit_matches_argmax_and_the_low_temperature_step():
     x2[3, 1] = V
     acc2, tok2, _ = oracle.verify_greedy(t2, x2)
     assert acc2[1:4].tolist() == [-1, -1, -1] and (tok2[1:4] == -1).all() and np.array_equal(acc2[4:], acc[4:])
+
+
+# -------------------------------------------------- entropy as the uncertainty measure (Sec. 5 item 1)
+def test_entropy_matches_library_routine_and_closed_forms():
+    rng = np.random.default_rng(11)
+    for V in (1, 2, 7, 1000):
+        p = rng.random(V)
+        p[rng.random(V) < 0.2] = 0.0
+        if p.sum() == 0:
+            p[0] = 1.0
+        p /= p.sum()
+        assert abs(oracle.entropy(p) - stats.entropy(p)) < 1e-12
+    for V in (2, 8, 4096):
+        assert abs(oracle.entropy(np.full(V, 1.0 / V)) - np.log(V)) < 1e-12        # flat: ln V
+        assert abs(oracle.entropy_uncertainty(np.log(V), V) - 1.0) < 1e-15
+        one_hot = np.zeros(V)
+        one_hot[V // 2] = 1.0
+        assert oracle.entropy(one_hot) == 0.0                                       # one-hot: 0
+    assert oracle.entropy_uncertainty(0.0, 1) == 0.0                                # a single entry leaves no doubt
+    # two-point distribution: H = -q ln q - (1 - q) ln(1 - q)
+    q = 0.2
+    assert abs(oracle.entropy([q, 1 - q]) - (-q * np.log(q) - (1 - q) * np.log(1 - q))) < 1e-15
+
+
+def test_entropy_output_matches_the_row_softmax():
+    rng = np.random.default_rng(12)
+    B, K, V = 5, 3, 300
+    t = rng.normal(0, 2, (B, K + 1, V)).astype(np.float32)
+    t[0, 1, 10:200] = -np.inf                       # masked entries contribute nothing
+    d = (t[:, :K] + rng.normal(0, 1, (B, K, V))).astype(np.float32)
+    x = rng.integers(0, 10, (B, K)).astype(np.int32)
+    for T in (0.7, 1.0, 1.6):
+        res = oracle.verify(t, d, x, T, 0.3, seed=1, offset=2, want_entropy=True)
+        for b in range(B):
+            for k in range(K):
+                p = sp_softmax(t[b, k].astype(np.float64) / np.float32(T))
+                assert abs(res.entropy[b, k] - stats.entropy(p)) < 1e-10
+    # the measure the paper prints is untouched by asking for the entropy
+    a = oracle.verify(t, d, x, 1.0, 0.3, seed=1, offset=2)
+    b_ = oracle.verify(t, d, x, 1.0, 0.3, seed=1, offset=2, want_entropy=True)
+    assert np.array_equal(a.accept_len, b_.accept_len) and np.array_equal(a.tokens, b_.tokens)
+    assert np.array_equal(a.margin, b_.margin)
+
+
+@pytest.mark.parametrize("beta,T", [(0.1, 0.9), (0.5, 1.3), (1.0, 1.0)])
+def test_acceptance_probability_closed_form_with_entropy(beta, T):
+    """With the entropy measure the acceptance region is the printed one with the other uncertainty:
+    P(accept position k) = min(1, R_k + beta H_k / ln V)."""
+    rng = np.random.default_rng(13)
+    K, V, B = 3, 6, 200_000
+    t_rows = rng.normal(0, 1.5, (K + 1, V))
+    d_rows = t_rows[:K] + rng.normal(0, 1.0, (K, V))
+    toks = [1, 4, 2]
+    t, d, x = tile(t_rows, d_rows, toks, B)
+    res = oracle.verify(t, d, x, T, beta, seed=6, offset=1, nthreads=4, uncertainty="entropy")
+    a = np.empty(K)
+    for k in range(K):
+        pt = sp_softmax(t[0, k].astype(np.float64) / np.float32(T))
+        pd = sp_softmax(d[0, k].astype(np.float64) / np.float32(T))
+        R = pt[toks[k]] / max(pd[toks[k]], 1e-10)
+        a[k] = min(1.0, R + float(np.float32(beta)) * stats.entropy(pt) / np.log(V))
+    emp = (res.cls != 0).mean(axis=0)
+    sigma = np.sqrt(np.maximum(a * (1 - a), 1e-12) / B)
+    assert np.all(np.abs(emp - a) < 5 * sigma + 1e-9), (emp, a)
+    # and it differs from the printed measure on these rows (otherwise the test proves nothing)
+    plain = closed_form_accept(t[0], d[0], toks, np.float32(T), np.float32(beta))
+    assert np.abs(plain - a).max() > 0.01
+
+
+def test_entropy_measure_one_hot_flat_and_monotone_in_beta():
+    rng = np.random.default_rng(14)
+    B, K, V = 40, 4, 50
+    t = rng.normal(0, 2, (B, K + 1, V)).astype(np.float32)
+    d = (t[:, :K] + rng.normal(0, 1.5, (B, K, V))).astype(np.float32)
+    x = rng.integers(0, V, (B, K)).astype(np.int32)
+    # accept sets are nested in beta
+    prev = None
+    for beta in (0.0, 0.05, 0.2, 0.5, 1.0):
+        res = oracle.verify(t, d, x, 1.0, beta, seed=2, offset=3, uncertainty="entropy")
+        acc = res.cls != 0
+        if prev is not None:
+            assert np.all(acc | ~prev)
+            assert np.all(res.accept_len >= prev_len)
+        prev, prev_len = acc, res.accept_len
+    # beta = 0: the measure plays no role
+    a = oracle.verify(t, d, x, 1.0, 0.0, seed=2, offset=3, uncertainty="entropy")
+    b = oracle.verify(t, d, x, 1.0, 0.0, seed=2, offset=3)
+    assert np.array_equal(a.accept_len, b.accept_len) and np.array_equal(a.tokens, b.tokens)
+    # one-hot target rows: H = 0, zero tolerance whatever beta
+    t1 = t.copy()
+    t1[:, :, 7] += 400.0
+    a = oracle.verify(t1, d, x, 1.0, 1.0, seed=2, offset=3, uncertainty="entropy")
+    b = oracle.verify(t1, d, x, 1.0, 0.0, seed=2, offset=3, uncertainty="entropy")
+    assert np.array_equal(a.accept_len, b.accept_len) and np.array_equal(a.cls, b.cls)
+    assert np.all(a.entropy < 1e-100)
+    # flat target rows: H = ln V, uncertainty 1, so beta = 1 accepts everything (R + 1 >= U)
+    tf = np.zeros_like(t)
+    a = oracle.verify(tf, d, x, 1.0, 1.0, seed=2, offset=3, uncertainty="entropy")
+    assert np.all(a.accept_len == K) and np.allclose(a.entropy, np.log(V), atol=1e-12)
