@@ -147,7 +147,8 @@ int ears_verify_ex(int dtype, const void* target_logits, const void* draft_logit
  *   A value the scalar form would refuse (temperature not finite or <= 0, beta not finite or
  *   < 0) cannot be seen by the host: it marks that one sequence invalid (out_accept_len = -1,
  *   tokens -1, EARS_DEV_INVALID_INPUT), the others are unaffected.
- *   flags       0 or EARS_FLAG_STOP_AT_FIRST_REJECT.  Sec. 3.1: rejecting x_i discards every later
+ *   flags       0, EARS_FLAG_STOP_AT_FIRST_REJECT and / or EARS_FLAG_ENTROPY_UNCERTAINTY (for the latter
+ *               see ears_verify_entropy).  Sec. 3.1: rejecting x_i discards every later
  *               draft token.  With the flag, what lies after a sequence's first rejected position
  *               (later rows and tokens, and the extra target row unless everything was accepted)
  *               is not part of the step: it is not validated and the optional per-position
@@ -159,7 +160,8 @@ int ears_verify_ex(int dtype, const void* target_logits, const void* draft_logit
  * Everything else is as in ears_verify_ex.
  */
 #define EARS_FLAG_STOP_AT_FIRST_REJECT 1u
-#define EARS_FLAGS_ALL (EARS_FLAG_STOP_AT_FIRST_REJECT)
+#define EARS_FLAG_ENTROPY_UNCERTAINTY 2u   /* see ears_verify_entropy */
+#define EARS_FLAGS_ALL (EARS_FLAG_STOP_AT_FIRST_REJECT | EARS_FLAG_ENTROPY_UNCERTAINTY)
 int ears_verify_var(int dtype, const void* target_logits, const void* draft_logits,
                     const int32_t* draft_tokens, int B, int K, int V,
                     float temperature, float beta,
@@ -169,6 +171,32 @@ int ears_verify_var(int dtype, const void* target_logits, const void* draft_logi
                     double* out_pt_tok, double* out_pd_tok, double* out_max_pt,
                     uint8_t* out_class, double* out_resid_mass,
                     void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * ears_verify_var with the entropy of the target distribution.  Sec. 3.2 measures the target
+ * model's uncertainty at a position as 1 - max_v P_t(v); Sec. 5 (future work, item 1) names the
+ * distribution's entropy as a more refined measure and gives no formula.  Here
+ *     H = -sum_v P_t(v) ln P_t(v)   (nats; masked entries contribute nothing)
+ * comes out of the same sweep over the target row that yields its normaliser (one more
+ * multiply-add per logit), and
+ *   out_entropy [B,K] double, optional (NULL to skip): H of target row k, for every position
+ *               (with EARS_FLAG_STOP_AT_FIRST_REJECT: up to the first rejection);
+ *   flags may include EARS_FLAG_ENTROPY_UNCERTAINTY: the tolerance of Sec. 3.2 becomes
+ *               beta * H / ln V in place of beta * (1 - max P_t).  H / ln V lies in [0, 1] like
+ *               the printed measure (1 for a flat row, 0 for a one-hot row or V = 1); dividing by
+ *               ln V is this library's reading of "entropy as the uncertainty measure".
+ * Without the flag and with out_entropy = NULL this is ears_verify_var.  Everything else
+ * (arguments, outputs, errors, workspace) as there; out_entropy must be 8-byte aligned.
+ */
+int ears_verify_entropy(int dtype, const void* target_logits, const void* draft_logits,
+                        const int32_t* draft_tokens, int B, int K, int V,
+                        float temperature, float beta,
+                        const float* seq_temperature, const float* seq_beta, unsigned flags,
+                        uint64_t seed, uint64_t offset,
+                        int64_t b_first, int32_t* out_accept_len, int32_t* out_tokens,
+                        double* out_pt_tok, double* out_pd_tok, double* out_max_pt,
+                        uint8_t* out_class, double* out_resid_mass, double* out_entropy,
+                        void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * The temperature -> 0 limit of the step (Sec. 1 names temperature = 0 as the deterministic

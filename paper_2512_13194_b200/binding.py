@@ -46,6 +46,9 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ears_verify_var.argtypes = ([c.c_int] + common[:8] + [c.c_void_p, c.c_void_p, c.c_uint] + common[8:] + [c.c_int64]
                                     + [c.c_void_p] * 7 + [c.c_void_p, c.c_size_t, c.c_void_p])
     lib.ears_verify_var.restype = c.c_int
+    lib.ears_verify_entropy.argtypes = ([c.c_int] + common[:8] + [c.c_void_p, c.c_void_p, c.c_uint] + common[8:] + [c.c_int64]
+                                        + [c.c_void_p] * 8 + [c.c_void_p, c.c_size_t, c.c_void_p])
+    lib.ears_verify_entropy.restype = c.c_int
     lib.ears_verify_greedy.argtypes = [c.c_int, c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p,
                                        c.c_void_p, c.c_size_t, c.c_void_p]
     lib.ears_verify_greedy.restype = c.c_int
@@ -137,11 +140,14 @@ def verify(target_logits: torch.Tensor, draft_logits: torch.Tensor, draft_tokens
            temperature: float, beta: float, seed: int = 0, offset: int = 0, *, b_first: int = 0,
            stats: bool = False, workspace: Optional[torch.Tensor] = None, stream=None,
            seq_temperature: Optional[torch.Tensor] = None, seq_beta: Optional[torch.Tensor] = None,
-           stop_at_first_reject: bool = False):
+           stop_at_first_reject: bool = False, uncertainty: str = "maxprob", entropy: bool = False):
     """One EARS verification step on the current CUDA device.
 
     Returns (accept_len [B] int32, tokens [B,K+1] int32) and, with ``stats=True``, a dict with
     pt_tok, pd_tok, max_pt [B,K] float64, cls [B,K] uint8 and resid_mass [B] float64.
+    ``uncertainty="entropy"`` scales the tolerance by H(P_t) / ln V instead of 1 - max P_t
+    (EARS_FLAG_ENTROPY_UNCERTAINTY); ``entropy=True`` adds H(P_t) [B,K] float64 to the returned dict
+    (which is then returned even without ``stats``).
     ``seq_temperature`` / ``seq_beta``: optional float32 CUDA tensors [B] that replace the scalar
     for each sequence (ears_verify_var).  ``stop_at_first_reject``: rows after a sequence's first
     rejection are not part of the step (EARS_FLAG_STOP_AT_FIRST_REJECT).
@@ -168,7 +174,14 @@ def verify(target_logits: torch.Tensor, draft_logits: torch.Tensor, draft_tokens
                       resid_mass=torch.zeros(B, dtype=torch.float64, device=dev))
             ptrs = [st[k].data_ptr() for k in ("pt_tok", "pd_tok", "max_pt", "cls", "resid_mass")]
         ws_ptr, ws_bytes = (None, 0) if workspace is None else (workspace.data_ptr(), workspace.numel() * workspace.element_size())
-        if seq_temperature is None and seq_beta is None and not stop_at_first_reject:
+        if uncertainty not in ("maxprob", "entropy"):
+            raise ValueError("uncertainty must be 'maxprob' or 'entropy'")
+        ent = None
+        if entropy:
+            ent = torch.empty((B, K), dtype=torch.float64, device=dev)
+            st = {} if st is None else st
+            st["entropy"] = ent
+        if seq_temperature is None and seq_beta is None and not stop_at_first_reject and uncertainty == "maxprob" and ent is None:
             rc = lib.ears_verify_ex(_dtype_code(t), t.data_ptr(), d.data_ptr(), x.data_ptr(), B, K, V,
                                     float(temperature), float(beta), int(seed), int(offset), int(b_first),
                                     acc.data_ptr(), tok.data_ptr(), *ptrs, ws_ptr, ws_bytes, _stream_ptr(stream))
@@ -180,15 +193,17 @@ def verify(target_logits: torch.Tensor, draft_logits: torch.Tensor, draft_tokens
                         raise ValueError("per-sequence arrays must be float32 CUDA tensors of shape [B]")
                     a = a.contiguous()
                 arrs.append(a)
-            rc = lib.ears_verify_var(_dtype_code(t), t.data_ptr(), d.data_ptr(), x.data_ptr(), B, K, V,
-                                     float(temperature), float(beta),
-                                     None if arrs[0] is None else arrs[0].data_ptr(),
-                                     None if arrs[1] is None else arrs[1].data_ptr(),
-                                     1 if stop_at_first_reject else 0,
-                                     int(seed), int(offset), int(b_first),
-                                     acc.data_ptr(), tok.data_ptr(), *ptrs, ws_ptr, ws_bytes, _stream_ptr(stream))
+            flags = (1 if stop_at_first_reject else 0) | (2 if uncertainty == "entropy" else 0)
+            head = (_dtype_code(t), t.data_ptr(), d.data_ptr(), x.data_ptr(), B, K, V, float(temperature), float(beta),
+                    None if arrs[0] is None else arrs[0].data_ptr(), None if arrs[1] is None else arrs[1].data_ptr(),
+                    flags, int(seed), int(offset), int(b_first), acc.data_ptr(), tok.data_ptr())
+            if uncertainty == "entropy" or ent is not None:
+                rc = lib.ears_verify_entropy(*head, *ptrs, None if ent is None else ent.data_ptr(), ws_ptr, ws_bytes,
+                                             _stream_ptr(stream))
+            else:
+                rc = lib.ears_verify_var(*head, *ptrs, ws_ptr, ws_bytes, _stream_ptr(stream))
     _check(rc)
-    return (acc, tok, st) if stats else (acc, tok)
+    return (acc, tok, st) if st is not None else (acc, tok)
 
 
 def verify_greedy(target_logits: torch.Tensor, draft_tokens: torch.Tensor, *, workspace: Optional[torch.Tensor] = None,

@@ -169,7 +169,7 @@ Plan make_plan(int B, int K, int V, int esize, bool aligned, int sms, const Plan
 
 struct Layout {
     size_t ticket1, ticket2, job_ctr, ticket_row, ready, heads, wq, counters_bytes;
-    size_t partial, rowstat, pt_tok, pd_tok, max_pt, cls, resid, seg, seg_stride, total;
+    size_t partial, rowstat, partial_w, roww, pt_tok, pd_tok, max_pt, cls, resid, seg, seg_stride, total;
 };
 
 Layout make_layout(int B, int K, int V, int parts1) {
@@ -188,6 +188,8 @@ Layout make_layout(int B, int K, int V, int parts1) {
     o = align_up(o, 256);
     L.partial = o; o = align_up(o + rows * parts1 * sizeof(float2), 256);
     L.rowstat = o; o = align_up(o + rows * sizeof(float2), 256);
+    L.partial_w = o; o = align_up(o + rows * parts1 * sizeof(float), 256);   // (entropy kernels)
+    L.roww = o; o = align_up(o + rows * sizeof(float), 256);
     L.pt_tok = o; o = align_up(o + (size_t)B * K * 8, 256);
     L.pd_tok = o; o = align_up(o + (size_t)B * K * 8, 256);
     L.max_pt = o; o = align_up(o + (size_t)B * K * 8, 256);
@@ -359,9 +361,12 @@ int profile_mark(cudaStream_t stream, bool timed) {
 
 template <typename E>
 int set_attrs_streamed(bool* cluster16) {
-    EARS_CUDA(cudaFuncSetAttribute(ears_cstream_kernel<E>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    EARS_CUDA(cudaFuncSetAttribute(ears_cstream_kernel<E, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    (int)(streamed_smem(0) + kStreamedSegBytes)));
-    if (cudaFuncSetAttribute(ears_cstream_kernel<E>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
+    EARS_CUDA(cudaFuncSetAttribute(ears_cstream_kernel<E, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)(streamed_smem(0) + kStreamedSegBytes)));
+    if (cudaFuncSetAttribute(ears_cstream_kernel<E, false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
+        cudaFuncSetAttribute(ears_cstream_kernel<E, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
         (void)cudaGetLastError();
         *cluster16 = false;
     }
@@ -372,17 +377,20 @@ template <typename E>
 int set_attrs(bool* cluster16) {
     int rc = set_attrs_streamed<E>(cluster16);
     if (rc) return rc;
-    EARS_CUDA(cudaFuncSetAttribute(ears_verify_kernel<E, kStages, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   (int)smem_bytes()));
-    EARS_CUDA(cudaFuncSetAttribute(ears_verify_kernel<E, kStages, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   (int)smem_bytes()));
-    EARS_CUDA(cudaFuncSetAttribute(ears_resident_kernel<E>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   (int)kResidentSmem2));
+    EARS_CUDA(cudaFuncSetAttribute(ears_verify_kernel<E, kStages, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes()));
+    EARS_CUDA(cudaFuncSetAttribute(ears_verify_kernel<E, kStages, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes()));
+    EARS_CUDA(cudaFuncSetAttribute(ears_verify_kernel<E, kStages, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes()));
+    EARS_CUDA(cudaFuncSetAttribute(ears_verify_kernel<E, kStages, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes()));
+    EARS_CUDA(cudaFuncSetAttribute(ears_resident_kernel<E, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kResidentSmem2));
+    EARS_CUDA(cudaFuncSetAttribute(ears_resident_kernel<E, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kResidentSmem2));
     // several CTAs per SM only fit when the SM's memory is configured as shared memory
-    EARS_CUDA(cudaFuncSetAttribute(ears_resident_kernel<E>, cudaFuncAttributePreferredSharedMemoryCarveout,
+    EARS_CUDA(cudaFuncSetAttribute(ears_resident_kernel<E, false>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                   (int)cudaSharedmemCarveoutMaxShared));
+    EARS_CUDA(cudaFuncSetAttribute(ears_resident_kernel<E, true>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                    (int)cudaSharedmemCarveoutMaxShared));
     // clusters of more than 8 CTAs are an opt-in; without it the plans stop at 8
-    if (cudaFuncSetAttribute(ears_resident_kernel<E>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
+    if (cudaFuncSetAttribute(ears_resident_kernel<E, false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
+        cudaFuncSetAttribute(ears_resident_kernel<E, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
         (void)cudaGetLastError();
         *cluster16 = false;
     }
@@ -408,8 +416,9 @@ int resident_clusters(DeviceInfo* di, const RPlan& rp, int dtype, int* out) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int n = 0;
-    const cudaError_t qe = rp.streamed ? cudaOccupancyMaxActiveClusters(&n, ears_cstream_kernel<E>, &cfg)
-                                       : cudaOccupancyMaxActiveClusters(&n, ears_resident_kernel<E>, &cfg);
+    // (the entropy variants have the same footprint)
+    const cudaError_t qe = rp.streamed ? cudaOccupancyMaxActiveClusters(&n, ears_cstream_kernel<E, false>, &cfg)
+                                       : cudaOccupancyMaxActiveClusters(&n, ears_resident_kernel<E, false>, &cfg);
     if (qe != cudaSuccess) {
         (void)cudaGetLastError();
         n = 0;
@@ -437,8 +446,11 @@ int launch_resident(RParams& p, const RPlan& rp, int max_clusters, cudaStream_t 
     const bool timed = profile_wanted();
     int rc = profile_mark(stream, timed);
     if (rc) return rc;
-    if (rp.streamed) EARS_CUDA(cudaLaunchKernelEx(&cfg, ears_cstream_kernel<E>, p));
-    else EARS_CUDA(cudaLaunchKernelEx(&cfg, ears_resident_kernel<E>, p));
+    const bool ent = p.unc_entropy || p.entropy;
+    if (rp.streamed && ent) EARS_CUDA(cudaLaunchKernelEx(&cfg, ears_cstream_kernel<E, true>, p));
+    else if (rp.streamed) EARS_CUDA(cudaLaunchKernelEx(&cfg, ears_cstream_kernel<E, false>, p));
+    else if (ent) EARS_CUDA(cudaLaunchKernelEx(&cfg, ears_resident_kernel<E, true>, p));
+    else EARS_CUDA(cudaLaunchKernelEx(&cfg, ears_resident_kernel<E, false>, p));
     return profile_mark(stream, timed);
 }
 
@@ -450,15 +462,22 @@ int launch(const Params& p, int sms, bool direct, cudaStream_t stream) {
     const bool timed = profile_wanted();
     int rc = profile_mark(stream, timed);
     if (rc) return rc;
+    const bool ent = p.unc_entropy || p.entropy;
     if (direct) {
         const long long dcap = (long long)sms * kDCtasPerSm;
         const int dgrid = (int)(units < dcap ? units : dcap);
-        if (p.seq_T) ears_direct_kernel<E, true><<<dgrid, kDThreads + 32, 0, stream>>>(p);
-        else ears_direct_kernel<E, false><<<dgrid, kDThreads + 32, 0, stream>>>(p);
+        if (p.seq_T && ent) ears_direct_kernel<E, true, true><<<dgrid, kDThreads + 32, 0, stream>>>(p);
+        else if (p.seq_T) ears_direct_kernel<E, true, false><<<dgrid, kDThreads + 32, 0, stream>>>(p);
+        else if (ent) ears_direct_kernel<E, false, true><<<dgrid, kDThreads + 32, 0, stream>>>(p);
+        else ears_direct_kernel<E, false, false><<<dgrid, kDThreads + 32, 0, stream>>>(p);
+    } else if (p.seq_T && ent) {
+        ears_verify_kernel<E, kStages, true, true><<<grid, kThreads, smem_bytes(), stream>>>(p);
     } else if (p.seq_T) {
-        ears_verify_kernel<E, kStages, true><<<grid, kThreads, smem_bytes(), stream>>>(p);
+        ears_verify_kernel<E, kStages, true, false><<<grid, kThreads, smem_bytes(), stream>>>(p);
+    } else if (ent) {
+        ears_verify_kernel<E, kStages, false, true><<<grid, kThreads, smem_bytes(), stream>>>(p);
     } else {
-        ears_verify_kernel<E, kStages, false><<<grid, kThreads, smem_bytes(), stream>>>(p);
+        ears_verify_kernel<E, kStages, false, false><<<grid, kThreads, smem_bytes(), stream>>>(p);
     }
     EARS_CUDA(cudaGetLastError());
     return profile_mark(stream, timed);
@@ -624,10 +643,12 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
                 float temperature, float beta, const float* seq_T, const float* seq_beta, unsigned flags,
                 uint64_t seed, uint64_t offset, int64_t b_first,
                 int32_t* out_len, int32_t* out_tok, double* o_pt, double* o_pd, double* o_max,
-                uint8_t* o_cls, double* o_resid, void* workspace, size_t workspace_bytes, void* stream_) {
+                uint8_t* o_cls, double* o_resid, void* workspace, size_t workspace_bytes, void* stream_,
+                double* o_entropy = nullptr) {
     int rc = check_arguments(dtype, t, d, x, B, K, V, temperature, beta, seq_T, seq_beta, flags, b_first, out_len, out_tok);
     if (rc) return rc;
     const int stop_first = (flags & EARS_FLAG_STOP_AT_FIRST_REJECT) ? 1 : 0;
+    const int unc_entropy = (flags & EARS_FLAG_ENTROPY_UNCERTAINTY) ? 1 : 0;
     if (seq_T) temperature = 1.0f;
     if (seq_beta) beta = 0.0f;
     const int esize = dtype_size(dtype);
@@ -688,6 +709,8 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
         p.n_clusters = 0;
         p.want_stats = (o_pt || o_pd || o_max || o_cls) ? 1 : 0;
         p.ordered = stop_first;
+        p.unc_entropy = unc_entropy;
+        p.entropy = o_entropy;
         rc = by_dtype(dtype, [&](auto* e) {
             return launch_resident<std::remove_pointer_t<decltype(e)>>(p, rp, max_clusters, stream);
         });
@@ -733,6 +756,10 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
     p.seg_base = (unsigned char*)(w + L.seg);
     p.seg_stride = L.seg_stride;
     p.stop_first = stop_first;
+    p.unc_entropy = unc_entropy;
+    p.entropy = o_entropy;
+    p.partial_w = (float*)(w + L.partial_w);
+    p.roww = (float*)(w + L.roww);
     p.plan = plan;
     rc = by_dtype(dtype, [&](auto* e) { return launch<std::remove_pointer_t<decltype(e)>>(p, di->sms, direct, stream); });
     if (rc && !workspace) forget_clean_counters(dev, stream_);
@@ -912,6 +939,19 @@ int ears_verify_var(int dtype, const void* target_logits, const void* draft_logi
     return verify_impl(dtype, target_logits, draft_logits, draft_tokens, B, K, V, temperature, beta,
                        seq_temperature, seq_beta, flags, seed, offset, b_first, out_accept_len, out_tokens, out_pt_tok,
                        out_pd_tok, out_max_pt, out_class, out_resid_mass, workspace, workspace_bytes, stream);
+}
+
+int ears_verify_entropy(int dtype, const void* target_logits, const void* draft_logits,
+                        const int32_t* draft_tokens, int B, int K, int V, float temperature, float beta,
+                        const float* seq_temperature, const float* seq_beta, unsigned flags,
+                        uint64_t seed, uint64_t offset, int64_t b_first, int32_t* out_accept_len,
+                        int32_t* out_tokens, double* out_pt_tok, double* out_pd_tok, double* out_max_pt,
+                        uint8_t* out_class, double* out_resid_mass, double* out_entropy,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+    if ((uintptr_t)out_entropy % 8) return EARS_ERR_ALIGN;
+    return verify_impl(dtype, target_logits, draft_logits, draft_tokens, B, K, V, temperature, beta,
+                       seq_temperature, seq_beta, flags, seed, offset, b_first, out_accept_len, out_tokens, out_pt_tok,
+                       out_pd_tok, out_max_pt, out_class, out_resid_mass, workspace, workspace_bytes, stream, out_entropy);
 }
 
 int ears_verify_greedy(int dtype, const void* target_logits, const int32_t* draft_tokens, int B, int K, int V,
@@ -1134,8 +1174,8 @@ int ears_describe_plan(int dtype, int B, int K, int V, char* out, size_t out_byt
         int per_sm = 0;
         by_dtype(dtype, [&](auto* e) {
             using El = std::remove_pointer_t<decltype(e)>;
-            return rp.streamed ? (int)cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ears_cstream_kernel<El>, kCThreads, rp.smem)
-                               : (int)cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ears_resident_kernel<El>, kRThreads, rp.smem);
+            return rp.streamed ? (int)cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ears_cstream_kernel<El, false>, kCThreads, rp.smem)
+                               : (int)cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ears_resident_kernel<El, false>, kRThreads, rp.smem);
         });
         snprintf(out, out_bytes, rp.streamed ? "cluster-streamed: cluster=%d slice_elems=%d smem_bytes=%zu ctas_per_sm=%d clusters_resident=%d clusters_launched=%lld" :
                  "resident: cluster=%d slice_elems=%d smem_bytes=%zu ctas_per_sm=%d clusters_resident=%d clusters_launched=%lld",

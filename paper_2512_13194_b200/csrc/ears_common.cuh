@@ -85,6 +85,10 @@ struct Params {
     unsigned char* seg_base;
     size_t seg_stride;
     int stop_first;       // 1: what lies after a sequence's first rejection is neither validated nor reported
+    int unc_entropy;      // 1: the tolerance is scaled by H(P_t) / ln V instead of 1 - max P_t [Sec. 5 item 1]
+    double* entropy;      // [B,K] H(P_t) of every target row, or NULL; the entropy kernels (ENT) fill it
+    float* partial_w;     // [B*(2K+1)*parts1] sum e t per row piece (ENT kernels)
+    float* roww;          // [B*(2K+1)] sum e t per row (ENT kernels)
     int* zero_ptr;        // counter block of the next call, cleared by this kernel (zero_words ints; may be 0)
     int zero_words;
     Plan plan;

@@ -47,6 +47,7 @@ struct CSmem {
     alignas(8) uint64_t xbar[2];          // statistics exchange, alternating by round
     uint64_t mbar2[2];                    // mass-total exchange, alternating by mass round
     alignas(16) float4 xstat[2][kRMaxCluster * kCWarps];   // (m_t, s_t, m_d, s_d) of every warp of every peer
+    float xw[2][kRMaxCluster * kCWarps];  // sum e t of the target slice of every warp of every peer (entropy kernels)
     double xmass[2][kRMaxCluster];        // mass totals of every peer
     int xnext[2];                         // next queue entry of the cluster (written by rank 0)
     int2 xjob[2][kRMaxCluster];           // second-pass job each peer announces: (sequence, position) or (-1, 0)
@@ -202,7 +203,7 @@ __device__ __forceinline__ int finish_streamed_sequence(const RParams& p, int b,
     return n;
 }
 
-template <typename E>
+template <typename E, bool ENT>
 __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(const RParams p) {
     extern __shared__ unsigned char smem_raw[];
     CSmem& sm = *reinterpret_cast<CSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
@@ -284,9 +285,10 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
         // ---- 1. statistics of this CTA's slices
         if (tid == 0) trace_mark(1, work ? b * (K + 1) + j : -1);
         float2 pt2 = make_float2(-INFINITY, 0.f), pd2 = make_float2(-INFINITY, 0.f);
+        float wv = 0.f;   // ENT: the thread's sum e t over the target slice
         if (work) {
             if (pair) {
-                pt2 = stream_piece<E, kCThreads>(trow, e0, e0 + n, vec, cb, tid);
+                pt2 = stream_piece<E, kCThreads, ENT>(trow, e0, e0 + n, vec, cb, tid, &wv);
                 pd2 = stream_piece<E, kCThreads>(drow, e0, e0 + n, vec, cb, tid);
             } else {
                 pt2 = stream_bonus_piece<E>(trow, e0, e0 + n, vec, cb, warp, lane, bseg - e0 / BSEG);
@@ -302,11 +304,13 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
                 Mt = fmaxf(Mt, __shfl_xor_sync(0xffffffffu, Mt, off));
                 Md = fmaxf(Md, __shfl_xor_sync(0xffffffffu, Md, off));
             }
-            float St = rebase_sum(pt2.x, pt2.y, Mt, cb), Sd = rebase_sum(pd2.x, pd2.y, Md, cb);
+            const float2 sw = ENT ? rebase_sum_w(pt2.x, pt2.y, wv, Mt, cb) : make_float2(rebase_sum(pt2.x, pt2.y, Mt, cb), 0.f);
+            float St = sw.x, Wt = sw.y, Sd = rebase_sum(pd2.x, pd2.y, Md, cb);
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) {
                 St += __shfl_xor_sync(0xffffffffu, St, off);
                 Sd += __shfl_xor_sync(0xffffffffu, Sd, off);
+                if (ENT) Wt += __shfl_xor_sync(0xffffffffu, Wt, off);
             }
             // ---- 2. every warp hands its partial result to every CTA of the cluster (itself included);
             //         warp 0 adds the next queue entry (rank 0) and the job this CTA has to announce
@@ -314,6 +318,7 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
             if (lane < C) {
                 peer_store(map_to_peer(smem_u32(&sm.xstat[par][rank * kCWarps + warp]), (uint32_t)lane),
                            make_float4(Mt, St, Md, Sd));
+                if (ENT) peer_store(map_to_peer(smem_u32(&sm.xw[par][rank * kCWarps + warp]), (uint32_t)lane), Wt);
                 if (warp == 0) {
                     if (rank == 0) peer_store(map_to_peer(smem_u32(&sm.xnext[par]), (uint32_t)lane), nx);
                     peer_store(map_to_peer(smem_u32(&sm.xjob[par][rank]), (uint32_t)lane), make_int2(sm.my_job_b, sm.my_job_n));
@@ -339,58 +344,15 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
         const int qj = (q_have && !ordered) ? (int)(nxt % (K + 1)) : 0;
         // ---- 3. the rows' (max, Z) and the decision
         if (work && warp == 0) {
-            // C x 8 partial results, lane i takes entries i, i + 32, ...: the same in every CTA, hence identical bits
-            const int parts = C * kCWarps;
-            float mt = -INFINITY, md = -INFINITY;
-            for (int i = lane; i < parts; i += 32) {
-                mt = fmaxf(mt, sm.xstat[par][i].x);
-                md = fmaxf(md, sm.xstat[par][i].z);
-            }
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-                mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, off));
-                md = fmaxf(md, __shfl_xor_sync(0xffffffffu, md, off));
-            }
-            float zt = 0.f, zd = 0.f;
-            for (int i = lane; i < parts; i += 32) {
-                const float4 v = sm.xstat[par][i];
-                zt += rebase_sum(v.x, v.y, mt, cb);
-                zd += rebase_sum(v.z, v.w, md, cb);
-            }
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-                zt += __shfl_xor_sync(0xffffffffu, zt, off);
-                zd += __shfl_xor_sync(0xffffffffu, zd, off);
-            }
+            float mt, zt, md, zd, wt;
+            merge_exchanged<ENT>(sm.xstat[par], sm.xw[par], C * kCWarps, cb, lane, mt, zt, md, zd, wt);
             if (lane == 0) {
                 const double Tb = seq_temperature(p, b), betab = seq_beta(p, b);
                 int dec = 1;
                 if (!rowstat_ok(mt, zt) || (pair && (!rowstat_ok(md, zd) || !tok_ok)) || !seq_params_ok(Tb, betab)) dec = -1;
                 sm.rs_t = make_float2(mt, zt);
                 sm.rs_d = pair ? make_float2(md, zd) : make_float2(0.f, 1.f);
-                if (pair && dec >= 0) {
-                    // fp32 first; it stands unless R comes close to the threshold (the band is some 25 times
-                    // the fp32 error) or the caller wants the probabilities: then fp64.  Every CTA of the
-                    // cluster runs the same arithmetic on the same numbers.
-                    const float pt32 = ex2_approx((lt - mt) * cb) / zt;
-                    const float pd32 = ex2_approx((ld - md) * cb) / zd;
-                    const float ratio32 = pt32 / fmaxf(pd32, (float)kEps);
-                    const float thr32 = fmaxf((float)U - (float)betab * (1.0f - 1.0f / zt), 0.0f);
-                    const float diff = ratio32 - thr32;
-                    if (!p.want_stats && fabsf(diff) > 1e-4f * (ratio32 + thr32) + 1e-6f) {
-                        dec = diff > 0.0f ? 1 : 0;
-                    } else {
-                        const Decision dc = decide_position((double)lt, (double)ld, sm.rs_t, sm.rs_d, Tb, betab, U);
-                        dec = dc.accept ? 1 : 0;
-                        if (rank == 0 && p.want_stats) {
-                            const size_t i = (size_t)b * K + j;
-                            p.pt_tok[i] = dc.pt;
-                            p.pd_tok[i] = dc.pd;
-                            p.max_pt[i] = dc.maxp;
-                            p.cls[i] = (uint8_t)dc.cls;
-                        }
-                    }
-                }
+                if (pair && dec >= 0) dec = cluster_decide<ENT>(p, b, j, lt, ld, U, sm.rs_t, sm.rs_d, wt, cb, Tb, betab, rank == 0);
                 sm.dec = dec;
             }
         }

@@ -62,11 +62,11 @@ __device__ __forceinline__ uint4 ld_stream16(const void* p) {
 }
 
 // An ordinary row piece [e0, e1): THREADS threads (tid = 0 .. THREADS-1) stride over it.
-// -> the thread's (m, s).
-template <typename E, int THREADS = kDThreads>
-__device__ __forceinline__ float2 stream_piece(const E* row, int e0, int e1, bool vec, float c, int tid) {
+// -> the thread's (m, s); ENT: also *w_out = its sum e t (see RowAccT).
+template <typename E, int THREADS = kDThreads, bool ENT = false>
+__device__ __forceinline__ float2 stream_piece(const E* row, int e0, int e1, bool vec, float c, int tid, float* w_out = nullptr) {
     constexpr int N = Words<E>::N;
-    RowAcc a;
+    RowAccT<ENT> a;
     acc_open(a);
     if (vec) {
         const uint4* vs = reinterpret_cast<const uint4*>(row + e0);
@@ -76,15 +76,15 @@ __device__ __forceinline__ float2 stream_piece(const E* row, int e0, int e1, boo
             uint4 w[kDUnroll];
 #pragma unroll
             for (int j = 0; j < kDUnroll; ++j) w[j] = ld_stream16(vs + v + j * THREADS);
-            fold_vectors<E, kDUnroll>(w, c, a);
+            fold_vectors<E, kDUnroll, ENT>(w, c, a);
         }
         for (; v + THREADS < nvec; v += 2 * THREADS) {   // what is left of a piece: two, then one at a time
             uint4 w[2] = {ld_stream16(vs + v), ld_stream16(vs + v + THREADS)};
-            fold_vectors<E, 2>(w, c, a);
+            fold_vectors<E, 2, ENT>(w, c, a);
         }
         for (; v < nvec; v += THREADS) {
             uint4 w[1] = {ld_stream16(vs + v)};
-            fold_vectors<E, 1>(w, c, a);
+            fold_vectors<E, 1, ENT>(w, c, a);
         }
     } else {  // rows that are not 16-byte aligned: element by element
         for (int i = e0 + tid; i < e1; i += THREADS) {
@@ -93,7 +93,7 @@ __device__ __forceinline__ float2 stream_piece(const E* row, int e0, int e1, boo
             acc_add_one(a, x, c);
         }
     }
-    return acc_close(a, c);
+    return acc_close(a, c, w_out);
 }
 
 // A piece [e0, e1) of the extra target row: warp w takes the segments w, w + kDWarps, ... of
@@ -263,7 +263,7 @@ __device__ __forceinline__ void arrive_B(int it) { if (it & 1) nb_arrive_id<4>()
 
 // Control-warp side of a finished work item: publish and count the piece, and do what falls to
 // the CTA that delivered a sequence's last piece.
-template <typename E, bool PER_SEQ>
+template <typename E, bool PER_SEQ, bool ENT>
 __device__ __forceinline__ void direct_epilogue(const Params& p, const DWork& wk, const float4* red, int lane) {
     const int K = p.K, R = 2 * K + 1, P = p.plan.parts1, P2 = p.plan.parts2;
     if (wk.kind == kDUnit) {
@@ -276,12 +276,17 @@ __device__ __forceinline__ void direct_epilogue(const Params& p, const DWork& wk
         float MM = v.x;
 #pragma unroll
         for (int off = kDWarps / 2; off > 0; off >>= 1) MM = fmaxf(MM, __shfl_xor_sync(0xffffffffu, MM, off));
-        float SS = rebase_sum(v.x, v.y, MM, c);
+        const float2 sw = ENT ? rebase_sum_w(v.x, v.y, v.z, MM, c) : make_float2(rebase_sum(v.x, v.y, MM, c), 0.f);
+        float SS = sw.x, WW = sw.y;
 #pragma unroll
-        for (int off = kDWarps / 2; off > 0; off >>= 1) SS += __shfl_xor_sync(0xffffffffu, SS, off);
+        for (int off = kDWarps / 2; off > 0; off >>= 1) {
+            SS += __shfl_xor_sync(0xffffffffu, SS, off);
+            if (ENT) WW += __shfl_xor_sync(0xffffffffu, WW, off);
+        }
         int last_b = -1;
         if (lane == 0) {
             p.partial[((size_t)b * R + ridx) * P + part] = make_float2(MM, SS);
+            if (ENT) p.partial_w[((size_t)b * R + ridx) * P + part] = WW;
             // two-level count (row, then sequence) keeps same-address atomics rare; the atomics
             // release this piece and acquire the others
             bool row_done = true;
@@ -292,7 +297,7 @@ __device__ __forceinline__ void direct_epilogue(const Params& p, const DWork& wk
         if (last_b >= 0) {
             // this CTA delivered the sequence's last piece: decide it
             __threadfence();
-            const int n = finalize_sequence<E>(p, last_b, lane);
+            const int n = finalize_sequence<E, ENT>(p, last_b, lane);
             __threadfence();
             __syncwarp();
             if (n == K) {
@@ -329,7 +334,7 @@ __device__ __forceinline__ void direct_epilogue(const Params& p, const DWork& wk
 //             arrive on B(it) and go on.
 // A and B alternate between two barrier ids by the parity of `it`; a generation always gets
 // exactly one arrival from every streaming thread and every control lane, on every path.
-template <typename E, bool PER_SEQ>
+template <typename E, bool PER_SEQ, bool ENT>
 __global__ void __launch_bounds__(kDThreads + 32, kDCtasPerSm) ears_direct_kernel(const Params p) {
     __shared__ DSmem sm;
     constexpr int CHUNK_ELEMS = kChunkBytes / (int)sizeof(E);
@@ -402,7 +407,7 @@ __global__ void __launch_bounds__(kDThreads + 32, kDCtasPerSm) ears_direct_kerne
                 if (!prev_done) {
                     sync_B(it - 1);
                     if (lane == 0) trace_mark(15, 1);
-                    direct_epilogue<E, PER_SEQ>(p, prev, sm.red[(it - 1) & 1], lane);
+                    direct_epilogue<E, PER_SEQ, ENT>(p, prev, sm.red[(it - 1) & 1], lane);
                     if (lane == 0) trace_mark(16, 1);
                     prev_done = true;
                     continue;
@@ -435,7 +440,7 @@ __global__ void __launch_bounds__(kDThreads + 32, kDCtasPerSm) ears_direct_kerne
             if (!prev_done) {
                 sync_B(it - 1);                               // B(it - 1): the previous item's results are in
                 if (lane == 0) trace_mark(15, 0);
-                direct_epilogue<E, PER_SEQ>(p, prev, sm.red[(it - 1) & 1], lane);
+                direct_epilogue<E, PER_SEQ, ENT>(p, prev, sm.red[(it - 1) & 1], lane);
                 if (lane == 0) trace_mark(16, 0);
             }
             if (wk.kind == kDExit) break;
@@ -460,16 +465,22 @@ __global__ void __launch_bounds__(kDThreads + 32, kDCtasPerSm) ears_direct_kerne
                 const int e0 = min(V, part * cpp * CHUNK_ELEMS);
                 const int e1 = min(V, min(chunks_per_row, (part + 1) * cpp) * CHUNK_ELEMS);
                 float2 ms;
+                float wv = 0.f;   // ENT: the thread's sum e t (target rows of positions only; the others do not need it)
                 if (bonus) ms = stream_bonus_piece<E>(row, e0, e1, vec, c, warp, lane, bonus_segs(p, b));
+                else if (ENT && !(ridx & 1)) ms = stream_piece<E, kDThreads, true>(row, e0, e1, vec, c, tid, &wv);
                 else ms = stream_piece<E>(row, e0, e1, vec, c, tid);
                 // (max, sum) of the warp: the maximum first, one rescale per thread, then a sum
                 float M = ms.x;
 #pragma unroll
                 for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
-                float S = rebase_sum(ms.x, ms.y, M, c);
+                const float2 sw = ENT ? rebase_sum_w(ms.x, ms.y, wv, M, c) : make_float2(rebase_sum(ms.x, ms.y, M, c), 0.f);
+                float S = sw.x, W = sw.y;
 #pragma unroll
-                for (int off = 16; off > 0; off >>= 1) S += __shfl_xor_sync(0xffffffffu, S, off);
-                if (lane == 0) sm.red[it & 1][warp] = make_float4(M, S, 0.f, 0.f);
+                for (int off = 16; off > 0; off >>= 1) {
+                    S += __shfl_xor_sync(0xffffffffu, S, off);
+                    if (ENT) W += __shfl_xor_sync(0xffffffffu, W, off);
+                }
+                if (lane == 0) sm.red[it & 1][warp] = make_float4(M, S, W, 0.f);
             } else {
                 // second pass: one piece of the two rows of sequence b's first rejected position n
                 __threadfence();

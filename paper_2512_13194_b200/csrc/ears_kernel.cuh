@@ -141,7 +141,7 @@ struct PipeSmem {
     uint64_t empty[STAGES];
     uint64_t unit_bar[kUnitSlots];
     StageMeta meta[STAGES];
-    float2 scratch[kUnitSlots][kConsumerWarps];
+    float4 scratch[kUnitSlots][kConsumerWarps];   // (m, s, sum e t, -) of each consumer warp at a unit's end
     volatile int units_read;   // unit ends the epilogue warp has taken out of the slots
     Mailbox<kEpiCap> epi;
     Mailbox<kSeqCap> seq;
@@ -229,9 +229,9 @@ __device__ __forceinline__ void loader_fill(PipeSmem<STAGES>& sm, int stage, con
 // of its eighth of the chunk together with the reference the terms were taken against.  If every
 // draft token turns out to be accepted, the final token is drawn from exactly these sums and the
 // row is not read again.
-template <typename E, bool BONUS>
+template <typename E, bool BONUS, bool ENT>
 __device__ __forceinline__ void chunk_stats(const unsigned char* buf, int nelem, int warp, int lane, float c,
-                                            RowAcc& a, BonusSeg* warp_chunk_out) {
+                                            RowAccT<ENT>& a, BonusSeg* warp_chunk_out) {
     constexpr int N = Words<E>::N, PN = N / 2;
     constexpr int VECS = kChunkBytes / 16 / kConsumers;  // 16-byte vectors per thread per chunk
     constexpr int CHUNK_ELEMS = kChunkBytes / (int)sizeof(E);
@@ -243,7 +243,7 @@ __device__ __forceinline__ void chunk_stats(const unsigned char* buf, int nelem,
         for (int j = 0; j < VECS; ++j) w[j] = Words<E>::mask_tail(w[j], nelem - ((warp * VECS + j) * 32 + lane) * N);
     }
     if (!BONUS) {
-        fold_vectors<E, VECS>(w, c, a);
+        fold_vectors<E, VECS, ENT>(w, c, a);
         return;
     }
     float cm = Words<E>::template vmax_all<VECS>(w);
@@ -337,7 +337,7 @@ __device__ __forceinline__ void chunk_segments(const unsigned char* bt, const un
 // Merges the pieces of all 2K+1 rows, writes (m, Z) per row, decides every position
 // (Sec. 3.2 steps 1-5 with the guards of Sec. 3.3 item 2) and writes the accepted
 // prefix (Sec. 3.1).  Returns the accepted length n, or -1 for an invalid sequence.
-template <typename E>
+template <typename E, bool ENT>
 __device__ int finalize_sequence(const Params& p, int b, int lane) {
     const int K = p.K, R = 2 * K + 1, V = p.V, P = p.plan.parts1;
     const E* t = reinterpret_cast<const E*>(p.t);
@@ -358,6 +358,16 @@ __device__ int finalize_sequence(const Params& p, int b, int lane) {
         }
         if (!rowstat_ok(m, s) && !stop_first) bad = true;
         p.rowstat[(size_t)b * R + r] = make_float2(m, s);
+        if (ENT && !(r & 1) && r < 2 * K) {
+            // sum e t of a target row: its pieces brought to the row maximum (known now)
+            const float* pw = p.partial_w + ((size_t)b * R + r) * P;
+            float w = 0.f;
+            for (int i = 0; i < P; ++i) {
+                const float2 v = __ldcg(pp + i);
+                w += rebase_sum_w(v.x, v.y, __ldcg(pw + i), m, cb).y;
+            }
+            p.roww[(size_t)b * R + r] = w;
+        }
     }
     __syncwarp();
     int first_reject = K;
@@ -376,7 +386,13 @@ __device__ int finalize_sequence(const Params& p, int b, int lane) {
                 const double lt = (double)load_logit(t + (size_t)target_row(b, k, K) * V + tok);
                 const double ld = (double)load_logit(d + (size_t)draft_row(b, k, K) * V + tok);
                 const double U = uniform_accept(p.seed, p.offset, (uint32_t)(p.b_first + b), (uint32_t)k);
-                const Decision dc = decide_position(lt, ld, st, sd, Tb, betab, U);
+                double unc = -1.0;   // < 0: the printed measure, 1 - max P_t
+                if (ENT) {
+                    const double H = row_entropy(st.y, __ldcg(&p.roww[(size_t)b * R + 2 * k]));
+                    if (p.entropy) p.entropy[(size_t)b * K + k] = H;
+                    if (p.unc_entropy) unc = entropy_uncertainty(H, V);
+                }
+                const Decision dc = decide_position(lt, ld, st, sd, Tb, betab, U, unc);
                 reject = !dc.accept;
                 const size_t i = (size_t)b * K + k;
                 p.pt_tok[i] = dc.pt;
@@ -610,7 +626,7 @@ __device__ void select_token(const Params& p, int b, int n, int lane) {
 // ---- the kernel -------------------------------------------------------------------
 // PER_SEQ: the call carries per-sequence temperatures, so log2(e)/T comes with every slot;
 // otherwise it is the kernel parameter (kept apart: the consumers' code is sensitive to it).
-template <typename E, int STAGES, bool PER_SEQ>
+template <typename E, int STAGES, bool PER_SEQ, bool ENT>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const Params p) {
     extern __shared__ unsigned char smem_raw[];
     using Smem = PipeSmem<STAGES>;
@@ -789,12 +805,18 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
                 slot_ok = mbar_wait(&sm.unit_bar[m.c % kUnitSlots], (m.c / kUnitSlots) & 1, &sm.abort_flag);
                 top = m.c;
             }
-            float pm = -INFINITY, ps = 0.f;
+            float pm = -INFINITY, ps = 0.f, pw = 0.f;
             if (m.kind == kMsgPiece && slot_ok) {
                 const float cu = PER_SEQ ? seq_c(p, m.a / (R * P)) : p.c;
                 for (int w = 0; w < kConsumerWarps; ++w) {
-                    const float2 v = sm.scratch[m.c % kUnitSlots][w];
+                    const float4 v = sm.scratch[m.c % kUnitSlots][w];
                     merge_ms(pm, ps, v.x, v.y, cu);
+                }
+                if (ENT) {   // sum e t of the piece, relative to the piece's maximum (known now)
+                    for (int w = 0; w < kConsumerWarps; ++w) {
+                        const float4 v = sm.scratch[m.c % kUnitSlots][w];
+                        pw += rebase_sum_w(v.x, v.y, v.z, pm, cu).y;
+                    }
                 }
             }
 #pragma unroll
@@ -808,6 +830,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
                 const int b = m.a / (R * P);
                 const int rem = m.a % (R * P);
                 p.partial[((size_t)b * R + rem / P) * P + rem % P] = make_float2(pm, ps);
+                if (ENT) p.partial_w[((size_t)b * R + rem / P) * P + rem % P] = pw;
                 // two-level count (row, then sequence) spreads the atomics over many addresses
                 bool row_done = true;
                 if (P > 1) row_done = ticket_add(&p.ticket_row[(size_t)b * R + rem / P]) == P - 1;
@@ -883,7 +906,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
             idle_t0 = 0;
             __threadfence();
             if (kind == 0) {
-                n = finalize_sequence<E>(p, b, lane);
+                n = finalize_sequence<E, ENT>(p, b, lane);
                 if (n == K) {
                     // every draft accepted: the sums of the extra row are already there
                     __threadfence();
@@ -909,7 +932,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
         }
     } else {
         // =============================== consumer warps
-        RowAcc acc;
+        RowAccT<ENT> acc;
         acc_open(acc);
         int unit_ends = 0;   // ends of units and pieces seen so far (same in every consumer warp)
         RowNorm rn{0.f, 0.f, 0.f, 0.f, 0.0};
@@ -925,9 +948,9 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
                 if (mt.flags & 1) acc_open(acc);
                 if (mt.aux) {  // a piece of the extra target row
                     BonusSeg* out = bonus_segs(p, mt.id / (R * P)) + (size_t)(mt.elem0 / CHUNK_ELEMS) * kConsumerWarps + warp;
-                    chunk_stats<E, true>(sm.buf[stage], mt.nelem, warp, lane, PER_SEQ ? mt.c : p.c, acc, out);
+                    chunk_stats<E, true, ENT>(sm.buf[stage], mt.nelem, warp, lane, PER_SEQ ? mt.c : p.c, acc, out);
                 } else {
-                    chunk_stats<E, false>(sm.buf[stage], mt.nelem, warp, lane, PER_SEQ ? mt.c : p.c, acc, nullptr);
+                    chunk_stats<E, false, ENT>(sm.buf[stage], mt.nelem, warp, lane, PER_SEQ ? mt.c : p.c, acc, nullptr);
                 }
                 if (!(mt.flags & 2)) {
                     __syncwarp();
@@ -937,16 +960,21 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) ears_verify_kernel(const
                 // last chunk of the unit: (max, sum) of the warp -- the maximum first (shuffles only),
                 // then one rescale per thread and a sum
                 const float cu = PER_SEQ ? mt.c : p.c;
-                const float2 ms = acc_close(acc, cu);
+                float wv = 0.f;
+                const float2 ms = acc_close(acc, cu, &wv);
                 float m = ms.x;
 #pragma unroll
                 for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
-                float sum = rebase_sum(ms.x, ms.y, m, cu);
+                const float2 sw = ENT ? rebase_sum_w(ms.x, ms.y, wv, m, cu) : make_float2(rebase_sum(ms.x, ms.y, m, cu), 0.f);
+                float sum = sw.x, wsum = sw.y;
 #pragma unroll
-                for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+                for (int off = 16; off > 0; off >>= 1) {
+                    sum += __shfl_xor_sync(0xffffffffu, sum, off);
+                    if (ENT) wsum += __shfl_xor_sync(0xffffffffu, wsum, off);
+                }
                 if (lane == 0) {
                     const int us = unit_ends % kUnitSlots;
-                    sm.scratch[us][warp] = make_float2(m, sum);
+                    sm.scratch[us][warp] = make_float4(m, sum, wsum, 0.f);
                     mbar_arrive(&sm.unit_bar[us]);
                     if (warp == 0) push_unit_end(sm, Msg{kMsgPiece, mt.id, 0, unit_ends});
                     mbar_arrive(&sm.empty[stage]);

@@ -77,16 +77,20 @@ __device__ __forceinline__ double warp_inclusive_scan(double v, int lane) {
 // P_t(x), P_d(x) from the token's logits and the rows' (max, Z); max P_t = 1/Z_t (the largest
 // term of Z is exp(0)); R = P_t(x) / max(P_d(x), eps); Tolerance = beta (1 - max P_t);
 // accept iff R >= max(U - Tolerance, 0).  cls: 0 reject, 1 direct accept (R >= U), 2 pardon.
+//
+// The uncertainty that scales the tolerance is 1 - max P_t as printed (Sec. 3.2), or -- when the
+// caller asks for it and passes unc >= 0 -- the normalised entropy H(P_t) / ln V (Sec. 5 names the
+// entropy as a more refined measure; the normalisation is this library's reading).
 struct Decision { double pt, pd, maxp; int cls; bool accept; };
 
 __device__ __forceinline__ Decision decide_position(double lt, double ld, float2 st, float2 sd, double T,
-                                                    double beta, double U) {
+                                                    double beta, double U, double unc = -1.0) {
     Decision r;
     r.pt = exp((lt - (double)st.x) / T) / (double)st.y;
     r.pd = exp((ld - (double)sd.x) / T) / (double)sd.y;
     r.maxp = 1.0 / (double)st.y;
     const double ratio = r.pt / fmax(r.pd, kEps);
-    const double tol = beta * (1.0 - r.maxp);
+    const double tol = beta * (unc >= 0.0 ? unc : 1.0 - r.maxp);
     const double thr = fmax(U - tol, 0.0);
     r.accept = ratio >= thr;
     r.cls = ratio >= U ? 1 : (r.accept ? 2 : 0);
@@ -158,15 +162,36 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 // Running (m, s) of one thread: s = sum exp2(fl(l c - mu)), mu = fl(m c) (0 while m = -inf).
 // One fused multiply-add per entry; the rounding of m c is taken out again in acc_close.
 // The sum is kept in four lanes (two register pairs) so that consecutive additions overlap.
-struct RowAcc { float m, mu; f32x2 s[2]; };
+//
+// ENT: the entropy of the row comes out of the same sweep.  With t = l c - mu (log2 units below
+// the reference) and e = 2^t, the thread also carries w = sum e t (one more multiply-add per
+// entry): H = ln Z - ln 2 * (sum e t) / Z.  Every t is <= 0 up to rounding, so nothing cancels.
+// Masked entries (l = -inf) would give 0 * -inf; the ENT loops therefore read their logits through
+// a clamp at a large negative finite value (NaNs pass the clamp and still reach the sums).
+template <bool ENT> struct RowAccT { float m, mu; f32x2 s[2]; f32x2 w[ENT ? 2 : 1]; };
+typedef RowAccT<false> RowAcc;
 
-__device__ __forceinline__ void acc_open(RowAcc& a) { a.m = -INFINITY; a.mu = 0.f; a.s[0] = a.s[1] = pack2(0.f, 0.f); }
+constexpr float kLogitFloor = -1.0e30f;   // what -inf logits are read as where products with them must stay finite
 
-__device__ __forceinline__ void acc_raise(RowAcc& a, float cm, float c) {
+template <bool ENT>
+__device__ __forceinline__ void acc_open(RowAccT<ENT>& a) {
+    a.m = -INFINITY; a.mu = 0.f; a.s[0] = a.s[1] = pack2(0.f, 0.f);
+    if (ENT) a.w[0] = a.w[ENT ? 1 : 0] = pack2(0.f, 0.f);
+}
+
+template <bool ENT>
+__device__ __forceinline__ void acc_raise(RowAccT<ENT>& a, float cm, float c) {
     if (cm > a.m) {  // false for NaN: a NaN entry reaches the sum instead
         const float mu_new = cm * c;
         const float sc = (a.m == -INFINITY) ? 0.f : ex2_approx(a.mu - mu_new);
         const f32x2 sc2 = pack2(sc, sc);
+        if (ENT) {
+            // every t drops by mu_new - mu and every e shrinks by sc: w <- sc (w - (mu_new - mu) s)
+            const float dl = (a.m == -INFINITY) ? 0.f : a.mu - mu_new;
+            const f32x2 dl2 = pack2(dl, dl);
+            a.w[0] = mul2(fma2(dl2, a.s[0], a.w[0]), sc2);
+            a.w[ENT ? 1 : 0] = mul2(fma2(dl2, a.s[1], a.w[ENT ? 1 : 0]), sc2);
+        }
         a.s[0] = mul2(a.s[0], sc2);
         a.s[1] = mul2(a.s[1], sc2);
         a.m = cm;
@@ -175,25 +200,50 @@ __device__ __forceinline__ void acc_raise(RowAcc& a, float cm, float c) {
 }
 
 // One more entry (loops that go element by element: rows that are not 16-byte aligned).
-__device__ __forceinline__ void acc_add_one(RowAcc& a, float x, float c) {
-    a.s[0] = add2(a.s[0], pack2(ex2_approx(__fmaf_rn(x, c, -a.mu)), 0.f));
+template <bool ENT>
+__device__ __forceinline__ void acc_add_one(RowAccT<ENT>& a, float x, float c) {
+    if (ENT) x = fmaxf(x, kLogitFloor) + (x != x ? x : 0.f);   // -inf -> floor; NaN stays NaN
+    const float t = __fmaf_rn(x, c, -a.mu), e = ex2_approx(t);
+    a.s[0] = add2(a.s[0], pack2(e, 0.f));
+    if (ENT) a.w[0] = add2(a.w[0], pack2(e * t, 0.f));
 }
 
 // Two more pairs of entries: sum += exp2(x c - mu) in each of the four lanes.
-__device__ __forceinline__ void acc_add_pairs(RowAcc& a, f32x2 x01, f32x2 x23, f32x2 c2, f32x2 nmu2) {
-    a.s[0] = add2(a.s[0], ex2_pair(fma2(x01, c2, nmu2)));
-    a.s[1] = add2(a.s[1], ex2_pair(fma2(x23, c2, nmu2)));
+template <bool ENT>
+__device__ __forceinline__ void acc_add_pairs(RowAccT<ENT>& a, f32x2 x01, f32x2 x23, f32x2 c2, f32x2 nmu2) {
+    const f32x2 t0 = fma2(x01, c2, nmu2), t1 = fma2(x23, c2, nmu2);
+    const f32x2 e0 = ex2_pair(t0), e1 = ex2_pair(t1);
+    a.s[0] = add2(a.s[0], e0);
+    a.s[1] = add2(a.s[1], e1);
+    if (ENT) {
+        a.w[0] = fma2(e0, t0, a.w[0]);
+        a.w[ENT ? 1 : 0] = fma2(e1, t1, a.w[ENT ? 1 : 0]);
+    }
 }
 
 // -> (m, s) with s relative to the exact product m c: fl(m c) differs from m c by
 // delta = fma(m, c, -fl(m c)) exactly; the terms were taken relative to fl(m c) = m c - delta, so
 // every one carries the factor 2^delta, which is divided out: 2^-delta = 1 - delta ln 2 to first
 // order (|delta| < 1e-5).
-__device__ __forceinline__ float2 acc_close(const RowAcc& a, float c) {
+// ENT: *w_out = sum e t relative to the exact product as well: the terms used t + delta and
+// e 2^delta, so w_used = 2^delta (w + delta s); both effects are taken out to first order.
+template <bool ENT>
+__device__ __forceinline__ float2 acc_close(const RowAccT<ENT>& a, float c, float* w_out = nullptr) {
     float s0, s1;
     unpack2(add2(a.s[0], a.s[1]), s0, s1);
-    float s = s0 + s1;
-    if (a.m > -INFINITY && a.m < INFINITY) s = __fmaf_rn(s, -0.6931471805599453f * __fmaf_rn(a.m, c, -a.mu), s);
+    float s = s0 + s1, w = 0.f;
+    if (ENT) {
+        float w0, w1;
+        unpack2(add2(a.w[0], a.w[ENT ? 1 : 0]), w0, w1);
+        w = w0 + w1;
+    }
+    if (a.m > -INFINITY && a.m < INFINITY) {
+        const float delta = __fmaf_rn(a.m, c, -a.mu);
+        const float k = -0.6931471805599453f * delta;
+        s = __fmaf_rn(s, k, s);
+        if (ENT) w = __fmaf_rn(-delta, s, __fmaf_rn(w, k, w));
+    }
+    if (ENT && w_out) *w_out = w;
     return make_float2(a.m, s);
 }
 
@@ -204,6 +254,41 @@ __device__ __forceinline__ float rebase_sum(float m, float s, float M, float c) 
     return s * sc;
 }
 
+// The same for the pair (s, w = sum e t): relative to M every t is lower by (M - m) c.
+__device__ __forceinline__ float2 rebase_sum_w(float m, float s, float w, float M, float c) {
+    if (m == -INFINITY) return make_float2(s * 0.f, 0.f);
+    const float dl = (m - M) * c;
+    const float sc = exp2f(dl);
+    return make_float2(s * sc, sc * __fmaf_rn(dl, s, w));
+}
+
+// Entropy (nats) of a row from Z = sum e and w = sum e t (t in log2 units below the row maximum):
+// ln p = t ln 2 - ln Z, hence H = ln Z - ln 2 * w / Z.  fp64: called once per position.
+__device__ __forceinline__ double row_entropy(float Z, float w) {
+    return log((double)Z) - 0.6931471805599453 * (double)w / (double)Z;
+}
+// H / ln V, the uncertainty in [0, 1] that the entropy gives (0 for a vocabulary of one entry).
+__device__ __forceinline__ double entropy_uncertainty(double H, int V) {
+    return V > 1 ? fmin(fmax(H / log((double)V), 0.0), 1.0) : 0.0;
+}
+
+// larger of two, a NaN operand wins (so that a clamp from below lets NaNs through)
+__device__ __forceinline__ float max_nan(float a, float b) {
+    float r;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ uint32_t max_nan_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+__device__ __forceinline__ uint32_t max_nan_f16x2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("max.NaN.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+
 // ---- packed 16-byte vectors of logits ---------------------------------------------
 // A vector stays packed (four 32-bit words, as loaded) until it is used.  Per element type:
 //   N            entries per vector
@@ -212,6 +297,7 @@ __device__ __forceinline__ float rebase_sum(float m, float s, float M, float c) 
 //                sum instead
 //   pairs        the entries widened to fp32, two per 64-bit register
 //   unpack       the entries widened to fp32, one per register
+//   floor_inf    the vector with its -inf entries raised to a large negative finite value (NaNs stay)
 //   minus_inf    a vector of -inf entries;  mask_tail: entries from index `keep` on become -inf
 //   gather       up to N entries fetched one by one (rows that are not 16-byte aligned)
 template <typename E> struct Words;
@@ -234,6 +320,10 @@ template <> struct Words<float> {
     }
     __device__ static __forceinline__ void unpack(uint4 w, float (&x)[4]) {
         x[0] = __uint_as_float(w.x); x[1] = __uint_as_float(w.y); x[2] = __uint_as_float(w.z); x[3] = __uint_as_float(w.w);
+    }
+    __device__ static __forceinline__ uint4 floor_inf(uint4 w) {
+        return make_uint4(__float_as_uint(max_nan(__uint_as_float(w.x), kLogitFloor)), __float_as_uint(max_nan(__uint_as_float(w.y), kLogitFloor)),
+                          __float_as_uint(max_nan(__uint_as_float(w.z), kLogitFloor)), __float_as_uint(max_nan(__uint_as_float(w.w), kLogitFloor)));
     }
     __device__ static __forceinline__ uint4 minus_inf() { return make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u); }
     __device__ static __forceinline__ uint4 mask_tail(uint4 w, int keep) {
@@ -282,6 +372,10 @@ template <> struct Words<uint16_t> {
         x[4] = __uint_as_float(w.z << 16); x[5] = __uint_as_float(w.z & 0xffff0000u);
         x[6] = __uint_as_float(w.w << 16); x[7] = __uint_as_float(w.w & 0xffff0000u);
     }
+    __device__ static __forceinline__ uint4 floor_inf(uint4 w) {   // 0xf149: about -1e30 as bfloat16
+        return make_uint4(max_nan_bf16x2(w.x, 0xf149f149u), max_nan_bf16x2(w.y, 0xf149f149u), max_nan_bf16x2(w.z, 0xf149f149u),
+                          max_nan_bf16x2(w.w, 0xf149f149u));
+    }
     __device__ static __forceinline__ uint4 minus_inf() { return make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u); }
     __device__ static __forceinline__ uint4 mask_tail(uint4 w, int keep) { return mask_tail16(w, keep, 0xff80u); }
     __device__ static __forceinline__ uint4 gather(const uint16_t* p, int left) {
@@ -306,6 +400,10 @@ template <> struct Words<f16_t> {
         p[0] = widen(w.x); p[1] = widen(w.y); p[2] = widen(w.z); p[3] = widen(w.w);
     }
     __device__ static __forceinline__ void unpack(uint4 w, float (&x)[8]) { Vec<f16_t>::unpack(w, x); }
+    __device__ static __forceinline__ uint4 floor_inf(uint4 w) {   // 0xfbff: -65504, the lowest finite binary16
+        return make_uint4(max_nan_f16x2(w.x, 0xfbfffbffu), max_nan_f16x2(w.y, 0xfbfffbffu), max_nan_f16x2(w.z, 0xfbfffbffu),
+                          max_nan_f16x2(w.w, 0xfbfffbffu));
+    }
     __device__ static __forceinline__ uint4 minus_inf() { return make_uint4(0xfc00fc00u, 0xfc00fc00u, 0xfc00fc00u, 0xfc00fc00u); }
     __device__ static __forceinline__ uint4 mask_tail(uint4 w, int keep) { return mask_tail16(w, keep, 0xfc00u); }
     __device__ static __forceinline__ uint4 gather(const f16_t* p, int left) {
@@ -318,15 +416,15 @@ template <> struct Words<f16_t> {
 
 // G vectors of one thread: maximum first, one rescale of the running sums if it grew, then one
 // multiply-add, one exp2 and one addition per entry, the first and the last on pairs.
-template <typename E, int G>
-__device__ __forceinline__ void fold_vectors(const uint4 (&w)[G], float c, RowAcc& a) {
+template <typename E, int G, bool ENT>
+__device__ __forceinline__ void fold_vectors(const uint4 (&w)[G], float c, RowAccT<ENT>& a) {
     constexpr int PN = Words<E>::N / 2;
     acc_raise(a, Words<E>::template vmax_all<G>(w), c);
     const f32x2 c2 = pack2(c, c), nmu2 = pack2(-a.mu, -a.mu);
 #pragma unroll
     for (int j = 0; j < G; ++j) {
         f32x2 p[PN];
-        Words<E>::pairs(w[j], p);
+        Words<E>::pairs(ENT ? Words<E>::floor_inf(w[j]) : w[j], p);
 #pragma unroll
         for (int i = 0; i < PN; i += 2) acc_add_pairs(a, p[i], p[i + 1], c2, nmu2);
     }
@@ -334,15 +432,15 @@ __device__ __forceinline__ void fold_vectors(const uint4 (&w)[G], float c, RowAc
 
 // Two 16-byte vectors (indices v0, v1) of a staged row piece holding n valid entries from its
 // start; `full` says that both vectors lie wholly inside the piece.
-template <typename E>
-__device__ __forceinline__ void stats_two_vectors(const unsigned char* buf, int v0, int v1, bool full, int n, float c, RowAcc& a) {
+template <typename E, bool ENT>
+__device__ __forceinline__ void stats_two_vectors(const unsigned char* buf, int v0, int v1, bool full, int n, float c, RowAccT<ENT>& a) {
     constexpr int N = Words<E>::N;
     uint4 w[2] = {reinterpret_cast<const uint4*>(buf)[v0], reinterpret_cast<const uint4*>(buf)[v1]};
     if (!full) {  // ragged end: what lies beyond the piece counts as -inf
         w[0] = Words<E>::mask_tail(w[0], n - v0 * N);
         w[1] = Words<E>::mask_tail(w[1], n - v1 * N);
     }
-    fold_vectors<E, 2>(w, c, a);
+    fold_vectors<E, 2, ENT>(w, c, a);
 }
 
 }  // namespace ears

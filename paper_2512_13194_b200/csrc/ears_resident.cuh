@@ -60,6 +60,8 @@ struct RParams {
     double* cand_mass;    // [B,K+1] mass that token was drawn from
     float4* rowstat;      // [B,K+1] (max, Z) of the item's target and draft rows (streaming clusters only)
     unsigned long long* seqmask;  // [B] positions decided (low word) and accepted (high word), K <= 30 (streaming clusters only)
+    int unc_entropy;      // 1: the tolerance is scaled by H(P_t) / ln V instead of 1 - max P_t [Sec. 5 item 1]
+    double* entropy;      // [B,K] H(P_t) of every target row, or NULL; the entropy kernels (ENT) fill it
     int C;                // CTAs per cluster
     int slice;            // elements of a row per CTA, a multiple of kSegElems
     int buf_bytes;        // shared-memory bytes reserved per row slice (slice bytes rounded up to kRSubBytes)
@@ -77,6 +79,7 @@ struct RSmem {
     uint64_t xbar[2];                    // statistics exchange, alternating by round
     uint64_t mbar2[2];                   // mass-total exchange, alternating by mass round
     alignas(16) float4 xstat[2][kRMaxCluster * kRWarps];   // (m_t, s_t, m_d, s_d) of every warp of every peer
+    float xw[2][kRMaxCluster * kRWarps]; // sum e t of the target slice of every warp of every peer (entropy kernels)
     double xmass[2][kRMaxCluster];       // mass totals of every peer
     int xnext[2];                        // next item of the cluster (written by rank 0)
     double segsum[kRMaxSeg];
@@ -148,11 +151,83 @@ __device__ __forceinline__ void cluster_sync_all() {
 }
 
 // Sub-chunk q of a slice of n valid entries: every thread takes two 16-byte vectors.
-template <typename E>
-__device__ __forceinline__ void stats_sub(const unsigned char* buf, int q, int n, int tid, float c, RowAcc& a) {
+template <typename E, bool ENT>
+__device__ __forceinline__ void stats_sub(const unsigned char* buf, int q, int n, int tid, float c, RowAccT<ENT>& a) {
     constexpr int SUB_VECS = kRSubBytes / 16;
     const int v0 = q * SUB_VECS + tid, v1 = v0 + kRThreads;
-    stats_two_vectors<E>(buf, v0, v1, (q + 1) * SUB_VECS * Vec<E>::N <= n, n, c, a);
+    stats_two_vectors<E, ENT>(buf, v0, v1, (q + 1) * SUB_VECS * Vec<E>::N <= n, n, c, a);
+}
+
+__device__ __forceinline__ void peer_store(uint32_t addr, float v) {
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+
+// Warp 0 of every CTA after the exchange: the C x 8 partial results -> the rows' (max, Z) and, ENT, the
+// target row's sum e t.  Lane i takes entries i, i + 32, ...: the same in every CTA, hence identical bits.
+template <bool ENT>
+__device__ __forceinline__ void merge_exchanged(const float4* xs, const float* xw, int parts, float cb, int lane,
+                                                float& mt, float& zt, float& md, float& zd, float& wt) {
+    mt = -INFINITY; md = -INFINITY;
+    for (int i = lane; i < parts; i += 32) {
+        mt = fmaxf(mt, xs[i].x);
+        md = fmaxf(md, xs[i].z);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, off));
+        md = fmaxf(md, __shfl_xor_sync(0xffffffffu, md, off));
+    }
+    zt = 0.f; zd = 0.f; wt = 0.f;
+    for (int i = lane; i < parts; i += 32) {
+        const float4 v = xs[i];
+        if (ENT) {
+            const float2 sw = rebase_sum_w(v.x, v.y, xw[i], mt, cb);
+            zt += sw.x;
+            wt += sw.y;
+        } else {
+            zt += rebase_sum(v.x, v.y, mt, cb);
+        }
+        zd += rebase_sum(v.z, v.w, md, cb);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        zt += __shfl_xor_sync(0xffffffffu, zt, off);
+        zd += __shfl_xor_sync(0xffffffffu, zd, off);
+        if (ENT) wt += __shfl_xor_sync(0xffffffffu, wt, off);
+    }
+}
+
+// Lane 0 of warp 0 of every CTA: the decision of one position from the rows' statistics (the same
+// arithmetic on the same numbers in every CTA of the cluster).  fp32 first; it stands unless R comes
+// close to the threshold (the band is some 25 times the fp32 error), the caller wants the
+// probabilities, or the entropy scales the tolerance: then fp64 (decide_position).
+// -> 1 accept, 0 reject.  `report`: this CTA writes the optional per-position outputs.
+template <bool ENT, class P>
+__device__ __forceinline__ int cluster_decide(const P& p, int b, int j, float lt, float ld, double U, float2 rs_t, float2 rs_d,
+                                              float wt, float cb, double Tb, double betab, bool report) {
+    const int K = p.K;
+    double unc = -1.0, H = 0.0;
+    if (ENT) {
+        H = row_entropy(rs_t.y, wt);
+        if (p.unc_entropy) unc = entropy_uncertainty(H, p.V);
+        if (report && p.entropy) p.entropy[(size_t)b * K + j] = H;
+    }
+    const float pt32 = ex2_approx((lt - rs_t.x) * cb) / rs_t.y;
+    const float pd32 = ex2_approx((ld - rs_d.x) * cb) / rs_d.y;
+    const float ratio32 = pt32 / fmaxf(pd32, (float)kEps);
+    const float unc32 = unc >= 0.0 ? (float)unc : 1.0f - 1.0f / rs_t.y;
+    const float thr32 = fmaxf((float)U - (float)betab * unc32, 0.0f);
+    const float diff = ratio32 - thr32;
+    if (!p.want_stats && fabsf(diff) > 1e-4f * (ratio32 + thr32) + 1e-6f) return diff > 0.0f ? 1 : 0;
+    const Decision dc = decide_position((double)lt, (double)ld, rs_t, rs_d, Tb, betab, U, unc);
+    if (report && p.want_stats) {
+        const size_t i = (size_t)b * K + j;
+        p.pt_tok[i] = dc.pt;
+        p.pd_tok[i] = dc.pd;
+        p.max_pt[i] = dc.maxp;
+        p.cls[i] = (uint8_t)dc.cls;
+    }
+    return dc.accept ? 1 : 0;
 }
 
 // ---- masses of a slice ------------------------------------------------------------
@@ -299,7 +374,7 @@ __device__ void finish_sequence(const RParams& p, int b, int lane) {
 }
 
 // ---- the kernel -----------------------------------------------------------------------
-template <typename E>
+template <typename E, bool ENT>
 __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RParams p) {
     extern __shared__ unsigned char smem_raw[];
     RSmem& sm = *reinterpret_cast<RSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
@@ -395,7 +470,8 @@ __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RPara
     while (have) {
         // ---- 1. statistics of the slices as the copies land
         const float cb = seq_c(p, b);   // log2(e) / temperature of this sequence
-        RowAcc at, ad;
+        RowAccT<ENT> at;   // ENT: the target slice also yields its sum e t
+        RowAcc ad;
         acc_open(at);
         acc_open(ad);
         for (int q = 0; q < nsub; ++q) {
@@ -403,32 +479,36 @@ __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RPara
                 if (!mbar_wait(&sm.full[q], (full_phase >> q) & 1u, &sm.abort_flag)) failed = true;
             }
             if (failed) break;
-            stats_sub<E>(buf_t, q, n, tid, cb, at);
-            if (pair) stats_sub<E>(buf_d, q, n, tid, cb, ad);
+            stats_sub<E, ENT>(buf_t, q, n, tid, cb, at);
+            if (pair) stats_sub<E, false>(buf_d, q, n, tid, cb, ad);
         }
         if (use_tma) full_phase ^= issued;
         // (max, sum) of the warp's share: the maximum first (shuffles only), then one rescale per
         // thread and a sum -- a much shorter dependent chain than merging (m, s) pairs step by step
         const int par = round & 1;
         {
-            const float2 pt2 = acc_close(at, cb), pd2 = acc_close(ad, cb);
+            float wv = 0.f;
+            const float2 pt2 = acc_close(at, cb, &wv), pd2 = acc_close(ad, cb);
             float Mt = pt2.x, Md = pd2.x;
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) {
                 Mt = fmaxf(Mt, __shfl_xor_sync(0xffffffffu, Mt, off));
                 Md = fmaxf(Md, __shfl_xor_sync(0xffffffffu, Md, off));
             }
-            float St = rebase_sum(pt2.x, pt2.y, Mt, cb), Sd = rebase_sum(pd2.x, pd2.y, Md, cb);
+            const float2 sw = ENT ? rebase_sum_w(pt2.x, pt2.y, wv, Mt, cb) : make_float2(rebase_sum(pt2.x, pt2.y, Mt, cb), 0.f);
+            float St = sw.x, Wt = sw.y, Sd = rebase_sum(pd2.x, pd2.y, Md, cb);
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) {
                 St += __shfl_xor_sync(0xffffffffu, St, off);
                 Sd += __shfl_xor_sync(0xffffffffu, Sd, off);
+                if (ENT) Wt += __shfl_xor_sync(0xffffffffu, Wt, off);
             }
             // ---- 2. every warp hands its partial result to every CTA of the cluster (itself included)
             const int nx = __shfl_sync(0xffffffffu, next_item, 0);
             if (lane < C) {
                 peer_store(map_to_peer(smem_u32(&sm.xstat[par][rank * kRWarps + warp]), (uint32_t)lane),
                            make_float4(Mt, St, Md, Sd));
+                if (ENT) peer_store(map_to_peer(smem_u32(&sm.xw[par][rank * kRWarps + warp]), (uint32_t)lane), Wt);
                 if (rank == 0 && warp == 0) peer_store(map_to_peer(smem_u32(&sm.xnext[par]), (uint32_t)lane), nx);
                 peer_arrive(map_to_peer(smem_u32(&sm.xbar[par]), (uint32_t)lane));
             }
@@ -437,61 +517,17 @@ __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RPara
         ++round;
         // ---- 3. the rows' (max, Z) and the decision
         if (ok && warp == 0) {
-            // C x 8 partial results, lane i takes entries i, i + 32, ...: the same in every CTA, hence identical bits
-            const int parts = C * kRWarps;
-            float mt = -INFINITY, md = -INFINITY;
-            for (int i = lane; i < parts; i += 32) {
-                mt = fmaxf(mt, sm.xstat[par][i].x);
-                md = fmaxf(md, sm.xstat[par][i].z);
+            float mt, zt, md, zd, wt;
+            merge_exchanged<ENT>(sm.xstat[par], sm.xw[par], C * kRWarps, cb, lane, mt, zt, md, zd, wt);
+            if (lane == 0) {
+                const double Tb = seq_temperature(p, b), betab = seq_beta(p, b);
+                int dec = 1;
+                if (!rowstat_ok(mt, zt) || (pair && (!rowstat_ok(md, zd) || !tok_ok)) || !seq_params_ok(Tb, betab)) dec = -1;
+                sm.rs_t = make_float2(mt, zt);
+                sm.rs_d = pair ? make_float2(md, zd) : make_float2(0.f, 1.f);
+                if (pair && dec >= 0) dec = cluster_decide<ENT>(p, b, j, lt, ld, U, sm.rs_t, sm.rs_d, wt, cb, Tb, betab, rank == 0);
+                sm.dec = dec;
             }
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-                mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, off));
-                md = fmaxf(md, __shfl_xor_sync(0xffffffffu, md, off));
-            }
-            float zt = 0.f, zd = 0.f;
-            for (int i = lane; i < parts; i += 32) {
-                const float4 v = sm.xstat[par][i];
-                zt += rebase_sum(v.x, v.y, mt, cb);
-                zd += rebase_sum(v.z, v.w, md, cb);
-            }
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-                zt += __shfl_xor_sync(0xffffffffu, zt, off);
-                zd += __shfl_xor_sync(0xffffffffu, zd, off);
-            }
-          if (lane == 0) {
-            const double Tb = seq_temperature(p, b), betab = seq_beta(p, b);
-            int dec = 1;
-            if (!rowstat_ok(mt, zt) || (pair && (!rowstat_ok(md, zd) || !tok_ok)) || !seq_params_ok(Tb, betab)) dec = -1;
-            sm.rs_t = make_float2(mt, zt);
-            sm.rs_d = pair ? make_float2(md, zd) : make_float2(0.f, 1.f);
-            if (pair && dec >= 0) {
-                // The decision in fp32 first; it stands unless R comes close to the threshold (the
-                // band is some 25 times the fp32 error), in which case -- or when the caller wants
-                // the probabilities -- it is taken in fp64.  Either way every CTA of the cluster
-                // runs the same arithmetic on the same numbers.
-                const float pt32 = ex2_approx((lt - mt) * cb) / zt;
-                const float pd32 = ex2_approx((ld - md) * cb) / zd;
-                const float ratio32 = pt32 / fmaxf(pd32, (float)kEps);
-                const float thr32 = fmaxf((float)U - (float)betab * (1.0f - 1.0f / zt), 0.0f);
-                const float diff = ratio32 - thr32;
-                if (!p.want_stats && fabsf(diff) > 1e-4f * (ratio32 + thr32) + 1e-6f) {
-                    dec = diff > 0.0f ? 1 : 0;
-                } else {
-                    const Decision dc = decide_position((double)lt, (double)ld, sm.rs_t, sm.rs_d, Tb, betab, U);
-                    dec = dc.accept ? 1 : 0;
-                    if (rank == 0 && p.want_stats) {
-                        const size_t i = (size_t)b * K + j;
-                        p.pt_tok[i] = dc.pt;
-                        p.pd_tok[i] = dc.pd;
-                        p.max_pt[i] = dc.maxp;
-                        p.cls[i] = (uint8_t)dc.cls;
-                    }
-                }
-            }
-            sm.dec = dec;
-          }
         }
         if (__syncthreads_or(ok ? 0 : 1)) { failed = true; break; }
         const int dec = sm.dec;

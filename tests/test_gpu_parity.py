@@ -583,3 +583,57 @@ def test_decision_class_counts_match_the_oracle(ears):
             want[("reject", "direct", "pardon")[int(ora.cls[b, k])]] += 1
     assert got == want and got["pardon"] > 0 and got["reject"] > 0
     assert got["reject"] == int((ora.accept_len < 4).sum())
+
+
+@pytest.mark.parametrize("path,cluster", [(1, 0), (3, 0), (2, 0), (2, 4), (4, 0), (4, 2)])
+@pytest.mark.parametrize("B,K,V,dtype", [(6, 3, 9000, "fp32"), (5, 4, 20001, "bf16"), (3, 2, 70000, "fp16"), (200, 2, 700, "bf16")])
+def test_parity_entropy_measure(ears, forced_path, B, K, V, dtype, path, cluster):
+    """H(P_t) out of the same sweep against the oracle's (1e-5 relative, or 5e-7 absolute: H = ln Z - ...
+    with Z an fp32 sum good to a few 1e-7, so that much of ln Z is the floor), and the step with H / ln V
+    as the uncertainty (Sec. 5 item 1) against the oracle in the same mode; masked entries (-inf) must
+    not disturb either; asking for the entropy alone leaves the printed rule's results untouched."""
+    forced_path(path, cluster)
+    dev = "cuda:0"
+    w, t, d, x = synth.tiny_inputs(B, K, V, dtype, seed=700 + K, noise=1.2)
+    t, d = t.clone(), d.clone()
+    t[0, 0, 5:V // 2] = float("-inf")
+    d[0, 0, 5:V // 2] = float("-inf")
+    t[1 % B, 1, :] = 0.0                      # a flat row: H = ln V
+    t[2 % B, K - 1, 3] += 60.0                # a (nearly) one-hot row: H ~ 0
+    x = x.clone()
+    x[0, 0] = 2
+    tg, dg, xg = t.to(dev), d.to(dev), x.to(dev)
+    tally = Tally()
+    for offset, (T, beta) in enumerate([(1.0, 0.3), (0.8, 1.0), (1.4, 0.05)]):
+        acc, tok, st = ears.verify(tg, dg, xg, T, beta, 9, offset, stats=True, uncertainty="entropy", entropy=True)
+        acc2, tok2, st2 = ears.verify(tg, dg, xg, T, beta, 9, offset, uncertainty="entropy", entropy=True)
+        torch.cuda.synchronize()
+        assert ears.last_device_status() == 0
+        assert torch.equal(acc, acc2) and torch.equal(tok, tok2)
+        ora = oracle.verify(t, d, x, T, beta, seed=9, offset=offset, nthreads=8, uncertainty="entropy")
+        tally.merge(compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, K, {k: v.cpu().numpy() for k, v in st.items() if k != "entropy"},
+                            inputs=(t, d, T)))
+        H = st["entropy"].cpu().numpy()
+        np.testing.assert_allclose(H, ora.entropy, rtol=1e-5, atol=5e-7)
+        np.testing.assert_allclose(st2["entropy"].cpu().numpy(), ora.entropy, rtol=1e-5, atol=5e-7)
+        assert abs(H[1 % B, 1] - np.log(V)) < 1e-5 * np.log(V)
+        # the printed rule with the entropy as a by-product only
+        ref = ears.verify(tg, dg, xg, T, beta, 9, offset)
+        a3, k3, st3 = ears.verify(tg, dg, xg, T, beta, 9, offset, entropy=True)
+        assert torch.equal(ref[0], a3) and torch.equal(ref[1], k3)
+        np.testing.assert_allclose(st3["entropy"].cpu().numpy(), ora.entropy, rtol=1e-5, atol=5e-7)
+    assert_parity(tally, max_explained=1)
+    assert tally.max_rel_prob_err < 1e-5
+
+
+def test_parity_entropy_measure_workload_rows(ears):
+    """Rows of workloads 3 and 4 (peaked, flat and Zipf-shaped distributions at full vocabulary), in the
+    automatic launch configuration."""
+    from dataclasses import replace
+    for idx, B in ((3, 32), (4, 48)):
+        w = replace(synth.workload(idx), B=B)
+        t, d, x = synth.make_inputs(w, "cpu")
+        acc, tok, st = ears.verify(t.cuda(), d.cuda(), x.cuda(), w.temperature, w.beta, 0, 2, uncertainty="entropy", entropy=True)
+        ora = oracle.verify(t, d, x, w.temperature, w.beta, seed=0, offset=2, nthreads=oracle.max_threads(), uncertainty="entropy")
+        assert_parity(compare(acc.cpu().numpy(), tok.cpu().numpy(), ora, w.K, inputs=(t, d, w.temperature)))
+        np.testing.assert_allclose(st["entropy"].cpu().numpy(), ora.entropy, rtol=1e-5, atol=5e-7)
