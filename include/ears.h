@@ -341,6 +341,21 @@ int ears_last_device_status(void* stream);
 int ears_workspace_device_status(void* workspace, void* stream);
 
 /*
+ * How the most recent call on the library-owned workspace of (current device, stream) decided its
+ * positions -- the three-way decision of Sec. 3.2 step 5 as production telemetry, counted on the
+ * device by the kernels themselves (no optional output is needed for it):
+ *   out_counts[0] direct acceptances (R >= U), [1] acceptances by pardon (U - Tolerance <= R < U),
+ *   [2] rejections, [3] sequences marked invalid.
+ * A sequence contributes the positions it really decided: its accepted prefix and, if there is
+ * one, its first rejection (so [2] is the number of sequences that ended in a rejection).  Waits
+ * for `stream`; out_counts is a HOST array of four words.  The greedy form counts [3] only.
+ */
+int ears_last_decision_counts(void* stream, uint32_t out_counts[4]);
+
+/* Same for a caller-owned workspace that was passed to a verification call on `stream`. */
+int ears_workspace_decision_counts(void* workspace, void* stream, uint32_t out_counts[4]);
+
+/*
  * Self-test of the kernels' bounded waits (every device-side wait in this library gives up
  * after a time limit, sets EARS_DEV_TIMEOUT and lets the kernel return; nothing can hang
  * the GPU).  Launches a tiny kernel that waits limit_ms (1..2000) on a barrier no thread ever

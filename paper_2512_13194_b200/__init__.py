@@ -6,12 +6,14 @@ synthetic workloads, ``shard`` the batch partition used across GPUs and
 the driver of the vocabulary-sharded step.
 """
 from . import shard, synth  # noqa: F401
+from .sampler import EarsSampler, StepResult  # noqa: F401
 from .binding import (  # noqa: F401
     DEV_INVALID_INPUT,
     DEV_TIMEOUT,
     EarsError,
     ShardStep,
     class_counts,
+    decision_counts,
     describe_plan,
     last_device_status,
     load_library,

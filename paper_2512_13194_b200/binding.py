@@ -74,6 +74,10 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.ears_last_device_status.restype = c.c_int
     lib.ears_workspace_device_status.argtypes = [c.c_void_p, c.c_void_p]
     lib.ears_workspace_device_status.restype = c.c_int
+    lib.ears_last_decision_counts.argtypes = [c.c_void_p, c.POINTER(c.c_uint32)]
+    lib.ears_last_decision_counts.restype = c.c_int
+    lib.ears_workspace_decision_counts.argtypes = [c.c_void_p, c.c_void_p, c.POINTER(c.c_uint32)]
+    lib.ears_workspace_decision_counts.restype = c.c_int
     lib.ears_selftest_bounded_wait.argtypes = [c.c_int, c.c_void_p]
     lib.ears_selftest_bounded_wait.restype = c.c_int
     lib.ears_philox_device.argtypes = [c.c_void_p, c.c_void_p, c.c_int, c.c_void_p]
@@ -323,6 +327,18 @@ def last_device_status(stream=None) -> int:
     if rc < 0:
         _check(rc)
     return rc
+
+
+def decision_counts(stream=None, workspace: Optional[torch.Tensor] = None) -> dict:
+    """Device-side counts of the three-way decision (Sec. 3.2 step 5) of the most recent call on
+    ``stream`` (or on ``workspace``): {"direct", "pardon", "reject", "invalid"}; waits for the stream."""
+    out = (ctypes.c_uint32 * 4)()
+    lib = load_library()
+    if workspace is None:
+        _check(lib.ears_last_decision_counts(_stream_ptr(stream), out))
+    else:
+        _check(lib.ears_workspace_decision_counts(workspace.data_ptr(), _stream_ptr(stream), out))
+    return {"direct": int(out[0]), "pardon": int(out[1]), "reject": int(out[2]), "invalid": int(out[3])}
 
 
 def workspace_device_status(workspace: torch.Tensor, stream=None) -> int:

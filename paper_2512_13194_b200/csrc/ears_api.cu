@@ -176,7 +176,7 @@ Layout make_layout(int B, int K, int V, int parts1) {
     Layout L;
     const size_t rows = (size_t)B * (2 * K + 1);
     size_t o = 0;
-    L.heads = o; o += 32;  // fixed place: the status word is heads[2] of any workspace
+    L.heads = o; o += kHeadsWords * 4;  // fixed place: the status word is heads[2] of any workspace, the decision counts heads[8..11]
     L.wq = o; o += (size_t)B * 16;
     L.ticket1 = o; o += (size_t)B * 4;
     L.ticket2 = o; o += (size_t)B * 4;
@@ -279,7 +279,7 @@ struct RLayout { size_t heads, ticket, seqmask, counters_bytes, flag, cand, cand
 RLayout make_rlayout(int B, int K) {
     RLayout L;
     size_t o = 0;
-    L.heads = o; o += 32;   // the status word is heads[2] of any workspace
+    L.heads = o; o += kHeadsWords * 4;   // the status word is heads[2] of any workspace
     L.ticket = o; o += (size_t)B * 4;
     o = align_up(o, 8);
     L.seqmask = o; o += (size_t)B * 8;
@@ -317,7 +317,7 @@ GLayout make_glayout(int B, int K, int V, int esize, int sms) {
     L.piece_elems = (int)pe;
     L.P = (int)((V + pe - 1) / pe);
     size_t o = 0;
-    L.heads = o; o += 32;
+    L.heads = o; o += kHeadsWords * 4;
     L.ticket = o; o += (size_t)B * 4;
     L.counters_bytes = o;
     o = align_up(o, 256);
@@ -1116,6 +1116,35 @@ int ears_last_device_status(void* stream_) {
 int ears_workspace_device_status(void* workspace, void* stream_) {
     if (!workspace) return EARS_ERR_NULL;
     return read_status((int*)workspace, (cudaStream_t)stream_);
+}
+
+static int read_counts(const int* heads, cudaStream_t stream, uint32_t out_counts[4]) {
+    EARS_CUDA(cudaMemcpyAsync(out_counts, heads + kCountDirect, 4 * sizeof(uint32_t), cudaMemcpyDeviceToHost, stream));
+    EARS_CUDA(cudaStreamSynchronize(stream));
+    return EARS_OK;
+}
+
+int ears_last_decision_counts(void* stream_, uint32_t out_counts[4]) {
+    if (!out_counts) return EARS_ERR_NULL;
+    int dev = 0;
+    EARS_CUDA(cudaGetDevice(&dev));
+    void* word = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        auto it = g_workspaces.find(std::make_pair(dev, stream_));
+        if (it != g_workspaces.end()) word = it->second.status_word;
+    }
+    out_counts[0] = out_counts[1] = out_counts[2] = out_counts[3] = 0;
+    if (!word) {
+        EARS_CUDA(cudaStreamSynchronize((cudaStream_t)stream_));
+        return EARS_OK;
+    }
+    return read_counts((const int*)word - 2, (cudaStream_t)stream_, out_counts);
+}
+
+int ears_workspace_decision_counts(void* workspace, void* stream_, uint32_t out_counts[4]) {
+    if (!workspace || !out_counts) return EARS_ERR_NULL;
+    return read_counts((const int*)workspace, (cudaStream_t)stream_, out_counts);
 }
 
 int ears_selftest_bounded_wait(int limit_ms, void* stream_) {

@@ -33,6 +33,32 @@ constexpr double kTinyMass = 1e-300;                 // below this a residual is
 constexpr int kDevInvalidInput = 1;
 constexpr int kDevTimeout = 2;
 
+// Words of the `heads` block (16 ints at the start of every workspace) that every kernel shares:
+// [2] the status word; [8..11] how the call's positions were decided, counted over what each
+// sequence really decided (up to and including its first rejection): direct acceptances,
+// pardons, rejections [Sec. 3.2 step 5], and [11] sequences marked invalid.
+constexpr int kHeadsWords = 16;
+constexpr int kCountDirect = 8, kCountPardon = 9, kCountReject = 10, kCountInvalid = 11;
+
+// One warp: classes cls(k) in {0 reject, 1 direct, 2 pardon} of positions k < upto are added to the
+// call's counters (cls_of: int(int k), evaluated by lane k % 32).
+template <class F>
+__device__ __forceinline__ void count_decisions(int* heads, int upto, int lane, F cls_of) {
+    int nd = 0, np = 0, nr = 0;
+    for (int k0 = 0; k0 < upto; k0 += 32) {
+        const int k = k0 + lane;
+        const int c = k < upto ? cls_of(k) : -1;
+        nd += __popc(__ballot_sync(0xffffffffu, c == 1));
+        np += __popc(__ballot_sync(0xffffffffu, c == 2));
+        nr += __popc(__ballot_sync(0xffffffffu, c == 0));
+    }
+    if (lane == 0) {
+        if (nd) atomicAdd(&heads[kCountDirect], nd);
+        if (np) atomicAdd(&heads[kCountPardon], np);
+        if (nr) atomicAdd(&heads[kCountReject], nr);
+    }
+}
+
 // Sum of exp2(l c - mu) over one consumer warp's share of a chunk of the extra target row; mu is
 // the fp32 product (running maximum) x c that the terms were taken relative to.
 struct BonusSeg { double sum; float mu; float pad; };

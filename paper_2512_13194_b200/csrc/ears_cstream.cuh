@@ -186,10 +186,12 @@ __device__ __forceinline__ int finish_streamed_sequence(const RParams& p, int b,
         if (lane == 0) {
             p.out_len[b] = -1;
             atomicOr(&p.heads[2], kDevInvalidInput);
+            atomicAdd(&p.heads[kCountInvalid], 1);
         }
         return -1;
     }
     const int n = first_reject;
+    count_decisions(p.heads, min(n + 1, K), lane, [fl](int k) { return (int)*reinterpret_cast<const volatile signed char*>(fl + k); });
     const bool mine = n == K || !job_pending;   // the slot n is filled here
     for (int q = lane; q <= K; q += 32) {
         if (q < n) ot[q] = p.x[(size_t)b * K + q];
@@ -387,6 +389,9 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
         if (work && ordered) {
             seq_goes_on = dec > 0 && pair;
             if (dec == 0) { job_b = b; job_n = j; }        // the first rejection of a sequence walked in order: its masses now
+            // every position a cluster reaches while walking a sequence in order is one the sequence decided
+            if (rank == 0 && tid == 0 && pair && dec >= 0)
+                atomicAdd(&p.heads[dec == 1 ? kCountDirect : (dec == 2 ? kCountPardon : kCountReject)], 1);
             if (rank == writer && warp == 0 && !seq_goes_on) {
                 int32_t* ot = p.out_tok + (size_t)b * (K + 1);
                 if (dec < 0) {
@@ -394,6 +399,7 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
                     if (lane == 0) {
                         p.out_len[b] = -1;
                         atomicOr(&p.heads[2], kDevInvalidInput);
+                        atomicAdd(&p.heads[kCountInvalid], 1);
                     }
                 } else {
                     for (int q = lane; q <= K; q += 32) {

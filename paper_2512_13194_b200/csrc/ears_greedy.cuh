@@ -132,6 +132,7 @@ __device__ void greedy_finish(const GParams& p, int b, int lane, int* row_top /*
         if (lane == 0) {
             p.out_len[b] = -1;
             atomicOr(&p.heads[2], kDevInvalidInput);
+            atomicAdd(&p.heads[kCountInvalid], 1);
         }
         return;
     }

@@ -422,11 +422,16 @@ __device__ int finalize_sequence(const Params& p, int b, int lane) {
         if (lane == 0) {
             p.out_len[b] = -1;
             atomicOr(&p.heads[2], kDevInvalidInput);
+            atomicAdd(&p.heads[kCountInvalid], 1);
         }
         return -1;
     }
     for (int j = lane; j <= K; j += 32) ot[j] = j < first_reject ? p.x[(size_t)b * K + j] : -1;
     if (lane == 0) p.out_len[b] = first_reject;
+    // what this sequence decided: the accepted prefix and, if there is one, the first rejection
+    // (each lane reads back the classes it wrote itself above)
+    const uint8_t* cl = p.cls + (size_t)b * K;
+    count_decisions(p.heads, min(first_reject + 1, K), lane, [cl](int k) { return (int)cl[k]; });
     return first_reject;
 }
 

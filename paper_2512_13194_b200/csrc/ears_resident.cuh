@@ -55,7 +55,7 @@ struct RParams {
     double* resid;
     int* heads;           // [0] item queue, [2] status word
     int* ticket;          // [B] items of the sequence that are done
-    signed char* flag;    // [B,K+1] 1 accepted / row usable, 0 rejected, -1 invalid
+    signed char* flag;    // [B,K+1] 1 accepted directly / row usable, 2 accepted by pardon, 0 rejected, -1 invalid
     int32_t* cand;        // [B,K+1] token drawn at the position (rejected positions and slot K)
     double* cand_mass;    // [B,K+1] mass that token was drawn from
     float4* rowstat;      // [B,K+1] (max, Z) of the item's target and draft rows (streaming clusters only)
@@ -201,7 +201,8 @@ __device__ __forceinline__ void merge_exchanged(const float4* xs, const float* x
 // arithmetic on the same numbers in every CTA of the cluster).  fp32 first; it stands unless R comes
 // close to the threshold (the band is some 25 times the fp32 error), the caller wants the
 // probabilities, or the entropy scales the tolerance: then fp64 (decide_position).
-// -> 1 accept, 0 reject.  `report`: this CTA writes the optional per-position outputs.
+// -> the class of Sec. 3.2 step 5: 1 direct accept (R >= U), 2 pardon, 0 reject.
+// `report`: this CTA writes the optional per-position outputs.
 template <bool ENT, class P>
 __device__ __forceinline__ int cluster_decide(const P& p, int b, int j, float lt, float ld, double U, float2 rs_t, float2 rs_d,
                                               float wt, float cb, double Tb, double betab, bool report) {
@@ -218,7 +219,7 @@ __device__ __forceinline__ int cluster_decide(const P& p, int b, int j, float lt
     const float unc32 = unc >= 0.0 ? (float)unc : 1.0f - 1.0f / rs_t.y;
     const float thr32 = fmaxf((float)U - (float)betab * unc32, 0.0f);
     const float diff = ratio32 - thr32;
-    if (!p.want_stats && fabsf(diff) > 1e-4f * (ratio32 + thr32) + 1e-6f) return diff > 0.0f ? 1 : 0;
+    if (!p.want_stats && fabsf(diff) > 1e-4f * (ratio32 + thr32) + 1e-6f) return diff > 0.0f ? (ratio32 >= (float)U ? 1 : 2) : 0;
     const Decision dc = decide_position((double)lt, (double)ld, rs_t, rs_d, Tb, betab, U, unc);
     if (report && p.want_stats) {
         const size_t i = (size_t)b * K + j;
@@ -227,7 +228,7 @@ __device__ __forceinline__ int cluster_decide(const P& p, int b, int j, float lt
         p.max_pt[i] = dc.maxp;
         p.cls[i] = (uint8_t)dc.cls;
     }
-    return dc.accept ? 1 : 0;
+    return dc.cls;
 }
 
 // ---- masses of a slice ------------------------------------------------------------
@@ -357,10 +358,12 @@ __device__ void finish_sequence(const RParams& p, int b, int lane) {
         if (lane == 0) {
             p.out_len[b] = -1;
             atomicOr(&p.heads[2], kDevInvalidInput);
+            atomicAdd(&p.heads[kCountInvalid], 1);
         }
         return;
     }
     const int n = first_reject;
+    count_decisions(p.heads, min(n + 1, K), lane, [fl](int k) { return (int)*reinterpret_cast<const volatile signed char*>(fl + k); });
     for (int j = lane; j <= K; j += 32) {
         int v = -1;
         if (j < n) v = p.x[(size_t)b * K + j];
@@ -638,6 +641,9 @@ __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RPara
             }
         }
         if (ordered) {
+            // every position a cluster reaches while walking a sequence in order is one the sequence decided
+            if (rank == 0 && tid == 0 && rj < K && dec >= 0)
+                atomicAdd(&p.heads[dec == 1 ? kCountDirect : (dec == 2 ? kCountPardon : kCountReject)], 1);
             // the cluster owns the whole sequence: one CTA writes its outputs when it ends
             if (rank == writer && warp == 0 && (dec < 0 || rj == K || dec == 0)) {
                 int32_t* ot = p.out_tok + (size_t)rb * (K + 1);
@@ -646,6 +652,7 @@ __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RPara
                     if (lane == 0) {
                         p.out_len[rb] = -1;
                         atomicOr(&p.heads[2], kDevInvalidInput);
+                        atomicAdd(&p.heads[kCountInvalid], 1);
                     }
                 } else {
                     for (int q = lane; q <= K; q += 32) ot[q] = q < rj ? p.x[(size_t)rb * K + q] : (q == rj ? token : -1);

@@ -571,18 +571,64 @@ def test_workspace_recorded_in_a_graph_outlives_a_larger_call(ears):
     assert ears.last_device_status(side) == 0
 
 
+def oracle_class_counts(ora, K):
+    want = {"direct": 0, "pardon": 0, "reject": 0, "invalid": int((ora.accept_len < 0).sum())}
+    for b in range(len(ora.accept_len)):
+        if ora.accept_len[b] >= 0:
+            for k in range(min(int(ora.accept_len[b]) + 1, K)):
+                want[("reject", "direct", "pardon")[int(ora.cls[b, k])]] += 1
+    return want
+
+
 def test_decision_class_counts_match_the_oracle(ears):
-    """direct / pardon / reject (Sec. 3.2 step 5) counted over the decided positions."""
+    """direct / pardon / reject (Sec. 3.2 step 5) counted over the decided positions, from the class output."""
     w, t, d, x = synth.tiny_inputs(64, 4, 3000, "fp32", seed=77, noise=1.2)
     acc, tok, st = ears.verify(t.cuda(), d.cuda(), x.cuda(), 1.0, 0.3, 2, 0, stats=True)
     got = ears.class_counts(st, acc)
     ora = oracle.verify(t, d, x, 1.0, 0.3, seed=2, offset=0)
-    want = {"direct": 0, "pardon": 0, "reject": 0}
-    for b in range(64):
-        for k in range(min(int(ora.accept_len[b]) + 1, 4)):
-            want[("reject", "direct", "pardon")[int(ora.cls[b, k])]] += 1
+    want = oracle_class_counts(ora, 4)
+    want.pop("invalid")
     assert got == want and got["pardon"] > 0 and got["reject"] > 0
     assert got["reject"] == int((ora.accept_len < 4).sum())
+
+
+@pytest.mark.parametrize("stop_first", [False, True])
+@pytest.mark.parametrize("path,cluster", [(1, 0), (3, 0), (2, 0), (2, 4), (4, 0), (4, 2)])
+def test_device_side_decision_counters(ears, forced_path, path, cluster, stop_first):
+    """The counters the kernels keep themselves (no optional output asked for): direct / pardon /
+    reject over what each sequence decided, and invalid sequences; with a caller workspace too; and
+    every call starts them from zero."""
+    forced_path(path, cluster)
+    dev = "cuda:0"
+    for dtype, V in (("fp32", 3000), ("bf16", 20001)):
+        w, t, d, x = synth.tiny_inputs(96, 4, V, dtype, seed=78, noise=1.2)
+        x = x.clone()
+        x[5, 1] = V + 3
+        x[17, 0] = -1
+        tg, dg, xg = t.to(dev), d.to(dev), x.to(dev)
+        ora = oracle.verify(t, d, x, 1.0, 0.3, seed=2, offset=0, nthreads=8, stop_at_first_reject=stop_first)
+        # (a decision within 1e-5 of its threshold, or a ratio that close to U, could be classed either way)
+        near = (np.abs(ora.margin) < 1e-5).any() or (np.abs(ora.pt_tok / np.maximum(ora.pd_tok, 1e-10)
+                                                               - np.vectorize(lambda b, k: oracle.uniform_accept(2, 0, b, k))(
+                                                                   *np.indices(ora.margin.shape))) < 1e-5).any()
+        want = oracle_class_counts(ora, 4)
+        for rep in range(2):
+            ears.verify(tg, dg, xg, 1.0, 0.3, 2, 0, stop_at_first_reject=stop_first)
+            got = ears.decision_counts()
+            assert got["invalid"] == want["invalid"] >= 1
+            if not near:
+                assert got == want, (got, want)
+            assert got["pardon"] > 0 and got["reject"] > 0
+        ws = torch.empty(ears.workspace_bytes(96, 4, V) + 256, dtype=torch.uint8, device=dev)
+        ws = ws[(-ws.data_ptr()) % 256:]
+        ears.verify(tg, dg, xg, 1.0, 0.3, 2, 0, workspace=ws, stop_at_first_reject=stop_first)
+        got_ws = ears.decision_counts(workspace=ws)
+        if not near:
+            assert got_ws == want
+        # a clean batch afterwards: nothing left over
+        ears.verify(tg[20:40], dg[20:40], xg[20:40], 1.0, 50.0, 2, 0, b_first=20, stop_at_first_reject=stop_first)
+        clean = ears.decision_counts()
+        assert clean["invalid"] == 0 and clean["reject"] == 0 and clean["direct"] + clean["pardon"] == 20 * 4
 
 
 @pytest.mark.parametrize("path,cluster", [(1, 0), (3, 0), (2, 0), (2, 4), (4, 0), (4, 2)])
