@@ -29,6 +29,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     if _lib is not None and path is None:
         return _lib
     if path is None:
+        path = os.environ.get("EARS_LIBRARY")      # another build of the same library (a variant under test)
+    if path is None:
         path = _build.LIB
         if not os.path.exists(path):
             path = _build.build()

@@ -42,7 +42,10 @@ namespace ears {
 constexpr int kDThreads = EARS_D_THREADS;
 constexpr int kDWarps = kDThreads / 32;
 constexpr int kDCtasPerSm = EARS_D_CTAS;
-constexpr int kDUnroll = 8;                        // 16-byte loads in flight per thread
+#ifndef EARS_D_UNROLL
+#define EARS_D_UNROLL 8
+#endif
+constexpr int kDUnroll = EARS_D_UNROLL;            // 16-byte loads in flight per thread
 constexpr int kBonusSegBytes = kChunkBytes / kConsumerWarps;   // bytes of the extra row per stored sum (2 KB)
 
 enum DWorkKind : int { kDUnit = 0, kDJob = 1, kDIdle = 2, kDExit = 3 };

@@ -349,25 +349,50 @@ __device__ int finalize_sequence(const Params& p, int b, int lane) {
     // tracked per position in `stop` (the first position that is rejected or unusable ends the scan).
     const bool stop_first = p.stop_first != 0;
     bool bad = !seq_params_ok(Tb, betab);
+    // Dependent round trips through L2 are what this function costs (it runs on one warp while the
+    // sequence's CTAs wait for nobody, but every sequence passes through it), so loads go out in
+    // batches and as early as their addresses are known: the draft tokens first, then the pieces of
+    // the rows, then the tokens' logits; with at most 32 rows the rows' statistics then travel between
+    // lanes by shuffle instead of through memory.
+    const bool rows_fit = R <= 32;
+    int tok_early = -1;
+    if (rows_fit && lane < K) tok_early = p.x[(size_t)b * K + lane];
+    float m_mine = -INFINITY, s_mine = 0.0f, w_mine = 0.0f;   // rows_fit: row `lane`
     for (int r = lane; r < R; r += 32) {
         float m = -INFINITY, s = 0.0f;
         const float2* pp = p.partial + ((size_t)b * R + r) * P;
-        for (int i = 0; i < P; ++i) {
-            float2 v = __ldcg(pp + i);
-            merge_ms(m, s, v.x, v.y, cb);
+        for (int i0 = 0; i0 < P; i0 += 8) {
+            float2 v[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = i0 + i < P ? __ldcg(pp + i0 + i) : make_float2(-INFINITY, 0.f);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) merge_ms(m, s, v[i].x, v[i].y, cb);
         }
         if (!rowstat_ok(m, s) && !stop_first) bad = true;
         p.rowstat[(size_t)b * R + r] = make_float2(m, s);
+        float w = 0.f;
         if (ENT && !(r & 1) && r < 2 * K) {
             // sum e t of a target row: its pieces brought to the row maximum (known now)
             const float* pw = p.partial_w + ((size_t)b * R + r) * P;
-            float w = 0.f;
-            for (int i = 0; i < P; ++i) {
-                const float2 v = __ldcg(pp + i);
-                w += rebase_sum_w(v.x, v.y, __ldcg(pw + i), m, cb).y;
+            for (int i0 = 0; i0 < P; i0 += 8) {
+                float2 v[8];
+                float q[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    v[i] = i0 + i < P ? __ldcg(pp + i0 + i) : make_float2(-INFINITY, 0.f);
+                    q[i] = i0 + i < P ? __ldcg(pw + i0 + i) : 0.f;
+                }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) w += rebase_sum_w(v[i].x, v[i].y, q[i], m, cb).y;
             }
             p.roww[(size_t)b * R + r] = w;
         }
+        m_mine = m; s_mine = s; w_mine = w;
+    }
+    float lt_early = 0.f, ld_early = 0.f;
+    if (rows_fit && lane < K && tok_early >= 0 && tok_early < V) {
+        lt_early = load_logit(t + (size_t)target_row(b, lane, K) * V + tok_early);
+        ld_early = load_logit(d + (size_t)draft_row(b, lane, K) * V + tok_early);
     }
     __syncwarp();
     int first_reject = K;
@@ -375,20 +400,31 @@ __device__ int finalize_sequence(const Params& p, int b, int lane) {
     for (int k0 = 0; k0 < K; k0 += 32) {
         const int k = k0 + lane;
         bool reject = false, posbad = false;
+        // the statistics of this position's two rows: from the lanes that merged them, or from memory
+        float2 st, sd;
+        float wt = 0.f;
+        if (rows_fit) {
+            const int src = k < K ? 2 * k : 0;
+            st = make_float2(__shfl_sync(0xffffffffu, m_mine, src), __shfl_sync(0xffffffffu, s_mine, src));
+            sd = make_float2(__shfl_sync(0xffffffffu, m_mine, src + 1), __shfl_sync(0xffffffffu, s_mine, src + 1));
+            if (ENT) wt = __shfl_sync(0xffffffffu, w_mine, src);
+        } else if (k < K) {
+            st = __ldcg(&p.rowstat[(size_t)b * R + 2 * k]);
+            sd = __ldcg(&p.rowstat[(size_t)b * R + 2 * k + 1]);
+            if (ENT) wt = __ldcg(&p.roww[(size_t)b * R + 2 * k]);
+        }
         if (k < K) {
-            const int tok = p.x[(size_t)b * K + k];
-            const float2 st = __ldcg(&p.rowstat[(size_t)b * R + 2 * k]);
-            const float2 sd = __ldcg(&p.rowstat[(size_t)b * R + 2 * k + 1]);
+            const int tok = rows_fit ? tok_early : p.x[(size_t)b * K + k];
             posbad = tok < 0 || tok >= V || !rowstat_ok(st.x, st.y) || !rowstat_ok(sd.x, sd.y);
             if (tok < 0 || tok >= V) {
                 if (!stop_first) bad = true;
             } else {
-                const double lt = (double)load_logit(t + (size_t)target_row(b, k, K) * V + tok);
-                const double ld = (double)load_logit(d + (size_t)draft_row(b, k, K) * V + tok);
+                const double lt = (double)(rows_fit ? lt_early : load_logit(t + (size_t)target_row(b, k, K) * V + tok));
+                const double ld = (double)(rows_fit ? ld_early : load_logit(d + (size_t)draft_row(b, k, K) * V + tok));
                 const double U = uniform_accept(p.seed, p.offset, (uint32_t)(p.b_first + b), (uint32_t)k);
                 double unc = -1.0;   // < 0: the printed measure, 1 - max P_t
                 if (ENT) {
-                    const double H = row_entropy(st.y, __ldcg(&p.roww[(size_t)b * R + 2 * k]));
+                    const double H = row_entropy(st.y, wt);
                     if (p.entropy) p.entropy[(size_t)b * K + k] = H;
                     if (p.unc_entropy) unc = entropy_uncertainty(H, V);
                 }
