@@ -37,7 +37,9 @@ FALLBACK_HBM_GBS = 6650.0
 # out (None) whenever its kernel changes after the capture.
 NCU_DRAM_BYTES_PER_SEQUENCE = {
     # kernel name: (bytes per sequence, what was captured)
-    "ears_verify_kernel": None,
+    "ears_verify_kernel": ((691050496 + 5236992) / 96,
+                           "ncu dram__bytes_read.sum + dram__bytes_write.sum of ears_verify_kernel<float,6,false,false> on a 96-sequence "
+                           "batch of this workload (profiles/ears_verify_kernel_cfg5.md), scaled by sequences"),
 }
 
 

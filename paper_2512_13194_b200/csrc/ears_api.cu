@@ -246,7 +246,11 @@ size_t streamed_area(int slice) {
     const size_t bonus4 = ((size_t)slice * 4 / kBonusSegBytes + kCBonusPad) * sizeof(BonusSeg);
     return std::max(job, std::max(bonus, bonus4));
 }
-size_t streamed_smem(int slice) { return ((sizeof(CSmem) + 127) & ~size_t(127)) + streamed_area(slice) + 128; }
+// behind the sums, 128-byte aligned: the copy ring
+size_t streamed_ring_offset(int slice) { return align_up(streamed_area(slice), 128); }
+size_t streamed_smem(int slice, int esize) {   // (only 4-byte logits use the ring)
+    return ((sizeof(CSmem) + 127) & ~size_t(127)) + streamed_ring_offset(slice) + (esize == 4 ? (size_t)kCStages * kCStageBytes : 0) + 128;
+}
 
 RPlan make_splan(int B, int K, int V, int esize, int sms, int max_cluster, int forced_cluster, bool ordered) {
     RPlan best;
@@ -266,7 +270,7 @@ RPlan make_splan(int B, int K, int V, int esize, int sms, int max_cluster, int f
         const double t_item = item_bytes / C / std::min(share, 60e9) + 2.5e-6;
         const double t = rounds * t_item * (ordered ? K + 1 : 1);   // walking a sequence in order: up to K+1 positions in a row
         if (!best.ok || t < best_t) {
-            best.ok = true; best.C = C; best.slice = slice; best.buf_bytes = 0; best.smem = streamed_smem(slice);
+            best.ok = true; best.C = C; best.slice = slice; best.buf_bytes = (int)streamed_ring_offset(slice); best.smem = streamed_smem(slice, esize);
             best.roomy = true; best.streamed = true;
             best_t = t;
         }
@@ -362,9 +366,9 @@ int profile_mark(cudaStream_t stream, bool timed) {
 template <typename E>
 int set_attrs_streamed(bool* cluster16) {
     EARS_CUDA(cudaFuncSetAttribute(ears_cstream_kernel<E, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   (int)(streamed_smem(0) + kStreamedSegBytes)));
+                                   (int)(streamed_smem(0, (int)sizeof(E)) + kStreamedSegBytes)));
     EARS_CUDA(cudaFuncSetAttribute(ears_cstream_kernel<E, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   (int)(streamed_smem(0) + kStreamedSegBytes)));
+                                   (int)(streamed_smem(0, (int)sizeof(E)) + kStreamedSegBytes)));
     if (cudaFuncSetAttribute(ears_cstream_kernel<E, false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
         cudaFuncSetAttribute(ears_cstream_kernel<E, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
         (void)cudaGetLastError();

@@ -1,4 +1,4 @@
-// The verification step with thread-block clusters that stream their rows: nothing is staged.
+// The verification step with thread-block clusters that stream their rows.
 //
 // Work item = one position of one sequence, as in the resident kernel: the pair (target row k,
 // draft row k), or the extra target row K.  A cluster of C CTAs takes an item from a queue; CTA j
@@ -20,7 +20,12 @@
 // read again (usually from L2).  A rejected position that is not the sequence's first costs nothing.
 // There is no global queue of second-pass work, no publication and no hand-over between clusters; a
 // cluster never waits for another cluster.  Without a shared-memory footprint several clusters share
-// an SM and hide each other's exchanges.  Ordered mode (EARS_FLAG_STOP_AT_FIRST_REJECT): the queue
+// an SM and hide each other's exchanges.  What a thread's own loads can keep in flight (eight 16-byte
+// loads, 32 KB per CTA) bounds a CTA to some 20 GB/s; whenever few CTAs are at work (a batch that
+// does not fill the machine, a second-pass job, the end of a launch) that bound is the speed of the
+// launch.  Rows of 4-byte logits that are 16-byte aligned therefore pass, for their statistics,
+// through a small ring of shared-memory stages filled by bulk asynchronous copies (64 KB in flight
+// per CTA, no registers held) and read by all threads of the CTA.  Ordered mode (EARS_FLAG_STOP_AT_FIRST_REJECT): the queue
 // holds sequences, a cluster walks one position by position and stops at its first rejection, whose
 // masses it computes at once; rows after it are never read.
 #pragma once
@@ -41,10 +46,13 @@ constexpr int kCBonusPad = 8;             // stream_bonus_piece may clear up to 
 #ifndef EARS_C_CTAS
 #define EARS_C_CTAS 3
 #endif
-constexpr int kCCtasPerSm = EARS_C_CTAS;  // no shared-memory footprint to speak of: registers set the limit
+constexpr int kCCtasPerSm = EARS_C_CTAS;
+constexpr int kCStages = 4;               // stages of the CTA's copy ring
+constexpr int kCStageBytes = 16384;       // per stage: 16 KB of one row, or 8 KB of each of two rows
 
 struct CSmem {
-    alignas(8) uint64_t xbar[2];          // statistics exchange, alternating by round
+    alignas(8) uint64_t full[kCStages];   // copy ring: bytes of a stage have landed
+    uint64_t xbar[2];                     // statistics exchange, alternating by round
     uint64_t mbar2[2];                    // mass-total exchange, alternating by mass round
     alignas(16) float4 xstat[2][kRMaxCluster * kCWarps];   // (m_t, s_t, m_d, s_d) of every warp of every peer
     float xw[2][kRMaxCluster * kCWarps];  // sum e t of the target slice of every warp of every peer (entropy kernels)
@@ -61,6 +69,57 @@ struct CSmem {
 
 __device__ __forceinline__ void peer_store(uint32_t addr, int2 v) {
     asm volatile("st.shared::cluster.v2.s32 [%0], {%1, %2};" ::"r"(addr), "r"(v.x), "r"(v.y) : "memory");
+}
+
+// ---- the copy ring ----------------------------------------------------------------------
+// All threads of the CTA sweep entries [e0, e0 + n) of one row (r1 = nullptr: 16 KB per stage) or of
+// two rows side by side (8 KB of each per stage).  Thread 0 keeps kCStages bulk copies in flight;
+// every thread waits for a stage, `process(first half, second half, entries before this stage,
+// entries per row in it)` reads it, and after a block-wide barrier the stage is filled again.
+// q: stage fills so far (the same in every thread).  -> false if a wait gave up.
+// Rows must be 16-byte aligned, e0 and n whole 16-byte vectors.
+template <typename E, class F>
+__device__ __forceinline__ bool staged_sweep(CSmem& sm, unsigned char* ring, uint32_t& q, const E* r0, const E* r1, int e0, int n,
+                                             F process) {
+    const int ce = (r1 ? kCStageBytes / 2 : kCStageBytes) / (int)sizeof(E);   // entries per row and stage
+    const int nchunks = (n + ce - 1) / ce;
+    auto issue = [&](int c) {   // thread 0
+        const int stage = (int)((q + (uint32_t)c) % kCStages);
+        const uint32_t bytes = (uint32_t)min(ce, n - c * ce) * (uint32_t)sizeof(E);
+        unsigned char* dst = ring + (size_t)stage * kCStageBytes;
+        mbar_arrive_expect_tx(&sm.full[stage], r1 ? 2 * bytes : bytes);
+        bulk_load(dst, r0 + e0 + (size_t)c * ce, bytes, &sm.full[stage]);
+        if (r1) bulk_load(dst + kCStageBytes / 2, r1 + e0 + (size_t)c * ce, bytes, &sm.full[stage]);
+    };
+    if (threadIdx.x == 0)
+        for (int c = 0; c < nchunks && c < kCStages; ++c) issue(c);
+    bool ok = true;
+    for (int c = 0; c < nchunks; ++c) {
+        const uint32_t qq = q + (uint32_t)c;
+        const int stage = (int)(qq % kCStages);
+        if (ok && !mbar_wait(&sm.full[stage], (qq / kCStages) & 1u, &sm.abort_flag)) ok = false;
+        const unsigned char* src = ring + (size_t)stage * kCStageBytes;
+        if (ok) process(src, src + kCStageBytes / 2, c * ce, min(ce, n - c * ce));
+        // everyone is through with the stage (or has given up: then the copies that are still in flight
+        // are waited for below, and nothing more is issued)
+        if (__syncthreads_or(ok ? 0 : 1)) { ok = false; }
+        if (ok && threadIdx.x == 0 && c + kCStages < nchunks) issue(c + kCStages);
+        if (!ok) {
+            // bounded wait for what was issued beyond this stage, so that no copy lands in memory the CTA has left
+            if (threadIdx.x == 0) {
+                for (int cc = c + 1; cc < nchunks && cc < c + kCStages; ++cc) {
+                    const uint32_t q2 = q + (uint32_t)cc;
+                    const unsigned long long t0 = global_timer_ns();
+                    while (!mbar_try_wait(&sm.full[q2 % kCStages], (q2 / kCStages) & 1u)) {
+                        if (global_timer_ns() - t0 > kWaitLimitNs) break;
+                    }
+                }
+            }
+            break;
+        }
+    }
+    q += (uint32_t)nchunks;
+    return ok;
 }
 
 // A segment sum of the extra row, taken relative to mu, brought to the row's own maximum (mc = m c,
@@ -212,6 +271,8 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
     unsigned char* area = reinterpret_cast<unsigned char*>(&sm) + ((sizeof(CSmem) + 127) & ~size_t(127));
     double* const segsum = reinterpret_cast<double*>(area);     // a job's sums per kSegElems entries
     BonusSeg* const bseg = reinterpret_cast<BonusSeg*>(area);   // the extra row's sums per 2 KB (never in use together)
+    unsigned char* const ring = area + p.buf_bytes;             // the copy ring (behind the sums; 128-byte aligned)
+    uint32_t ring_q = 0;                                        // stage fills so far
     constexpr int BSEG = kBonusSegBytes / (int)sizeof(E);       // entries per bonus segment
     const int K = p.K, V = p.V, C = p.C;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -229,6 +290,7 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
     clear_next_counters(p);
     if (tid == 0) {
         for (int i = 0; i < 2; ++i) { mbar_init(&sm.xbar[i], (unsigned)(C * kCWarps)); mbar_init(&sm.mbar2[i], (unsigned)C); }
+        for (int i = 0; i < kCStages; ++i) mbar_init(&sm.full[i], 1u);
         sm.abort_flag = 0;
         sm.my_job_b = -1;
         sm.my_job_n = 0;
@@ -288,7 +350,78 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
         if (tid == 0) trace_mark(1, work ? b * (K + 1) + j : -1);
         float2 pt2 = make_float2(-INFINITY, 0.f), pd2 = make_float2(-INFINITY, 0.f);
         float wv = 0.f;   // ENT: the thread's sum e t over the target slice
-        if (work) {
+        // 4-byte logits take the copy ring (measured on B200, 64 sequences of 1 MB rows: 121 us against 184);
+        // 2-byte logits do twice the arithmetic per staged byte and lose to their own loads there
+        // (32 sequences of 256 KB rows: 55 us against 47), so they keep the register path
+        const bool staged = vec && sizeof(E) == 4;
+        if (work && staged && pair) {
+            // through the copy ring: 8 KB of each row per stage, two vectors of each per thread
+            constexpr int N = Words<E>::N;
+            RowAccT<ENT> at;
+            RowAcc ad;
+            acc_open(at);
+            acc_open(ad);
+            const bool swept = staged_sweep<E>(sm, ring, ring_q, trow, drow, e0, n,
+                [&](const unsigned char* bt, const unsigned char* bd, int, int cnt) {
+                    const int nv = cnt / N;   // whole vectors: rows and slices are
+                    uint4 wt[2], wd[2];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int v = tid + h * kCThreads;
+                        wt[h] = v < nv ? reinterpret_cast<const uint4*>(bt)[v] : Words<E>::minus_inf();
+                        wd[h] = v < nv ? reinterpret_cast<const uint4*>(bd)[v] : Words<E>::minus_inf();
+                    }
+                    fold_vectors<E, 2, ENT>(wt, cb, at);
+                    fold_vectors<E, 2, false>(wd, cb, ad);
+                });
+            if (!swept) { failed = true; break; }
+            pt2 = acc_close(at, cb, &wv);
+            pd2 = acc_close(ad, cb);
+        } else if (work && staged) {
+            // the extra row through the copy ring: 16 KB per stage, warp w takes its 2 KB block w, keeps a
+            // warp-uniform running maximum and leaves (sum, reference) of the block behind
+            constexpr int N = Words<E>::N, PN = N / 2, VPL = BSEG / N / 32;
+            RowAcc a;
+            acc_open(a);
+            const f32x2 c2 = pack2(cb, cb);
+            const bool swept = staged_sweep<E>(sm, ring, ring_q, trow, (const E*)nullptr, e0, n,
+                [&](const unsigned char* bt, const unsigned char*, int before, int cnt) {
+                    const int first = warp * BSEG;   // this warp's block within the stage
+                    if (first >= cnt) return;
+                    uint4 w[VPL];
+#pragma unroll
+                    for (int i = 0; i < VPL; ++i) {
+                        const int k0 = first + (i * 32 + lane) * N;
+                        w[i] = k0 < cnt ? reinterpret_cast<const uint4*>(bt)[k0 / N] : Words<E>::minus_inf();
+                    }
+                    float cm = Words<E>::template vmax_all<VPL>(w);
+#pragma unroll
+                    for (int off = 16; off > 0; off >>= 1) cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, off));
+                    acc_raise(a, cm, cb);
+                    const f32x2 nmu2 = pack2(-a.mu, -a.mu);
+                    f32x2 cs[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
+#pragma unroll
+                    for (int i = 0; i < VPL; ++i) {
+                        f32x2 q2[PN];
+                        Words<E>::pairs(w[i], q2);
+#pragma unroll
+                        for (int u = 0; u < PN; u += 2) {
+                            cs[0] = add2(cs[0], ex2_pair(fma2(q2[u], c2, nmu2)));
+                            cs[1] = add2(cs[1], ex2_pair(fma2(q2[u + 1], c2, nmu2)));
+                        }
+                    }
+                    a.s[0] = add2(a.s[0], cs[0]);
+                    a.s[1] = add2(a.s[1], cs[1]);
+                    float q0, q1;
+                    unpack2(add2(cs[0], cs[1]), q0, q1);
+                    double tot = (double)(q0 + q1);   // a lane's few terms in fp32, lanes in fp64
+#pragma unroll
+                    for (int off = 16; off > 0; off >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, off);
+                    if (lane == 0) bseg[(before + first) / BSEG] = BonusSeg{tot, a.mu, 0.f};
+                });
+            if (!swept) { failed = true; break; }
+            pt2 = acc_close(a, cb);
+        } else if (work) {
             if (pair) {
                 pt2 = stream_piece<E, kCThreads, ENT>(trow, e0, e0 + n, vec, cb, tid, &wv);
                 pd2 = stream_piece<E, kCThreads>(drow, e0, e0 + n, vec, cb, tid);
@@ -464,8 +597,11 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
             bool resid = true;
             __syncthreads();                         // the bonus sums of step 4 (same memory) are no longer needed
             for (;;) {
-                if (resid) stream_job_piece<E, true>(jt, jd, e0, e0 + n, vec, rn, cj, warp, lane, so);
-                else stream_job_piece<E, false>(jt, jt, e0, e0 + n, vec, rn, cj, warp, lane, so);
+                if (resid) {
+                    stream_job_piece<E, true>(jt, jd, e0, e0 + n, vec, rn, cj, warp, lane, so);
+                } else {
+                    stream_job_piece<E, false>(jt, jt, e0, e0 + n, vec, rn, cj, warp, lane, so);
+                }
                 __syncthreads();
                 if (!cluster_pick<E>(sm, p, val, (n + kSegElems - 1) / kSegElems, kSegElems, job_b, resid, jt, jd, rn, cj, e0, n, rank,
                                      C, mround, jtoken)) {
