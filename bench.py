@@ -689,6 +689,133 @@ def run_greedy_table(args):
         del t, x
 
 
+def run_early_table(args):
+    """Leaving out what follows a sequence's first rejection (EARS_FLAG_STOP_AT_FIRST_REJECT) at large
+    batches: the rows a step needs, and the time with the flag off and on (identical results
+    required), L2 flushed before every step.  Not the benchmark line."""
+    import torch
+
+    import paper_2512_13194_b200 as ears
+    from dataclasses import replace
+    from paper_2512_13194_b200 import synth
+
+    torch.cuda.set_device(0)
+    ears.load_library()
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+
+    def timed(fn, n=21):
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+        for a, b in ev:
+            flush.zero_(); a.record(); fn(); b.record()
+        torch.cuda.synchronize()
+        return statistics.median(a.elapsed_time(b) * 1e3 for a, b in ev)
+
+    print("| workload | B | beta | rows needed / rows | flag off: kernel, us | flag on: us |")
+    print("|---|---|---|---|---|---|")
+    for idx, B in ((4, 1024), (4, 256), (2, 4096), (3, 512), (5, 512)):
+        w = replace(synth.workload(idx), B=B)
+        t, d, x = synth.make_inputs(w, "cuda:0")
+        for beta in (w.beta, 0.0):
+            off = lambda: ears.verify(t, d, x, w.temperature, beta, 0, 1)
+            on = lambda: ears.verify(t, d, x, w.temperature, beta, 0, 1, stop_at_first_reject=True)
+            a0, t0 = off()
+            p_off = ears.describe_plan(w.dtype, w.B, w.K, w.V).split(":")[0]
+            a1, t1 = on()
+            torch.cuda.synchronize()
+            assert torch.equal(a0, a1) and torch.equal(t0, t1)
+            n = a0.clamp(min=0)
+            need = int((2 * torch.clamp(n + 1, max=w.K) + (n == w.K)).sum())
+            print(f"| {idx} | {B} | {beta} | {need} / {w.rows} ({need / w.rows:.2f}) | {p_off}, {timed(off):.1f} | {timed(on):.1f} |", flush=True)
+        del t, d, x
+
+
+def run_read_ceiling(args):
+    """What library reductions reach on this GPU over a tensor of the benchmark workload's size
+    (read-only traffic, unlike the read + write copy behind the measured peak): context for the
+    roofline fraction.  Not the benchmark line."""
+    import torch
+
+    torch.cuda.set_device(0)
+    peak, peak_kind = measured_peak()
+    print(f"| dtype | GB | op | median ms | GB/s | of {peak:.0f} ({peak_kind}) |")
+    print("|---|---|---|---|---|---|")
+    for dt, n in ((torch.float32, 917504000), (torch.bfloat16, 1835008000)):
+        x = torch.empty(n, dtype=dt, device="cuda").normal_()
+        y = torch.empty_like(x)
+        gb = x.numel() * x.element_size() / 1e9
+        for name, fn, mult in (("sum (read only)", lambda: x.sum(), 1), ("max (read only)", lambda: x.max(), 1),
+                               ("copy_ (read + write)", lambda: y.copy_(x), 2)):
+            for _ in range(3):
+                fn()
+            ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(20)]
+            for a, b in ev:
+                a.record(); fn(); b.record()
+            torch.cuda.synchronize()
+            med = statistics.median(a.elapsed_time(b) for a, b in ev)
+            print(f"| {str(dt).split('.')[-1]} | {gb:.2f} | {name} | {med:.3f} | {mult * gb / med * 1e3:.0f} | {mult * gb / med * 1e3 / peak:.2f} |", flush=True)
+        del x, y
+
+
+def run_path_table(args):
+    """Every kernel forced in turn (ears_set_path) on the workloads and on larger batches of their
+    shapes, L2 flushed before every step, median of 21 event-timed steps.  '-': that kernel cannot
+    take the shape.  Not the benchmark line."""
+    import torch
+
+    import paper_2512_13194_b200 as ears
+    from dataclasses import replace
+    from paper_2512_13194_b200 import synth
+
+    torch.cuda.set_device(0)
+    ears.load_library()
+    peak, peak_kind = measured_peak()
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    names = {0: "automatic", 1: "ring", 2: "resident", 3: "direct", 4: "cluster-streamed"}
+    print(f"| shape | logits GB | beta | rejected sequences | automatic choice | " + " | ".join(f"{names[q]} us" for q in range(5))
+          + f" | best GB/s (of {peak:.0f} {peak_kind}) |")
+    print("|---|---|---|---|---|" + "---|" * 6)
+    cases = ((1, 0, None), (2, 0, None), (3, 0, None), (4, 0, None), (5, 0, None), (4, 1024, 50.0), (4, 1024, None), (4, 1024, 0.0),
+             (3, 512, None), (2, 4096, None), (1, 2048, None), (5, 512, 0.0))
+    if args.batch:
+        cases = ((args.workload, args.batch, args.beta),)
+    for idx, B, beta in cases:
+        w = synth.workload(idx)
+        if B:
+            w = replace(w, B=B)
+        beta = w.beta if beta is None else beta
+        t, d, x = synth.make_inputs(w, "cuda:0")
+        nbytes = t.numel() * t.element_size() + d.numel() * d.element_size()
+        cells, ref, best = [], None, None
+        for q in range(5):
+            ears.set_path(q, 0)
+            try:
+                acc, tok = ears.verify(t, d, x, w.temperature, beta, w.verify_seed, 1)
+            except ears.EarsError:
+                cells.append("-")
+                continue
+            torch.cuda.synchronize()
+            if ref is None:
+                ref = (acc, tok, ears.describe_plan(w.dtype, w.B, w.K, w.V).split(":")[0])
+            else:   # every kernel must give the automatic choice's result (a sanity check, not the parity test: near-ties may differ)
+                assert (acc != ref[0]).sum() <= 2 and (tok != ref[1]).any(-1).sum() <= 8
+            ts = []
+            for it in range(3 + 21):
+                flush.zero_()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); ears.verify(t, d, x, w.temperature, beta, w.verify_seed, 1); b.record()
+                torch.cuda.synchronize()
+                if it >= 3:
+                    ts.append(a.elapsed_time(b) * 1e3)
+            us = statistics.median(ts)
+            best = us if best is None else min(best, us)
+            cells.append(f"{us:.1f}")
+        ears.set_path(0, 0)
+        rej = int((ref[0] < w.K).sum())
+        print(f"| workload {idx} at B={w.B} | {nbytes / 1e9:.3f} | {beta} | {rej} | {ref[2]} | " + " | ".join(cells)
+              + f" | {nbytes / best / 1e3:.0f} ({nbytes / best / 1e3 / peak:.2f}) |", flush=True)
+        del t, d, x
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -714,6 +841,9 @@ def main():
     ap.add_argument("--shard-table", action="store_true",
                     help="print per-phase times of one rank of the vocabulary-sharded step instead")
     ap.add_argument("--greedy-table", action="store_true", help="print times of the temperature -> 0 form instead")
+    ap.add_argument("--path-table", action="store_true", help="print the time of every kernel, forced in turn, on a list of shapes instead")
+    ap.add_argument("--early-table", action="store_true", help="print times with / without stopping at the first rejection instead")
+    ap.add_argument("--read-ceiling", action="store_true", help="print what library reductions reach on this GPU instead")
     args = ap.parse_args()
     if args.timeline:
         run_timeline(args)
@@ -721,6 +851,12 @@ def main():
         run_series(args)
     elif args.greedy_table:
         run_greedy_table(args)
+    elif args.path_table:
+        run_path_table(args)
+    elif args.early_table:
+        run_early_table(args)
+    elif args.read_ceiling:
+        run_read_ceiling(args)
     elif args.shard_table:
         run_shard_table(args)
     elif args.table:

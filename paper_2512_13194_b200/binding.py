@@ -444,7 +444,9 @@ class ShardStep:
 
 def set_path(path: int = 0, cluster: int = 0) -> None:
     """0 = automatic; path 1 streaming kernel with the shared-memory ring, 2 resident (cluster) kernel,
-    3 streaming kernel reading straight from global memory; cluster = CTAs per cluster."""
+    3 streaming kernel reading straight from global memory, 4 cluster-streamed kernel; cluster = CTAs
+    per cluster (paths 2 and 4; 0 = chosen by the library).  A forced path that cannot take a call's
+    shape makes that call fail with EARS_ERR_SHAPE."""
     _check(load_library().ears_set_path(path, cluster))
 
 

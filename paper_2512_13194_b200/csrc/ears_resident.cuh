@@ -470,8 +470,10 @@ __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RPara
     // barriers of every CTA are initialised before any peer arrives on them; the first copies
     // (into this CTA's own memory only) are already under way
     cluster_sync_all();
+    if (tid == 0) trace_mark(0, 0);
     while (have) {
         // ---- 1. statistics of the slices as the copies land
+        if (tid == 0) trace_mark(1, b * (K + 1) + j);
         const float cb = seq_c(p, b);   // log2(e) / temperature of this sequence
         RowAccT<ENT> at;   // ENT: the target slice also yields its sum e t
         RowAcc ad;
@@ -486,6 +488,7 @@ __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RPara
             if (pair) stats_sub<E, false>(buf_d, q, n, tid, cb, ad);
         }
         if (use_tma) full_phase ^= issued;
+        if (tid == 0) trace_mark(2, 0);
         // (max, sum) of the warp's share: the maximum first (shuffles only), then one rescale per
         // thread and a sum -- a much shorter dependent chain than merging (m, s) pairs step by step
         const int par = round & 1;
@@ -518,6 +521,7 @@ __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RPara
         }
         bool ok = !failed && mbar_wait_cluster(&sm.xbar[par], (uint32_t)(round >> 1) & 1u, &sm.abort_flag);
         ++round;
+        if (tid == 0) trace_mark(3, 0);
         // ---- 3. the rows' (max, Z) and the decision
         if (ok && warp == 0) {
             float mt, zt, md, zd, wt;
@@ -535,6 +539,7 @@ __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RPara
         if (__syncthreads_or(ok ? 0 : 1)) { failed = true; break; }
         const int dec = sm.dec;
         const long long nxt = sm.xnext[par];
+        if (tid == 0) trace_mark(4, dec);
         // ---- 4. the token of a rejected position / the bonus token, from the resident slices
         int writer = (b + j) % C, token = -1;   // reports are spread over the CTAs of the cluster
         double mass = 0.0;
@@ -630,6 +635,7 @@ __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RPara
         // ---- 5. the slices and segment sums are free: start the next item's copies, then let one
         //         CTA report this item and count it; the sequence's last item finishes the sequence
         __syncthreads();
+        if (tid == 0) trace_mark(5, token);
         const int rb = b, rj = j;
         if (ordered && dec > 0 && pair) {
             issue_item(b, j + 1);          // accepted: on to the next position (or the extra row) of this sequence
@@ -693,6 +699,7 @@ __global__ void __launch_bounds__(kRThreads, 3) ears_resident_kernel(const RPara
         if (tid == 0) atomicOr(&p.heads[2], kDevTimeout);
     }
     __syncthreads();
+    if (tid == 0) trace_mark(6, 0);
     cluster_sync_all();
 }
 
