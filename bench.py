@@ -559,14 +559,14 @@ def run_timeline(args):
     ears.set_path(args.path, args.cluster)
     flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
     for i in range(3):
-        ears.verify(t, d, x, w.temperature, beta, w.verify_seed, i)
+        ears.verify(t, d, x, w.temperature, beta, w.verify_seed, i, stop_at_first_reject=args.stop_first)
     torch.cuda.synchronize()
     flush.zero_()
     torch.cuda.synchronize()
     assert lib.ears_trace_reset() == 0
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    acc, _ = ears.verify(t, d, x, w.temperature, beta, w.verify_seed, 7)
+    acc, _ = ears.verify(t, d, x, w.temperature, beta, w.verify_seed, 7, stop_at_first_reject=args.stop_first)
     e1.record()
     torch.cuda.synchronize()
     n_ctas, n_ev = ctypes.c_int(), ctypes.c_int()
@@ -722,7 +722,8 @@ def run_early_table(args):
             p_off = ears.describe_plan(w.dtype, w.B, w.K, w.V).split(":")[0]
             a1, t1 = on()
             torch.cuda.synchronize()
-            assert torch.equal(a0, a1) and torch.equal(t0, t1)
+            # the two calls may run different kernels: equal up to near-ties (a sanity check, not the parity test)
+            assert (a0 != a1).sum() <= 2 and (t0 != t1).any(-1).sum() <= 8
             n = a0.clamp(min=0)
             need = int((2 * torch.clamp(n + 1, max=w.K) + (n == w.K)).sum())
             print(f"| {idx} | {B} | {beta} | {need} / {w.rows} ({need / w.rows:.2f}) | {p_off}, {timed(off):.1f} | {timed(on):.1f} |", flush=True)
@@ -775,7 +776,10 @@ def run_path_table(args):
           + f" | best GB/s (of {peak:.0f} {peak_kind}) |")
     print("|---|---|---|---|---|" + "---|" * 6)
     cases = ((1, 0, None), (2, 0, None), (3, 0, None), (4, 0, None), (5, 0, None), (4, 1024, 50.0), (4, 1024, None), (4, 1024, 0.0),
-             (3, 512, None), (2, 4096, None), (1, 2048, None), (5, 512, 0.0))
+             (3, 512, None), (2, 4096, None), (1, 2048, None), (5, 512, 0.0),
+             # between the workloads' sizes: where the automatic choice changes hands
+             (1, 64, None), (2, 64, None), (2, 512, None), (3, 64, None), (3, 128, None), (3, 256, None),
+             (4, 32, None), (4, 64, None), (4, 256, None), (4, 512, None), (5, 32, None), (5, 128, None))
     if args.batch:
         cases = ((args.workload, args.batch, args.beta),)
     for idx, B, beta in cases:
@@ -832,6 +836,7 @@ def main():
     ap.add_argument("--path", type=int, default=0, help="with --timeline: force a kernel (ears_set_path)")
     ap.add_argument("--cluster", type=int, default=0, help="with --timeline: CTAs per cluster")
     ap.add_argument("--beta", type=float, default=None, help="with --timeline: override the workload's beta")
+    ap.add_argument("--stop-first", action="store_true", help="with --timeline: leave out what follows a first rejection")
     ap.add_argument("--series", type=int, default=0,
                     help="instead of the benchmark line: this many steps back to back, kernel time per launch "
                          "binned by the SM clock sampled beside it")

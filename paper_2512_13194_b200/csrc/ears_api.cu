@@ -206,7 +206,13 @@ Layout make_layout(int B, int K, int V, int parts1) {
 }
 
 // ---- the resident path: one position's rows held in the shared memory of a cluster ----
-struct RPlan { bool ok = false; int C = 0, slice = 0, buf_bytes = 0; size_t smem = 0; bool roomy = false; bool streamed = false; };
+struct RPlan {
+    bool ok = false;
+    int C = 0, slice = 0, buf_bytes = 0;
+    size_t smem = 0;
+    bool roomy = false, streamed = false;
+    int job_elems = 0, parts2 = 0;   // streaming clusters: entries per second-pass piece, pieces per job
+};
 
 size_t resident_smem(int buf_bytes) { return ((sizeof(RSmem) + 127) & ~size_t(127)) + 2 * (size_t)buf_bytes + 128; }
 
@@ -232,19 +238,19 @@ RPlan make_rplan(int B, int K, int V, int esize, int sms, int max_cluster, int f
     return best;
 }
 
-// The streamed form of the cluster kernel: nothing is staged, a CTA only keeps the segment sums of
-// its slice (8 bytes per 256 entries).  The cluster size is the one a small model of the launch
-// likes best: clusters pull positions from a queue, so the kernel takes
-// rounds x (time to stream a position + its exchange, decision and report), where the CTAs that are
-// active share the memory bandwidth and at least two rounds' worth of them hide each other's waits.
+// The streamed form of the cluster kernel: nothing is staged, a CTA only keeps the extra row's
+// sums per 2 KB of its slice.  Cluster size: a CTA pulls some 20 GB/s on its own, so positions are
+// split over as many CTAs as it takes to fill the CTA slots of the device in one round, and no
+// further -- a second, mostly empty round costs more than longer slices do (measured on B200, us for
+// clusters of 1 / 2 / 4: 32 x 8 positions of 2 x 256 KB: 60 / 73 / 79; 64 x 8: 95 / 97 / 119;
+// 128 x 5 of 2 x 304 KB: 111 / 115 / 145; 32 x 4 of 2 x 1 MB (4-byte): 97 / 72 / 86).  When sequences
+// are walked in order a small model of the launch picks the size instead: rounds x positions in a row
+// x (time to stream a position + its exchange, decision and report).
 constexpr size_t kStreamedSegBytes = 48 * 1024;   // segment sums of a slice: at most this much shared memory
 
-// bytes behind CSmem: a job's sums per 256 entries, or the extra row's per 2 KB (the larger of the two)
+// bytes behind CSmem: the extra row's sums per 2 KB of the slice (sized for 4-byte entries, which give the most)
 size_t streamed_area(int slice) {
-    const size_t job = (size_t)(slice / kSegElems) * sizeof(double);
-    const size_t bonus = ((size_t)slice * 2 / kBonusSegBytes + kCBonusPad) * sizeof(BonusSeg);   // 2-byte entries give the fewest, 4-byte: slice * 4
-    const size_t bonus4 = ((size_t)slice * 4 / kBonusSegBytes + kCBonusPad) * sizeof(BonusSeg);
-    return std::max(job, std::max(bonus, bonus4));
+    return ((size_t)slice * 4 / kBonusSegBytes + kCBonusPad) * sizeof(BonusSeg);
 }
 // behind the sums, 128-byte aligned: the copy ring
 size_t streamed_ring_offset(int slice) { return align_up(streamed_area(slice), 128); }
@@ -268,25 +274,40 @@ RPlan make_splan(int B, int K, int V, int esize, int sms, int max_cluster, int f
         // one CTA can pull on its own (~60 GB/s), plus ~2.5 us of exchange, decision and report
         const double share = 6.5e12 / (double)(clusters * C);
         const double t_item = item_bytes / C / std::min(share, 60e9) + 2.5e-6;
-        const double t = rounds * t_item * (ordered ? K + 1 : 1);   // walking a sequence in order: up to K+1 positions in a row
+        double t = rounds * t_item * (K + 1);   // walking a sequence in order: up to K+1 positions in a row
+        if (!ordered) t = items <= resident ? -(double)C : (double)C;   // the largest size whose clusters all run in one round, else the smallest
         if (!best.ok || t < best_t) {
             best.ok = true; best.C = C; best.slice = slice; best.buf_bytes = (int)streamed_ring_offset(slice); best.smem = streamed_smem(slice, esize);
             best.roomy = true; best.streamed = true;
             best_t = t;
         }
     }
+    if (best.ok) {
+        // Pieces of a job (a sequence's first rejected position) in the shared queue: 16 KB of each row
+        // (32 KB for 4-byte entries: one sweep of a CTA's warps), so that the many CTAs waiting at the end
+        // of a small batch finish a job in one short step.
+        const int chunk_elems = kChunkBytes / esize;
+        best.job_elems = (esize == 4 ? 2 : 1) * chunk_elems;
+        best.parts2 = (V + best.job_elems - 1) / best.job_elems;
+    }
     return best;
 }
 
-struct RLayout { size_t heads, ticket, seqmask, counters_bytes, flag, cand, cand_mass, rowstat, pt_tok, pd_tok, max_pt, cls, resid, total; };
+struct RLayout {
+    size_t heads, ticket, ticket2, seqmask, ready, counters_bytes, flag, cand, cand_mass, rowstat, pt_tok, pd_tok, max_pt, cls, resid,
+        seg, total;
+    int nseg;
+};
 
-RLayout make_rlayout(int B, int K) {
+RLayout make_rlayout(int B, int K, int V) {
     RLayout L;
     size_t o = 0;
     L.heads = o; o += kHeadsWords * 4;   // the status word is heads[2] of any workspace
     L.ticket = o; o += (size_t)B * 4;
+    L.ticket2 = o; o += (size_t)B * 4;
     o = align_up(o, 8);
     L.seqmask = o; o += (size_t)B * 8;
+    L.ready = o; o += (size_t)B * 8;
     L.counters_bytes = o;
     o = align_up(o, 256);
     L.flag = o; o = align_up(o + (size_t)B * (K + 1), 256);
@@ -298,6 +319,8 @@ RLayout make_rlayout(int B, int K) {
     L.max_pt = o; o = align_up(o + (size_t)B * K * 8, 256);
     L.cls = o; o = align_up(o + (size_t)B * K, 256);
     L.resid = o; o = align_up(o + (size_t)B * 8, 256);
+    L.nseg = (V + kSegElems - 1) / kSegElems;   // (streaming clusters: the second pass's sums per segment)
+    L.seg = o; o = align_up(o + (size_t)B * L.nseg * 8, 256);
     L.total = o;
     return L;
 }
@@ -564,43 +587,68 @@ int pick_counters(void* caller_ws, int dev, void* stream_, int kind, size_t coun
     return EARS_OK;
 }
 
-// The resident plan for this shape, if its rows fit a cluster and the device can hold one.
+// The cluster plan for this shape (rows resident in shared memory, or streamed by the clusters), if
+// one of the two is the kernel to take.
 int choose_resident(int dtype, int B, int K, int V, bool ordered, DeviceInfo* di, const PlanOverride& ov, RPlan* rp,
                     int* max_clusters) {
     *rp = RPlan();
     *max_clusters = 0;
     if (ov.path == 1 || ov.path == 3 || ov.parts1 != 0) return EARS_OK;
     const int esize = dtype_size(dtype);
-    if (ov.path == 4) *rp = make_splan(B, K, V, esize, di->sms, di->cluster16 ? kRMaxCluster : 8, ov.cluster, ordered);
-    else *rp = make_rplan(B, K, V, esize, di->sms, di->cluster16 ? kRMaxCluster : 8, ov.cluster);
-    if (ov.path == 0 && ordered && B >= 4 * di->sms) {
-        // Asked to leave out what follows a first rejection, and enough sequences to give every SM
-        // four clusters of its own (fewer leave the last round half empty): clusters that stream walk one sequence each and read nothing after
-        // its first rejection, where the other streaming kernels read every row and discard.  (Rows
-        // short enough to stay in shared memory keep the resident kernel, which does the same.)
-        const long long items = (long long)B * (K + 1);
-        const bool resident_takes_it = rp->ok && items <= (!rp->roomy ? 64 : (rp->C >= 8 ? 256 : 3072));
-        if (!resident_takes_it) {
-            const RPlan sp = make_splan(B, K, V, esize, di->sms, di->cluster16 ? kRMaxCluster : 8, ov.cluster, true);
-            if (sp.ok) *rp = sp;
+    const int cmax = di->cluster16 ? kRMaxCluster : 8;
+    const long long items = (long long)B * (K + 1);
+    const long long slots = (long long)kCCtasPerSm * di->sms;
+    auto clusters_of = [&](const RPlan& plan, int* out) {
+        return by_dtype(dtype, [&](auto* e) { return resident_clusters<std::remove_pointer_t<decltype(e)>>(di, plan, dtype, out); });
+    };
+    if (ov.path == 4) {
+        *rp = make_splan(B, K, V, esize, di->sms, cmax, ov.cluster, ordered);
+    } else {
+        *rp = make_rplan(B, K, V, esize, di->sms, cmax, ov.cluster);
+        if (rp->ok) {
+            const int rc = clusters_of(*rp, max_clusters);
+            if (rc) return rc;
+            if (*max_clusters < 1) rp->ok = false;
         }
     }
-    if (rp->ok && ov.path == 0 && !rp->streamed) {
-        // Holding rows in shared memory costs a few microseconds of latency per position that
-        // nothing else in that CTA can hide.  It wins when rows are short (a cluster of at most
-        // four CTAs holds a pair) and when there are few positions, where the streaming kernel's
-        // second pass and its queues dominate; long rows in large batches stream faster.
-        // Measured on B200 (B, K, V, dtype: us resident / best streaming kernel): 8,5,32000,bf16: 19 / 43;
-        // 512,5,32000,bf16: 148 / 150; 4096,5,32000,bf16: 1009 / 910; 32,7,128256,bf16: 72 / 75;
-        // 64,7,128256,bf16: 123 / 102; 128,4,152064,bf16: 195 / 120.
-        const long long items = (long long)B * (K + 1);
-        const long long limit = !rp->roomy ? 64 : (rp->C >= 8 ? 256 : 3072);
-        if (items > limit) rp->ok = false;
+    if (ov.path == 0) {
+        // Holding rows in shared memory costs a cluster about 6.5 us per position when it starts fresh and
+        // 13 us in steady state, which nothing else in its CTAs can hide.  It wins when rows are short (a
+        // cluster of at most four CTAs holds a pair: many clusters fit the device) and, with larger
+        // clusters, while the positions take the resident clusters no more than two to three rounds.
+        // Measured on B200 (B, K, V, dtype: us resident / cluster-streamed / best of ring and direct):
+        // 8,5,32000,bf16: 19 / 25 / 38;  512,5,32000,bf16: 155 / 166 / 153;  4096,5,32000,bf16: 1048 / 1024 / 832;
+        // 8,7,128256,bf16: 41 / 45 / 53;  16,7,128256,bf16: 49 / 49 / 61;  24,7,128256,bf16: 66 / 51 / 70;
+        // 32,7,128256,bf16: 77 / 60 / 75;  8,4,152064,bf16: 37 / 45 / 50;  16,4,152064,bf16: 55 / 48 / 59.
+        bool resident = rp->ok;
+        if (resident) {
+            const long long limit = !rp->roomy ? 64 : (rp->C >= 8 ? std::min<long long>(256, 8LL * *max_clusters / 3) : 3072);
+            resident = items <= limit;
+        }
+        if (!resident) {
+            // Clusters that stream their slices.  Their sweep is the fastest there is on 2-byte logits, and
+            // a batch that gives the device's CTA slots only a few rounds of positions has the shortest tail
+            // with them (the second pass of a first rejection is shared out piece by piece among all CTAs);
+            // the streaming kernels' finer units win in larger batches, the ring kernel on long 4-byte rows
+            // once the positions outnumber what two CTAs per SM take in one round.  Measured on B200 (B, K, V, dtype: us cluster-streamed /
+            // best of ring and direct): 64,7,128256,bf16: 96 / 105;  128,..: 143 / 143;  160,..: 160 / 168;
+            // 256,..: 231 / 229;  512,..: 430 / 399;  32,4,152064,bf16: 55 / 68;  64,..: 72 / 94;  128,..: 113 / 125;
+            // 256,..: 169 / 186;  320,..: 209 / 220;  384,..: 239 / 246;  512,..: 306 / 309;  1024,..: 559 / 552;
+            // 8,3,256000,fp32: 35 / 57;  32,..: 72 / 90;  64,..: 119 / 129;  96,..: 221 / 161;  128,..: 213 / 192.
+            // With the flag that leaves out what follows a first rejection they also skip the reads, which
+            // pays from four sequences per SM on.
+            // (With the flag these clusters always walk sequences in order, a chain of up to K+1 positions
+            // that a small batch cannot hide: below that size a flagged call goes to the streaming kernels.)
+            const bool few = !ordered && (esize == 2 ? 2 * items <= 9 * slots : items <= 2LL * di->sms);
+            const bool skip_reads = ordered && B >= 4 * di->sms;
+            RPlan sp;
+            if (few || skip_reads) sp = make_splan(B, K, V, esize, di->sms, cmax, ov.cluster, ordered);
+            *rp = sp;   // (not ok: a streaming kernel takes the call)
+            *max_clusters = 0;
+        }
     }
-    if (rp->ok) {
-        const int rc = by_dtype(dtype, [&](auto* e) {
-            return resident_clusters<std::remove_pointer_t<decltype(e)>>(di, *rp, dtype, max_clusters);
-        });
+    if (rp->ok && *max_clusters == 0) {
+        const int rc = clusters_of(*rp, max_clusters);
         if (rc) return rc;
         if (*max_clusters < 1) rp->ok = false;
     }
@@ -682,7 +730,7 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
     rc = choose_resident(dtype, B, K, V, stop_first != 0, di, ov, &rp, &max_clusters);
     if (rc) return rc;
     if (rp.ok) {
-        const RLayout L = make_rlayout(B, K);
+        const RLayout L = make_rlayout(B, K, V);
         if (workspace && workspace_bytes < L.total) return EARS_ERR_WORKSPACE;
         char *w = nullptr, *cw = nullptr;
         RParams p;
@@ -708,6 +756,12 @@ int verify_impl(int dtype, const void* t, const void* d, const int32_t* x, int B
         p.cand_mass = (double*)(w + L.cand_mass);
         p.rowstat = (float4*)(w + L.rowstat);
         p.seqmask = (unsigned long long*)(cw + L.seqmask);
+        p.ready = (unsigned long long*)(cw + L.ready);
+        p.ticket2 = (int*)(cw + L.ticket2);
+        p.segsums = (double*)(w + L.seg);
+        p.nseg = L.nseg;
+        p.job_elems = rp.job_elems;
+        p.parts2 = rp.parts2;
         p.C = rp.C; p.slice = rp.slice; p.buf_bytes = rp.buf_bytes;
         p.use_tma = aligned && ov.loader != 2;
         p.n_clusters = 0;
@@ -786,7 +840,7 @@ size_t workspace_bound(int B, int K, int V) {
             const size_t tot = make_layout(B, K, V, pl.parts1).total;
             if (tot > best) best = tot;
         }
-    const size_t res = make_rlayout(B, K).total;
+    const size_t res = make_rlayout(B, K, V).total;
     if (res > best) best = res;
     for (int esize = 2; esize <= 4; esize += 2)
         for (int s = 0; s < 2; ++s) {
@@ -1210,9 +1264,12 @@ int ears_describe_plan(int dtype, int B, int K, int V, char* out, size_t out_byt
             return rp.streamed ? (int)cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ears_cstream_kernel<El, false>, kCThreads, rp.smem)
                                : (int)cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ears_resident_kernel<El, false>, kRThreads, rp.smem);
         });
-        snprintf(out, out_bytes, rp.streamed ? "cluster-streamed: cluster=%d slice_elems=%d smem_bytes=%zu ctas_per_sm=%d clusters_resident=%d clusters_launched=%lld" :
-                 "resident: cluster=%d slice_elems=%d smem_bytes=%zu ctas_per_sm=%d clusters_resident=%d clusters_launched=%lld",
-                 rp.C, rp.slice, rp.smem, per_sm, max_clusters, items < max_clusters ? items : (long long)max_clusters);
+        if (rp.streamed)
+            snprintf(out, out_bytes, "cluster-streamed: cluster=%d slice_elems=%d smem_bytes=%zu ctas_per_sm=%d clusters_resident=%d clusters_launched=%lld second_pass_pieces=%d",
+                     rp.C, rp.slice, rp.smem, per_sm, max_clusters, items < max_clusters ? items : (long long)max_clusters, rp.parts2);
+        else
+            snprintf(out, out_bytes, "resident: cluster=%d slice_elems=%d smem_bytes=%zu ctas_per_sm=%d clusters_resident=%d clusters_launched=%lld",
+                     rp.C, rp.slice, rp.smem, per_sm, max_clusters, items < max_clusters ? items : (long long)max_clusters);
     } else {
         const bool direct = use_direct(ov, esize, V, (long long)B * (K + 1));
         const Plan pl = make_plan(B, K, V, esize, true, di->sms, ov, direct);

@@ -6,28 +6,34 @@
 //
 //   1. softmax statistics (max, sum exp2) of the slices [Sec. 3.1]; for the extra row the sums of
 //      2 KB segments are kept in shared memory as well, so that a bonus token needs no second read;
-//   2. the partial results, the cluster's next queue entry and any pending second-pass job travel
-//      through distributed shared memory (remote stores plus a remote mbarrier arrive per peer);
+//   2. the partial results and the cluster's next queue entry travel through distributed shared
+//      memory (remote stores plus a remote mbarrier arrive per peer);
 //   3. every CTA takes the decision of Sec. 3.2 (guards of Sec. 3.3 item 2) from identical numbers;
 //   4. the extra row draws its bonus token at once from the segment sums of step 1;
 //   5. one CTA reports the item in a per-sequence word of decided / accepted positions.  The report
-//      that settles the sequence's first rejection [Sec. 3.1] (every earlier position accepted) leaves
-//      a job: the two rows of that one position are read a second time -- by this cluster, in its
-//      next round, while they are still in L2 -- for the masses max(0, P_t - P_d) and the
-//      inverse-CDF pick.  Whoever reports last (an item or the job) writes the sequence's outputs.
+//      that settles the sequence's first rejection [Sec. 3.1] (every earlier position accepted)
+//      publishes a job: the two rows of that one position are read a second time, for the masses
+//      max(0, P_t - P_d) and the inverse-CDF pick.  A job is cut into pieces of 16-32 KB per row
+//      that the CTAs of the whole launch serve, at most one per round beside their own items and,
+//      once their cluster has run out of items, for as long as any sequence is unfinished (one CTA
+//      alone is bound by its special-function unit to some 13-19 GB/s on such rows, so a job left
+//      to one cluster took 30-40 us).  Whoever reports last (an item or the job) writes the
+//      sequence's outputs.
 //
 // So every logit crosses HBM once for the statistics, and per sequence at most one pair of rows is
 // read again (usually from L2).  A rejected position that is not the sequence's first costs nothing.
-// There is no global queue of second-pass work, no publication and no hand-over between clusters; a
-// cluster never waits for another cluster.  Without a shared-memory footprint several clusters share
-// an SM and hide each other's exchanges.  What a thread's own loads can keep in flight (eight 16-byte
-// loads, 32 KB per CTA) bounds a CTA to some 20 GB/s; whenever few CTAs are at work (a batch that
-// does not fill the machine, a second-pass job, the end of a launch) that bound is the speed of the
-// launch.  Rows of 4-byte logits that are 16-byte aligned therefore pass, for their statistics,
-// through a small ring of shared-memory stages filled by bulk asynchronous copies (64 KB in flight
-// per CTA, no registers held) and read by all threads of the CTA.  Ordered mode (EARS_FLAG_STOP_AT_FIRST_REJECT): the queue
-// holds sequences, a cluster walks one position by position and stops at its first rejection, whose
-// masses it computes at once; rows after it are never read.
+// A cluster never waits for another cluster while it has items; the only cross-cluster wait is the
+// one at the end (CTAs stay to serve pieces until every sequence is finished), which cannot deadlock
+// (whoever finishes a sequence waits for nobody) and is time-limited.  Without a shared-memory
+// footprint several clusters share an SM and hide each other's exchanges.  What a thread's own
+// loads can keep in flight (eight 16-byte loads, 32 KB per CTA) bounds a CTA to some 20 GB/s;
+// whenever few CTAs are at work (a batch that does not fill the machine, the end of a launch) that
+// bound is the speed of the launch.  Rows of 4-byte logits that are 16-byte aligned therefore pass,
+// for their statistics, through a small ring of shared-memory stages filled by bulk asynchronous
+// copies (64 KB in flight per CTA, no registers held) and read by all threads of the CTA.
+// Ordered mode (EARS_FLAG_STOP_AT_FIRST_REJECT): the queue holds sequences, a cluster walks one
+// position by position and stops at its first rejection, whose masses it takes at once (each CTA
+// over its slice, without the queue); rows after it are never read.
 #pragma once
 #include "ears_common.cuh"
 #include "ears_math.cuh"
@@ -58,18 +64,15 @@ struct CSmem {
     float xw[2][kRMaxCluster * kCWarps];  // sum e t of the target slice of every warp of every peer (entropy kernels)
     double xmass[2][kRMaxCluster];        // mass totals of every peer
     int xnext[2];                         // next queue entry of the cluster (written by rank 0)
-    int2 xjob[2][kRMaxCluster];           // second-pass job each peer announces: (sequence, position) or (-1, 0)
-    int my_job_b, my_job_n;               // job this CTA will announce with the next exchange
+    int job_b, job_n, job_piece;          // second-pass piece this CTA serves next (job_b < 0: none)
+    int my_ticket;                        // ticket of the shared queue this CTA holds (-1: none)
+    int drain_state;                      // end of the launch: 0 go on, 1 every sequence is finished, -1 give up
     float2 rs_t, rs_d;                    // (max, Z) of the item's rows
     int dec;                              // 1 accept / row usable, 0 reject, -1 invalid
     int pick_rank;                        // CTA that holds u*S (-1: no mass anywhere)
     double pick_tin, pick_S;
     int abort_flag;
 };
-
-__device__ __forceinline__ void peer_store(uint32_t addr, int2 v) {
-    asm volatile("st.shared::cluster.v2.s32 [%0], {%1, %2};" ::"r"(addr), "r"(v.x), "r"(v.y) : "memory");
-}
 
 // ---- the copy ring ----------------------------------------------------------------------
 // All threads of the CTA sweep entries [e0, e0 + n) of one row (r1 = nullptr: 16 KB per stage) or of
@@ -221,6 +224,26 @@ __device__ __forceinline__ int settled_first_rejection(unsigned long long m, int
     return (decided & below) == below ? n : -1;
 }
 
+// The word of a sequence: bit k of the low half = position k (K = the extra row) has reported, bit k of
+// the high half = it was not rejected; the top bit = the second-pass job has reported.  The sequence is
+// complete with the report that makes "all K+1 positions in, and the job too if a position was
+// rejected" true; reports only add bits, so exactly one report sees it (none follows it).
+constexpr unsigned long long kJobReported = 1ull << 63;
+__device__ __forceinline__ bool sequence_complete(unsigned long long m, int K) {
+    const uint32_t decided = (uint32_t)m, accepted = (uint32_t)(m >> 32);
+    const uint32_t items = (2u << K) - 1u;   // K <= 30
+    if ((decided & items) != items) return false;
+    const bool rejected = (decided & ~accepted & ((1u << K) - 1u)) != 0;
+    return !rejected || (m & kJobReported) != 0;
+}
+// Adds bits to that word with release + acquire semantics at device scope in the atomic itself: the
+// reporter's stores are visible to whoever sees the bits, and earlier reporters' stores to the reporter.
+__device__ __forceinline__ unsigned long long seqmask_or(unsigned long long* addr, unsigned long long bits) {
+    unsigned long long old;
+    asm volatile("atom.or.acq_rel.gpu.b64 %0, [%1], %2;" : "=l"(old) : "l"(addr), "l"(bits) : "memory");
+    return old;
+}
+
 // Called by one warp once everything of sequence b is in: first rejection [Sec. 3.1], the accepted
 // prefix and the token drawn at that position (or the bonus token).  With job_pending the slot of a
 // rejected position is left to the second-pass job that is yet to run (K > 30 only).
@@ -264,13 +287,159 @@ __device__ __forceinline__ int finish_streamed_sequence(const RParams& p, int b,
     return n;
 }
 
+// ---- second-pass jobs, shared by all CTAs of the launch --------------------------------
+// A job = (sequence b, its first rejected position n); its rows' statistics are in p.rowstat before
+// it is published.  Published jobs form a queue (p.ready, filled in the order of p.heads[3]); a job
+// has p.parts2 pieces of p.job_elems entries.  Pieces are handed out by one counter for the whole
+// queue (p.heads[4]): ticket i stands for piece i % parts2 of the job in slot i / parts2, whether or
+// not that job has been published yet.  A CTA with nothing else to do takes a ticket and waits for
+// its slot: when a job appears, the parts2 CTAs that hold its tickets serve it at once, with no
+// contention and one atomic per piece.  A CTA that still has items takes a ticket only while the
+// counter is behind the publications, i.e. when a piece is there to be served right away.
+// p.ticket2[b] counts the pieces of b's job that are done; the CTA that completes the last one
+// draws the token.
+
+// One thread publishes a job (its rowstat entry and whatever else a server reads were written
+// before by this thread, or are ordered before by a fence of the caller).
+__device__ __forceinline__ void publish_job(const RParams& p, int b, int n) {
+    __threadfence();
+    const int slot = atomicAdd(&p.heads[3], 1);
+    *reinterpret_cast<volatile unsigned long long*>(&p.ready[slot]) = ((unsigned long long)(b + 1) << 32) | (unsigned)n;
+}
+
+// A sequence is finished (its outputs are complete): lets the CTAs that stay to serve pieces leave.
+__device__ __forceinline__ void count_finished(const RParams& p) {
+    __threadfence();
+    atomicAdd(&p.heads[1], 1);
+}
+
+// What lane 0 of warp 0 reads of the queue at the start of a round, so that it costs no wait later:
+// jobs published, tickets given out, and the entry of the slot of the ticket this CTA holds.
+struct JobPoll { int published, given; unsigned long long e; };
+
+__device__ __forceinline__ unsigned long long ticket_slot_entry(const RParams& p, int ticket) {
+    const int slot = ticket / p.parts2;
+    return slot < p.B ? *reinterpret_cast<const volatile unsigned long long*>(&p.ready[slot]) : 0ull;
+}
+
+__device__ __forceinline__ JobPoll poll_jobs(const RParams& p, const CSmem& sm) {
+    JobPoll q;
+    q.published = *reinterpret_cast<const volatile int*>(&p.heads[3]);
+    q.given = *reinterpret_cast<const volatile int*>(&p.heads[4]);
+    q.e = sm.my_ticket >= 0 ? ticket_slot_entry(p, sm.my_ticket) : 0ull;
+    return q;
+}
+
+// Thread 0 decides which second-pass piece the CTA serves next and leaves it in shared memory
+// (job_b < 0: none): the piece of the ticket it holds, once that piece's job is published.
+// turn < 0: the CTA has no items left, so it takes a ticket whatever the state of the queue.  Otherwise (turn = its round) it takes one only if the
+// polled counters say pieces are waiting, and only if it is among as many CTAs as there are such
+// pieces (a window of CTA indices that moves with the round): the CTAs of a launch poll at about
+// the same time and see the same counters, and if all of them took a ticket most would end up
+// holding one for a job that is yet to come, which then has to wait for a busy CTA.
+__device__ __forceinline__ void claim_job(const RParams& p, CSmem& sm, const JobPoll& q, int turn) {
+    const int P2 = p.parts2;
+    int jb = -1, jn = 0, piece = 0;
+    {
+        unsigned long long e = q.e;
+        const int waiting = q.published * P2 - q.given;
+        const bool idle = turn < 0;
+        if (sm.my_ticket < 0 && (idle || (int)((blockIdx.x + (unsigned)turn * 37u) % gridDim.x) < waiting)) {
+            sm.my_ticket = atomicAdd(&p.heads[4], 1);
+            e = ticket_slot_entry(p, sm.my_ticket);
+        }
+        if (sm.my_ticket >= 0 && e != 0) {
+            jb = (int)(e >> 32) - 1;
+            jn = (int)(unsigned)e;
+            piece = sm.my_ticket % P2;
+            sm.my_ticket = -1;
+        }
+    }
+    sm.job_b = jb; sm.job_n = jn; sm.job_piece = piece;
+}
+
+// The CTA that completed a job's last piece draws the token from the stored segment sums (one warp):
+// token = smallest j with u S < C_j over max(0, P_t - P_d) of position n [Sec. 3.1; speculative
+// sampling's residual draw], from P_t if rounding left the residual without mass.
+template <typename E>
+__device__ __forceinline__ int select_job_token(const RParams& p, int b, int n, int lane, double* mass_out) {
+    const int K = p.K, V = p.V;
+    const float cj = seq_c(p, b);
+    const E* trow = reinterpret_cast<const E*>(p.t) + (size_t)target_row(b, n, K) * V;
+    const E* drow = reinterpret_cast<const E*>(p.d) + (size_t)draft_row(b, n, K) * V;
+    const float4 rs = __ldcg(&p.rowstat[(size_t)b * (K + 1) + n]);
+    const RowNorm rn = make_rownorm(make_float2(rs.x, rs.y), make_float2(rs.z, rs.w));
+    const double u = uniform_final(p.seed, p.offset, (uint32_t)(p.b_first + b), (uint32_t)K);
+    const double* ss = p.segsums + (size_t)b * p.nseg;
+    double S = 0.0, before = 0.0;
+    const int seg = pick_block([ss](int g) { return __ldcg(ss + g); }, p.nseg, u, lane, &S, &before);
+    int tok;
+    double S_used = S;
+    if (seg < 0 || !(S * rn.izt >= kTinyMass)) tok = warp_sample_pt_slow<E>(trow, V, rn, cj, u, lane, &S_used);
+    else tok = pick_in_range<E>(trow, drow, true, rn, cj, seg * kSegElems, kSegElems, u * S - before, V, lane);
+    *mass_out = S_used * rn.izt;
+    return tok;
+}
+
+// All threads of the CTA: the piece that thread 0 left in shared memory (claim_job, then a block-wide
+// barrier).  -> false if there was none.
+template <typename E>
+__device__ __forceinline__ bool serve_claimed_piece(const RParams& p, CSmem& sm, bool vec, bool early) {
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int jb = sm.job_b, jn = sm.job_n, piece = sm.job_piece;
+    if (jb < 0) return false;
+    const int K = p.K, V = p.V;
+    __threadfence();   // the publication was seen: what preceded it (the rows' statistics) is visible
+    const float cj = seq_c(p, jb);
+    const E* jt = reinterpret_cast<const E*>(p.t) + (size_t)target_row(jb, jn, K) * V;
+    const E* jd = reinterpret_cast<const E*>(p.d) + (size_t)draft_row(jb, jn, K) * V;
+    const float4 rs = __ldcg(&p.rowstat[(size_t)jb * (K + 1) + jn]);
+    const RowNorm rn = make_rownorm(make_float2(rs.x, rs.y), make_float2(rs.z, rs.w));
+    const int e0 = min(V, piece * p.job_elems), e1 = min(V, e0 + p.job_elems);
+    stream_job_piece<E, true>(jt, jd, e0, e1, vec, rn, cj, warp, lane, p.segsums + (size_t)jb * p.nseg);
+    __threadfence();   // the sums are visible before the piece counts as done
+    __syncthreads();
+    if (warp == 0) {
+        int last = 0;
+        if (lane == 0) last = ticket_add(&p.ticket2[jb]) == p.parts2 - 1 ? 1 : 0;
+        last = __shfl_sync(0xffffffffu, last, 0);
+        if (last) {
+            __threadfence();
+            double mass = 0.0;
+            const int jtoken = select_job_token<E>(p, jb, jn, lane, &mass);
+            if (early) {
+                // the job reports like an item; if it is the last of the sequence to do so it finishes it
+                int fin = 0;
+                if (lane == 0) {
+                    const size_t s = (size_t)jb * (K + 1) + jn;
+                    p.cand[s] = jtoken;
+                    p.cand_mass[s] = mass;
+                    fin = sequence_complete(seqmask_or(p.seqmask + jb, kJobReported) | kJobReported, K) ? 1 : 0;
+                }
+                fin = __shfl_sync(0xffffffffu, fin, 0);
+                if (fin) {
+                    __threadfence();
+                    finish_streamed_sequence(p, jb, lane, false);
+                    if (lane == 0) count_finished(p);
+                }
+            } else if (lane == 0) {
+                // the rest of the sequence's outputs were written by whoever published the job
+                p.out_tok[(size_t)jb * (K + 1) + jn] = jtoken;
+                p.resid[jb] = mass;
+                count_finished(p);
+            }
+            if (lane == 0) trace_mark(7, jtoken);
+        }
+    }
+    return true;
+}
+
 template <typename E, bool ENT>
 __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(const RParams p) {
     extern __shared__ unsigned char smem_raw[];
     CSmem& sm = *reinterpret_cast<CSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     unsigned char* area = reinterpret_cast<unsigned char*>(&sm) + ((sizeof(CSmem) + 127) & ~size_t(127));
-    double* const segsum = reinterpret_cast<double*>(area);     // a job's sums per kSegElems entries
-    BonusSeg* const bseg = reinterpret_cast<BonusSeg*>(area);   // the extra row's sums per 2 KB (never in use together)
+    BonusSeg* const bseg = reinterpret_cast<BonusSeg*>(area);   // the extra row's sums per 2 KB
     unsigned char* const ring = area + p.buf_bytes;             // the copy ring (behind the sums; 128-byte aligned)
     uint32_t ring_q = 0;                                        // stage fills so far
     constexpr int BSEG = kBonusSegBytes / (int)sizeof(E);       // entries per bonus segment
@@ -292,8 +461,9 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
         for (int i = 0; i < 2; ++i) { mbar_init(&sm.xbar[i], (unsigned)(C * kCWarps)); mbar_init(&sm.mbar2[i], (unsigned)C); }
         for (int i = 0; i < kCStages; ++i) mbar_init(&sm.full[i], 1u);
         sm.abort_flag = 0;
-        sm.my_job_b = -1;
-        sm.my_job_n = 0;
+        sm.job_b = -1;
+        sm.my_ticket = -1;
+        sm.drain_state = 0;
         mbar_init_fence();
     }
     __syncthreads();
@@ -340,21 +510,23 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
     // barriers of every CTA are initialised before any peer arrives on them
     cluster_sync_all();
 
-    for (;;) {
-        const bool work = have;          // the same in every CTA of the cluster
+    while (have) {
         const bool pair = j < K;
-        const float cb = work ? seq_c(p, b) : 1.0f;   // log2(e) / temperature of this sequence
-        const E* const trow = tbase + (size_t)target_row(work ? b : 0, work ? j : 0, K) * V;
-        const E* const drow = dbase + (size_t)draft_row(work ? b : 0, (work && pair) ? j : 0, K) * V;
+        const float cb = seq_c(p, b);    // log2(e) / temperature of this sequence
+        const E* const trow = tbase + (size_t)target_row(b, j, K) * V;
+        const E* const drow = dbase + (size_t)draft_row(b, pair ? j : 0, K) * V;
+        // a look at the queue of second-pass jobs, taken now so that it costs no wait after the sweep
+        JobPoll polled{0, 0, 0ull};
+        if (tid == 0) polled = poll_jobs(p, sm);
         // ---- 1. statistics of this CTA's slices
-        if (tid == 0) trace_mark(1, work ? b * (K + 1) + j : -1);
+        if (tid == 0) trace_mark(1, b * (K + 1) + j);
         float2 pt2 = make_float2(-INFINITY, 0.f), pd2 = make_float2(-INFINITY, 0.f);
         float wv = 0.f;   // ENT: the thread's sum e t over the target slice
         // 4-byte logits take the copy ring (measured on B200, 64 sequences of 1 MB rows: 121 us against 184);
         // 2-byte logits do twice the arithmetic per staged byte and lose to their own loads there
         // (32 sequences of 256 KB rows: 55 us against 47), so they keep the register path
         const bool staged = vec && sizeof(E) == 4;
-        if (work && staged && pair) {
+        if (staged && pair) {
             // through the copy ring: 8 KB of each row per stage, two vectors of each per thread
             constexpr int N = Words<E>::N;
             RowAccT<ENT> at;
@@ -377,7 +549,7 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
             if (!swept) { failed = true; break; }
             pt2 = acc_close(at, cb, &wv);
             pd2 = acc_close(ad, cb);
-        } else if (work && staged) {
+        } else if (staged) {
             // the extra row through the copy ring: 16 KB per stage, warp w takes its 2 KB block w, keeps a
             // warp-uniform running maximum and leaves (sum, reference) of the block behind
             constexpr int N = Words<E>::N, PN = N / 2, VPL = BSEG / N / 32;
@@ -421,7 +593,7 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
                 });
             if (!swept) { failed = true; break; }
             pt2 = acc_close(a, cb);
-        } else if (work) {
+        } else {
             if (pair) {
                 pt2 = stream_piece<E, kCThreads, ENT>(trow, e0, e0 + n, vec, cb, tid, &wv);
                 pd2 = stream_piece<E, kCThreads>(drow, e0, e0 + n, vec, cb, tid);
@@ -448,37 +620,27 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
                 if (ENT) Wt += __shfl_xor_sync(0xffffffffu, Wt, off);
             }
             // ---- 2. every warp hands its partial result to every CTA of the cluster (itself included);
-            //         warp 0 adds the next queue entry (rank 0) and the job this CTA has to announce
+            //         warp 0 of rank 0 adds the cluster's next queue entry
             const int nx = __shfl_sync(0xffffffffu, next_item, 0);
             if (lane < C) {
                 peer_store(map_to_peer(smem_u32(&sm.xstat[par][rank * kCWarps + warp]), (uint32_t)lane),
                            make_float4(Mt, St, Md, Sd));
                 if (ENT) peer_store(map_to_peer(smem_u32(&sm.xw[par][rank * kCWarps + warp]), (uint32_t)lane), Wt);
-                if (warp == 0) {
-                    if (rank == 0) peer_store(map_to_peer(smem_u32(&sm.xnext[par]), (uint32_t)lane), nx);
-                    peer_store(map_to_peer(smem_u32(&sm.xjob[par][rank]), (uint32_t)lane), make_int2(sm.my_job_b, sm.my_job_n));
-                }
+                if (warp == 0 && rank == 0) peer_store(map_to_peer(smem_u32(&sm.xnext[par]), (uint32_t)lane), nx);
                 peer_arrive(map_to_peer(smem_u32(&sm.xbar[par]), (uint32_t)lane));
             }
         }
         bool ok = mbar_wait_cluster(&sm.xbar[par], (uint32_t)(round >> 1) & 1u, &sm.abort_flag);
         ++round;
         if (tid == 0) trace_mark(3, 0);
-        if (__syncthreads_or(ok ? 0 : 1)) { failed = true; break; }   // (also: every warp has sent before my_job is cleared)
-        if (tid == 0) sm.my_job_b = -1;
-        // the job announced in this round, if any (at most one CTA reported an item last round)
-        int job_b = -1, job_n = 0;
-        for (int i = 0; i < C; ++i) {
-            const int2 q = sm.xjob[par][i];
-            if (q.x >= 0) { job_b = q.x; job_n = q.y; }
-        }
+        if (__syncthreads_or(ok ? 0 : 1)) { failed = true; break; }
         // the cluster's next queue entry, known to every CTA now
         const long long nxt = sm.xnext[par];
-        const bool q_have = work && nxt < n_items;
+        const bool q_have = nxt < n_items;
         const int qb = q_have ? (ordered ? (int)nxt : (int)(nxt / (K + 1))) : 0;
         const int qj = (q_have && !ordered) ? (int)(nxt % (K + 1)) : 0;
         // ---- 3. the rows' (max, Z) and the decision
-        if (work && warp == 0) {
+        if (warp == 0) {
             float mt, zt, md, zd, wt;
             merge_exchanged<ENT>(sm.xstat[par], sm.xw[par], C * kCWarps, cb, lane, mt, zt, md, zd, wt);
             if (lane == 0) {
@@ -492,18 +654,18 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
             }
         }
         __syncthreads();
-        const int dec = work ? sm.dec : 1;
+        const int dec = sm.dec;
         if (tid == 0) {
             trace_mark(4, dec);
             // the next item's token, fetched now that the others are released: the loads land while this
             // item is reported (walking a sequence in order, an accepted position is followed by the next one)
-            if (work && ordered && pair && dec > 0) fetch_token(b, j + 1);
+            if (ordered && pair && dec > 0) fetch_token(b, j + 1);
             else if (q_have) fetch_token(qb, qj);
         }
         // ---- 4. the extra row draws its bonus token at once from the segment sums of step 1
-        int writer = work ? (b + j) % C : 0, token = -1;   // reports are spread over the CTAs of the cluster
+        int writer = (b + j) % C, token = -1;   // reports are spread over the CTAs of the cluster
         double mass = 0.0;
-        if (work && !pair && dec >= 0) {
+        if (!pair && dec >= 0) {
             const RowNorm rn = make_rownorm(sm.rs_t, sm.rs_d);
             const double mc = (double)rn.mt * (double)cb;   // exact: two fp32 factors
             const BonusSeg* bs = bseg;
@@ -516,12 +678,11 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
             if (sm.pick_rank >= 0) writer = sm.pick_rank;
             mass = sm.pick_S * rn.izt;
         }
-        // ---- 5. one CTA reports the item and counts it; the sequence's last item finishes the sequence
-        //         and, after a rejection, leaves the second-pass job for the cluster's next round
+        // ---- 5. one CTA reports the item and counts it; the sequence's last item finishes the sequence;
+        //         a first rejection is published as a second-pass job
         bool seq_goes_on = false;
-        if (work && ordered) {
+        if (ordered) {
             seq_goes_on = dec > 0 && pair;
-            if (dec == 0) { job_b = b; job_n = j; }        // the first rejection of a sequence walked in order: its masses now
             // every position a cluster reaches while walking a sequence in order is one the sequence decided
             if (rank == 0 && tid == 0 && pair && dec >= 0)
                 atomicAdd(&p.heads[dec == 1 ? kCountDirect : (dec == 2 ? kCountPardon : kCountReject)], 1);
@@ -533,6 +694,7 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
                         p.out_len[b] = -1;
                         atomicOr(&p.heads[2], kDevInvalidInput);
                         atomicAdd(&p.heads[kCountInvalid], 1);
+                        count_finished(p);
                     }
                 } else {
                     for (int q = lane; q <= K; q += 32) {
@@ -542,11 +704,17 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
                     }
                     if (lane == 0) {
                         p.out_len[b] = j;
-                        if (!pair) p.resid[b] = mass;
+                        if (!pair) {
+                            p.resid[b] = mass;
+                            count_finished(p);
+                        } else {
+                            // the first rejection of a sequence walked in order: whoever draws its token below reads this
+                            p.rowstat[(size_t)b * (K + 1) + j] = make_float4(sm.rs_t.x, sm.rs_t.y, sm.rs_d.x, sm.rs_d.y);
+                        }
                     }
                 }
             }
-        } else if (work && rank == writer && warp == 0) {
+        } else if (rank == writer && warp == 0) {
             int last = 0;
             if (lane == 0) {
                 const size_t s = (size_t)b * (K + 1) + j;
@@ -556,19 +724,15 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
                 p.rowstat[s] = make_float4(sm.rs_t.x, sm.rs_t.y, sm.rs_d.x, sm.rs_d.y);
                 if (early) {
                     // decided, and accepted unless rejected (an unusable position counts as accepted here: it
-                    // must not ask for masses; the flag array remembers it and invalidates the sequence)
+                    // must not ask for masses; the flag array remembers it and invalidates the sequence).
+                    // One atomic on the sequence's word does it all: it releases the stores above, tells
+                    // whether this report settles the first rejection, and whether it is the sequence's last.
                     const unsigned long long bit = 1ull << j;
                     const unsigned long long add = bit | (dec != 0 ? bit << 32 : 0ull);
-                    __threadfence();   // the row statistics above are visible before the position counts as decided
-                    const unsigned long long old = atomicOr(p.seqmask + b, add);
+                    const unsigned long long old = seqmask_or(p.seqmask + b, add);
                     const int n_now = settled_first_rejection(old | add, K);
-                    if (n_now >= 0 && settled_first_rejection(old, K) < 0) { sm.my_job_b = b; sm.my_job_n = n_now; }   // settled by this report
-                    const int done = ticket_add(&p.ticket[b]) + 1;
-                    // K+1 items report, and the job if a position was rejected; the last of them finishes
-                    const unsigned long long all = *reinterpret_cast<volatile unsigned long long*>(p.seqmask + b);
-                    const bool every = (uint32_t)all == (K + 1 >= 32 ? 0xffffffffu : (1u << (K + 1)) - 1u);
-                    const bool none_rejected = ((uint32_t)all & ~(uint32_t)(all >> 32) & ((1u << K) - 1u)) == 0;
-                    last = (done == K + 2 || (done == K + 1 && every && none_rejected)) ? 1 : 0;
+                    if (n_now >= 0 && settled_first_rejection(old, K) < 0) publish_job(p, b, n_now);   // settled by this report
+                    last = sequence_complete(old | add, K) ? 1 : 0;
                 } else {
                     last = ticket_add(&p.ticket[b]) == K ? 1 : 0;
                 }
@@ -577,73 +741,81 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
             if (last) {
                 __threadfence();
                 const int nfirst = finish_streamed_sequence(p, b, lane, !early);
-                if (!early && lane == 0 && nfirst >= 0 && nfirst < K) { sm.my_job_b = b; sm.my_job_n = nfirst; }
+                if (lane == 0) {
+                    if (!early && nfirst >= 0 && nfirst < K) publish_job(p, b, nfirst);   // the job fills slot nfirst
+                    else count_finished(p);
+                }
             }
         }
         if (tid == 0) trace_mark(5, token);
-        // ---- 6. the second-pass job of this round: the masses of one rejected position and its token
-        if (job_b >= 0) {
-            const float cj = seq_c(p, job_b);
-            const E* const jt = tbase + (size_t)target_row(job_b, job_n, K) * V;
-            const E* const jd = dbase + (size_t)draft_row(job_b, job_n, K) * V;
-            float4 rs;
-            if (ordered) rs = make_float4(sm.rs_t.x, sm.rs_t.y, sm.rs_d.x, sm.rs_d.y);
-            else rs = __ldcg(&p.rowstat[(size_t)job_b * (K + 1) + job_n]);   // stored before the ticket that made the job
-            const RowNorm rn = make_rownorm(make_float2(rs.x, rs.y), make_float2(rs.z, rs.w));
-            double* so = segsum - e0 / kSegElems;    // sums land at index (entry - e0) / kSegElems
-            const double* ss = segsum;
-            auto val = [ss](int g) { return ss[g]; };
-            int jtoken = -1;
-            bool resid = true;
-            __syncthreads();                         // the bonus sums of step 4 (same memory) are no longer needed
-            for (;;) {
-                if (resid) {
-                    stream_job_piece<E, true>(jt, jd, e0, e0 + n, vec, rn, cj, warp, lane, so);
-                } else {
-                    stream_job_piece<E, false>(jt, jt, e0, e0 + n, vec, rn, cj, warp, lane, so);
-                }
-                __syncthreads();
-                if (!cluster_pick<E>(sm, p, val, (n + kSegElems - 1) / kSegElems, kSegElems, job_b, resid, jt, jd, rn, cj, e0, n, rank,
-                                     C, mround, jtoken)) {
-                    failed = true;
-                    break;
-                }
-                // a rejection implies residual mass; if rounding erased it, draw from P_t instead
-                if (resid && !(sm.pick_S * rn.izt >= kTinyMass)) { resid = false; __syncthreads(); continue; }
-                break;
-            }
-            if (failed) break;
-            if (warp == 0 && (rank == sm.pick_rank || (sm.pick_rank < 0 && rank == 0))) {
-                if (early) {
-                    // the job reports like an item; if it is the last of the sequence to do so it finishes it
-                    int last = 0;
+        if (ordered && dec == 0) {
+            // The first rejection of a sequence walked in order: every CTA of the cluster knows it, so the
+            // cluster takes the masses of that position at once, each CTA over its own slice, without the
+            // queue; the CTA that is done last draws the token.
+            const RowNorm rn = make_rownorm(sm.rs_t, sm.rs_d);
+            stream_job_piece<E, true>(trow, drow, e0, e0 + n, vec, rn, cb, warp, lane, p.segsums + (size_t)b * p.nseg);
+            __threadfence();   // the sums (and the writer's rowstat entry) are visible before this CTA counts as done
+            __syncthreads();
+            if (warp == 0) {
+                int last = 0;
+                if (lane == 0) last = ticket_add(&p.ticket2[b]) == C - 1 ? 1 : 0;
+                last = __shfl_sync(0xffffffffu, last, 0);
+                if (last) {
+                    __threadfence();
+                    double jmass = 0.0;
+                    const int jtoken = select_job_token<E>(p, b, j, lane, &jmass);
                     if (lane == 0) {
-                        const size_t s = (size_t)job_b * (K + 1) + job_n;
-                        p.cand[s] = jtoken;
-                        p.cand_mass[s] = sm.pick_S * rn.izt;
-                        last = ticket_add(&p.ticket[job_b]) + 1 == K + 2 ? 1 : 0;
+                        p.out_tok[(size_t)b * (K + 1) + j] = jtoken;
+                        p.resid[b] = jmass;
+                        count_finished(p);
+                        trace_mark(7, jtoken);
                     }
-                    last = __shfl_sync(0xffffffffu, last, 0);
-                    if (last) {
-                        __threadfence();
-                        finish_streamed_sequence(p, job_b, lane, false);
-                    }
-                } else if (lane == 0) {
-                    p.out_tok[(size_t)job_b * (K + 1) + job_n] = jtoken;
-                    p.resid[job_b] = sm.pick_S * rn.izt;
                 }
             }
-            if (tid == 0) trace_mark(7, jtoken);
         }
-        __syncthreads();     // shared memory of this round (decision, sums) is free again
-        if (!work) break;    // that was the round after the last item: its job, if any, is done
+        // ---- 6. one piece of a published second-pass job, if the look at the start of the round found one waiting
+        if (tid == 0) claim_job(p, sm, polled, round);
+        __syncthreads();     // the claim is known; shared memory of this round (decision, sums) is free again
+        serve_claimed_piece<E>(p, sm, vec, early);
         // ---- on to the next item
         if (seq_goes_on) {
             take_item(b, j + 1);
         } else {
             have = q_have;
             if (have) take_item(qb, qj);
-            else j = 0;
+        }
+    }
+    // ---- the cluster has run out of items: its CTAs stay and serve second-pass pieces until every
+    //      sequence of the batch is finished (by whichever CTA).  A sequence is finished by CTAs that
+    //      wait for nobody, so this cannot deadlock; it is time-limited like every other wait.
+    if (!failed) {
+        unsigned long long wait_t0 = 0;
+        for (;;) {
+            if (tid == 0) {
+                const JobPoll q{0, 0, sm.my_ticket >= 0 ? ticket_slot_entry(p, sm.my_ticket) : 0ull};
+                claim_job(p, sm, q, -1);
+                int st = 0;
+                if (sm.job_b < 0) {
+                    if (*reinterpret_cast<volatile int*>(&p.heads[1]) >= p.B) {
+                        st = 1;
+                    } else if (*reinterpret_cast<volatile int*>(&p.heads[2]) & kDevTimeout) {
+                        st = -1;   // another CTA gave up: the count will never be reached
+                    } else {
+                        const unsigned long long now = global_timer_ns();
+                        if (wait_t0 == 0) wait_t0 = now;
+                        else if (now - wait_t0 > kIdleLimitNs) st = -1;
+                        __nanosleep(200);
+                    }
+                }
+                sm.drain_state = st;
+            }
+            __syncthreads();
+            const int st = sm.drain_state;
+            const bool served = serve_claimed_piece<E>(p, sm, vec, early);
+            __syncthreads();   // everyone has read the claim and the state before warp 0 writes them again
+            if (served) continue;
+            if (st > 0) break;
+            if (st < 0) { failed = true; break; }
         }
     }
     if (tid == 0) trace_mark(6, 0);

@@ -53,13 +53,18 @@ struct RParams {
     double* max_pt;
     uint8_t* cls;
     double* resid;
-    int* heads;           // [0] item queue, [2] status word
+    int* heads;           // [0] item queue, [1] finished sequences, [2] status word, [3] published jobs, [4] piece tickets given out ([1], [3], [4]: streaming clusters)
     int* ticket;          // [B] items of the sequence that are done
     signed char* flag;    // [B,K+1] 1 accepted directly / row usable, 2 accepted by pardon, 0 rejected, -1 invalid
     int32_t* cand;        // [B,K+1] token drawn at the position (rejected positions and slot K)
     double* cand_mass;    // [B,K+1] mass that token was drawn from
     float4* rowstat;      // [B,K+1] (max, Z) of the item's target and draft rows (streaming clusters only)
     unsigned long long* seqmask;  // [B] positions decided (low word) and accepted (high word), K <= 30 (streaming clusters only)
+    // second-pass jobs of the streaming clusters (a sequence's first rejected position), served by every CTA:
+    unsigned long long* ready;    // [B] published jobs in the order of heads[3]: (b + 1) << 32 | n
+    int* ticket2;                 // [B] pieces of the sequence's job that are done
+    double* segsums;              // [B, nseg] masses per kSegElems entries of the job's rows
+    int nseg, job_elems, parts2;  // segments per row; entries per piece; pieces per job
     int unc_entropy;      // 1: the tolerance is scaled by H(P_t) / ln V instead of 1 - max P_t [Sec. 5 item 1]
     double* entropy;      // [B,K] H(P_t) of every target row, or NULL; the entropy kernels (ENT) fill it
     int C;                // CTAs per cluster
