@@ -287,7 +287,10 @@ RPlan make_splan(int B, int K, int V, int esize, int sms, int max_cluster, int f
         // (32 KB for 4-byte entries: one sweep of a CTA's warps), so that the many CTAs waiting at the end
         // of a small batch finish a job in one short step.
         const int chunk_elems = kChunkBytes / esize;
-        best.job_elems = (esize == 4 ? 2 : 1) * chunk_elems;
+        // (twice that once the positions give every CTA four rounds or more: CTAs are busy then, and the
+        // round trips around a piece weigh more than the wait for a job's last piece)
+        const int job_chunks = (esize == 4 ? 2 : 1) * (items >= 4LL * kCCtasPerSm * sms ? 2 : 1);
+        best.job_elems = job_chunks * chunk_elems;
         best.parts2 = (V + best.job_elems - 1) / best.job_elems;
     }
     return best;
