@@ -286,7 +286,8 @@ def run_ours(args):
     step_bytes = logits_bytes + rs_formula
     k_avg = statistics.fmean(kernel_ms)
     plan = ears.describe_plan(w.dtype, w.B, K, V)
-    kernel_name = {"resident": "ears_resident_kernel", "direct": "ears_direct_kernel"}.get(plan.split(":")[0], "ears_verify_kernel")
+    kernel_name = {"resident": "ears_resident_kernel", "direct": "ears_direct_kernel",
+                   "cluster-streamed": "ears_cstream_kernel"}.get(plan.split(":")[0], "ears_verify_kernel")
     if kernel_name == "ears_resident_kernel":
         rs_again = 0     # the rows of a position stay in shared memory until its token is drawn
     peak, peak_kind = measured_peak()
