@@ -251,6 +251,38 @@ __device__ __forceinline__ unsigned long long seqmask_or(unsigned long long* add
 __device__ __forceinline__ int finish_streamed_sequence(const RParams& p, int b, int lane, bool job_pending) {
     const int K = p.K;
     const signed char* fl = p.flag + (size_t)b * (K + 1);
+    int32_t* ot = p.out_tok + (size_t)b * (K + 1);
+    if (K < 32) {
+        // one lane per position: everything the outputs need is asked for at once (this runs at the very
+        // end of a launch, where every dependent round trip shows)
+        int f = 1, xk = -1, ck = -1;
+        double cm = 0.0;
+        if (lane <= K) {
+            f = *reinterpret_cast<const volatile signed char*>(fl + lane);
+            ck = __ldcg(p.cand + (size_t)b * (K + 1) + lane);
+            cm = __ldcg(p.cand_mass + (size_t)b * (K + 1) + lane);
+            if (lane < K) xk = p.x[(size_t)b * K + lane];
+        }
+        const unsigned rej = __ballot_sync(0xffffffffu, lane < K && f == 0);
+        const bool bad = __any_sync(0xffffffffu, f < 0);
+        if (bad) {
+            if (lane <= K) ot[lane] = -1;
+            if (lane == 0) {
+                p.out_len[b] = -1;
+                atomicOr(&p.heads[2], kDevInvalidInput);
+                atomicAdd(&p.heads[kCountInvalid], 1);
+            }
+            return -1;
+        }
+        const int n = rej ? __ffs(rej) - 1 : K;
+        count_decisions(p.heads, min(n + 1, K), lane, [f](int) { return f; });
+        const bool mine = n == K || !job_pending;   // the slot n is filled here
+        if (lane < n) ot[lane] = xk;
+        else if (lane > n && lane <= K) ot[lane] = -1;
+        else if (lane == n && mine) { ot[lane] = ck; p.resid[b] = cm; }
+        if (lane == 0) p.out_len[b] = n;
+        return n;
+    }
     int first_reject = K;
     bool bad = false;
     for (int k0 = 0; k0 <= K; k0 += 32) {
@@ -262,7 +294,6 @@ __device__ __forceinline__ int finish_streamed_sequence(const RParams& p, int b,
         if (rej != 0 && first_reject == K) first_reject = k0 + __ffs(rej) - 1;
     }
     bad = __any_sync(0xffffffffu, bad);
-    int32_t* ot = p.out_tok + (size_t)b * (K + 1);
     if (bad) {
         for (int q = lane; q <= K; q += 32) ot[q] = -1;
         if (lane == 0) {
