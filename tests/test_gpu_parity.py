@@ -62,8 +62,8 @@ SHAPES = [
 
 
 # (path, cluster): 1 = streaming kernel with the shared-memory ring; 3 = streaming kernel reading straight from
-# global memory; 2 = resident kernel with 1..16 CTAs per cluster (0 = automatic); 4 = the cluster kernel in its
-# streamed form (nothing staged, slices read twice)
+# global memory; 2 = resident kernel with 1..16 CTAs per cluster (0 = automatic); 4 = the cluster-streamed kernel
+# (clusters stream their slices; the second pass of a first rejection is shared out among all CTAs)
 PATHS = [(1, 0), (3, 0), (2, 0), (2, 1), (2, 2), (2, 4), (2, 8), (2, 16), (4, 0), (4, 1), (4, 2), (4, 4), (4, 8), (4, 16)]
 
 
@@ -100,7 +100,7 @@ def test_parity_shapes(ears, forced_path, B, K, V, dtype, path, cluster):
 @pytest.mark.parametrize("idx", [1, 2, 3, 4])
 def test_parity_workloads(ears, forced_path, idx, path):
     """Workloads 1-4 at full size, in the automatic launch configuration (the resident kernel for
-    workloads 1-3, the streaming kernel for workload 4) and with the streaming kernel forced."""
+    workloads 1-2, the cluster-streamed kernel for workloads 3-4) and with the other kernels forced."""
     forced_path(path)
     w = synth.workload(idx)
     temps = w.temperatures or (w.temperature,)
@@ -118,6 +118,31 @@ def test_parity_workloads(ears, forced_path, idx, path):
     assert tally.max_rel_prob_err < 1e-5
     print(f"\n{w.name}: rows={tally.rows} explained={tally.explained} flagged_dec={tally.flagged_decisions} "
           f"flagged_tok={tally.flagged_tokens} max_rel={tally.max_rel_prob_err:.2e} mean_len={np.mean(lens):.2f}")
+
+
+@pytest.mark.parametrize("cluster", [0, 1, 2, 4])
+@pytest.mark.parametrize("B,K,V,dtype,beta", [(96, 7, 20000, "bf16", 0.0), (600, 3, 9000, "fp32", 0.0), (40, 31, 3000, "bf16", 0.05),
+                                              (130, 2, 70001, "fp16", 0.0)])
+def test_parity_shared_second_pass(ears, forced_path, B, K, V, dtype, beta, cluster):
+    """The cluster-streamed kernel with most sequences rejected somewhere and more positions than CTA
+    slots: many second-pass jobs in the queue at once, pieces served between items and by CTAs that have
+    run out of them, for every cluster size; K = 31 takes the path without the per-sequence word; the
+    device-side counters see every sequence exactly once."""
+    forced_path(4, cluster)
+    w, t, d, x = synth.tiny_inputs(B, K, V, dtype, seed=77, temperature=1.1)
+    tally, _, _, ora = run_both(ears, w, t, d, x, 1.1, beta, seed=5, offset=11)
+    assert_parity(tally, max_explained=2)
+    if beta == 0.0:
+        assert (ora.accept_len < K).sum() >= B // 4   # many second-pass jobs
+    got = ears.decision_counts()        # of run_both's last call (the one without the optional outputs)
+    want = oracle_class_counts(ora, K)
+    assert got["invalid"] == 0
+    # (a decision the oracle flags as a near-tie could be classed either way; a flipped decision also
+    # changes which later positions count)
+    if tally.flagged_decisions == 0:
+        assert got == want, (got, want)
+    else:
+        assert abs(sum(got.values()) - sum(want.values())) <= K * tally.flagged_decisions
 
 
 @pytest.mark.parametrize("path", [0, 1, 3, 4])
