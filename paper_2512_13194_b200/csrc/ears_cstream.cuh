@@ -653,7 +653,14 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
             // ---- 2. every warp hands its partial result to every CTA of the cluster (itself included);
             //         warp 0 of rank 0 adds the cluster's next queue entry
             const int nx = __shfl_sync(0xffffffffu, next_item, 0);
-            if (lane < C) {
+            if (C == 1) {
+                // a cluster of one: plain shared memory and the block-wide barrier below do
+                if (lane == 0) {
+                    sm.xstat[par][warp] = make_float4(Mt, St, Md, Sd);
+                    if (ENT) sm.xw[par][warp] = Wt;
+                    if (warp == 0) sm.xnext[par] = nx;
+                }
+            } else if (lane < C) {
                 peer_store(map_to_peer(smem_u32(&sm.xstat[par][rank * kCWarps + warp]), (uint32_t)lane),
                            make_float4(Mt, St, Md, Sd));
                 if (ENT) peer_store(map_to_peer(smem_u32(&sm.xw[par][rank * kCWarps + warp]), (uint32_t)lane), Wt);
@@ -661,7 +668,7 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
                 peer_arrive(map_to_peer(smem_u32(&sm.xbar[par]), (uint32_t)lane));
             }
         }
-        bool ok = mbar_wait_cluster(&sm.xbar[par], (uint32_t)(round >> 1) & 1u, &sm.abort_flag);
+        bool ok = C == 1 || mbar_wait_cluster(&sm.xbar[par], (uint32_t)(round >> 1) & 1u, &sm.abort_flag);
         ++round;
         if (tid == 0) trace_mark(3, 0);
         if (__syncthreads_or(ok ? 0 : 1)) { failed = true; break; }
