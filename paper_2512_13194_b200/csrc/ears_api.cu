@@ -635,14 +635,14 @@ int choose_resident(int dtype, int B, int K, int V, bool ordered, DeviceInfo* di
             // the streaming kernels' finer units win in larger batches, the ring kernel on long 4-byte rows
             // once the positions outnumber what two CTAs per SM take in one round.  Measured on B200 (B, K, V, dtype: us cluster-streamed /
             // best of ring and direct): 64,7,128256,bf16: 96 / 105;  128,..: 143 / 143;  160,..: 160 / 168;
-            // 256,..: 231 / 229;  512,..: 430 / 399;  32,4,152064,bf16: 55 / 68;  64,..: 72 / 94;  128,..: 113 / 125;
-            // 256,..: 169 / 186;  320,..: 209 / 220;  384,..: 239 / 246;  512,..: 306 / 309;  1024,..: 559 / 552;
+            // 256,..: 225 / 229;  512,..: 428 / 399;  32,4,152064,bf16: 55 / 68;  64,..: 72 / 94;  128,..: 113 / 125;
+            // 256,..: 164 / 186;  320,..: 209 / 220;  384,..: 239 / 246;  512,..: 295 / 309;  1024,..: 541 / 551 (643 / 621 at beta = 0);
             // 8,3,256000,fp32: 35 / 57;  32,..: 72 / 90;  64,..: 119 / 129;  96,..: 221 / 161;  128,..: 213 / 192.
             // With the flag that leaves out what follows a first rejection they also skip the reads, which
             // pays from four sequences per SM on.
             // (With the flag these clusters always walk sequences in order, a chain of up to K+1 positions
             // that a small batch cannot hide: below that size a flagged call goes to the streaming kernels.)
-            const bool few = !ordered && (esize == 2 ? 2 * items <= 9 * slots : items <= 2LL * di->sms);
+            const bool few = !ordered && (esize == 2 ? items <= 6 * slots : items <= 2LL * di->sms);
             const bool skip_reads = ordered && B >= 4 * di->sms;
             RPlan sp;
             if (few || skip_reads) sp = make_splan(B, K, V, esize, di->sms, cmax, ov.cluster, ordered);

@@ -53,6 +53,7 @@ constexpr int kCBonusPad = 8;             // stream_bonus_piece may clear up to 
 #define EARS_C_CTAS 3
 #endif
 constexpr int kCCtasPerSm = EARS_C_CTAS;
+constexpr int kCFetcher = 32;             // the thread that fetches the next item's token and logits (lane 0 of warp 1)
 constexpr int kCStages = 4;               // stages of the CTA's copy ring
 constexpr int kCStageBytes = 16384;       // per stage: 16 KB of one row, or 8 KB of each of two rows
 
@@ -66,6 +67,9 @@ struct CSmem {
     int xnext[2];                         // next queue entry of the cluster (written by rank 0)
     int job_b, job_n, job_piece;          // second-pass piece this CTA serves next (job_b < 0: none)
     int my_ticket;                        // ticket of the shared queue this CTA holds (-1: none)
+    float tk_lt, tk_ld;                   // the item's token logits and uniform, fetched a round ahead by thread kCFetcher
+    double tk_U;
+    int tk_ok;
     int drain_state;                      // end of the launch: 0 go on, 1 every sequence is finished, -1 give up
     float2 rs_t, rs_d;                    // (max, Z) of the item's rows
     int dec;                              // 1 accept / row usable, 0 reject, -1 invalid
@@ -504,13 +508,13 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
     int round = 0, mround = 0;                             // exchanges so far (the same in every CTA of the cluster)
     bool failed = false;
     int b = 0, j = 0;
-    // what thread 0 fetches ahead for an item's decision: the token's two logits and the uniform
+    // what thread kCFetcher fetches ahead for an item's decision: the token's two logits and the uniform
     float lt = 0.f, ld = 0.f, nx_lt = 0.f, nx_ld = 0.f;
     double U = 0.0, nx_U = 0.0;
     bool tok_ok = true, nx_tok_ok = true;
     int next_item = 0;
 
-    auto fetch_token = [&](int fb, int fj) {   // thread 0
+    auto fetch_token = [&](int fb, int fj) {   // thread kCFetcher
         nx_tok_ok = true;
         if (fj < K) {
             const int tok = p.x[(size_t)fb * K + fj];
@@ -526,7 +530,6 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
         b = nb;
         j = nj;
         if (tid == 0) {
-            lt = nx_lt; ld = nx_ld; U = nx_U; tok_ok = nx_tok_ok;
             // the cluster's next queue entry: one per position, or one per sequence when ordered
             if (rank == 0 && (!ordered || j == 0)) next_item = atomicAdd(&p.heads[0], 1) + p.n_clusters;
         }
@@ -535,7 +538,7 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
     bool have = cluster_id < n_items;
     if (have) {
         const int fb = ordered ? cluster_id : cluster_id / (K + 1), fj = ordered ? 0 : cluster_id % (K + 1);
-        if (tid == 0) fetch_token(fb, fj);
+        if (tid == kCFetcher) fetch_token(fb, fj);
         take_item(fb, fj);
     }
     // barriers of every CTA are initialised before any peer arrives on them
@@ -633,6 +636,9 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
             }
         }
         if (tid == 0) trace_mark(2, 0);
+        // what was fetched ahead for this item goes to shared memory now that the sweep is over (the barrier
+        // of the exchange below orders it before the decision)
+        if (tid == kCFetcher) { sm.tk_lt = nx_lt; sm.tk_ld = nx_ld; sm.tk_U = nx_U; sm.tk_ok = nx_tok_ok ? 1 : 0; }
         // (max, sum) of the warp's share: the maximum first (shuffles only), then one rescale per thread and a sum
         const int par = round & 1;
         {
@@ -682,6 +688,9 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
             float mt, zt, md, zd, wt;
             merge_exchanged<ENT>(sm.xstat[par], sm.xw[par], C * kCWarps, cb, lane, mt, zt, md, zd, wt);
             if (lane == 0) {
+                // what was fetched ahead for this item is taken over only now: the loads (two dependent
+                // misses for the first item of a launch) have had the whole sweep to land
+                lt = sm.tk_lt; ld = sm.tk_ld; U = sm.tk_U; tok_ok = sm.tk_ok != 0;
                 const double Tb = seq_temperature(p, b), betab = seq_beta(p, b);
                 int dec = 1;
                 if (!rowstat_ok(mt, zt) || (pair && (!rowstat_ok(md, zd) || !tok_ok)) || !seq_params_ok(Tb, betab)) dec = -1;
@@ -693,10 +702,12 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
         }
         __syncthreads();
         const int dec = sm.dec;
-        if (tid == 0) {
-            trace_mark(4, dec);
-            // the next item's token, fetched now that the others are released: the loads land while this
-            // item is reported (walking a sequence in order, an accepted position is followed by the next one)
+        if (tid == 0) trace_mark(4, dec);
+        if (tid == kCFetcher) {
+            // the next item's token and its two logits, asked for by a thread of a warp that has nothing to do
+            // until this item is reported (the address of the logits waits for the token: a round trip that the
+            // deciding warp does not have to sit through); the loads land during the next sweep
+            // (walking a sequence in order, an accepted position is followed by the next one)
             if (ordered && pair && dec > 0) fetch_token(b, j + 1);
             else if (q_have) fetch_token(qb, qj);
         }
