@@ -1,5 +1,5 @@
 // Shared-memory pipeline primitives for sm_100a: mbarrier wrappers with bounded
-// waits and the 1-D bulk asynchronous copy (TMA, no multicast) that feeds the
+// waits and the 1-D bulk asynchronous copy (TMA, each CTA for itself) that feeds the
 // streaming kernels.  Every wait gives up after a time limit, records it in a
 // block-wide abort flag and lets the caller unwind; nothing here can spin forever.
 #pragma once

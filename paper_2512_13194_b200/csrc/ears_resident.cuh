@@ -2,8 +2,8 @@
 //
 // Work item = one position of one sequence: the pair (target row k, draft row k), or the
 // extra target row K.  A thread-block cluster of C CTAs takes an item; CTA j brings the j-th
-// slice of the row(s) into its own shared memory with 1-D bulk asynchronous copies (no
-// multicast; element-wise copies when the rows are not 16-byte aligned) and everything else
+// slice of the row(s) into its own shared memory with 1-D bulk asynchronous copies (each
+// CTA fetches for itself; element-wise copies when the rows are not 16-byte aligned) and everything else
 // is computed from there, so that every logit crosses HBM exactly once:
 //
 //   1. softmax statistics (max, sum exp2) of the slices while the copies land [Sec. 3.1];
