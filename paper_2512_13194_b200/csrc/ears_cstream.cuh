@@ -756,10 +756,7 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
                         if (!pair) {
                             p.resid[b] = mass;
                             count_finished(p);
-                        } else {
-                            // the first rejection of a sequence walked in order: whoever draws its token below reads this
-                            p.rowstat[(size_t)b * (K + 1) + j] = make_float4(sm.rs_t.x, sm.rs_t.y, sm.rs_d.x, sm.rs_d.y);
-                        }
+                        }   // (the first rejection of a sequence walked in order: its token is drawn below)
                     }
                 }
             }
@@ -799,27 +796,35 @@ __global__ void __launch_bounds__(kCThreads, kCCtasPerSm) ears_cstream_kernel(co
         if (tid == 0) trace_mark(5, token);
         if (ordered && dec == 0) {
             // The first rejection of a sequence walked in order: every CTA of the cluster knows it, so the
-            // cluster takes the masses of that position at once, each CTA over its own slice, without the
-            // queue; the CTA that is done last draws the token.
+            // cluster takes the masses of that position at once, without the queue: each CTA over its own
+            // slice into shared memory (the area of the extra row's sums is as large and not in use: a
+            // rejected position is not followed by that row), then the cluster-wide pick of step 4.
             const RowNorm rn = make_rownorm(sm.rs_t, sm.rs_d);
-            stream_job_piece<E, true>(trow, drow, e0, e0 + n, vec, rn, cb, warp, lane, p.segsums + (size_t)b * p.nseg);
-            __threadfence();   // the sums (and the writer's rowstat entry) are visible before this CTA counts as done
-            __syncthreads();
-            if (warp == 0) {
-                int last = 0;
-                if (lane == 0) last = ticket_add(&p.ticket2[b]) == C - 1 ? 1 : 0;
-                last = __shfl_sync(0xffffffffu, last, 0);
-                if (last) {
-                    __threadfence();
-                    double jmass = 0.0;
-                    const int jtoken = select_job_token<E>(p, b, j, lane, &jmass);
-                    if (lane == 0) {
-                        p.out_tok[(size_t)b * (K + 1) + j] = jtoken;
-                        p.resid[b] = jmass;
-                        count_finished(p);
-                        trace_mark(7, jtoken);
-                    }
+            double* const segsum = reinterpret_cast<double*>(area);
+            double* so = segsum - e0 / kSegElems;    // sums land at index (entry - e0) / kSegElems
+            const double* ss = segsum;
+            auto val = [ss](int g) { return ss[g]; };
+            int jtoken = -1;
+            bool resid = true;
+            for (;;) {
+                if (resid) stream_job_piece<E, true>(trow, drow, e0, e0 + n, vec, rn, cb, warp, lane, so);
+                else stream_job_piece<E, false>(trow, trow, e0, e0 + n, vec, rn, cb, warp, lane, so);
+                __syncthreads();
+                if (!cluster_pick<E>(sm, p, val, (n + kSegElems - 1) / kSegElems, kSegElems, b, resid, trow, drow, rn, cb, e0, n, rank, C,
+                                     mround, jtoken)) {
+                    failed = true;
+                    break;
                 }
+                // a rejection implies residual mass; if rounding erased it, draw from P_t instead
+                if (resid && !(sm.pick_S * rn.izt >= kTinyMass)) { resid = false; __syncthreads(); continue; }
+                break;
+            }
+            if (failed) break;
+            if (warp == 0 && lane == 0 && (rank == sm.pick_rank || (sm.pick_rank < 0 && rank == 0))) {
+                p.out_tok[(size_t)b * (K + 1) + j] = jtoken;
+                p.resid[b] = sm.pick_S * rn.izt;
+                count_finished(p);
+                trace_mark(7, jtoken);
             }
         }
         // ---- 6. one piece of a published second-pass job, if the look at the start of the round found one waiting
