@@ -380,18 +380,24 @@ int ears_philox_device(const uint32_t* ctr_key, uint32_t* out, int n, void* stre
 int ears_set_plan(int loader, int parts);
 
 /*
- * Choice between the two kernels, for tests and measurements (0 = automatic for both fields):
+ * Choice among the four kernels, for tests and measurements (0 = automatic for both fields):
  *   path 1 = streaming kernel with a ring of shared-memory slots filled by bulk copies (the rows of
- *            a rejected position are read a second time), 3 = streaming kernel whose warps read
- *            straight from global memory (same second pass), 2 = resident kernel (the two rows of a
- *            position stay in the shared memory of a thread-block cluster; every logit is read
- *            once).  Forcing path 2 on a shape whose rows do not fit a cluster makes the
- *            verification calls return EARS_ERR_SHAPE.  A non-zero `parts` of ears_set_plan
- *            also selects the streaming kernel.
- *   cluster = CTAs per cluster of the resident kernel: 1, 2, 4, 8 or 16.
- * Both kernels implement the same step (Sec. 3.1-3.3); results differ only through
+ *            a rejected position are read a second time);
+ *        3 = streaming kernel whose warps read straight from global memory (same second pass);
+ *        2 = resident kernel (the two rows of a position stay in the shared memory of a
+ *            thread-block cluster; every logit is read once);
+ *        4 = cluster-streamed kernel (the same clusters stream their slices instead of holding
+ *            them; per sequence only the rows of the first rejected position are read again, in
+ *            pieces that all CTAs of the launch serve; with EARS_FLAG_STOP_AT_FIRST_REJECT nothing
+ *            after a first rejection is read).
+ *            Forcing path 2 or 4 on a shape it cannot take (rows that do not fit a cluster's
+ *            shared memory) makes the verification calls return EARS_ERR_SHAPE.  A non-zero
+ *            `parts` of ears_set_plan also selects the ring kernel.
+ *   cluster = CTAs per cluster of paths 2 and 4: 1, 2, 4, 8 or 16.
+ * All kernels implement the same step (Sec. 3.1-3.3); results differ only through
  * floating-point summation order.  The initial values can also come from the environment,
- * read once when the library is loaded: EARS_PATH=streaming|resident|direct, EARS_CLUSTER=1|2|4|8|16.
+ * read once when the library is loaded: EARS_PATH=streaming|resident|direct|cluster-streamed (or 1..4),
+ * EARS_CLUSTER=1|2|4|8|16.
  */
 int ears_set_path(int path, int cluster);
 

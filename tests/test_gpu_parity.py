@@ -80,7 +80,7 @@ def forced_path(ears):
 @pytest.mark.parametrize("B,K,V,dtype", SHAPES)
 def test_parity_shapes(ears, forced_path, B, K, V, dtype, path, cluster):
     """Tiny to medium cases: several chunks, ragged tails, unaligned rows (element-wise loader),
-    empty slices in large clusters; under both kernels."""
+    empty slices in large clusters; under every kernel and cluster size."""
     forced_path(path, cluster)
     tally = Tally()
     for seed, (T, beta) in enumerate([(1.0, 0.0), (0.8, 0.3), (1.3, 1.0)]):
