@@ -153,10 +153,11 @@ int ears_verify_ex(int dtype, const void* target_logits, const void* draft_logit
  *               (later rows and tokens, and the extra target row unless everything was accepted)
  *               is not part of the step: it is not validated and the optional per-position
  *               outputs are not written there; lengths and tokens are the same as without the
- *               flag on valid data.  Where the resident kernel runs (see ears_set_path) those rows
- *               are not even read -- a cluster then walks a sequence position by position -- which
- *               saves their HBM traffic at the price of a longer chain per sequence; the
- *               streaming kernel reads them anyway and ignores them.
+ *               flag on valid data.  Where a cluster kernel runs (the resident kernel for short
+ *               rows, the cluster-streamed kernel from four sequences per SM on; see
+ *               ears_set_path) those rows are not even read -- a cluster then walks a sequence
+ *               position by position -- which saves their HBM traffic at the price of a longer
+ *               chain per sequence; the other streaming kernels read them anyway and ignore them.
  * Everything else is as in ears_verify_ex.
  */
 #define EARS_FLAG_STOP_AT_FIRST_REJECT 1u
